@@ -1,0 +1,223 @@
+"""ctypes front end of the CPU checker (``ec_oracle.cpp``).  TEST INFRASTRUCTURE ONLY.
+
+Only the tests, the smoke check and the benchmark's CPU-baseline leg may import
+this package; the GPU library and its Python binding never do.  All arguments
+are numpy arrays in host memory.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "ec_oracle.cpp")
+_LIB = os.path.join(_HERE, "libec_oracle.so")
+
+F32, BF16, I64, F64 = 0, 1, 2, 3
+SUM, MAX, MIN = 0, 1, 2
+ORDER_FIXED, ORDER_PAIRWISE = 0, 1
+
+_IN_NP = {F32: np.float32, BF16: np.uint16, I64: np.int64, F64: np.float64}
+_OUT_NP = {F32: np.float32, BF16: np.float32, I64: np.int64, F64: np.float64}
+
+CXXFLAGS = ["-O2", "-ffp-contract=off", "-fno-fast-math", "-fopenmp", "-fPIC", "-shared", "-std=c++17"]
+
+
+def build(force: bool = False) -> str:
+    """Compile the checker with g++ (plain -O2, no contraction, no fast-math)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        subprocess.check_call(["g++", *CXXFLAGS, "-o", _LIB, _SRC])
+    return _LIB
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    global _lib
+    if _lib is None:
+        L = C.CDLL(build())
+        L.oracle_allreduce_new.restype = C.c_void_p
+        L.oracle_allreduce_new.argtypes = [C.c_int, C.c_size_t, C.c_int, C.c_int, C.c_size_t]
+        L.oracle_allreduce_free.argtypes = [C.c_void_p]
+        L.oracle_allreduce_reset.argtypes = [C.c_void_p]
+        L.oracle_allreduce_apply.restype = C.c_int
+        L.oracle_allreduce_apply.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                             C.c_int, C.c_int]
+        L.oracle_allreduce_applied.argtypes = [C.c_void_p, C.c_void_p]
+        L.oracle_allreduce_oneshot.restype = C.c_int
+        L.oracle_allreduce_oneshot.argtypes = [C.c_int, C.c_size_t, C.c_int, C.c_int, C.c_size_t,
+                                               C.c_void_p, C.c_void_p, C.c_void_p]
+        L.oracle_allreduce_ref64.restype = C.c_int
+        L.oracle_allreduce_ref64.argtypes = [C.c_int, C.c_size_t, C.c_int, C.c_size_t, C.c_void_p,
+                                             C.c_void_p, C.c_void_p, C.c_void_p]
+        L.oracle_allgatherv.restype = C.c_int
+        L.oracle_allgatherv.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_size_t, C.c_void_p,
+                                        C.c_void_p, C.c_void_p, C.c_size_t]
+        L.oracle_kmeans_assign.argtypes = [C.c_void_p, C.c_size_t, C.c_int, C.c_void_p, C.c_int,
+                                           C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int]
+        L.oracle_kmeans_partials.argtypes = [C.c_void_p, C.c_size_t, C.c_int, C.c_int, C.c_int,
+                                             C.c_void_p, C.c_void_p, C.c_int]
+        L.oracle_kmeans_update.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p]
+        L.oracle_max_threads.restype = C.c_int
+        _lib = L
+    return _lib
+
+
+def max_threads() -> int:
+    return int(lib().oracle_max_threads())
+
+
+def _ptr(a):
+    return None if a is None else a.ctypes.data_as(C.c_void_p)
+
+
+def _ptr_table(bufs, dtype_np):
+    keep = [np.ascontiguousarray(b, dtype=dtype_np) for b in bufs]
+    table = (C.c_void_p * len(keep))(*[b.ctypes.data for b in keep])
+    return keep, table
+
+
+class Allreduce:
+    """State of one eventually consistent allreduce (which contributions are
+    already folded into ``result``) plus the apply/reset calls."""
+
+    def __init__(self, P: int, n: int, dtype: int, op: int, segment_size: int):
+        self.P, self.n, self.dtype, self.op, self.seg = P, n, dtype, op, segment_size
+        self.S = (n + segment_size - 1) // segment_size
+        self.W = (P + 63) // 64
+        self._h = lib().oracle_allreduce_new(P, n, dtype, op, segment_size)
+        if not self._h:
+            raise ValueError("bad allreduce parameters")
+
+    def __del__(self):
+        if getattr(self, "_h", None):
+            lib().oracle_allreduce_free(self._h)
+            self._h = None
+
+    def reset(self) -> None:
+        lib().oracle_allreduce_reset(self._h)
+
+    def apply(self, bufs, arrival_mask, result: np.ndarray, contrib_count: np.ndarray | None = None,
+              order: int = ORDER_FIXED, threads: int = 1) -> None:
+        """Fold the newly notified contributions into ``result`` (in place)."""
+        assert len(bufs) == self.P
+        keep, table = _ptr_table(bufs, _IN_NP[self.dtype])
+        for b in keep:
+            assert b.size >= self.n
+        assert result.dtype == _OUT_NP[self.dtype] and result.flags.c_contiguous and result.size >= self.n
+        if arrival_mask is not None:
+            arrival_mask = np.ascontiguousarray(arrival_mask, dtype=np.uint64)
+            assert arrival_mask.size == self.S * self.W
+        if contrib_count is not None:
+            assert contrib_count.dtype == np.uint32 and contrib_count.size >= self.S
+        rc = lib().oracle_allreduce_apply(self._h, table, _ptr(arrival_mask), _ptr(result),
+                                          _ptr(contrib_count), order, threads)
+        if rc != 0:
+            raise RuntimeError("oracle_allreduce_apply failed")
+
+    def applied(self) -> np.ndarray:
+        out = np.zeros((self.P, self.S), dtype=np.uint8)
+        lib().oracle_allreduce_applied(self._h, _ptr(out))
+        return out.astype(bool)
+
+
+def allreduce_oneshot(bufs, dtype: int, op: int, segment_size: int, order: np.ndarray) -> np.ndarray:
+    """Fold each segment once, left to right through ``order`` (int32 [S][P], -1 ends a row)."""
+    P = len(bufs)
+    keep, table = _ptr_table(bufs, _IN_NP[dtype])
+    n = keep[0].size
+    order = np.ascontiguousarray(order, dtype=np.int32)
+    result = np.empty(n, dtype=_OUT_NP[dtype])
+    rc = lib().oracle_allreduce_oneshot(P, n, dtype, op, segment_size, table, _ptr(order), _ptr(result))
+    if rc != 0:
+        raise RuntimeError("oracle_allreduce_oneshot failed")
+    return result
+
+
+def allreduce_ref64(bufs, dtype: int, segment_size: int, arrival_mask=None):
+    """(double-precision sum over notified ranks, sum of magnitudes) per element."""
+    P = len(bufs)
+    keep, table = _ptr_table(bufs, _IN_NP[dtype])
+    n = keep[0].size
+    if arrival_mask is not None:
+        arrival_mask = np.ascontiguousarray(arrival_mask, dtype=np.uint64)
+    ref = np.empty(n, dtype=np.float64)
+    mag = np.empty(n, dtype=np.float64)
+    rc = lib().oracle_allreduce_ref64(P, n, dtype, segment_size, table, _ptr(arrival_mask), _ptr(ref), _ptr(mag))
+    if rc != 0:
+        raise RuntimeError("oracle_allreduce_ref64 failed")
+    return ref, mag
+
+
+def allgatherv(bufs, counts: np.ndarray, arrival_mask, out: np.ndarray):
+    """Returns (displs int64 [P+1], status); copies notified ranks into ``out`` in place."""
+    P = len(bufs)
+    counts = np.ascontiguousarray(counts, dtype=np.int64)
+    keep = [np.ascontiguousarray(b) for b in bufs]
+    for r, b in enumerate(keep):
+        assert b.dtype == out.dtype and b.size >= counts[r]
+    table = (C.c_void_p * P)(*[b.ctypes.data for b in keep])
+    if arrival_mask is not None:
+        arrival_mask = np.ascontiguousarray(arrival_mask, dtype=np.uint64)
+    displs = np.empty(P + 1, dtype=np.int64)
+    assert out.flags.c_contiguous
+    status = lib().oracle_allgatherv(table, _ptr(counts), P, out.dtype.itemsize, _ptr(arrival_mask),
+                                     _ptr(displs), _ptr(out), out.size)
+    return displs, int(status)
+
+
+def kmeans_assign(points: np.ndarray, centroids: np.ndarray, threads: int = 1):
+    """Returns (labels int32, best d^2, second-best d^2, second-best label)."""
+    points = np.ascontiguousarray(points, dtype=np.float32)
+    centroids = np.ascontiguousarray(centroids, dtype=np.float32)
+    N, D = points.shape
+    K = centroids.shape[0]
+    labels = np.empty(N, dtype=np.int32)
+    best = np.empty(N, dtype=np.float64)
+    second = np.empty(N, dtype=np.float64)
+    second_label = np.empty(N, dtype=np.int32)
+    lib().oracle_kmeans_assign(_ptr(points), N, D, _ptr(centroids), K, _ptr(labels), _ptr(best),
+                               _ptr(second), _ptr(second_label), threads)
+    return labels, best, second, second_label
+
+
+def kmeans_partials(points: np.ndarray, labels: np.ndarray, K: int, P: int, threads: int = 1) -> np.ndarray:
+    """fp32 [P][K][D+4]: per rank and centroid the coordinate sums, the point count, three zeros."""
+    points = np.ascontiguousarray(points, dtype=np.float32)
+    labels = np.ascontiguousarray(labels, dtype=np.int32)
+    N, D = points.shape
+    out = np.empty((P, K, D + 4), dtype=np.float32)
+    lib().oracle_kmeans_partials(_ptr(points), N, D, K, P, _ptr(labels), _ptr(out), threads)
+    return out
+
+
+def kmeans_update(reduced: np.ndarray, old_centroids: np.ndarray) -> np.ndarray:
+    reduced = np.ascontiguousarray(reduced, dtype=np.float32)
+    old_centroids = np.ascontiguousarray(old_centroids, dtype=np.float32)
+    K, D = old_centroids.shape
+    assert reduced.shape == (K, D + 4)
+    new = np.empty_like(old_centroids)
+    lib().oracle_kmeans_update(_ptr(reduced), D, K, _ptr(old_centroids), _ptr(new))
+    return new
+
+
+def kmeans_iterate(points: np.ndarray, centroids: np.ndarray, P: int, arrival_mask, threads: int = 1):
+    """One Lloyd iteration whose combine step is one eventually consistent
+    allreduce epoch with one segment per centroid row: assignment, per-rank
+    partials, a single apply with this iteration's notifications (late rows are
+    dropped; the next iteration supersedes them), centroid update.
+    Returns (new centroids, labels, reduced [K][D+4], contrib_count [K])."""
+    K, D = centroids.shape
+    labels, _, _, _ = kmeans_assign(points, centroids, threads)
+    partials = kmeans_partials(points, labels, K, P, threads)
+    n = K * (D + 4)
+    ar = Allreduce(P, n, F32, SUM, D + 4)
+    reduced = np.empty(n, dtype=np.float32)
+    count = np.empty(K, dtype=np.uint32)
+    ar.apply([partials[r].reshape(-1) for r in range(P)], arrival_mask, reduced, count)
+    reduced = reduced.reshape(K, D + 4)
+    return kmeans_update(reduced, centroids), labels, reduced, count
