@@ -1,0 +1,234 @@
+/*
+ * ec.h - eventually consistent collectives on one B200: C ABI.
+ *
+ * P simulated ranks live as buffers in one GPU's memory.  Every (rank, segment)
+ * contribution carries an arrival notification (one bit).  The collectives
+ * produce their result from whatever has arrived, report how much took part,
+ * and fold late contributions in when they land.
+ *
+ * General rules for every entry point
+ *   - extern "C"; returns int: EC_OK (0) or a negative EC_ERR_* code.  Nothing
+ *     throws, exits, or synchronises the device.
+ *   - "device" pointers are CUDA device addresses valid on the current device;
+ *     "host" pointers are ordinary process memory.  The caller owns every buffer
+ *     it passes; the library owns only its context objects (and a workspace it
+ *     allocated itself when the caller passed none).
+ *   - All device work is enqueued on `stream` (a cudaStream_t; NULL = the legacy
+ *     default stream).  Buffers and notification words must stay valid and
+ *     unmodified until that work has completed.  Notification words are read on
+ *     the device when the kernel runs, so a producer may set bits in stream
+ *     order right up to the call ("write early, check late", Sec. II).
+ *   - A context is not thread-safe and expects its calls in one stream order;
+ *     distinct contexts are independent.
+ *
+ * Notification words (Sec. II: data is usable once its notification is
+ * visible): uint64 [S][W] on the device, W = ceil(P/64); the notification of
+ * rank r for segment s is bit (r % 64) of word [s][r / 64].  Bits at or above P
+ * are ignored.  Words are cumulative inside an epoch; a bit that is cleared
+ * after its contribution was folded in is ignored (nothing is un-applied).
+ * A contribution whose bit is 0 is never read.
+ */
+#ifndef EC_H_
+#define EC_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct CUstream_st* ec_stream_t; /* the same type as cudaStream_t */
+
+typedef enum {
+    EC_F32 = 0,  /* fp32 in, fp32 accumulate, fp32 out */
+    EC_BF16 = 1, /* raw bfloat16 bits in, widened exactly, fp32 accumulate, fp32 out */
+    EC_I64 = 2,  /* int64 in/out; sum wraps modulo 2^64 */
+    EC_F64 = 3   /* fp64 in/out (the element type of the paper's experiments) */
+} ec_dtype_t;
+
+typedef enum {
+    EC_SUM = 0, /* the paper's "global sum" (Sec. IV-A) */
+    EC_MAX = 1, /* acc = (x > acc) ? x : acc */
+    EC_MIN = 2  /* acc = (x < acc) ? x : acc */
+} ec_op_t;
+
+typedef enum {
+    EC_ORDER_FIXED = 0,   /* each apply folds its new ranks in ascending rank order: reproducible bits */
+    EC_ORDER_PAIRWISE = 1 /* balanced tree over the rank index (float sum only): smaller rounding error */
+} ec_order_t;
+
+enum {
+    EC_OK = 0,
+    EC_ERR_INVALID = -1,     /* NULL / zero / inconsistent argument */
+    EC_ERR_UNSUPPORTED = -2, /* combination of dtype, op and order that is not implemented */
+    EC_ERR_CUDA = -3,        /* a CUDA runtime call failed; see ec_last_cuda_error() */
+    EC_ERR_STATE = -4,       /* call not allowed in the context's current state */
+    EC_ERR_CAPACITY = -5     /* a size exceeds a stated limit or a workspace is too small */
+};
+
+#define EC_MAX_RANKS 1024 /* largest P any call accepts */
+
+typedef struct ec_ctx ec_ctx_t;
+typedef struct ec_kmeans ec_kmeans_t;
+
+/* ------------------------------------------------------------------------- *
+ * Eventually consistent allreduce.
+ *
+ * Follows the Scatter-Reduce stage of the segmented pipelined ring (Sec. IV-A):
+ * the vector is cut into segments that are reduced independently, here all on
+ * one device, so the P-1 ring steps of a segment collapse into one pass over
+ * the P rank buffers.  The consistency rule is the paper's (Sec. II, Sec. III):
+ * only notified contributions are used; the status output says how many ranks
+ * are in each segment's result ("threshold" and "status" parameters); once
+ * every notification has been seen the result is the complete reduction
+ * (end of Sec. IV-A).
+ *
+ * n elements per rank, segments of segment_size elements (the last may be
+ * short), S = ceil(n / segment_size).
+ * ------------------------------------------------------------------------- */
+
+/* Bytes of device workspace a context needs (two copies of the "already folded
+ * in" words, 256-byte aligned).  0 on invalid arguments. */
+size_t ec_allreduce_workspace_bytes(int P, size_t n, size_t segment_size);
+
+/* Create a context.  `workspace` is device memory of at least
+ * ec_allreduce_workspace_bytes() bytes, 256-byte aligned, owned by the caller
+ * and kept alive until destroy; NULL lets the library cudaMalloc it (and free it
+ * in destroy).  The workspace is cleared with a cudaMemsetAsync on the legacy
+ * default stream followed by a stream synchronise, so init must not be called
+ * during stream capture.  Pairwise order is accepted only for EC_SUM on a
+ * floating dtype (else EC_ERR_UNSUPPORTED). */
+int ec_allreduce_init(ec_ctx_t** ctx, int P, size_t n, ec_dtype_t dtype, ec_op_t op, size_t segment_size,
+                      ec_order_t order, void* workspace, size_t workspace_bytes);
+
+/* One apply = one round: fold every contribution that is notified now and was
+ * not folded in by an earlier apply of this epoch.
+ *
+ *   rank_bufs      HOST array of P DEVICE pointers; rank r's vector of n elements
+ *                  of the context's input type.  Read during the call (copied
+ *                  into the launch), so it may be reused at once.
+ *   P, n, dtype, op, segment_size
+ *                  must equal the values given to init (EC_ERR_INVALID if not).
+ *   arrival_mask   device uint64 [S][W]; NULL means everything has arrived.
+ *   result         device, n elements of the output type (fp32 for EC_F32 and
+ *                  EC_BF16, int64, fp64).  In/out across the applies of an epoch.
+ *                  Must not alias a rank buffer.
+ *   contrib_count  device uint32 [S], or NULL.  After the call contrib_count[s]
+ *                  = number of ranks folded into segment s so far this epoch
+ *                  (= popcount of the cumulative words restricted to bits < P).
+ *
+ * Per segment: if no rank was folded in before, the accumulator starts from the
+ * operator's identity (+0.0; -inf / +inf; 0; INT64_MIN / INT64_MAX) and `result`
+ * is not read; otherwise it starts from `result`.  The new ranks are folded in
+ * ascending rank order (EC_ORDER_FIXED) or as a balanced tree whose root is then
+ * added (EC_ORDER_PAIRWISE).  The first apply of an epoch writes the identity to
+ * segments without any contribution, so `result` is fully defined after it;
+ * later applies neither read nor write segments without new arrivals.
+ *
+ * 16-byte aligned pointers together with segment_size * sizeof(input element)
+ * divisible by 16 take the 128-bit path; anything else is still correct through
+ * an element-wise path.  One kernel launch, no allocation. */
+int ec_allreduce_apply(ec_ctx_t* ctx, const void* const* rank_bufs, int P, size_t n, ec_dtype_t dtype,
+                       ec_op_t op, size_t segment_size, const uint64_t* arrival_mask, void* result,
+                       uint32_t* contrib_count, ec_stream_t stream);
+
+/* Start a new epoch: forget which contributions were folded in (the counterpart
+ * of resetting notifications, Sec. II / Sec. IV-B).  `result` is not touched; the
+ * next apply overwrites it. */
+int ec_allreduce_reset(ec_ctx_t* ctx, ec_stream_t stream);
+
+/* Expert knob: elements of one segment handled per thread block (rounded to the
+ * vector width) and threads per block (64..512, multiple of 32).  0 keeps the
+ * current value.  Affects speed only, never results. */
+int ec_allreduce_set_tile(ec_ctx_t* ctx, int threads, size_t tile_elems);
+
+/* Free the context (and its workspace if the library allocated it).  The caller
+ * makes sure no work of this context is still running. */
+int ec_allreduce_destroy(ec_ctx_t* ctx);
+
+/* ------------------------------------------------------------------------- *
+ * Eventually consistent allgatherv.
+ *
+ * Every rank owns a fixed slot, as every chunk has a fixed place in the ring's
+ * Allgather stage (Sec. IV-A) and every writer its own target and notification
+ * in the AlltoAll (Sec. IV-B): displs is the exclusive prefix sum of the counts
+ * of ALL ranks, arrived or not, and displs[P] the total.  Ranks whose bit is
+ * set are copied into their slot; the slots of the others are left untouched
+ * (a late rank is one more call with its bit set).  Stateless.
+ *
+ *   bufs           HOST array of P DEVICE pointers (rank r: counts[r] elements).
+ *                  Entries of ranks that are not notified may be NULL.
+ *   counts         device int64 [P], each >= 0.
+ *   dtype          element type (sets the element size: 4, 2, 8, 8 bytes).
+ *   arrival_mask   device uint64 [W], one bit per rank; NULL = all arrived.
+ *   displs         device int64 [P+1], written.
+ *   out            device, out_capacity_elems elements.
+ *   status         device uint32, written: 0 = done; 1 = the total exceeds
+ *                  out_capacity_elems or a count is negative - then displs is
+ *                  still written but not a byte of `out`.
+ * One kernel launch (prefix sum and copy fused), no allocation. */
+int ec_allgatherv(const void* const* bufs, const int64_t* counts, int P, ec_dtype_t dtype,
+                  const uint64_t* arrival_mask, int64_t* displs, void* out, size_t out_capacity_elems,
+                  uint32_t* status, ec_stream_t stream);
+
+/* ------------------------------------------------------------------------- *
+ * K-means driver: Lloyd iterations whose combine step is the allreduce above.
+ * (The paper's iterative-convergent ML workload is a matrix factorisation on a
+ * data set that is not available; K-means takes its place as the data-parallel
+ * solver that tolerates missing contributions, Sec. I and Sec. III.)
+ *
+ * N points of D coordinates, row-major fp32 [N][D]; K centroids fp32 [K][D];
+ * rank r owns points [r*N/P, (r+1)*N/P).  Per-rank partials are fp32
+ * [P][K][D+4]: columns 0..D-1 the coordinate sums of the rank's points with that
+ * label, column D their number, D+1..D+3 zero.  One iteration = assignment
+ * (label = nearest centroid by squared Euclidean distance computed as
+ * sum_d (x-c)^2 in fp32, lowest index on a tie), partials, one allreduce epoch
+ * (reset + one apply, segment = one centroid row of D+4 elements, so a rank's
+ * sums and count for a centroid arrive together; contributions that are not
+ * notified are dropped for this iteration), centroid update (sum / points; a
+ * centroid without points stays where it was).
+ * Limits: 1 <= D <= 128 and D % 4 == 0; 1 <= K <= 1024; 1 <= P <= EC_MAX_RANKS.
+ * ------------------------------------------------------------------------- */
+size_t ec_kmeans_workspace_bytes(size_t N, int D, int K, int P);
+
+/* points and init_centroids are device pointers; points must stay valid for the
+ * life of the context (they are not copied), init_centroids are copied in on the
+ * legacy default stream (synchronised before return).  workspace as for the
+ * allreduce (NULL = library allocates). */
+int ec_kmeans_init(ec_kmeans_t** km, const float* points, size_t N, int D, int K, int P,
+                   const float* init_centroids, void* workspace, size_t workspace_bytes);
+
+/* Assignment alone: labels[j] for the given device centroids [K][D]. */
+int ec_kmeans_assign(ec_kmeans_t* km, const float* centroids, int32_t* labels, ec_stream_t stream);
+
+/* Partials alone: device labels [N] -> device partials [P][K][D+4].  Sums are
+ * accumulated in a fixed order (no floating-point atomics): same bits every run. */
+int ec_kmeans_partials(ec_kmeans_t* km, const int32_t* labels, float* partials, ec_stream_t stream);
+
+/* One full iteration on the context's own centroids.  arrival_mask: device
+ * uint64 [K][W] for this iteration, NULL = all arrived. */
+int ec_kmeans_iterate(ec_kmeans_t* km, const uint64_t* arrival_mask, ec_stream_t stream);
+
+/* Replace the context's centroids (device [K][D]); used for lock-step checks. */
+int ec_kmeans_set_centroids(ec_kmeans_t* km, const float* centroids, ec_stream_t stream);
+
+/* Copy out (device to device, on `stream`) whichever outputs are non-NULL:
+ * centroids [K][D], labels [N] and reduced [K][D+4] and contrib_count [K] of the
+ * last iteration. */
+int ec_kmeans_get(ec_kmeans_t* km, float* centroids, int32_t* labels, float* reduced,
+                  uint32_t* contrib_count, ec_stream_t stream);
+
+int ec_kmeans_destroy(ec_kmeans_t* km);
+
+/* ------------------------------------------------------------------------- */
+const char* ec_strerror(int code);
+/* The cudaError_t of the last failed CUDA call on this thread (0 if none). */
+int ec_last_cuda_error(void);
+/* Library version, major * 1000 + minor. */
+int ec_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* EC_H_ */

@@ -1,0 +1,201 @@
+"""Thin ctypes binding of ``libec_b200.so`` (the C ABI of ``include/ec.h``).
+
+Argument marshalling only: every step of the collectives runs in the CUDA
+kernels of the library.  PyTorch supplies device memory and streams.  There is
+no CPU fallback: if the library cannot be loaded, importing a symbol raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libec_b200.so")
+
+F32, BF16, I64, F64 = 0, 1, 2, 3
+SUM, MAX, MIN = 0, 1, 2
+ORDER_FIXED, ORDER_PAIRWISE = 0, 1
+MAX_RANKS = 1024
+
+OK, ERR_INVALID, ERR_UNSUPPORTED, ERR_CUDA, ERR_STATE, ERR_CAPACITY = 0, -1, -2, -3, -4, -5
+
+IN_TORCH = {F32: torch.float32, BF16: torch.bfloat16, I64: torch.int64, F64: torch.float64}
+OUT_TORCH = {F32: torch.float32, BF16: torch.float32, I64: torch.int64, F64: torch.float64}
+
+# every symbol include/ec.h declares: (restype, argtypes)
+_vp, _sz, _i, _u64 = C.c_void_p, C.c_size_t, C.c_int, C.c_uint64
+SYMBOLS = {
+    "ec_allreduce_workspace_bytes": (_sz, [_i, _sz, _sz]),
+    "ec_allreduce_init": (_i, [C.POINTER(_vp), _i, _sz, _i, _i, _sz, _i, _vp, _sz]),
+    "ec_allreduce_apply": (_i, [_vp, _vp, _i, _sz, _i, _i, _sz, _vp, _vp, _vp, _vp]),
+    "ec_allreduce_reset": (_i, [_vp, _vp]),
+    "ec_allreduce_set_tile": (_i, [_vp, _i, _sz]),
+    "ec_allreduce_destroy": (_i, [_vp]),
+    "ec_allgatherv": (_i, [_vp, _vp, _i, _i, _vp, _vp, _vp, _sz, _vp, _vp]),
+    "ec_kmeans_workspace_bytes": (_sz, [_sz, _i, _i, _i]),
+    "ec_kmeans_init": (_i, [C.POINTER(_vp), _vp, _sz, _i, _i, _i, _vp, _vp, _sz]),
+    "ec_kmeans_assign": (_i, [_vp, _vp, _vp, _vp]),
+    "ec_kmeans_partials": (_i, [_vp, _vp, _vp, _vp]),
+    "ec_kmeans_iterate": (_i, [_vp, _vp, _vp]),
+    "ec_kmeans_set_centroids": (_i, [_vp, _vp, _vp]),
+    "ec_kmeans_get": (_i, [_vp, _vp, _vp, _vp, _vp, _vp]),
+    "ec_kmeans_destroy": (_i, [_vp]),
+    "ec_strerror": (C.c_char_p, [_i]),
+    "ec_last_cuda_error": (_i, []),
+    "ec_version": (_i, []),
+}
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Load the CUDA library; raises if it was not built (no fallback exists)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2203_17063_b200.build` "
+                "(there is no CPU fallback)")
+        L = C.CDLL(LIB_PATH)
+        for name, (res, args) in SYMBOLS.items():
+            fn = getattr(L, name)
+            fn.restype = res
+            fn.argtypes = args
+        _lib = L
+    return _lib
+
+
+class EcError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        msg = lib().ec_strerror(code).decode()
+        if code == ERR_CUDA:
+            msg += f" [cudaError {lib().ec_last_cuda_error()}]"
+        super().__init__(f"{where}: {msg} ({code})")
+
+
+def _check(code: int, where: str) -> None:
+    if code != OK:
+        raise EcError(code, where)
+
+
+def _ptr(t) -> int | None:
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    return t.data_ptr()
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        return torch.cuda.current_stream().cuda_stream
+    if isinstance(stream, int):
+        return stream
+    return stream.cuda_stream
+
+
+def _table(bufs):
+    return (C.c_void_p * len(bufs))(*[_ptr(b) for b in bufs])
+
+
+class Allreduce:
+    """ec_allreduce_init / apply / reset / destroy for one (P, n, dtype, op, segment_size)."""
+
+    def __init__(self, P: int, n: int, dtype: int, op: int, segment_size: int, order: int = ORDER_FIXED,
+                 device="cuda"):
+        L = lib()
+        self.P, self.n, self.dtype, self.op, self.seg, self.order = P, n, dtype, op, segment_size, order
+        self.S = (n + segment_size - 1) // segment_size if segment_size else 0
+        self.W = (P + 63) // 64
+        need = L.ec_allreduce_workspace_bytes(P, n, segment_size)
+        self._ws = torch.empty(max(need, 256), dtype=torch.uint8, device=device) if need else None
+        h = C.c_void_p()
+        _check(L.ec_allreduce_init(C.byref(h), P, n, dtype, op, segment_size, order,
+                                   _ptr(self._ws), need), "ec_allreduce_init")
+        self._h = h
+
+    def apply(self, rank_bufs, arrival_mask, result, contrib_count=None, stream=None) -> None:
+        _check(lib().ec_allreduce_apply(self._h, _table(rank_bufs), len(rank_bufs), self.n, self.dtype, self.op,
+                                        self.seg, _ptr(arrival_mask), _ptr(result), _ptr(contrib_count),
+                                        _stream(stream)), "ec_allreduce_apply")
+
+    def apply_raw(self, table, arrival_mask_ptr, result_ptr, count_ptr, stream_ptr) -> int:
+        """Same call with pre-marshalled arguments (for timing loops); returns the status code."""
+        return lib().ec_allreduce_apply(self._h, table, self.P, self.n, self.dtype, self.op, self.seg,
+                                        arrival_mask_ptr, result_ptr, count_ptr, stream_ptr)
+
+    def reset(self, stream=None) -> None:
+        _check(lib().ec_allreduce_reset(self._h, _stream(stream)), "ec_allreduce_reset")
+
+    def set_tile(self, threads: int = 0, tile_elems: int = 0) -> None:
+        _check(lib().ec_allreduce_set_tile(self._h, threads, tile_elems), "ec_allreduce_set_tile")
+
+    def destroy(self) -> None:
+        if getattr(self, "_h", None):
+            lib().ec_allreduce_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+
+def allgatherv(bufs, counts, dtype: int, arrival_mask, displs, out, status, stream=None,
+               out_capacity_elems: int | None = None) -> None:
+    """ec_allgatherv: counts/displs/out/status are device tensors, bufs a list of device tensors (or None)."""
+    cap = out.numel() if out_capacity_elems is None else out_capacity_elems
+    _check(lib().ec_allgatherv(_table(bufs), _ptr(counts), len(bufs), dtype, _ptr(arrival_mask), _ptr(displs),
+                               _ptr(out), cap, _ptr(status), _stream(stream)), "ec_allgatherv")
+
+
+class KMeans:
+    """ec_kmeans_* on device tensors: points fp32 [N][D], centroids fp32 [K][D]."""
+
+    def __init__(self, points: torch.Tensor, K: int, P: int, init_centroids: torch.Tensor):
+        L = lib()
+        assert points.is_cuda and points.dtype == torch.float32 and points.is_contiguous()
+        assert init_centroids.is_cuda and init_centroids.dtype == torch.float32 and init_centroids.is_contiguous()
+        self.N, self.D = points.shape
+        self.K, self.P = K, P
+        self.points = points                      # keep alive: the library does not copy them
+        need = L.ec_kmeans_workspace_bytes(self.N, self.D, K, P)
+        self._ws = torch.empty(max(need, 256), dtype=torch.uint8, device=points.device) if need else None
+        h = C.c_void_p()
+        _check(L.ec_kmeans_init(C.byref(h), _ptr(points), self.N, self.D, K, P, _ptr(init_centroids),
+                                _ptr(self._ws), need), "ec_kmeans_init")
+        self._h = h
+
+    def assign(self, centroids, labels, stream=None) -> None:
+        _check(lib().ec_kmeans_assign(self._h, _ptr(centroids), _ptr(labels), _stream(stream)), "ec_kmeans_assign")
+
+    def partials(self, labels, partials, stream=None) -> None:
+        _check(lib().ec_kmeans_partials(self._h, _ptr(labels), _ptr(partials), _stream(stream)), "ec_kmeans_partials")
+
+    def iterate(self, arrival_mask=None, stream=None) -> None:
+        _check(lib().ec_kmeans_iterate(self._h, _ptr(arrival_mask), _stream(stream)), "ec_kmeans_iterate")
+
+    def iterate_raw(self, mask_ptr, stream_ptr) -> int:
+        return lib().ec_kmeans_iterate(self._h, mask_ptr, stream_ptr)
+
+    def set_centroids(self, centroids, stream=None) -> None:
+        _check(lib().ec_kmeans_set_centroids(self._h, _ptr(centroids), _stream(stream)), "ec_kmeans_set_centroids")
+
+    def get(self, centroids=None, labels=None, reduced=None, contrib_count=None, stream=None) -> None:
+        _check(lib().ec_kmeans_get(self._h, _ptr(centroids), _ptr(labels), _ptr(reduced), _ptr(contrib_count),
+                                   _stream(stream)), "ec_kmeans_get")
+
+    def destroy(self) -> None:
+        if getattr(self, "_h", None):
+            lib().ec_kmeans_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass

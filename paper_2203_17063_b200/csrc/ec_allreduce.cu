@@ -1,0 +1,544 @@
+// Eventually consistent allreduce: the segment-wise combine of P rank buffers.
+//
+// One launch per apply.  A thread block owns one tile of one segment.  Its first
+// warp reads the segment's notification words and the "already folded in" words,
+// takes the difference (what is new), and - by ballot - decides whether the
+// segment has news at all and whether it ever had a contributor.  The block then
+// streams the tile of every new rank with 128-bit loads, folds in ascending rank
+// order (or as a pairwise tree) and writes the result tile.  The block of tile 0
+// also writes the segment's updated words and its contributor count.  The folded
+// words are double buffered (read one copy, write the other) so that no block can
+// see another block's update: there is no inter-block dependency and no wait.
+//
+// Follows Sec. IV-A (each chunk of the vector is reduced independently, global
+// sum), Sec. II (a contribution is used only once its notification is visible)
+// and Sec. III (status output: how many took part).
+
+#include <new>
+
+#include "ec_common.cuh"
+
+namespace ec {
+
+thread_local int g_last_cuda_error = 0;
+
+namespace {
+
+// ---------------------------------------------------------------------------------------------
+// element types
+// ---------------------------------------------------------------------------------------------
+template <int DT> struct Elem;
+template <> struct Elem<EC_F32> {
+    typedef float In; typedef float Acc;
+    static constexpr int VEC = 4;  // elements per 16 input bytes
+    __device__ static __forceinline__ void unpack(const uint4& r, Acc (&x)[VEC]) {
+        x[0] = __uint_as_float(r.x); x[1] = __uint_as_float(r.y); x[2] = __uint_as_float(r.z); x[3] = __uint_as_float(r.w);
+    }
+    __device__ static __forceinline__ Acc widen(In v) { return v; }
+};
+template <> struct Elem<EC_BF16> {
+    typedef uint16_t In; typedef float Acc;
+    static constexpr int VEC = 8;
+    __device__ static __forceinline__ void unpack(const uint4& r, Acc (&x)[VEC]) {
+        // element 2k is the low half of word k, 2k+1 the high half; widening = bits << 16, exact
+        x[0] = __uint_as_float(r.x << 16); x[1] = __uint_as_float(r.x & 0xFFFF0000u);
+        x[2] = __uint_as_float(r.y << 16); x[3] = __uint_as_float(r.y & 0xFFFF0000u);
+        x[4] = __uint_as_float(r.z << 16); x[5] = __uint_as_float(r.z & 0xFFFF0000u);
+        x[6] = __uint_as_float(r.w << 16); x[7] = __uint_as_float(r.w & 0xFFFF0000u);
+    }
+    __device__ static __forceinline__ Acc widen(In v) { return __uint_as_float((uint32_t)v << 16); }
+};
+template <> struct Elem<EC_I64> {
+    typedef long long In; typedef long long Acc;
+    static constexpr int VEC = 2;
+    __device__ static __forceinline__ void unpack(const uint4& r, Acc (&x)[VEC]) {
+        x[0] = (long long)((unsigned long long)r.x | ((unsigned long long)r.y << 32));
+        x[1] = (long long)((unsigned long long)r.z | ((unsigned long long)r.w << 32));
+    }
+    __device__ static __forceinline__ Acc widen(In v) { return v; }
+};
+template <> struct Elem<EC_F64> {
+    typedef double In; typedef double Acc;
+    static constexpr int VEC = 2;
+    __device__ static __forceinline__ void unpack(const uint4& r, Acc (&x)[VEC]) {
+        x[0] = __longlong_as_double((long long)((unsigned long long)r.x | ((unsigned long long)r.y << 32)));
+        x[1] = __longlong_as_double((long long)((unsigned long long)r.z | ((unsigned long long)r.w << 32)));
+    }
+    __device__ static __forceinline__ Acc widen(In v) { return v; }
+};
+
+// ---------------------------------------------------------------------------------------------
+// operators.  Sums use the explicit round-to-nearest intrinsics: never contracted, never reordered.
+// ---------------------------------------------------------------------------------------------
+template <int OP> __device__ __forceinline__ float comb(float a, float x) {
+    if (OP == EC_SUM) return __fadd_rn(a, x);
+    if (OP == EC_MAX) return (x > a) ? x : a;
+    return (x < a) ? x : a;
+}
+template <int OP> __device__ __forceinline__ double comb(double a, double x) {
+    if (OP == EC_SUM) return __dadd_rn(a, x);
+    if (OP == EC_MAX) return (x > a) ? x : a;
+    return (x < a) ? x : a;
+}
+template <int OP> __device__ __forceinline__ long long comb(long long a, long long x) {
+    if (OP == EC_SUM) return (long long)((unsigned long long)a + (unsigned long long)x);
+    if (OP == EC_MAX) return (x > a) ? x : a;
+    return (x < a) ? x : a;
+}
+template <int OP> __device__ __forceinline__ float ident(float) {
+    return OP == EC_SUM ? 0.0f : OP == EC_MAX ? -__int_as_float(0x7f800000) : __int_as_float(0x7f800000);
+}
+template <int OP> __device__ __forceinline__ double ident(double) {
+    return OP == EC_SUM ? 0.0 : OP == EC_MAX ? -__longlong_as_double(0x7ff0000000000000LL)
+                                             : __longlong_as_double(0x7ff0000000000000LL);
+}
+template <int OP> __device__ __forceinline__ long long ident(long long) {
+    return OP == EC_SUM ? 0LL : OP == EC_MAX ? (long long)0x8000000000000000ULL : 0x7fffffffffffffffLL;
+}
+
+// accumulator vector <-> result memory (VEC accumulators = VEC*sizeof(Acc)/16 stores of 16 bytes)
+template <class Acc, int VEC>
+__device__ __forceinline__ void load_acc(const Acc* p, Acc (&acc)[VEC]) {
+    constexpr int PER = 16 / sizeof(Acc);
+#pragma unroll
+    for (int q = 0; q < VEC / PER; ++q) {
+        const uint4 r = ld_plain16(p + q * PER);
+        if (sizeof(Acc) == 4) {
+            acc[q * PER + 0] = (Acc)__uint_as_float(r.x); acc[q * PER + 1] = (Acc)__uint_as_float(r.y);
+            acc[q * PER + 2] = (Acc)__uint_as_float(r.z); acc[q * PER + 3] = (Acc)__uint_as_float(r.w);
+        } else {
+            const unsigned long long a = (unsigned long long)r.x | ((unsigned long long)r.y << 32);
+            const unsigned long long b = (unsigned long long)r.z | ((unsigned long long)r.w << 32);
+            memcpy(&acc[q * PER + 0], &a, 8);
+            memcpy(&acc[q * PER + 1], &b, 8);
+        }
+    }
+}
+template <class Acc, int VEC>
+__device__ __forceinline__ void store_acc(Acc* p, const Acc (&acc)[VEC]) {
+    constexpr int PER = 16 / sizeof(Acc);
+#pragma unroll
+    for (int q = 0; q < VEC / PER; ++q) {
+        uint4 r;
+        if (sizeof(Acc) == 4) {
+            uint32_t w[4];
+            memcpy(w, &acc[q * PER], 16);
+            r = make_uint4(w[0], w[1], w[2], w[3]);
+        } else {
+            unsigned long long w[2];
+            memcpy(w, &acc[q * PER], 16);
+            r = make_uint4((uint32_t)w[0], (uint32_t)(w[0] >> 32), (uint32_t)w[1], (uint32_t)(w[1] >> 32));
+        }
+        st_plain16(p + q * PER, r);
+    }
+}
+
+struct ApplyArgs {
+    size_t n, seg, tile;
+    const uint64_t* arrival;     // [S][W] or nullptr
+    const uint64_t* applied_in;  // [S][W]
+    uint64_t* applied_out;       // [S][W]
+    void* result;
+    uint32_t* contrib_count;     // [S] or nullptr
+    unsigned tiles_per_seg;
+    int P, W, first_apply;
+};
+
+constexpr int RU = 8;        // rank buffers whose loads are issued together (independent loads, ordered adds)
+constexpr int MAX_W = EC_MAX_RANKS / 64;
+constexpr int TREE_LEVELS = 7;  // 1024 ranks / 8 per leaf block = 128 blocks = 2^7
+
+// ---------------------------------------------------------------------------------------------
+// the apply kernel
+// ---------------------------------------------------------------------------------------------
+template <int DT, int OP, bool VECTOR, int CAP, int ORDER>
+__global__ void __launch_bounds__(512)
+apply_kernel(const ApplyArgs a, const __grid_constant__ PtrTable<CAP> tbl) {
+    typedef Elem<DT> E;
+    typedef typename E::In In;
+    typedef typename E::Acc Acc;
+    constexpr int VEC = E::VEC;
+
+    __shared__ const char* s_ptr[CAP];   // tile base of every new rank, ascending
+    __shared__ uint16_t s_rank[CAP];
+    __shared__ uint64_t s_new[MAX_W];
+    __shared__ int s_m, s_fresh;
+
+    const unsigned s = blockIdx.x / a.tiles_per_seg;
+    const unsigned t = blockIdx.x - s * a.tiles_per_seg;
+    const size_t lo = (size_t)s * a.seg + (size_t)t * a.tile;
+    size_t seg_hi = (size_t)(s + 1) * a.seg;
+    if (seg_hi > a.n) seg_hi = a.n;
+
+    if (threadIdx.x < 32) {
+        const int lane = threadIdx.x;
+        uint64_t nw = 0, old = 0;
+        if (lane < a.W) {
+            uint64_t arr = a.arrival ? a.arrival[(size_t)s * a.W + lane] : ~0ull;
+            if (lane == a.W - 1 && (a.P & 63)) arr &= (1ull << (a.P & 63)) - 1;   // bits >= P mean nothing
+            old = a.applied_in[(size_t)s * a.W + lane];
+            nw = arr & ~old;
+        }
+        const unsigned any_new = __ballot_sync(0xffffffffu, nw != 0);
+        const unsigned any_old = __ballot_sync(0xffffffffu, old != 0);
+        const int cnt_new = __popcll(nw);
+        int incl = cnt_new, total = __popcll(nw | old);
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const int y = __shfl_up_sync(0xffffffffu, incl, d);
+            if (lane >= d) incl += y;
+            total += __shfl_xor_sync(0xffffffffu, total, d);
+        }
+        if (t == 0) {
+            if (lane < a.W) a.applied_out[(size_t)s * a.W + lane] = old | nw;
+            if (lane == 0 && a.contrib_count) a.contrib_count[s] = (uint32_t)total;
+        }
+        if (lane < MAX_W) s_new[lane] = nw;
+        int j = incl - cnt_new;
+        uint64_t bits = nw;
+        while (bits) {
+            const int b = __ffsll((long long)bits) - 1;
+            bits &= bits - 1;
+            s_rank[j++] = (uint16_t)(lane * 64 + b);
+        }
+        if (lane == 31) s_m = incl;
+        if (lane == 0) s_fresh = (any_old == 0) ? 1 : 0;
+        (void)any_new;
+    }
+    __syncthreads();
+    const int m = s_m;
+    const bool fresh = s_fresh != 0;
+    if (m == 0 && !(fresh && a.first_apply)) return;   // nothing new: the segment is neither read nor written
+    if (lo >= seg_hi) return;                          // tile beyond a short last segment
+    size_t hi = lo + a.tile;
+    if (hi > seg_hi) hi = seg_hi;
+    const size_t cnt = hi - lo;
+    Acc* res = reinterpret_cast<Acc*>(a.result) + lo;
+    const int tid = threadIdx.x, nthr = blockDim.x;
+    const uint64_t pol = evict_first_policy();
+
+    if (ORDER == EC_ORDER_FIXED) {
+        for (int j = tid; j < m; j += nthr)
+            s_ptr[j] = reinterpret_cast<const char*>(tbl.p[s_rank[j]]) + lo * sizeof(In);
+        __syncthreads();
+        const size_t nvec = VECTOR ? cnt / VEC : 0;
+        for (size_t v = tid; v < nvec; v += nthr) {
+            Acc acc[VEC];
+            if (fresh) {
+#pragma unroll
+                for (int e = 0; e < VEC; ++e) acc[e] = ident<OP>(Acc());
+            } else {
+                load_acc<Acc, VEC>(res + v * VEC, acc);
+            }
+            const size_t boff = v * 16;
+            for (int j = 0; j < m; j += RU) {
+                uint4 raw[RU];
+#pragma unroll
+                for (int u = 0; u < RU; ++u)
+                    if (j + u < m) raw[u] = ld_stream16(s_ptr[j + u] + boff, pol);
+#pragma unroll
+                for (int u = 0; u < RU; ++u) {
+                    if (j + u < m) {
+                        Acc x[VEC];
+                        E::unpack(raw[u], x);
+#pragma unroll
+                        for (int e = 0; e < VEC; ++e) acc[e] = comb<OP>(acc[e], x[e]);
+                    }
+                }
+            }
+            store_acc<Acc, VEC>(res + v * VEC, acc);
+        }
+        // element-wise path: everything when the 128-bit path does not apply, else the ragged tail
+        for (size_t i = nvec * VEC + tid; i < cnt; i += nthr) {
+            Acc acc = fresh ? ident<OP>(Acc()) : res[i];
+            for (int j = 0; j < m; j += RU) {
+                In raw[RU];
+#pragma unroll
+                for (int u = 0; u < RU; ++u)
+                    if (j + u < m) raw[u] = reinterpret_cast<const In*>(s_ptr[j + u])[i];
+#pragma unroll
+                for (int u = 0; u < RU; ++u)
+                    if (j + u < m) acc = comb<OP>(acc, E::widen(raw[u]));
+            }
+            res[i] = acc;
+        }
+    } else {
+        // Pairwise: balanced binary tree over the rank index, P padded to a power of two, ranks that
+        // are not new contribute the identity.  Leaves are taken eight ranks at a time (a complete
+        // three-level subtree); the subtrees are merged with a binary counter, which reproduces the
+        // recursive halving tree exactly.
+        int P2 = 1;
+        while (P2 < a.P) P2 <<= 1;
+        const int leaf = P2 < 8 ? P2 : 8;
+        const int nblk = P2 / leaf;
+        int nlev = 0;
+        while ((1 << nlev) < nblk) ++nlev;
+        const size_t nvec = VECTOR ? cnt / VEC : 0;
+        const size_t nunits = nvec + (cnt - nvec * VEC);   // vectors first, then single elements
+        for (size_t w = tid; w < nunits; w += nthr) {
+            const bool isvec = w < nvec;
+            const size_t e0 = isvec ? w * VEC : nvec * VEC + (w - nvec);   // first element of this unit
+            Acc stack[TREE_LEVELS][VEC];
+            Acc node[VEC];
+            for (int blk = 0; blk < nblk; ++blk) {
+                const int r0 = blk * leaf;
+                const unsigned byte = (unsigned)(s_new[r0 >> 6] >> (r0 & 63)) & ((1u << leaf) - 1u);
+                Acc lv[8][VEC];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+#pragma unroll
+                    for (int e = 0; e < VEC; ++e) lv[u][e] = ident<OP>(Acc());
+                }
+                if (byte != 0) {
+                    if (isvec) {
+                        uint4 raw[8];
+#pragma unroll
+                        for (int u = 0; u < 8; ++u)
+                            if ((byte >> u) & 1u)
+                                raw[u] = ld_stream16(reinterpret_cast<const char*>(tbl.p[r0 + u]) + e0 * sizeof(In), pol);
+#pragma unroll
+                        for (int u = 0; u < 8; ++u)
+                            if ((byte >> u) & 1u) E::unpack(raw[u], lv[u]);
+                    } else {
+#pragma unroll
+                        for (int u = 0; u < 8; ++u)
+                            if ((byte >> u) & 1u) lv[u][0] = E::widen(reinterpret_cast<const In*>(tbl.p[r0 + u])[e0]);
+                    }
+                }
+#pragma unroll
+                for (int e = 0; e < VEC; ++e) {
+                    if (leaf == 8)
+                        node[e] = comb<OP>(comb<OP>(comb<OP>(lv[0][e], lv[1][e]), comb<OP>(lv[2][e], lv[3][e])),
+                                           comb<OP>(comb<OP>(lv[4][e], lv[5][e]), comb<OP>(lv[6][e], lv[7][e])));
+                    else if (leaf == 4)
+                        node[e] = comb<OP>(comb<OP>(lv[0][e], lv[1][e]), comb<OP>(lv[2][e], lv[3][e]));
+                    else if (leaf == 2)
+                        node[e] = comb<OP>(lv[0][e], lv[1][e]);
+                    else
+                        node[e] = lv[0][e];
+                }
+                bool carry = true;
+#pragma unroll
+                for (int l = 0; l < TREE_LEVELS; ++l) {
+                    if (l < nlev && carry) {
+                        if ((blk >> l) & 1) {
+#pragma unroll
+                            for (int e = 0; e < VEC; ++e) node[e] = comb<OP>(stack[l][e], node[e]);
+                        } else {
+#pragma unroll
+                            for (int e = 0; e < VEC; ++e) stack[l][e] = node[e];
+                            carry = false;
+                        }
+                    }
+                }
+            }
+            // node is the root now
+            if (isvec) {
+                if (!fresh) {
+                    Acc acc[VEC];
+                    load_acc<Acc, VEC>(res + e0, acc);
+#pragma unroll
+                    for (int e = 0; e < VEC; ++e) node[e] = comb<OP>(acc[e], node[e]);
+                }
+                store_acc<Acc, VEC>(res + e0, node);
+            } else {
+                res[e0] = fresh ? node[0] : comb<OP>(res[e0], node[0]);
+            }
+        }
+    }
+}
+
+template <int DT, int OP, bool VECTOR, int ORDER>
+int launch_cap(const ApplyArgs& a, const void* const* bufs, unsigned grid, int threads, cudaStream_t st) {
+    if (a.P <= 64) {
+        PtrTable<64> tbl;
+        for (int r = 0; r < 64; ++r) tbl.p[r] = r < a.P ? bufs[r] : nullptr;
+        apply_kernel<DT, OP, VECTOR, 64, ORDER><<<grid, threads, 0, st>>>(a, tbl);
+    } else {
+        PtrTable<EC_MAX_RANKS> tbl;
+        for (int r = 0; r < EC_MAX_RANKS; ++r) tbl.p[r] = r < a.P ? bufs[r] : nullptr;
+        apply_kernel<DT, OP, VECTOR, EC_MAX_RANKS, ORDER><<<grid, threads, 0, st>>>(a, tbl);
+    }
+    EC_CUDA(cudaGetLastError());
+    return EC_OK;
+}
+
+template <int DT, int OP>
+int launch_op(const ApplyArgs& a, const void* const* bufs, bool vector, int order, unsigned grid, int threads,
+              cudaStream_t st) {
+    if (order == EC_ORDER_FIXED)
+        return vector ? launch_cap<DT, OP, true, EC_ORDER_FIXED>(a, bufs, grid, threads, st)
+                      : launch_cap<DT, OP, false, EC_ORDER_FIXED>(a, bufs, grid, threads, st);
+    if constexpr (OP == EC_SUM && DT != EC_I64)
+        return vector ? launch_cap<DT, EC_SUM, true, EC_ORDER_PAIRWISE>(a, bufs, grid, threads, st)
+                      : launch_cap<DT, EC_SUM, false, EC_ORDER_PAIRWISE>(a, bufs, grid, threads, st);
+    return EC_ERR_UNSUPPORTED;
+}
+
+template <int DT>
+int launch_dt(const ApplyArgs& a, const void* const* bufs, int op, bool vector, int order, unsigned grid,
+              int threads, cudaStream_t st) {
+    switch (op) {
+        case EC_SUM: return launch_op<DT, EC_SUM>(a, bufs, vector, order, grid, threads, st);
+        case EC_MAX: return launch_op<DT, EC_MAX>(a, bufs, vector, order, grid, threads, st);
+        case EC_MIN: return launch_op<DT, EC_MIN>(a, bufs, vector, order, grid, threads, st);
+    }
+    return EC_ERR_INVALID;
+}
+
+size_t words_bytes(int P, size_t n, size_t seg) {
+    const size_t S = (n + seg - 1) / seg;
+    const size_t W = (size_t)(P + 63) / 64;
+    return align_up(S * W * sizeof(uint64_t), 256);
+}
+
+bool bad_shape(int P, size_t n, size_t seg) {
+    return P < 1 || P > EC_MAX_RANKS || n == 0 || seg == 0 || (n + seg - 1) / seg > 0x7fffffffull;
+}
+
+}  // namespace
+}  // namespace ec
+
+struct ec_ctx {
+    int P, W, dtype, op, order;
+    size_t n, seg, S;
+    void* ws;
+    bool own_ws;
+    uint64_t* applied[2];
+    int cur;           // which copy holds the current words
+    bool first_apply;  // no apply yet in this epoch
+    int threads;
+    size_t tile;       // elements per block
+};
+
+using namespace ec;
+
+extern "C" {
+
+size_t ec_allreduce_workspace_bytes(int P, size_t n, size_t segment_size) {
+    if (bad_shape(P, n, segment_size)) return 0;
+    return 2 * words_bytes(P, n, segment_size);
+}
+
+int ec_allreduce_init(ec_ctx_t** out, int P, size_t n, ec_dtype_t dtype, ec_op_t op, size_t segment_size,
+                      ec_order_t order, void* workspace, size_t workspace_bytes) {
+    if (!out) return EC_ERR_INVALID;
+    *out = nullptr;
+    if (bad_shape(P, n, segment_size)) return EC_ERR_INVALID;
+    if ((int)dtype < 0 || (int)dtype > EC_F64 || (int)op < 0 || (int)op > EC_MIN) return EC_ERR_INVALID;
+    if ((int)order != EC_ORDER_FIXED && (int)order != EC_ORDER_PAIRWISE) return EC_ERR_INVALID;
+    if (order == EC_ORDER_PAIRWISE && (op != EC_SUM || dtype == EC_I64)) return EC_ERR_UNSUPPORTED;
+    const size_t need = ec_allreduce_workspace_bytes(P, n, segment_size);
+    if (workspace && (workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 255u))) return EC_ERR_CAPACITY;
+    ec_ctx* c = new (std::nothrow) ec_ctx();
+    if (!c) return EC_ERR_INVALID;
+    c->P = P; c->W = (P + 63) / 64; c->dtype = dtype; c->op = op; c->order = order;
+    c->n = n; c->seg = segment_size; c->S = (n + segment_size - 1) / segment_size;
+    c->own_ws = workspace == nullptr;
+    c->ws = workspace;
+    if (c->own_ws) {
+        cudaError_t e = cudaMalloc(&c->ws, need);
+        if (e != cudaSuccess) { delete c; return cuda_fail(e); }
+    }
+    cudaError_t e = cudaMemsetAsync(c->ws, 0, need, 0);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(0);
+    if (e != cudaSuccess) {
+        if (c->own_ws) cudaFree(c->ws);
+        delete c;
+        return cuda_fail(e);
+    }
+    c->applied[0] = reinterpret_cast<uint64_t*>(c->ws);
+    c->applied[1] = reinterpret_cast<uint64_t*>(reinterpret_cast<char*>(c->ws) + need / 2);
+    c->cur = 0;
+    c->first_apply = true;
+    c->threads = 256;
+    c->tile = 8192 / in_bytes(dtype);   // 8 KB of every rank buffer per block
+    *out = c;
+    return EC_OK;
+}
+
+int ec_allreduce_set_tile(ec_ctx_t* c, int threads, size_t tile_elems) {
+    if (!c) return EC_ERR_INVALID;
+    if (threads != 0) {
+        if (threads < 64 || threads > 512 || threads % 32) return EC_ERR_INVALID;
+        c->threads = threads;
+    }
+    if (tile_elems != 0) {
+        const size_t vec = 16 / in_bytes(c->dtype);
+        c->tile = align_up(tile_elems, vec);
+    }
+    return EC_OK;
+}
+
+int ec_allreduce_apply(ec_ctx_t* c, const void* const* rank_bufs, int P, size_t n, ec_dtype_t dtype, ec_op_t op,
+                       size_t segment_size, const uint64_t* arrival_mask, void* result, uint32_t* contrib_count,
+                       ec_stream_t stream) {
+    if (!c || !rank_bufs || !result) return EC_ERR_INVALID;
+    if (P != c->P || n != c->n || (int)dtype != c->dtype || (int)op != c->op || segment_size != c->seg)
+        return EC_ERR_INVALID;
+    bool vector = aligned16(result) && (c->seg * in_bytes(c->dtype)) % 16 == 0;
+    for (int r = 0; r < P; ++r) {
+        if (!rank_bufs[r] || rank_bufs[r] == result) return EC_ERR_INVALID;
+        vector = vector && aligned16(rank_bufs[r]);
+    }
+    const size_t seg_len = c->seg < c->n ? c->seg : c->n;
+    const size_t tiles = (seg_len + c->tile - 1) / c->tile;
+    if (tiles * c->S > 0x7fffffffull) return EC_ERR_CAPACITY;
+    ApplyArgs a;
+    a.n = c->n; a.seg = c->seg; a.tile = c->tile;
+    a.arrival = arrival_mask;
+    a.applied_in = c->applied[c->cur];
+    a.applied_out = c->applied[c->cur ^ 1];
+    a.result = result;
+    a.contrib_count = contrib_count;
+    a.tiles_per_seg = (unsigned)tiles;
+    a.P = c->P; a.W = c->W; a.first_apply = c->first_apply ? 1 : 0;
+    const unsigned grid = (unsigned)(tiles * c->S);
+    int rc;
+    switch (c->dtype) {
+        case EC_F32: rc = launch_dt<EC_F32>(a, rank_bufs, c->op, vector, c->order, grid, c->threads, stream); break;
+        case EC_BF16: rc = launch_dt<EC_BF16>(a, rank_bufs, c->op, vector, c->order, grid, c->threads, stream); break;
+        case EC_I64: rc = launch_dt<EC_I64>(a, rank_bufs, c->op, vector, c->order, grid, c->threads, stream); break;
+        case EC_F64: rc = launch_dt<EC_F64>(a, rank_bufs, c->op, vector, c->order, grid, c->threads, stream); break;
+        default: rc = EC_ERR_INVALID;
+    }
+    if (rc != EC_OK) return rc;
+    c->cur ^= 1;
+    c->first_apply = false;
+    return EC_OK;
+}
+
+int ec_allreduce_reset(ec_ctx_t* c, ec_stream_t stream) {
+    if (!c) return EC_ERR_INVALID;
+    EC_CUDA(cudaMemsetAsync(c->applied[c->cur], 0, (size_t)c->S * c->W * sizeof(uint64_t), stream));
+    c->first_apply = true;
+    return EC_OK;
+}
+
+int ec_allreduce_destroy(ec_ctx_t* c) {
+    if (!c) return EC_ERR_INVALID;
+    int rc = EC_OK;
+    if (c->own_ws && c->ws) {
+        cudaError_t e = cudaFree(c->ws);
+        if (e != cudaSuccess) rc = cuda_fail(e);
+    }
+    delete c;
+    return rc;
+}
+
+const char* ec_strerror(int code) {
+    switch (code) {
+        case EC_OK: return "ok";
+        case EC_ERR_INVALID: return "invalid argument";
+        case EC_ERR_UNSUPPORTED: return "unsupported combination of dtype, op and order";
+        case EC_ERR_CUDA: return "CUDA runtime error (see ec_last_cuda_error)";
+        case EC_ERR_STATE: return "call not allowed in this state";
+        case EC_ERR_CAPACITY: return "size beyond a limit, or workspace too small";
+    }
+    return "unknown error code";
+}
+
+int ec_last_cuda_error(void) { return g_last_cuda_error; }
+int ec_version(void) { return 1000; }
+
+}  // extern "C"

@@ -1,0 +1,473 @@
+// K-means driver on top of the eventually consistent allreduce.
+//
+// The paper's iterative-convergent ML workload (Sec. I, Sec. V) tolerates contributions that are
+// missing or late; here Lloyd's iteration plays that role: every simulated rank assigns its shard
+// of points, forms per-centroid partial sums, and the partial sums are combined by one allreduce
+// epoch in which only the notified (rank, centroid-row) contributions take part.
+//
+// Kernels:
+//   assign    one thread per point, the point's coordinates in registers, centroids staged in
+//             shared memory and read as broadcasts; squared distance sum_d (x-c)^2 in fp32;
+//             bound by the fp32 pipes, not by memory.
+//   partials  one warp walks a contiguous run of points with lane = coordinate and keeps
+//             [K][D] running sums in its own shared-memory slab: plain read-add-write, no
+//             atomics, fixed order.  Warps, then blocks of a rank are folded in index order.
+//   update    centroid = sum / points where points > 0.
+
+#include <new>
+
+#include "ec_common.cuh"
+
+namespace ec {
+namespace {
+
+constexpr int AS_THREADS = 256;
+constexpr int PT_THREADS = 256;
+constexpr int PT_WARPS = PT_THREADS / 32;
+constexpr size_t SMEM_BUDGET = 200 * 1024;
+
+// ---------------------------------------------------------------------------------------------
+// assignment
+// ---------------------------------------------------------------------------------------------
+template <int D>
+__global__ void __launch_bounds__(AS_THREADS)
+assign_kernel(const float* __restrict__ points, size_t N, const float* __restrict__ centroids, int K, int kc,
+              int32_t* __restrict__ labels) {
+    extern __shared__ __align__(16) float s_c[];   // kc centroids of D floats
+    const int tid = threadIdx.x;
+    for (size_t base = (size_t)blockIdx.x * AS_THREADS; base < N; base += (size_t)gridDim.x * AS_THREADS) {
+        const size_t j = base + tid;
+        const bool live = j < N;
+        float x[D];
+        if (live) {
+            const float4* row = reinterpret_cast<const float4*>(points + j * D);
+#pragma unroll
+            for (int q = 0; q < D / 4; ++q) {
+                const float4 v = __ldg(row + q);
+                x[4 * q] = v.x; x[4 * q + 1] = v.y; x[4 * q + 2] = v.z; x[4 * q + 3] = v.w;
+            }
+        } else {
+#pragma unroll
+            for (int d = 0; d < D; ++d) x[d] = 0.0f;
+        }
+        float best = __int_as_float(0x7f800000);
+        int bi = 0;
+        for (int k0 = 0; k0 < K; k0 += kc) {
+            const int kn = K - k0 < kc ? K - k0 : kc;
+            __syncthreads();                         // previous chunk fully consumed
+            for (int i = tid; i < kn * D / 4; i += AS_THREADS)
+                reinterpret_cast<float4*>(s_c)[i] = __ldg(reinterpret_cast<const float4*>(centroids + (size_t)k0 * D) + i);
+            __syncthreads();
+            int k = 0;
+            for (; k + 1 < kn; k += 2) {             // two centroids at a time: two independent chains
+                const float4* c0 = reinterpret_cast<const float4*>(s_c + (size_t)k * D);
+                const float4* c1 = reinterpret_cast<const float4*>(s_c + (size_t)(k + 1) * D);
+                float d0 = 0.0f, d1 = 0.0f;
+#pragma unroll
+                for (int q = 0; q < D / 4; ++q) {
+                    const float4 a = c0[q], b = c1[q];
+                    float t;
+                    t = x[4 * q] - a.x; d0 = fmaf(t, t, d0);
+                    t = x[4 * q + 1] - a.y; d0 = fmaf(t, t, d0);
+                    t = x[4 * q + 2] - a.z; d0 = fmaf(t, t, d0);
+                    t = x[4 * q + 3] - a.w; d0 = fmaf(t, t, d0);
+                    t = x[4 * q] - b.x; d1 = fmaf(t, t, d1);
+                    t = x[4 * q + 1] - b.y; d1 = fmaf(t, t, d1);
+                    t = x[4 * q + 2] - b.z; d1 = fmaf(t, t, d1);
+                    t = x[4 * q + 3] - b.w; d1 = fmaf(t, t, d1);
+                }
+                if (d0 < best) { best = d0; bi = k0 + k; }          // strict <: the lowest index wins a tie
+                if (d1 < best) { best = d1; bi = k0 + k + 1; }
+            }
+            if (k < kn) {
+                const float4* c0 = reinterpret_cast<const float4*>(s_c + (size_t)k * D);
+                float d0 = 0.0f;
+#pragma unroll
+                for (int q = 0; q < D / 4; ++q) {
+                    const float4 a = c0[q];
+                    float t;
+                    t = x[4 * q] - a.x; d0 = fmaf(t, t, d0);
+                    t = x[4 * q + 1] - a.y; d0 = fmaf(t, t, d0);
+                    t = x[4 * q + 2] - a.z; d0 = fmaf(t, t, d0);
+                    t = x[4 * q + 3] - a.w; d0 = fmaf(t, t, d0);
+                }
+                if (d0 < best) { best = d0; bi = k0 + k; }
+            }
+        }
+        if (live) labels[j] = bi;
+    }
+}
+
+// Any D (multiple of 4, at most 128): coordinates are re-read from global memory (L1) per centroid chunk.
+__global__ void __launch_bounds__(AS_THREADS)
+assign_generic_kernel(const float* __restrict__ points, size_t N, int D, const float* __restrict__ centroids, int K,
+                      int kc, int32_t* __restrict__ labels) {
+    extern __shared__ __align__(16) float s_c[];
+    const int tid = threadIdx.x;
+    for (size_t base = (size_t)blockIdx.x * AS_THREADS; base < N; base += (size_t)gridDim.x * AS_THREADS) {
+        const size_t j = base + tid;
+        const bool live = j < N;
+        const float* row = points + (live ? j : 0) * (size_t)D;
+        float best = __int_as_float(0x7f800000);
+        int bi = 0;
+        for (int k0 = 0; k0 < K; k0 += kc) {
+            const int kn = K - k0 < kc ? K - k0 : kc;
+            __syncthreads();
+            for (int i = tid; i < kn * D; i += AS_THREADS) s_c[i] = centroids[(size_t)k0 * D + i];
+            __syncthreads();
+            for (int k = 0; k < kn; ++k) {
+                float d0 = 0.0f;
+                for (int d = 0; d < D; ++d) {
+                    const float t = row[d] - s_c[k * D + d];
+                    d0 = fmaf(t, t, d0);
+                }
+                if (d0 < best) { best = d0; bi = k0 + k; }
+            }
+        }
+        if (live) labels[j] = bi;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// per-rank partial sums
+// ---------------------------------------------------------------------------------------------
+// Block (r, c) covers the c-th of C equal runs of rank r's points; its `warps` warps split the run
+// again.  out: [P][C][K][D+4] (scratch) - or the partials themselves when C == 1.
+__global__ void __launch_bounds__(PT_THREADS)
+partials_kernel(const float* __restrict__ points, const int32_t* __restrict__ labels, size_t N, int D, int K, int P,
+                int C, int warps, float* __restrict__ out) {
+    extern __shared__ __align__(16) float s_acc[];                  // [warps][K][D] sums, then [warps][K] counts
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const int r = blockIdx.x / C, c = blockIdx.x - r * C;
+    const size_t KD = (size_t)K * D;
+    int* s_cnt = reinterpret_cast<int*>(s_acc + (size_t)warps * KD);
+    for (size_t i = threadIdx.x; i < (size_t)warps * KD; i += blockDim.x) s_acc[i] = 0.0f;
+    for (size_t i = threadIdx.x; i < (size_t)warps * K; i += blockDim.x) s_cnt[i] = 0;
+    __syncthreads();
+    const size_t j0 = (size_t)r * N / P, j1 = (size_t)(r + 1) * N / P;
+    const size_t len = j1 - j0;
+    const size_t b0 = j0 + len * c / C, b1 = j0 + len * (c + 1) / C;   // this block's run
+    if (w < warps) {
+        const size_t blen = b1 - b0;
+        const size_t p0 = b0 + blen * w / warps, p1 = b0 + blen * (w + 1) / warps;
+        float* acc = s_acc + (size_t)w * KD;
+        int* cnt = s_cnt + (size_t)w * K;
+        const int dims = (D + 31) / 32;                               // coordinates per lane
+        size_t j = p0;
+        for (; j + 4 <= p1; j += 4) {                                 // loads of four points in flight
+            int lab[4];
+            float v[4][4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                lab[u] = __ldg(labels + j + u);
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const int d = lane + 32 * q;
+                    v[u][q] = (q < dims && d < D) ? __ldg(points + (j + u) * (size_t)D + d) : 0.0f;
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int k = lab[u];
+                if ((unsigned)k < (unsigned)K) {
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const int d = lane + 32 * q;
+                        if (q < dims && d < D) acc[(size_t)k * D + d] = __fadd_rn(acc[(size_t)k * D + d], v[u][q]);
+                    }
+                    if (lane == 0) cnt[k] += 1;
+                }
+            }
+        }
+        for (; j < p1; ++j) {
+            const int k = __ldg(labels + j);
+            if ((unsigned)k < (unsigned)K) {
+                for (int d = lane; d < D; d += 32)
+                    acc[(size_t)k * D + d] = __fadd_rn(acc[(size_t)k * D + d], __ldg(points + j * (size_t)D + d));
+                if (lane == 0) cnt[k] += 1;
+            }
+        }
+    }
+    __syncthreads();
+    // fold the warps in index order and write rows of D+4
+    const int stride = D + 4;
+    float* dst = out + ((size_t)r * C + c) * (size_t)K * stride;
+    for (size_t i = threadIdx.x; i < (size_t)K * stride; i += blockDim.x) {
+        const int k = (int)(i / stride), d = (int)(i - (size_t)k * stride);
+        float val = 0.0f;
+        if (d < D) {
+            val = s_acc[(size_t)k * D + d];
+            for (int ww = 1; ww < warps; ++ww) val = __fadd_rn(val, s_acc[(size_t)ww * KD + (size_t)k * D + d]);
+        } else if (d == D) {
+            int n = 0;
+            for (int ww = 0; ww < warps; ++ww) n += s_cnt[(size_t)ww * K + k];
+            val = (float)n;                                            // exact: at most 2^24 points per block
+        }
+        dst[i] = val;
+    }
+}
+
+// partials[r][k][d] = scratch[r][0][k][d] + scratch[r][1][k][d] + ... in index order
+__global__ void partials_fold_kernel(const float* __restrict__ scratch, int C, size_t row_elems, size_t total,
+                                     float* __restrict__ partials) {
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+        const size_t r = i / row_elems, e = i - r * row_elems;
+        const float* src = scratch + r * (size_t)C * row_elems + e;
+        float v = src[0];
+        for (int c = 1; c < C; ++c) v = __fadd_rn(v, src[(size_t)c * row_elems]);
+        partials[i] = v;
+    }
+}
+
+__global__ void update_kernel(const float* __restrict__ reduced, int D, int K, float* __restrict__ centroids) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= K * D) return;
+    const int k = i / D, d = i - k * D;
+    const float pts = reduced[(size_t)k * (D + 4) + D];
+    if (pts > 0.0f) centroids[i] = __fdiv_rn(reduced[(size_t)k * (D + 4) + d], pts);
+}
+
+int sm_count_km() {
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) return 148;
+    return n;
+}
+
+}  // namespace
+}  // namespace ec
+
+struct ec_kmeans {
+    const float* points;
+    size_t N;
+    int D, K, P;
+    void* ws;
+    bool own_ws;
+    // carved out of ws
+    float* centroids;      // [K][D]
+    int32_t* labels;       // [N]
+    float* partials;       // [P][K][D+4]
+    float* scratch;        // [P][C][K][D+4]
+    float* reduced;        // [K][D+4]
+    uint32_t* contrib;     // [K]
+    void* ar_ws;
+    ec_ctx_t* ar;
+    const void* bufs[EC_MAX_RANKS];
+    int sms, C, warps, kc;
+    size_t assign_smem, part_smem;
+};
+
+using namespace ec;
+
+namespace {
+
+struct KmLayout {
+    size_t off_centroids, off_labels, off_partials, off_scratch, off_reduced, off_contrib, off_ar, total;
+    int C, warps;
+};
+
+// Blocks per rank (C) and warps per block for the partials kernel, from the shape alone.
+bool km_plan(size_t N, int D, int K, int P, int sms, KmLayout* L) {
+    const size_t KD = (size_t)K * D;
+    int warps = PT_WARPS;
+    while (warps > 1 && (size_t)warps * (KD + K) * 4 > SMEM_BUDGET / 2) warps >>= 1;   // two blocks per SM if possible
+    if ((size_t)warps * (KD + K) * 4 > SMEM_BUDGET) return false;
+    const size_t smem = (size_t)warps * (KD + K) * 4;
+    const int per_sm = (int)(SMEM_BUDGET / smem) < 2048 / PT_THREADS ? (int)(SMEM_BUDGET / smem) : 2048 / PT_THREADS;
+    int C = (sms * (per_sm < 1 ? 1 : per_sm)) / P;          // one wave of resident blocks
+    if (C < 1) C = 1;
+    const size_t shard = N / (size_t)P > 0 ? N / (size_t)P : 1;
+    while (C > 1 && shard / (size_t)C < 256) --C;            // keep runs long enough to be worth a block
+    L->C = C;
+    L->warps = warps;
+    const size_t stride = (size_t)D + 4;
+    size_t off = 0;
+    L->off_centroids = off; off = align_up(off + KD * 4, 256);
+    L->off_labels = off; off = align_up(off + N * 4, 256);
+    L->off_partials = off; off = align_up(off + (size_t)P * K * stride * 4, 256);
+    L->off_scratch = off; off = align_up(off + (size_t)P * C * K * stride * 4, 256);
+    L->off_reduced = off; off = align_up(off + (size_t)K * stride * 4, 256);
+    L->off_contrib = off; off = align_up(off + (size_t)K * 4, 256);
+    L->off_ar = off; off = align_up(off + ec_allreduce_workspace_bytes(P, (size_t)K * stride, stride), 256);
+    L->total = off;
+    return true;
+}
+
+bool km_bad_shape(size_t N, int D, int K, int P) {
+    return N == 0 || D < 1 || D > 128 || (D % 4) != 0 || K < 1 || K > 1024 || P < 1 || P > EC_MAX_RANKS ||
+           (size_t)P > N;
+}
+
+int km_assign(ec_kmeans* km, const float* centroids, int32_t* labels, cudaStream_t st) {
+    const size_t tiles = (km->N + AS_THREADS - 1) / AS_THREADS;
+    const size_t cap = (size_t)km->sms * 8;
+    const unsigned grid = (unsigned)(tiles < cap ? tiles : cap);
+    switch (km->D) {
+#define EC_ASSIGN_CASE(DD)                                                                                   \
+    case DD:                                                                                                  \
+        assign_kernel<DD><<<grid, AS_THREADS, km->assign_smem, st>>>(km->points, km->N, centroids, km->K, km->kc, labels); \
+        break;
+        EC_ASSIGN_CASE(4)
+        EC_ASSIGN_CASE(8)
+        EC_ASSIGN_CASE(16)
+        EC_ASSIGN_CASE(32)
+        EC_ASSIGN_CASE(64)
+#undef EC_ASSIGN_CASE
+        default:
+            assign_generic_kernel<<<grid, AS_THREADS, km->assign_smem, st>>>(km->points, km->N, km->D, centroids, km->K,
+                                                                             km->kc, labels);
+    }
+    EC_CUDA(cudaGetLastError());
+    return EC_OK;
+}
+
+int km_partials(ec_kmeans* km, const int32_t* labels, float* partials, cudaStream_t st) {
+    float* first = km->C == 1 ? partials : km->scratch;
+    partials_kernel<<<(unsigned)(km->P * km->C), PT_THREADS, km->part_smem, st>>>(km->points, labels, km->N, km->D, km->K,
+                                                                                  km->P, km->C, km->warps, first);
+    EC_CUDA(cudaGetLastError());
+    if (km->C > 1) {
+        const size_t row = (size_t)km->K * (km->D + 4), total = row * km->P;
+        const unsigned grid = (unsigned)((total + 255) / 256);
+        partials_fold_kernel<<<grid, 256, 0, st>>>(km->scratch, km->C, row, total, partials);
+        EC_CUDA(cudaGetLastError());
+    }
+    return EC_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t ec_kmeans_workspace_bytes(size_t N, int D, int K, int P) {
+    if (km_bad_shape(N, D, K, P)) return 0;
+    KmLayout L;
+    if (!km_plan(N, D, K, P, sm_count_km(), &L)) return 0;
+    return L.total;
+}
+
+int ec_kmeans_init(ec_kmeans_t** out, const float* points, size_t N, int D, int K, int P, const float* init_centroids,
+                   void* workspace, size_t workspace_bytes) {
+    if (!out) return EC_ERR_INVALID;
+    *out = nullptr;
+    if (!points || !init_centroids || km_bad_shape(N, D, K, P)) return EC_ERR_INVALID;
+    if (!aligned16(points)) return EC_ERR_INVALID;
+    KmLayout L;
+    const int sms = sm_count_km();
+    if (!km_plan(N, D, K, P, sms, &L)) return EC_ERR_CAPACITY;
+    if (workspace && (workspace_bytes < L.total || (reinterpret_cast<uintptr_t>(workspace) & 255u))) return EC_ERR_CAPACITY;
+    ec_kmeans* km = new (std::nothrow) ec_kmeans();
+    if (!km) return EC_ERR_INVALID;
+    km->points = points; km->N = N; km->D = D; km->K = K; km->P = P;
+    km->own_ws = workspace == nullptr;
+    km->ws = workspace;
+    km->ar = nullptr;
+    if (km->own_ws) {
+        cudaError_t e = cudaMalloc(&km->ws, L.total);
+        if (e != cudaSuccess) { delete km; return cuda_fail(e); }
+    }
+    char* base = reinterpret_cast<char*>(km->ws);
+    km->centroids = reinterpret_cast<float*>(base + L.off_centroids);
+    km->labels = reinterpret_cast<int32_t*>(base + L.off_labels);
+    km->partials = reinterpret_cast<float*>(base + L.off_partials);
+    km->scratch = reinterpret_cast<float*>(base + L.off_scratch);
+    km->reduced = reinterpret_cast<float*>(base + L.off_reduced);
+    km->contrib = reinterpret_cast<uint32_t*>(base + L.off_contrib);
+    km->ar_ws = base + L.off_ar;
+    km->sms = sms; km->C = L.C; km->warps = L.warps;
+    // centroid chunk for the assignment: as many as fit in 64 KB, all of them if possible
+    int kc = (int)((64 * 1024) / ((size_t)D * 4));
+    if (kc > K) kc = K;
+    if (kc > 1) kc &= ~1;
+    if (kc < 1) kc = 1;
+    km->kc = kc;
+    km->assign_smem = (size_t)kc * D * 4;
+    km->part_smem = (size_t)L.warps * ((size_t)K * D + K) * 4;
+    const size_t stride = (size_t)D + 4;
+    int rc = EC_OK;
+    cudaError_t e = cudaSuccess;
+    if (km->assign_smem > 48 * 1024) {
+        switch (D) {
+            case 4: e = cudaFuncSetAttribute(assign_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)km->assign_smem); break;
+            case 8: e = cudaFuncSetAttribute(assign_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)km->assign_smem); break;
+            case 16: e = cudaFuncSetAttribute(assign_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)km->assign_smem); break;
+            case 32: e = cudaFuncSetAttribute(assign_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)km->assign_smem); break;
+            case 64: e = cudaFuncSetAttribute(assign_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)km->assign_smem); break;
+            default: e = cudaFuncSetAttribute(assign_generic_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)km->assign_smem);
+        }
+    }
+    if (e == cudaSuccess && km->part_smem > 48 * 1024)
+        e = cudaFuncSetAttribute(partials_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)km->part_smem);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(km->centroids, init_centroids, (size_t)K * D * 4, cudaMemcpyDeviceToDevice, 0);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(0);
+    if (e != cudaSuccess) rc = cuda_fail(e);
+    if (rc == EC_OK)
+        rc = ec_allreduce_init(&km->ar, P, (size_t)K * stride, EC_F32, EC_SUM, stride, EC_ORDER_FIXED, km->ar_ws,
+                               ec_allreduce_workspace_bytes(P, (size_t)K * stride, stride));
+    if (rc != EC_OK) {
+        if (km->own_ws) cudaFree(km->ws);
+        delete km;
+        return rc;
+    }
+    for (int r = 0; r < P; ++r) km->bufs[r] = km->partials + (size_t)r * K * stride;
+    *out = km;
+    return EC_OK;
+}
+
+int ec_kmeans_assign(ec_kmeans_t* km, const float* centroids, int32_t* labels, ec_stream_t stream) {
+    if (!km || !centroids || !labels || !aligned16(centroids)) return EC_ERR_INVALID;
+    return km_assign(km, centroids, labels, stream);
+}
+
+int ec_kmeans_partials(ec_kmeans_t* km, const int32_t* labels, float* partials, ec_stream_t stream) {
+    if (!km || !labels || !partials) return EC_ERR_INVALID;
+    return km_partials(km, labels, partials, stream);
+}
+
+int ec_kmeans_iterate(ec_kmeans_t* km, const uint64_t* arrival_mask, ec_stream_t stream) {
+    if (!km) return EC_ERR_INVALID;
+    int rc = km_assign(km, km->centroids, km->labels, stream);
+    if (rc != EC_OK) return rc;
+    rc = km_partials(km, km->labels, km->partials, stream);
+    if (rc != EC_OK) return rc;
+    rc = ec_allreduce_reset(km->ar, stream);
+    if (rc != EC_OK) return rc;
+    const size_t stride = (size_t)km->D + 4;
+    rc = ec_allreduce_apply(km->ar, km->bufs, km->P, (size_t)km->K * stride, EC_F32, EC_SUM, stride, arrival_mask,
+                            km->reduced, km->contrib, stream);
+    if (rc != EC_OK) return rc;
+    const int total = km->K * km->D;
+    update_kernel<<<(total + 255) / 256, 256, 0, stream>>>(km->reduced, km->D, km->K, km->centroids);
+    EC_CUDA(cudaGetLastError());
+    return EC_OK;
+}
+
+int ec_kmeans_set_centroids(ec_kmeans_t* km, const float* centroids, ec_stream_t stream) {
+    if (!km || !centroids) return EC_ERR_INVALID;
+    EC_CUDA(cudaMemcpyAsync(km->centroids, centroids, (size_t)km->K * km->D * 4, cudaMemcpyDeviceToDevice, stream));
+    return EC_OK;
+}
+
+int ec_kmeans_get(ec_kmeans_t* km, float* centroids, int32_t* labels, float* reduced, uint32_t* contrib_count,
+                  ec_stream_t stream) {
+    if (!km) return EC_ERR_INVALID;
+    if (centroids) EC_CUDA(cudaMemcpyAsync(centroids, km->centroids, (size_t)km->K * km->D * 4, cudaMemcpyDeviceToDevice, stream));
+    if (labels) EC_CUDA(cudaMemcpyAsync(labels, km->labels, km->N * 4, cudaMemcpyDeviceToDevice, stream));
+    if (reduced) EC_CUDA(cudaMemcpyAsync(reduced, km->reduced, (size_t)km->K * (km->D + 4) * 4, cudaMemcpyDeviceToDevice, stream));
+    if (contrib_count) EC_CUDA(cudaMemcpyAsync(contrib_count, km->contrib, (size_t)km->K * 4, cudaMemcpyDeviceToDevice, stream));
+    return EC_OK;
+}
+
+int ec_kmeans_destroy(ec_kmeans_t* km) {
+    if (!km) return EC_ERR_INVALID;
+    int rc = EC_OK;
+    if (km->ar) ec_allreduce_destroy(km->ar);
+    if (km->own_ws && km->ws) {
+        cudaError_t e = cudaFree(km->ws);
+        if (e != cudaSuccess) rc = cuda_fail(e);
+    }
+    delete km;
+    return rc;
+}
+
+}  // extern "C"

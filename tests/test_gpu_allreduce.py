@@ -1,0 +1,292 @@
+"""GPU parity of ec_allreduce_* against the CPU checker, element by element, through the C ABI."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+pytestmark = pytest.mark.gpu
+
+import oracle
+from paper_2203_17063_b200 import inputs
+from tests.gpu_util import NP_OUT, bits, ec, run_schedule, sentinel, to_dev, to_host
+
+
+@pytest.fixture(autouse=True)
+def _need_gpu(cuda_device):
+    yield
+
+
+def _bufs(kind, seed, P, n, **kw):
+    return inputs.rank_buffers(kind, seed, P, n, **kw)
+
+
+# ---------------------------------------------------------------------------
+# the five workloads, reduced (several tiles, a ragged tail) and at full size
+# ---------------------------------------------------------------------------
+def test_config1_all_arrived_fixed_order_bit_exact():
+    P, n, seg = 4, 1 << 20, 16384
+    bufs = _bufs("uniform_f32", 1001, P, n)
+    (g, gc, c, cc), = run_schedule(P, n, seg, ec.F32, ec.SUM, bufs, [None])
+    assert (gc == P).all()
+    # all arrived: the result is the plain rank-order sum
+    acc = np.zeros(n, dtype=np.float32)
+    for b in bufs:
+        acc = acc + b
+    assert np.array_equal(bits(g), bits(acc))
+    # and the same with an explicit all-ones mask
+    S = n // seg
+    run_schedule(P, n, seg, ec.F32, ec.SUM, bufs, [np.full((S, 1), 0xF, dtype=np.uint64)])
+
+
+@pytest.mark.parametrize("n,seg", [((1 << 20) + 37, 65536), (1 << 24, 65536)], ids=["reduced", "full"])
+def test_config2_three_rounds(n, seg):
+    P = 16
+    S = (n + seg - 1) // seg
+    bufs = _bufs("normal_f32", 1002, P, n)
+    rounds = inputs.arrival_rounds(2002, P, S, 0.7)
+    masks = inputs.cumulative_masks(rounds)
+    outs = run_schedule(P, n, seg, ec.F32, ec.SUM, bufs, masks, oracle_threads=8)
+    g, gc, _, _ = outs[-1]
+    assert (gc == P).all()
+    # final result equals the one-shot fold in canonical order (round of arrival, rank)
+    order = np.argsort(rounds.T.astype(np.int32) * 1024 + np.arange(P)[None, :], axis=1, kind="stable").astype(np.int32)
+    one = oracle.allreduce_oneshot(bufs, oracle.F32, oracle.SUM, seg, order)
+    assert np.array_equal(bits(g), bits(one))
+    # and sits within the sequential-summation bound of the double sum
+    if n <= (1 << 21):
+        ref, mag = oracle.allreduce_ref64(bufs, oracle.F32, seg, None)
+        assert (np.abs(g.astype(np.float64) - ref) <= (P - 1) * 2.0 ** -24 * mag * 1.01).all()
+
+
+@pytest.mark.parametrize("n,seg", [((1 << 21) + 8 * 13, 131072), (1 << 25, 131072)], ids=["reduced", "full"])
+def test_config3_bf16_fixed_and_pairwise(n, seg):
+    P = 32
+    S = (n + seg - 1) // seg
+    bufs = _bufs("normal_bf16", 1003, P, n, sigma=1e-3)
+    rounds = inputs.arrival_rounds(2003, P, S, 0.9)
+    masks = inputs.cumulative_masks(rounds)
+    outs = run_schedule(P, n, seg, ec.BF16, ec.SUM, bufs, masks, oracle_threads=8)
+    assert (outs[-1][1] == P).all()
+    # pairwise variant: tolerance gate against the double-precision sum, on the round-1 subset and all-at-once
+    for m in (masks[0], None):
+        (g, gc, c, cc), = run_schedule(P, n, seg, ec.BF16, ec.SUM, bufs, [m], order=ec.ORDER_PAIRWISE,
+                                       oracle_threads=8, compare=False)
+        assert np.array_equal(gc, cc)
+        ref, mag = oracle.allreduce_ref64(bufs, oracle.BF16, seg, m)
+        tol = 1e-5 * math.log2(P) * mag
+        assert (np.abs(g.astype(np.float64) - ref) <= tol).all()
+        assert np.abs(g - ref).max() <= 1e-5 * math.log2(P) * np.abs(ref).max()
+        # the tree is the checker's tree: same bits
+        assert np.array_equal(bits(g), bits(c))
+
+
+@pytest.mark.parametrize("op", [ec.SUM, ec.MAX])
+def test_config4_int64_reductions(op):
+    P, n, seg = 256, 1 << 20, 8192
+    S = n // seg
+    bufs = _bufs("int64_below", 1004, P, n, bound=1 << 20)
+    rounds = inputs.arrival_rounds(2004, P, S, 0.8, last_round=2)
+    masks = inputs.cumulative_masks(rounds)
+    outs = run_schedule(P, n, seg, ec.I64, op, bufs, masks, oracle_threads=8)
+    g = outs[-1][0]
+    stack = np.stack(bufs)
+    assert np.array_equal(g, stack.sum(0) if op == ec.SUM else stack.max(0))
+
+
+def test_int64_full_range_wraps():
+    P, n, seg = 7, 50000, 4096
+    bufs = _bufs("int64_full", 5, P, n)
+    S = (n + seg - 1) // seg
+    masks = inputs.cumulative_masks(inputs.arrival_rounds(6, P, S, 0.5))
+    for op in (ec.SUM, ec.MAX, ec.MIN):
+        run_schedule(P, n, seg, ec.I64, op, bufs, masks)
+
+
+# ---------------------------------------------------------------------------
+# edge cases
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("P", [1, 2, 63, 64, 65, 128, 255, 256, 1024])
+def test_rank_counts_at_word_boundaries(P):
+    n, seg = 3000, 256
+    S = (n + seg - 1) // seg
+    bufs = _bufs("normal_f32", 100 + P, P, n)
+    rounds = inputs.arrival_rounds(200 + P, P, S, 0.6)
+    masks = inputs.cumulative_masks(rounds)
+    # garbage above bit P-1 must change nothing
+    if P % 64:
+        junk = np.uint64(((1 << 64) - 1) ^ ((1 << (P % 64)) - 1))
+        masks = [m.copy() for m in masks]
+        for m in masks:
+            m[:, -1] |= junk
+    poison = [rounds > t for t in (1, 2, 3)]
+    run_schedule(P, n, seg, ec.F32, ec.SUM, bufs, masks, poison=poison)
+
+
+@pytest.mark.parametrize("dtype,kind", [(ec.F32, "normal_f32"), (ec.BF16, "normal_bf16"), (ec.I64, "int64_full"),
+                                        (ec.F64, "f64")])
+@pytest.mark.parametrize("op", [ec.SUM, ec.MAX, ec.MIN])
+def test_every_dtype_and_op(dtype, kind, op):
+    P, n, seg = 5, 10000, 1024
+    S = (n + seg - 1) // seg
+    if kind == "f64":
+        bufs = [np.random.default_rng(r).standard_normal(n) for r in range(P)]
+    else:
+        bufs = _bufs(kind, 300, P, n)
+    rounds = inputs.arrival_rounds(301, P, S, 0.5)
+    rounds[:, 2] = 3                                   # a segment that is empty until the last round
+    masks = inputs.cumulative_masks(rounds)
+    run_schedule(P, n, seg, dtype, op, bufs, masks, poison=[rounds > t for t in (1, 2, 3)])
+
+
+@pytest.mark.parametrize("n,seg,off,roff", [
+    (1000, 64, 0, 0),        # aligned, vector path, n % seg != 0
+    (1000, 63, 0, 0),        # segment size not a multiple of the vector width: element-wise path
+    (1000, 64, 1, 0),        # rank buffers one element off 16-byte alignment
+    (1000, 64, 0, 1),        # result one element off
+    (50, 64, 0, 0),          # n < seg: a single short segment
+    (1001, 1, 0, 0),         # one element per segment
+    (4099, 4096, 0, 0),      # short last segment of 3 elements
+    (4103, 4100, 0, 0),      # vector path with a ragged tail inside every segment? (4100 % 4 == 0)
+])
+@pytest.mark.parametrize("dtype,kind", [(ec.F32, "normal_f32"), (ec.BF16, "normal_bf16"), (ec.I64, "int64_full")])
+def test_alignment_and_ragged_shapes(n, seg, off, roff, dtype, kind):
+    P = 6
+    S = (n + seg - 1) // seg
+    bufs = _bufs(kind, 400, P, n)
+    rounds = inputs.arrival_rounds(401 + n, P, S, 0.5)
+    masks = inputs.cumulative_masks(rounds)
+    run_schedule(P, n, seg, dtype, ec.SUM, bufs, masks, offset_elems=off, result_offset=roff)
+    run_schedule(P, n, seg, dtype, ec.SUM, bufs, masks, offset_elems=off, result_offset=roff, tile=(64, 96))
+
+
+@pytest.mark.parametrize("tile", [(64, 4), (128, 1000), (512, 1 << 16), (256, 12)])
+def test_tile_shapes_do_not_change_results(tile):
+    P, n, seg = 9, 70001, 9000
+    S = (n + seg - 1) // seg
+    bufs = _bufs("normal_f32", 500, P, n)
+    masks = inputs.cumulative_masks(inputs.arrival_rounds(501, P, S, 0.4))
+    run_schedule(P, n, seg, ec.F32, ec.SUM, bufs, masks, tile=tile)
+    run_schedule(P, n, seg, ec.F32, ec.SUM, bufs, masks[:1], tile=tile, order=ec.ORDER_PAIRWISE)
+
+
+@pytest.mark.parametrize("P", [1, 2, 3, 4, 5, 8, 9, 16, 31, 64, 100, 300])
+def test_pairwise_tree_matches_checker_bits(P):
+    n, seg = 2100, 512
+    S = (n + seg - 1) // seg
+    bufs = _bufs("normal_f32", 600 + P, P, n)
+    masks = inputs.cumulative_masks(inputs.arrival_rounds(601 + P, P, S, 0.6))
+    outs = run_schedule(P, n, seg, ec.F32, ec.SUM, bufs, masks, order=ec.ORDER_PAIRWISE)
+    ref, mag = oracle.allreduce_ref64(bufs, oracle.F32, seg, None)
+    g = outs[-1][0]
+    # three rounds, each a tree plus one add: error below (ceil(log2 P) + 3) rounding units of sum|x|
+    assert (np.abs(g - ref) <= (math.ceil(math.log2(max(P, 2))) + 3) * 2.0 ** -24 * mag * 1.01).all()
+    # bf16 and fp64 inputs through the same tree
+    b16 = _bufs("normal_bf16", 700 + P, P, n, sigma=1.0)
+    run_schedule(P, n, seg, ec.BF16, ec.SUM, b16, masks, order=ec.ORDER_PAIRWISE)
+    f64 = [np.random.default_rng(P * 10 + r).standard_normal(n) for r in range(P)]
+    run_schedule(P, n, seg, ec.F64, ec.SUM, f64, masks, order=ec.ORDER_PAIRWISE)
+
+
+def test_signed_zero_and_identity_rules():
+    n, seg = 64, 16
+    z = np.full(n, -0.0, dtype=np.float32)
+    outs = run_schedule(2, n, seg, ec.F32, ec.SUM, [z, z], [None])
+    assert not np.signbit(outs[0][0]).any()            # +0.0 + (-0.0) = +0.0
+    outs = run_schedule(2, n, seg, ec.F32, ec.MAX, [z, z], [None])
+    assert np.signbit(outs[0][0]).all()                # -0.0 > -inf
+    outs = run_schedule(2, n, seg, ec.F32, ec.SUM, [z, z], [None], order=ec.ORDER_PAIRWISE)
+    assert np.signbit(outs[0][0]).all()                # the tree adds -0.0 + -0.0 and nothing else
+    # nothing arrives in the first apply: identities everywhere, counts zero
+    none = np.zeros((4, 1), dtype=np.uint64)
+    for op, ident in ((ec.SUM, 0.0), (ec.MAX, -np.inf), (ec.MIN, np.inf)):
+        (g, gc, c, cc), = run_schedule(2, n, seg, ec.F32, op, [z, z], [none])
+        assert (g == ident).all() and (gc == 0).all()
+    (g, gc, _, _), = run_schedule(2, n, seg, ec.I64, ec.MAX, [np.zeros(n, np.int64)] * 2, [none])
+    assert (g == np.iinfo(np.int64).min).all()
+
+
+def test_idempotence_regress_reset_and_untouched_segments():
+    P, n, seg = 10, 5000, 500
+    S = 10
+    bufs = _bufs("normal_f32", 800, P, n)
+    rounds = inputs.arrival_rounds(801, P, S, 0.5)
+    rounds[:, 4] = 1                                   # segment 4 complete after round 1: idle afterwards
+    masks = inputs.cumulative_masks(rounds)
+    ar = ec.Allreduce(P, n, ec.F32, ec.SUM, seg)
+    d_bufs = [to_dev(b) for b in bufs]
+    d_res = to_dev(sentinel(np.float32, n))
+    d_cnt = torch.zeros(S, dtype=torch.int32, device="cuda")
+    d_masks = [to_dev(m) for m in masks]
+    ar.apply(d_bufs, d_masks[0], d_res, d_cnt)
+    first = to_host(d_res).copy()
+    assert not np.isnan(first).any()
+    # same mask again: not a byte changes
+    ar.apply(d_bufs, d_masks[0], d_res, d_cnt)
+    assert np.array_equal(bits(to_host(d_res)), bits(first))
+    # scribble into the idle segment: later applies must neither read nor write it
+    d_res[4 * seg:5 * seg] = 12345.0
+    ar.apply(d_bufs, d_masks[1], d_res, d_cnt)
+    assert (to_host(d_res)[4 * seg:5 * seg] == 12345.0).all()
+    # a mask with bits cleared (regress) un-applies nothing
+    before = to_host(d_res).copy()
+    cnt_before = d_cnt.cpu().numpy().copy()
+    ar.apply(d_bufs, to_dev(np.zeros_like(masks[0])), d_res, d_cnt)
+    assert np.array_equal(bits(to_host(d_res)), bits(before))
+    assert np.array_equal(d_cnt.cpu().numpy(), cnt_before)
+    ar.apply(d_bufs, d_masks[2], d_res, None)          # contrib_count may be NULL
+    # new epoch: the same schedule reproduces the same bits
+    runs = []
+    for _ in range(2):
+        ar.reset()
+        d_res.copy_(to_dev(sentinel(np.float32, n)))
+        for m in d_masks:
+            ar.apply(d_bufs, m, d_res, d_cnt)
+        runs.append(to_host(d_res).copy())
+    assert np.array_equal(bits(runs[0]), bits(runs[1]))
+    ref = oracle.Allreduce(P, n, oracle.F32, oracle.SUM, seg)
+    c = sentinel(np.float32, n)
+    for m in masks:
+        ref.apply(bufs, m, c, None)
+    assert np.array_equal(bits(runs[0]), bits(c))
+    ar.destroy()
+
+
+def test_argument_errors_on_device():
+    n, seg, P = 1000, 100, 3
+    ar = ec.Allreduce(P, n, ec.F32, ec.SUM, seg)
+    bufs = [torch.zeros(n, device="cuda") for _ in range(P)]
+    res = torch.zeros(n, device="cuda")
+    L = ec.lib()
+    tbl = (ec.C.c_void_p * P)(*[b.data_ptr() for b in bufs])
+    st = torch.cuda.current_stream().cuda_stream
+    assert L.ec_allreduce_apply(ar._h, tbl, P + 1, n, ec.F32, ec.SUM, seg, None, res.data_ptr(), None, st) == ec.ERR_INVALID
+    assert L.ec_allreduce_apply(ar._h, tbl, P, n, ec.I64, ec.SUM, seg, None, res.data_ptr(), None, st) == ec.ERR_INVALID
+    assert L.ec_allreduce_apply(ar._h, tbl, P, n, ec.F32, ec.SUM, seg, None, bufs[1].data_ptr(), None, st) == ec.ERR_INVALID
+    assert L.ec_allreduce_apply(ar._h, tbl, P, n, ec.F32, ec.SUM, seg, None, None, None, st) == ec.ERR_INVALID
+    assert L.ec_allreduce_apply(ar._h, tbl, P, n, ec.F32, ec.SUM, seg, None, res.data_ptr(), None, st) == ec.OK
+    torch.cuda.synchronize()
+    with pytest.raises(ec.EcError):
+        ec.Allreduce(P, n, ec.I64, ec.SUM, seg, ec.ORDER_PAIRWISE)
+    ar.destroy()
+
+
+def test_library_allocated_workspace():
+    """init with workspace = NULL lets the library allocate; results are the same."""
+    import ctypes as C
+    L = ec.lib()
+    P, n, seg = 4, 4096, 512
+    bufs = _bufs("normal_f32", 900, P, n)
+    d_bufs = [to_dev(b) for b in bufs]
+    h = C.c_void_p()
+    assert L.ec_allreduce_init(C.byref(h), P, n, ec.F32, ec.SUM, seg, ec.ORDER_FIXED, None, 0) == ec.OK
+    res = torch.empty(n, device="cuda")
+    tbl = (C.c_void_p * P)(*[b.data_ptr() for b in d_bufs])
+    assert L.ec_allreduce_apply(h, tbl, P, n, ec.F32, ec.SUM, seg, None, res.data_ptr(), None,
+                                torch.cuda.current_stream().cuda_stream) == ec.OK
+    torch.cuda.synchronize()
+    ref = oracle.Allreduce(P, n, oracle.F32, oracle.SUM, seg)
+    c = np.empty(n, dtype=np.float32)
+    ref.apply(bufs, None, c, None)
+    assert np.array_equal(bits(to_host(res)), bits(c))
+    assert L.ec_allreduce_destroy(h) == ec.OK

@@ -1,0 +1,156 @@
+"""GPU parity of the K-means driver against the CPU checker, through the C ABI.
+
+Labels must equal the checker's except at near-ties (relative gap between the two
+closest centroids below 1e-5), where the second-closest is also accepted;
+partial sums and centroids within 1e-4 relative (row norm); counts exact."""
+import numpy as np
+import pytest
+import torch
+
+pytestmark = pytest.mark.gpu
+
+import oracle
+from paper_2203_17063_b200 import inputs
+from tests.gpu_util import ec, to_dev, to_host
+
+
+@pytest.fixture(autouse=True)
+def _need_gpu(cuda_device):
+    yield
+
+
+def check_labels(g_labels, points, centroids, threads=8):
+    c_labels, d1, d2, second = oracle.kmeans_assign(points, centroids, threads)
+    diff = np.nonzero(g_labels != c_labels)[0]
+    if diff.size:
+        near = (d2[diff] - d1[diff]) <= 1e-5 * d2[diff]
+        assert near.all(), f"{(~near).sum()} label mismatches away from near-ties"
+        assert np.array_equal(g_labels[diff], second[diff]), "a mismatching label is not the second closest"
+    return c_labels, diff.size
+
+
+def rows_close(g, c, rel=1e-4):
+    num = np.linalg.norm(g.astype(np.float64) - c.astype(np.float64), axis=-1)
+    den = np.linalg.norm(c.astype(np.float64), axis=-1)
+    return (num <= rel * den + 1e-30).all()
+
+
+def lockstep(N, D, K, P, iters, seed, p_arrive=0.75):
+    points, comp, _ = inputs.kmeans_mixture(seed, N, D, K)
+    cents = inputs.kmeans_first_of_component(points, comp, K)
+    masks = inputs.kmeans_masks(seed + 1000, iters, P, K, p_arrive)
+    d_points = to_dev(points)
+    km = ec.KMeans(d_points, K, P, to_dev(cents))
+    d_labels = torch.empty(N, dtype=torch.int32, device="cuda")
+    d_part = torch.empty(P, K, D + 4, device="cuda")
+    d_cent = torch.empty(K, D, device="cuda")
+    d_red = torch.empty(K, D + 4, device="cuda")
+    d_cnt = torch.empty(K, dtype=torch.int32, device="cuda")
+    for t in range(iters):
+        # the GPU is fed the checker's current centroids
+        km.set_centroids(to_dev(cents))
+        km.assign(to_dev(cents), d_labels)
+        g_labels = to_host(d_labels)
+        c_labels, nmis = check_labels(g_labels, points, cents)
+        # partials from the checker's labels: sums within tolerance, counts exact
+        km.partials(to_dev(c_labels), d_part)
+        g_part = to_host(d_part)
+        c_part = oracle.kmeans_partials(points, c_labels, K, P, 8)
+        assert np.array_equal(g_part[:, :, D], c_part[:, :, D])
+        assert (g_part[:, :, D + 1:] == 0).all()
+        assert rows_close(g_part[:, :, :D], c_part[:, :, :D])
+        # whole iteration on the GPU vs the checker's iteration
+        km.iterate(to_dev(masks[t]))
+        km.get(d_cent, None, d_red, d_cnt)
+        torch.cuda.synchronize()
+        new, _, c_red, c_cnt = oracle.kmeans_iterate(points, cents, P, masks[t], 8)
+        assert np.array_equal(to_host(d_cnt).view(np.uint32), c_cnt)
+        if nmis == 0:
+            assert np.array_equal(to_host(d_red)[:, D], c_red[:, D])
+        assert rows_close(to_host(d_cent), new)
+        cents = new
+    km.destroy()
+
+
+def test_lockstep_small():
+    lockstep(N=1 << 15, D=32, K=64, P=64, iters=4, seed=1005)
+
+
+@pytest.mark.parametrize("N,D,K,P", [(5000, 8, 5, 3), (4099, 16, 7, 1), (3000, 4, 3, 7), (2048, 64, 9, 2),
+                                     (3001, 12, 6, 5), (2500, 128, 4, 2), (20000, 32, 200, 4)])
+def test_lockstep_shapes(N, D, K, P):
+    lockstep(N, D, K, P, iters=2, seed=77 + D)
+
+
+def test_exact_ties_take_the_lowest_index():
+    pts = np.zeros((300, 4), dtype=np.float32)
+    cents = np.array([[1, 0, 0, 0], [0, 1, 0, 0], [-1, 0, 0, 0], [0, 0, 0, 0.5]], dtype=np.float32)
+    cents = np.concatenate([cents[:3], cents[:3], cents[3:]])          # duplicates: exact ties
+    km = ec.KMeans(to_dev(pts), cents.shape[0], 1, to_dev(cents))
+    lab = torch.empty(300, dtype=torch.int32, device="cuda")
+    km.assign(to_dev(cents), lab)
+    assert (to_host(lab) == 6).all()
+    cents[6] = [0, 0, 0, 1]                                             # now seven centroids at distance 1
+    km.assign(to_dev(cents), lab)
+    assert (to_host(lab) == 0).all()
+    km.destroy()
+
+
+def test_free_running_config5_reduced():
+    """Both sides run their own trajectory for 20 iterations from the one-centroid-per-component start."""
+    N, D, K, P, iters = 1 << 17, 32, 64, 64, 20
+    points, comp, _ = inputs.kmeans_mixture(1005, N, D, K)
+    cents0 = inputs.kmeans_first_of_component(points, comp, K)
+    masks = inputs.kmeans_masks(2005, iters, P, K, 0.75)
+    km = ec.KMeans(to_dev(points), K, P, to_dev(cents0))
+    d_masks = [to_dev(m) for m in masks]
+    for t in range(iters):
+        km.iterate(d_masks[t])
+    d_cent = torch.empty(K, D, device="cuda")
+    d_labels = torch.empty(N, dtype=torch.int32, device="cuda")
+    km.get(d_cent, d_labels)
+    torch.cuda.synchronize()
+    cents = cents0
+    for t in range(iters):
+        prev = cents
+        cents, labels, _, _ = oracle.kmeans_iterate(points, cents, P, masks[t], 8)
+    assert rows_close(to_host(d_cent), cents)
+    # labels of the last iteration were taken against the centroids before the last update
+    check_labels(to_host(d_labels), points, prev)
+    km.destroy()
+
+
+def test_full_size_config5_one_iteration_sampled():
+    """N = 2^22 in the launch configuration the benchmark times; the checker labels a sample of points one by one."""
+    N, D, K, P = 1 << 22, 32, 64, 64
+    points, comp, _ = inputs.kmeans_mixture(1005, N, D, K)
+    cents = inputs.kmeans_first_of_component(points, comp, K)
+    mask = inputs.kmeans_masks(2005, 1, P, K, 0.75)[0]
+    km = ec.KMeans(to_dev(points), K, P, to_dev(cents))
+    km.iterate(to_dev(mask))
+    d_cent = torch.empty(K, D, device="cuda")
+    d_labels = torch.empty(N, dtype=torch.int32, device="cuda")
+    d_red = torch.empty(K, D + 4, device="cuda")
+    d_cnt = torch.empty(K, dtype=torch.int32, device="cuda")
+    km.get(d_cent, d_labels, d_red, d_cnt)
+    torch.cuda.synchronize()
+    g_labels = to_host(d_labels)
+    idx = np.random.default_rng(0).choice(N, size=1 << 16, replace=False)
+    idx.sort()
+    c_lab, d1, d2, second = oracle.kmeans_assign(points[idx], cents, 8)
+    diff = np.nonzero(g_labels[idx] != c_lab)[0]
+    assert ((d2[diff] - d1[diff]) <= 1e-5 * d2[diff]).all()
+    # properties that hold at any size: counts of arrived cells add up, centroids are means of labelled points
+    arrived = ((mask[:, 0][None, :] >> np.arange(P, dtype=np.uint64)[:, None]) & np.uint64(1)).astype(bool)   # [P][K]
+    assert np.array_equal(to_host(d_cnt).view(np.uint32), arrived.sum(0).astype(np.uint32))
+    shard = N // P
+    onehot_counts = np.stack([np.bincount(g_labels[r * shard:(r + 1) * shard], minlength=K) for r in range(P)])
+    assert np.array_equal(to_host(d_red)[:, D], (onehot_counts * arrived).sum(0).astype(np.float32))
+    k = int(np.argmax(arrived.sum(0)))
+    sel = np.zeros(N, dtype=bool)
+    for r in range(P):
+        if arrived[r, k]:
+            sel[r * shard:(r + 1) * shard] = g_labels[r * shard:(r + 1) * shard] == k
+    mean = points[sel].astype(np.float64).mean(0)
+    assert np.linalg.norm(to_host(d_cent)[k] - mean) <= 1e-4 * np.linalg.norm(mean)
+    km.destroy()
