@@ -295,14 +295,14 @@ apply_kernel(const ApplyArgs a, const __grid_constant__ PtrTable<CAP> tbl) {
 #pragma unroll
                         for (int u = 0; u < 8; ++u)
                             if ((byte >> u) & 1u)
-                                raw[u] = ld_stream16(reinterpret_cast<const char*>(tbl.p[r0 + u]) + e0 * sizeof(In), pol);
+                                raw[u] = ld_stream16(reinterpret_cast<const char*>(tbl.p[r0 + u]) + (lo + e0) * sizeof(In), pol);
 #pragma unroll
                         for (int u = 0; u < 8; ++u)
                             if ((byte >> u) & 1u) E::unpack(raw[u], lv[u]);
                     } else {
 #pragma unroll
                         for (int u = 0; u < 8; ++u)
-                            if ((byte >> u) & 1u) lv[u][0] = E::widen(reinterpret_cast<const In*>(tbl.p[r0 + u])[e0]);
+                            if ((byte >> u) & 1u) lv[u][0] = E::widen(reinterpret_cast<const In*>(tbl.p[r0 + u])[lo + e0]);
                     }
                 }
 #pragma unroll
