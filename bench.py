@@ -1,0 +1,585 @@
+#!/usr/bin/env python
+"""Benchmark of the eventually consistent collectives on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--no-extras]
+
+One "step" is one epoch of the headline workload (P=16 ranks, n=2^24 fp32 per
+rank, segments of 65536 elements, seeded three-round arrival schedule): a reset
+and three ec_allreduce_apply calls - the first produces the partial result from
+what has arrived, the next two fold the late segments in.  The metric is the
+algorithmic GB/s of those applies: bytes of every newly folded (rank, segment)
+plus bytes of result written (and read back, for segments that already held a
+partial result), computed from the actual masks.
+
+Prints ONE JSON line.  With --gpus N > 1 (under torchrun) every rank runs an
+independent replica on its own GPU - the path has no exchange between GPUs -
+and the line reports the sum over ranks divided by the slowest rank's time.
+"""
+from __future__ import annotations
+
+import argparse
+import ctypes as C
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+HEADLINE = dict(P=16, n=1 << 24, seg=65536, p_first=0.7, seed=1002, seed_sched=2002)
+NOMINAL_HBM_GBS = 8000.0
+
+# dram__bytes_read.sum + dram__bytes_write.sum of the three apply launches of one headline epoch, from
+# one ncu capture (see profiles/); None until a capture exists.
+NCU_TRAFFIC_BYTES_PER_EPOCH = None
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+# --------------------------------------------------------------------------------------------
+# algorithmic bytes of one apply, from the masks
+# --------------------------------------------------------------------------------------------
+def popcount64(a: np.ndarray) -> np.ndarray:
+    a = a.astype(np.uint64)
+    c = np.zeros(a.shape, dtype=np.int64)
+    for b in range(64):
+        c += ((a >> np.uint64(b)) & np.uint64(1)).astype(np.int64)
+    return c
+
+
+def apply_bytes(prev_mask, mask, P, n, seg, in_bytes, out_bytes, first_apply):
+    """Bytes one apply must move: inputs of the newly notified (rank, segment) pairs, the result
+    segments it writes, and the result segments it first reads (those that held a partial result)."""
+    S = (n + seg - 1) // seg
+    seg_len = np.minimum(seg, n - np.arange(S) * seg).astype(np.int64)
+    if mask is None:
+        mask = np.full((S, (P + 63) // 64), np.uint64(2 ** 64 - 1))
+        if P % 64:
+            mask[:, -1] = np.uint64((1 << (P % 64)) - 1)
+    prev = np.zeros_like(mask) if prev_mask is None else prev_mask
+    new = mask & ~prev
+    n_new = popcount64(new).sum(axis=1)
+    had = popcount64(prev).sum(axis=1) > 0
+    written = (n_new > 0) | (first_apply & ~had)
+    read_back = (n_new > 0) & had
+    total = (n_new * seg_len * in_bytes).sum() + (written * seg_len * out_bytes).sum() \
+        + (read_back * seg_len * out_bytes).sum()
+    words = mask.size * 8 * 2 + S * 4
+    return int(total + words)
+
+
+# --------------------------------------------------------------------------------------------
+# clocks during the timed region
+# --------------------------------------------------------------------------------------------
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.lines: list[str] = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._pump, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, smax, reasons = [], [], set()
+        for line in self.lines:
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                smax.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# --------------------------------------------------------------------------------------------
+# workloads
+# --------------------------------------------------------------------------------------------
+def make_headline_host(scale_n=None):
+    from paper_2203_17063_b200 import inputs
+    cfg = dict(HEADLINE)
+    if scale_n:
+        cfg["n"] = scale_n
+    S = (cfg["n"] + cfg["seg"] - 1) // cfg["seg"]
+    bufs = inputs.rank_buffers("normal_f32", cfg["seed"], cfg["P"], cfg["n"])
+    rounds = inputs.arrival_rounds(cfg["seed_sched"], cfg["P"], S, cfg["p_first"])
+    masks = inputs.cumulative_masks(rounds)
+    return cfg, bufs, masks
+
+
+def epoch_bytes(cfg, masks, in_b=4, out_b=4):
+    per_round, prev = [], None
+    for t, m in enumerate(masks):
+        per_round.append(apply_bytes(prev, m, cfg["P"], cfg["n"], cfg["seg"], in_b, out_b, t == 0))
+        prev = m
+    return per_round
+
+
+def ev_ms(pairs):
+    return [a.elapsed_time(b) for a, b in pairs]
+
+
+def mean_ci(xs):
+    m = statistics.fmean(xs)
+    if len(xs) < 2:
+        return m, 0.0
+    return m, 1.96 * statistics.stdev(xs) / (len(xs) ** 0.5)
+
+
+def run_ours(args, rank, world, local_rank):
+    import torch
+    from paper_2203_17063_b200 import binding as ec
+
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    peak, peak_kind = measured_peaks()
+    cfg, h_bufs, h_masks = make_headline_host()
+    P, n, seg = cfg["P"], cfg["n"], cfg["seg"]
+    S = n // seg
+    per_round_bytes = epoch_bytes(cfg, h_masks)
+    step_bytes = sum(per_round_bytes)
+
+    stream = torch.cuda.Stream(device=dev)
+    st = stream.cuda_stream
+    # pinned host copies (the end-to-end leg copies from these every step)
+    pin_bufs = [torch.from_numpy(b).pin_memory() for b in h_bufs]
+    d_bufs = [t.to(dev) for t in pin_bufs]
+    d_masks = [torch.from_numpy(m.view(np.int64)).to(dev) for m in h_masks]
+    d_res = torch.empty(n, dtype=torch.float32, device=dev)
+    d_cnt = torch.empty(S, dtype=torch.int32, device=dev)
+    pin_res = torch.empty(n, dtype=torch.float32).pin_memory()
+    pin_cnt = torch.empty(S, dtype=torch.int32).pin_memory()
+    ar = ec.Allreduce(P, n, ec.F32, ec.SUM, seg, device=dev)
+    if args.threads or args.tile:
+        ar.set_tile(args.threads, args.tile)
+    table = (C.c_void_p * P)(*[t.data_ptr() for t in d_bufs])
+    L = ec.lib()
+
+    def epoch(events=None):
+        L.ec_allreduce_reset(ar._h, st)
+        for t in range(len(d_masks)):
+            if events is not None:
+                events[t][0].record(stream)
+            rc = ar.apply_raw(table, d_masks[t].data_ptr(), d_res.data_ptr(), d_cnt.data_ptr(), st)
+            if events is not None:
+                events[t][1].record(stream)
+            if rc != 0:
+                raise ec.EcError(rc, "ec_allreduce_apply")
+
+    with torch.cuda.stream(stream):
+        for _ in range(args.warmup):
+            epoch()
+        barrier()
+        clocks = ClockSampler(local_rank)
+        clocks.start()
+        K = args.steps
+        step_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+        apply_ev = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+                     for _ in d_masks] for _ in range(K)]
+        t_all0 = torch.cuda.Event(enable_timing=True)
+        t_all1 = torch.cuda.Event(enable_timing=True)
+        t_all0.record(stream)
+        for k in range(K):
+            step_ev[k][0].record(stream)
+            epoch(apply_ev[k])
+            step_ev[k][1].record(stream)
+        t_all1.record(stream)
+        barrier()
+        clock_info = clocks.stop()
+    total_ms = t_all0.elapsed_time(t_all1)
+    steps_ms = ev_ms(step_ev)
+    round_ms = [[a.elapsed_time(b) for a, b in ev] for ev in apply_ev]        # [K][rounds]
+    kernel_ms_total = sum(sum(r) for r in round_ms)
+    launches = K * len(d_masks)
+
+    # ---- end to end: host buffers in, result out, copies inside the timed region ------------------
+    e2e_steps = max(3, min(10, K))
+    h2d = sum(t.numel() * t.element_size() for t in pin_bufs) + sum(m.numel() * 8 for m in d_masks)
+    d2h = pin_res.numel() * 4 + pin_cnt.numel() * 4
+    pin_masks = [torch.from_numpy(m.view(np.int64)).pin_memory() for m in h_masks]
+    with torch.cuda.stream(stream):
+        def e2e_epoch():
+            for r in range(P):
+                d_bufs[r].copy_(pin_bufs[r], non_blocking=True)
+            for t in range(len(d_masks)):
+                d_masks[t].copy_(pin_masks[t], non_blocking=True)
+            epoch()
+            pin_res.copy_(d_res, non_blocking=True)
+            pin_cnt.copy_(d_cnt, non_blocking=True)
+        e2e_epoch()
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(e2e_steps):
+            e2e_epoch()
+        e1.record(stream)
+        barrier()
+    e2e_ms = e0.elapsed_time(e1) / e2e_steps
+
+    # max over ranks
+    def max_over_ranks(x):
+        if dist is None:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    total_ms_max = max_over_ranks(total_ms)
+    e2e_ms_max = max_over_ranks(e2e_ms)
+    value = world * step_bytes * K / (total_ms_max * 1e-3) / 1e9
+    e2e_value = world * step_bytes / (e2e_ms_max * 1e-3) / 1e9
+    achieved = step_bytes * K / (kernel_ms_total * 1e-3) / 1e9
+    m_step, ci_step = mean_ci(steps_ms)
+
+    line = {
+        "metric": "ec_allreduce_apply_GBps",
+        "value": round(value, 2),
+        "unit": "GB/s",
+        "n_gpus": world,
+        "steps": K,
+        "warmup": args.warmup,
+        "ms_per_step": round(total_ms_max / K, 5),
+        "higher_is_better": True,
+        "scaling": "weak",
+        "vs_baseline": None,
+        "dtype": "f32",
+        "data": "synthetic",
+        "config": {
+            "workload": "config 2: P=16 ranks x n=2^24 fp32 N(0,1), segment 65536, op=sum, fixed rank order; "
+                        "3-round arrival schedule (70% round 1, rest round 2 or 3); step = reset + 3 applies",
+            "parallelism": "replicas only (no exchange between GPUs)" if world > 1 else "1 GPU",
+            "algorithmic_bytes_per_step": step_bytes,
+            "algorithmic_bytes_per_round": per_round_bytes,
+            "elements_per_s": round(world * n * K / (total_ms_max * 1e-3), 1),
+            "input_elements_per_s": round(world * P * n * K / (total_ms_max * 1e-3), 1),
+            "l2": "rank buffers (1 GiB) exceed L2 every step; the 64 MiB result is carried between rounds as in the workload",
+            "ms_per_step_mean_ci95": [round(m_step, 5), round(ci_step, 5)],
+            "ms_per_round_mean": [round(statistics.fmean(r[t] for r in round_ms), 5) for t in range(len(d_masks))],
+            "GBps_per_round": [round(per_round_bytes[t] / (statistics.fmean(r[t] for r in round_ms) * 1e-3) / 1e9, 1)
+                               for t in range(len(d_masks))],
+        },
+        "roofline": {
+            "bound": "hbm",
+            "kernel": "apply_kernel<f32,sum,vector,64,fixed> (all three launches of an epoch)",
+            "achieved": round(achieved, 1),
+            "peak": peak,
+            "peak_kind": f"of {peak_kind}",
+            "unit": "GB/s",
+            "frac": round(achieved / peak, 4),
+            "frac_of_nominal_8TBps": round(achieved / NOMINAL_HBM_GBS, 4),
+            "traffic": NCU_TRAFFIC_BYTES_PER_EPOCH,
+        },
+        "e2e": {"value": round(e2e_value, 2), "unit": "GB/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "ms_per_step": round(e2e_ms_max, 3), "steps": e2e_steps},
+        "gpu_launches": launches,
+        "clocks": clock_info,
+    }
+
+    if rank == 0 and world == 1:
+        line["cpu_baseline"] = cpu_baseline(cfg, h_bufs, h_masks, per_round_bytes, budget_s=args.cpu_seconds)
+        if not args.no_extras:
+            del h_bufs, pin_bufs, d_bufs
+            ar.destroy()
+            line["extras"] = extras(args, dev, stream, peak)
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps(line))
+
+
+# --------------------------------------------------------------------------------------------
+# the CPU checker as a timed baseline (never tuned for this)
+# --------------------------------------------------------------------------------------------
+def cpu_baseline(cfg, h_bufs, h_masks, per_round_bytes, budget_s=15.0):
+    import oracle
+    P, n, seg = cfg["P"], cfg["n"], cfg["seg"]
+    threads = oracle.max_threads()
+    ref = oracle.Allreduce(P, n, oracle.F32, oracle.SUM, seg)
+    res = np.empty(n, dtype=np.float32)
+    cnt = np.empty((n + seg - 1) // seg, dtype=np.uint32)
+    times = []
+    t_start = time.perf_counter()
+    while True:
+        ref.reset()
+        t0 = time.perf_counter()
+        for m in h_masks:
+            ref.apply(h_bufs, m, res, cnt, threads=threads)
+        times.append(time.perf_counter() - t0)
+        if time.perf_counter() - t_start > budget_s or len(times) >= 20:
+            break
+    best = min(times)
+    return {"value": round(sum(per_round_bytes) / best / 1e9, 3), "unit": "GB/s", "cores": threads, "kind": "oracle",
+            "sample": f"{len(times)} full epochs of the same workload (n={n}, 3 rounds), best of them; "
+                      f"mean {statistics.fmean(times) * 1e3:.1f} ms per epoch",
+            "host_cpus": os.cpu_count()}
+
+
+# --------------------------------------------------------------------------------------------
+# the other workloads (reported beside the headline; parity for them is in tests/)
+# --------------------------------------------------------------------------------------------
+def time_calls(stream, fn, reps, warm=3, before=None):
+    import torch
+    with torch.cuda.stream(stream):
+        for _ in range(warm):
+            if before:
+                before()
+            fn()
+        torch.cuda.synchronize()
+        evs = []
+        for _ in range(reps):
+            if before:
+                before()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            fn()
+            b.record(stream)
+            evs.append((a, b))
+        torch.cuda.synchronize()
+    return ev_ms(evs)
+
+
+def extras(args, dev, stream, peak):
+    import torch
+    from paper_2203_17063_b200 import binding as ec
+    from paper_2203_17063_b200 import inputs
+    out = {}
+    st = stream.cuda_stream
+    L = ec.lib()
+    reps = max(10, min(args.steps, 50))
+
+    def allreduce_case(name, P, n, seg, dtype, kind, seed, sched_seed, p_first, last_round, order=ec.ORDER_FIXED, **kw):
+        S = (n + seg - 1) // seg
+        h = inputs.rank_buffers(kind, seed, P, n, **kw)
+        if kind == "normal_bf16":
+            d = [torch.from_numpy(b.view(np.int16)).to(dev).view(torch.bfloat16) for b in h]
+        else:
+            d = [torch.from_numpy(b).to(dev) for b in h]
+        del h
+        in_b = d[0].element_size()
+        out_dt = ec.OUT_TORCH[dtype]
+        out_b = torch.empty(0, dtype=out_dt).element_size()
+        masks = inputs.cumulative_masks(inputs.arrival_rounds(sched_seed, P, S, p_first, last_round)) if last_round > 1 else [None]
+        d_masks = [None if m is None else torch.from_numpy(m.view(np.int64)).to(dev) for m in masks]
+        res = torch.empty(n, dtype=out_dt, device=dev)
+        cnt = torch.empty(S, dtype=torch.int32, device=dev)
+        ar = ec.Allreduce(P, n, dtype, ec.SUM, seg, order, device=dev)
+        if args.threads or args.tile:
+            ar.set_tile(args.threads, args.tile)
+        table = (C.c_void_p * P)(*[t.data_ptr() for t in d])
+        cfgd = dict(P=P, n=n, seg=seg)
+        rb = epoch_bytes(cfgd, masks, in_b, out_b) if masks[0] is not None else [apply_bytes(None, None, P, n, seg, in_b, out_b, True)]
+        entry = {}
+        # all at once
+        full_bytes = apply_bytes(None, None, P, n, seg, in_b, out_b, True)
+        ms = time_calls(stream, lambda: ar.apply_raw(table, None, res.data_ptr(), cnt.data_ptr(), st), reps,
+                        before=lambda: L.ec_allreduce_reset(ar._h, st))
+        m, ci = mean_ci(ms)
+        entry["all_at_once"] = {"ms": round(m, 5), "ci95": round(ci, 5), "GBps": round(full_bytes / m / 1e6, 1),
+                                "frac_measured": round(full_bytes / m / 1e6 / peak, 4),
+                                "frac_8TBps": round(full_bytes / m / 1e6 / NOMINAL_HBM_GBS, 4), "bytes": full_bytes}
+        if masks[0] is not None:
+            with torch.cuda.stream(stream):
+                per = [[] for _ in masks]
+                for k in range(reps + 3):
+                    L.ec_allreduce_reset(ar._h, st)
+                    evs = []
+                    for t, dm in enumerate(d_masks):
+                        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                        a.record(stream)
+                        ar.apply_raw(table, dm.data_ptr(), res.data_ptr(), cnt.data_ptr(), st)
+                        b.record(stream)
+                        evs.append((a, b))
+                    torch.cuda.synchronize()
+                    if k >= 3:
+                        for t, (a, b) in enumerate(evs):
+                            per[t].append(a.elapsed_time(b))
+            entry["rounds"] = [{"ms": round(statistics.fmean(p), 5), "GBps": round(rb[t] / statistics.fmean(p) / 1e6, 1),
+                                "frac_measured": round(rb[t] / statistics.fmean(p) / 1e6 / peak, 4), "bytes": rb[t]}
+                               for t, p in enumerate(per)]
+        ar.destroy()
+        out[name] = entry
+
+    allreduce_case("config1_P4_f32_n2^20", 4, 1 << 20, 16384, ec.F32, "uniform_f32", 1001, 0, 1.0, 1)
+    allreduce_case("config2_P16_f32_n2^24_all_at_once", 16, 1 << 24, 65536, ec.F32, "normal_f32", 1002, 2002, 0.7, 1)
+    allreduce_case("config3_P32_bf16_n2^25", 32, 1 << 25, 131072, ec.BF16, "normal_bf16", 1003, 2003, 0.9, 3, sigma=1e-3)
+    allreduce_case("config3_P32_bf16_n2^25_pairwise", 32, 1 << 25, 131072, ec.BF16, "normal_bf16", 1003, 2003, 0.9, 1,
+                   order=ec.ORDER_PAIRWISE, sigma=1e-3)
+    allreduce_case("config4_P256_i64_n2^20", 256, 1 << 20, 8192, ec.I64, "int64_below", 1004, 2004, 0.8, 2, bound=1 << 20)
+
+    # config 4 gather
+    P = 256
+    counts = inputs.gather_counts(1004, P)
+    hb = inputs.gather_buffers(1004, counts)
+    arrived = inputs.bernoulli_mask(2004, 0, P, 1, 0.8)[:, 0]
+    db = [torch.from_numpy(b).to(dev) for b in hb]
+    total = int(counts.sum())
+    d_counts = torch.from_numpy(counts).to(dev)
+    d_mask = torch.from_numpy(inputs.pack_mask(arrived[:, None]).reshape(-1).view(np.int64)).to(dev)
+    d_displs = torch.empty(P + 1, dtype=torch.int64, device=dev)
+    d_out = torch.empty(total, dtype=torch.int64, device=dev)
+    d_status = torch.empty(1, dtype=torch.int32, device=dev)
+    table = (C.c_void_p * P)(*[t.data_ptr() for t in db])
+    gbytes = 2 * 8 * int(counts[arrived].sum()) + P * 8 * 2
+    ms = time_calls(stream, lambda: L.ec_allgatherv(table, d_counts.data_ptr(), P, ec.I64, d_mask.data_ptr(),
+                                                    d_displs.data_ptr(), d_out.data_ptr(), total,
+                                                    d_status.data_ptr(), st), reps)
+    m, ci = mean_ci(ms)
+    out["config4_allgatherv_P256_i64"] = {"ms": round(m, 5), "ci95": round(ci, 5), "GBps": round(gbytes / m / 1e6, 1),
+                                          "bytes": gbytes, "note": "109 MB working set: L2-resident when repeated"}
+    del db, d_out
+
+    # config 5: K-means iterations per second
+    N, D, K, P = 1 << 22, 32, 64, 64
+    pts, comp, _ = inputs.kmeans_mixture(1005, N, D, K)
+    init = inputs.kmeans_first_of_component(pts, comp, K)
+    masks = [torch.from_numpy(m.view(np.int64)).to(dev) for m in inputs.kmeans_masks(2005, 20, P, K, 0.75)]
+    d_pts = torch.from_numpy(pts).to(dev)
+    d_init = torch.from_numpy(init).to(dev)
+    km = ec.KMeans(d_pts, K, P, d_init)
+    with torch.cuda.stream(stream):
+        for t in range(3):
+            km.iterate_raw(masks[t].data_ptr(), st)
+        runs = []
+        for rep in range(5):
+            km.set_centroids(d_init, stream)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            for t in range(20):
+                km.iterate_raw(masks[t].data_ptr(), st)
+            b.record(stream)
+            torch.cuda.synchronize()
+            runs.append(a.elapsed_time(b))
+        lab = torch.empty(N, dtype=torch.int32, device=dev)
+        ms_assign = time_calls(stream, lambda: km.assign(d_init, lab, stream), 10)
+        part = torch.empty(P, K, D + 4, device=dev)
+        ms_part = time_calls(stream, lambda: km.partials(lab, part, stream), 10)
+    m, ci = mean_ci(runs)
+    sm_clock_ghz = 1.965
+    alu_peak_lane_ops = 148 * 128 * sm_clock_ghz * 1e9
+    out["config5_kmeans_N2^22_D32_K64_P64"] = {
+        "iterations_per_s": round(20 / (m * 1e-3), 1), "ms_per_20_iterations": round(m, 3), "ci95": round(ci, 3),
+        "assign_ms": round(statistics.fmean(ms_assign), 4), "partials_ms": round(statistics.fmean(ms_part), 4),
+        "assign_frac_of_fp32_alu_bound": round((2.0 * N * K * D / alu_peak_lane_ops) / (statistics.fmean(ms_assign) * 1e-3), 4),
+        "note": "assign bound = 2*N*K*D lane-instructions (sub + fma) at 148 SMs x 128 lanes x 1.965 GHz",
+    }
+    km.destroy()
+    return out
+
+
+# --------------------------------------------------------------------------------------------
+# reference arm: the CPU checker, timed as it stands on the host cores
+# --------------------------------------------------------------------------------------------
+def run_reference(args, rank):
+    if rank != 0:
+        return
+    # bounded sample: the same workload with n cut to 2^21 per rank (1/8 of the elements), every step one epoch
+    sample_n = 1 << 21
+    cfg, h_bufs, h_masks = make_headline_host(scale_n=sample_n)
+    per_round = epoch_bytes(cfg, h_masks)
+    import oracle
+    threads = oracle.max_threads()
+    ref = oracle.Allreduce(cfg["P"], cfg["n"], oracle.F32, oracle.SUM, cfg["seg"])
+    res = np.empty(cfg["n"], dtype=np.float32)
+    cnt = np.empty((cfg["n"] + cfg["seg"] - 1) // cfg["seg"], dtype=np.uint32)
+
+    def epoch():
+        ref.reset()
+        for m in h_masks:
+            ref.apply(h_bufs, m, res, cnt, threads=threads)
+
+    for _ in range(args.warmup):
+        epoch()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        epoch()
+    dt = time.perf_counter() - t0
+    value = round(sum(per_round) * args.steps / dt / 1e9, 3)
+    sample = f"each step = one 3-round epoch of the headline workload cut to n={sample_n} per rank (1/8 of the elements)"
+    print(json.dumps({
+        "impl": "reference", "metric": "ec_allreduce_apply_GBps", "value": value, "unit": "GB/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(dt / args.steps * 1e3, 3),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": "config 2 (P=16, fp32, segment 65536, 3-round schedule) on the CPU checker; " + sample},
+        "cpu_baseline": {"value": value, "unit": "GB/s", "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-extras", action="store_true", help="headline workload only")
+    ap.add_argument("--cpu-seconds", type=float, default=15.0, help="time budget of the CPU baseline leg")
+    ap.add_argument("--threads", type=int, default=0, help="expert: threads per block of the apply kernel")
+    ap.add_argument("--tile", type=int, default=0, help="expert: elements per block of the apply kernel")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+    if world != args.gpus and world == 1 and args.gpus > 1:
+        raise SystemExit("launch with torchrun for --gpus > 1")
+    run_ours(args, rank, world, local_rank)
+
+
+if __name__ == "__main__":
+    main()
