@@ -105,31 +105,48 @@ class ClockSampler:
 
     def _pump(self):
         for line in self.proc.stdout:
-            self.lines.append(line.strip())
+            self.lines.append((time.perf_counter(), line.strip()))
 
-    def stop(self) -> dict:
+    def wait_first(self, timeout=8.0):
+        """Block until nvidia-smi has produced a sample (it takes a moment to start)."""
+        t0 = time.perf_counter()
+        while self.proc is not None and not self.lines and time.perf_counter() - t0 < timeout:
+            time.sleep(0.02)
+
+    def stop(self, t_begin=None, t_end=None) -> dict:
+        """Summary of the samples taken inside [t_begin, t_end] (host clock); if the window is too
+        short to hold three samples, of every sample since the sampler started (warm-up included)."""
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.12)
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
         except subprocess.TimeoutExpired:
             self.proc.kill()
-        sm, smax, reasons = [], [], set()
-        for line in self.lines:
+        rows = []
+        for ts, line in self.lines:
             f = [x.strip() for x in line.split(",")]
             if len(f) < 9:
                 continue
             try:
-                sm.append(float(f[1]))
-                smax.append(float(f[2]))
+                rows.append((ts, float(f[1]), float(f[2]), float(f[3]), f[5:9]))
             except ValueError:
                 continue
-            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+        inside = [r for r in rows if t_begin is not None and t_begin <= r[0] <= t_end]
+        window = "timed region"
+        if len(inside) < 3:
+            inside, window = rows, "warm-up + timed region + end-to-end leg (timed region shorter than 3 samples)"
+        reasons = set()
+        for r in inside:
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[4]):
                 if val.lower().startswith("active"):
                     reasons.add(name)
-        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
-                "reasons": sorted(reasons), "samples": len(sm)}
+        busy = [r for r in inside if r[3] > 300.0] or inside        # samples under load (power well above idle)
+        return {"sm_mhz": statistics.median(r[1] for r in busy) if busy else None,
+                "sm_max_mhz": max(r[2] for r in inside) if inside else None,
+                "power_w_max": max(r[3] for r in inside) if inside else None,
+                "reasons": sorted(reasons), "samples": len(inside), "window": window}
 
 
 # --------------------------------------------------------------------------------------------
@@ -218,11 +235,13 @@ def run_ours(args, rank, world, local_rank):
                 raise ec.EcError(rc, "ec_allreduce_apply")
 
     with torch.cuda.stream(stream):
+        clocks = ClockSampler(local_rank)
+        clocks.start()
+        clocks.wait_first()
         for _ in range(args.warmup):
             epoch()
         barrier()
-        clocks = ClockSampler(local_rank)
-        clocks.start()
+        t_host0 = time.perf_counter()
         K = args.steps
         step_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
         apply_ev = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
@@ -236,7 +255,12 @@ def run_ours(args, rank, world, local_rank):
             step_ev[k][1].record(stream)
         t_all1.record(stream)
         barrier()
-        clock_info = clocks.stop()
+        t_host1 = time.perf_counter()
+    if args.profile_only:
+        clocks.stop()
+        if rank == 0:
+            print(json.dumps({"profile_only": True, "steps": K, "ms_per_step": t_all0.elapsed_time(t_all1) / K}))
+        return
     total_ms = t_all0.elapsed_time(t_all1)
     steps_ms = ev_ms(step_ev)
     round_ms = [[a.elapsed_time(b) for a, b in ev] for ev in apply_ev]        # [K][rounds]
@@ -266,6 +290,7 @@ def run_ours(args, rank, world, local_rank):
         e1.record(stream)
         barrier()
     e2e_ms = e0.elapsed_time(e1) / e2e_steps
+    clock_info = clocks.stop(t_host0, t_host1)
 
     # max over ranks
     def max_over_ranks(x):
@@ -560,8 +585,9 @@ def run_reference(args, rank):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=100)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=50)
+    ap.add_argument("--profile-only", action="store_true", help="warm-up and timed steps only (for ncu captures)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-extras", action="store_true", help="headline workload only")
     ap.add_argument("--cpu-seconds", type=float, default=15.0, help="time budget of the CPU baseline leg")

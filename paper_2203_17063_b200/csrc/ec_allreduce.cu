@@ -98,11 +98,11 @@ template <int OP> __device__ __forceinline__ long long ident(long long) {
 
 // accumulator vector <-> result memory (VEC accumulators = VEC*sizeof(Acc)/16 stores of 16 bytes)
 template <class Acc, int VEC>
-__device__ __forceinline__ void load_acc(const Acc* p, Acc (&acc)[VEC]) {
+__device__ __forceinline__ void load_acc(const Acc* p, Acc (&acc)[VEC], uint64_t rpol) {
     constexpr int PER = 16 / sizeof(Acc);
 #pragma unroll
     for (int q = 0; q < VEC / PER; ++q) {
-        const uint4 r = ld_plain16(p + q * PER);
+        const uint4 r = ld_hint16(p + q * PER, rpol);
         if (sizeof(Acc) == 4) {
             acc[q * PER + 0] = (Acc)__uint_as_float(r.x); acc[q * PER + 1] = (Acc)__uint_as_float(r.y);
             acc[q * PER + 2] = (Acc)__uint_as_float(r.z); acc[q * PER + 3] = (Acc)__uint_as_float(r.w);
@@ -115,7 +115,7 @@ __device__ __forceinline__ void load_acc(const Acc* p, Acc (&acc)[VEC]) {
     }
 }
 template <class Acc, int VEC>
-__device__ __forceinline__ void store_acc(Acc* p, const Acc (&acc)[VEC]) {
+__device__ __forceinline__ void store_acc(Acc* p, const Acc (&acc)[VEC], uint64_t rpol) {
     constexpr int PER = 16 / sizeof(Acc);
 #pragma unroll
     for (int q = 0; q < VEC / PER; ++q) {
@@ -129,7 +129,7 @@ __device__ __forceinline__ void store_acc(Acc* p, const Acc (&acc)[VEC]) {
             memcpy(w, &acc[q * PER], 16);
             r = make_uint4((uint32_t)w[0], (uint32_t)(w[0] >> 32), (uint32_t)w[1], (uint32_t)(w[1] >> 32));
         }
-        st_plain16(p + q * PER, r);
+        st_hint16(p + q * PER, r, rpol);
     }
 }
 
@@ -142,11 +142,63 @@ struct ApplyArgs {
     uint32_t* contrib_count;     // [S] or nullptr
     unsigned tiles_per_seg;
     int P, W, first_apply;
+    int res_hint;                // reserved: cache policy of the result accesses
 };
 
 constexpr int RU = 8;        // rank buffers whose loads are issued together (independent loads, ordered adds)
 constexpr int MAX_W = EC_MAX_RANKS / 64;
 constexpr int TREE_LEVELS = 7;  // 1024 ranks / 8 per leaf block = 128 blocks = 2^7
+
+// Fold the m new ranks into VPT result vectors per thread, RU rank loads per vector in flight.
+// Loads are independent and issued together; the adds of one vector stay in ascending rank order.
+template <int DT, int OP, int VPT, int RUN>
+__device__ __forceinline__ void fold_vectors(const char* const* s_ptr, int m, typename Elem<DT>::Acc* res, size_t nvec,
+                                             bool fresh, int tid, int nthr, uint64_t pol, uint64_t rpol) {
+    typedef Elem<DT> E;
+    typedef typename E::Acc Acc;
+    constexpr int VEC = E::VEC;
+    for (size_t v0 = tid; v0 < nvec; v0 += (size_t)nthr * VPT) {
+        Acc acc[VPT][VEC];
+#pragma unroll
+        for (int p = 0; p < VPT; ++p) {
+            const size_t v = v0 + (size_t)p * nthr;
+            if (fresh || v >= nvec) {
+#pragma unroll
+                for (int e = 0; e < VEC; ++e) acc[p][e] = ident<OP>(Acc());
+            } else {
+                load_acc<Acc, VEC>(res + v * VEC, acc[p], rpol);
+            }
+        }
+        for (int j = 0; j < m; j += RUN) {
+            uint4 raw[VPT][RUN];
+#pragma unroll
+            for (int p = 0; p < VPT; ++p) {
+                const size_t v = v0 + (size_t)p * nthr;
+#pragma unroll
+                for (int u = 0; u < RUN; ++u)
+                    if (j + u < m && v < nvec) raw[p][u] = ld_stream16(s_ptr[j + u] + v * 16, pol);
+            }
+#pragma unroll
+            for (int p = 0; p < VPT; ++p) {
+                const size_t v = v0 + (size_t)p * nthr;
+#pragma unroll
+                for (int u = 0; u < RUN; ++u) {
+                    if (j + u < m && v < nvec) {
+                        Acc x[VEC];
+                        E::unpack(raw[p][u], x);
+#pragma unroll
+                        for (int e = 0; e < VEC; ++e) acc[p][e] = comb<OP>(acc[p][e], x[e]);
+                    }
+                }
+            }
+        }
+#pragma unroll
+        for (int p = 0; p < VPT; ++p) {
+            const size_t v = v0 + (size_t)p * nthr;
+            if (v < nvec) store_acc<Acc, VEC>(res + v * VEC, acc[p], rpol);
+        }
+    }
+}
 
 // ---------------------------------------------------------------------------------------------
 // the apply kernel
@@ -176,7 +228,8 @@ apply_kernel(const ApplyArgs a, const __grid_constant__ PtrTable<CAP> tbl) {
         if (lane < a.W) {
             uint64_t arr = a.arrival ? a.arrival[(size_t)s * a.W + lane] : ~0ull;
             if (lane == a.W - 1 && (a.P & 63)) arr &= (1ull << (a.P & 63)) - 1;   // bits >= P mean nothing
-            old = a.applied_in[(size_t)s * a.W + lane];
+            // the first apply of an epoch starts from "nothing folded in": no need to clear the words
+            old = a.first_apply ? 0ull : a.applied_in[(size_t)s * a.W + lane];
             nw = arr & ~old;
         }
         const unsigned any_new = __ballot_sync(0xffffffffu, nw != 0);
@@ -216,38 +269,20 @@ apply_kernel(const ApplyArgs a, const __grid_constant__ PtrTable<CAP> tbl) {
     Acc* res = reinterpret_cast<Acc*>(a.result) + lo;
     const int tid = threadIdx.x, nthr = blockDim.x;
     const uint64_t pol = evict_first_policy();
+    const uint64_t rpol = result_policy(a.res_hint);
 
     if (ORDER == EC_ORDER_FIXED) {
         for (int j = tid; j < m; j += nthr)
             s_ptr[j] = reinterpret_cast<const char*>(tbl.p[s_rank[j]]) + lo * sizeof(In);
         __syncthreads();
         const size_t nvec = VECTOR ? cnt / VEC : 0;
-        for (size_t v = tid; v < nvec; v += nthr) {
-            Acc acc[VEC];
-            if (fresh) {
-#pragma unroll
-                for (int e = 0; e < VEC; ++e) acc[e] = ident<OP>(Acc());
-            } else {
-                load_acc<Acc, VEC>(res + v * VEC, acc);
-            }
-            const size_t boff = v * 16;
-            for (int j = 0; j < m; j += RU) {
-                uint4 raw[RU];
-#pragma unroll
-                for (int u = 0; u < RU; ++u)
-                    if (j + u < m) raw[u] = ld_stream16(s_ptr[j + u] + boff, pol);
-#pragma unroll
-                for (int u = 0; u < RU; ++u) {
-                    if (j + u < m) {
-                        Acc x[VEC];
-                        E::unpack(raw[u], x);
-#pragma unroll
-                        for (int e = 0; e < VEC; ++e) acc[e] = comb<OP>(acc[e], x[e]);
-                    }
-                }
-            }
-            store_acc<Acc, VEC>(res + v * VEC, acc);
-        }
+        // Few new ranks (a late round): each thread keeps several result vectors in flight;
+        // many new ranks (a first round): one vector per thread, eight rank loads in flight.
+        // (Eight accumulators per bf16 vector: half as many vectors per thread keeps the registers at 64.)
+        constexpr int LATE = VEC > 4 ? 2 : 4, MID = VEC > 4 ? 1 : 2;
+        if (m <= 2) fold_vectors<DT, OP, LATE, 2>(s_ptr, m, res, nvec, fresh, tid, nthr, pol, rpol);
+        else if (m <= 4) fold_vectors<DT, OP, MID, 4>(s_ptr, m, res, nvec, fresh, tid, nthr, pol, rpol);
+        else fold_vectors<DT, OP, 1, 8>(s_ptr, m, res, nvec, fresh, tid, nthr, pol, rpol);
         // element-wise path: everything when the 128-bit path does not apply, else the ragged tail
         for (size_t i = nvec * VEC + tid; i < cnt; i += nthr) {
             Acc acc = fresh ? ident<OP>(Acc()) : res[i];
@@ -336,11 +371,11 @@ apply_kernel(const ApplyArgs a, const __grid_constant__ PtrTable<CAP> tbl) {
             if (isvec) {
                 if (!fresh) {
                     Acc acc[VEC];
-                    load_acc<Acc, VEC>(res + e0, acc);
+                    load_acc<Acc, VEC>(res + e0, acc, rpol);
 #pragma unroll
                     for (int e = 0; e < VEC; ++e) node[e] = comb<OP>(acc[e], node[e]);
                 }
-                store_acc<Acc, VEC>(res + e0, node);
+                store_acc<Acc, VEC>(res + e0, node, rpol);
             } else {
                 res[e0] = fresh ? node[0] : comb<OP>(res[e0], node[0]);
             }
@@ -409,6 +444,7 @@ struct ec_ctx {
     bool first_apply;  // no apply yet in this epoch
     int threads;
     size_t tile;       // elements per block
+    int res_hint;      // L2 policy of the result accesses
 };
 
 using namespace ec;
@@ -451,7 +487,8 @@ int ec_allreduce_init(ec_ctx_t** out, int P, size_t n, ec_dtype_t dtype, ec_op_t
     c->applied[1] = reinterpret_cast<uint64_t*>(reinterpret_cast<char*>(c->ws) + need / 2);
     c->cur = 0;
     c->first_apply = true;
-    c->threads = 256;
+    c->res_hint = 1;     // keep the partial result in L2 for the next round (measured: +2% per epoch)
+    c->threads = 128;    // many small blocks overlap their start-up latency best (measured)
     c->tile = 8192 / in_bytes(dtype);   // 8 KB of every rank buffer per block
     *out = c;
     return EC_OK;
@@ -493,6 +530,7 @@ int ec_allreduce_apply(ec_ctx_t* c, const void* const* rank_bufs, int P, size_t 
     a.contrib_count = contrib_count;
     a.tiles_per_seg = (unsigned)tiles;
     a.P = c->P; a.W = c->W; a.first_apply = c->first_apply ? 1 : 0;
+    a.res_hint = c->res_hint;
     const unsigned grid = (unsigned)(tiles * c->S);
     int rc;
     switch (c->dtype) {
@@ -510,7 +548,7 @@ int ec_allreduce_apply(ec_ctx_t* c, const void* const* rank_bufs, int P, size_t 
 
 int ec_allreduce_reset(ec_ctx_t* c, ec_stream_t stream) {
     if (!c) return EC_ERR_INVALID;
-    EC_CUDA(cudaMemsetAsync(c->applied[c->cur], 0, (size_t)c->S * c->W * sizeof(uint64_t), stream));
+    (void)stream;               // nothing to enqueue: the next apply ignores the stored words
     c->first_apply = true;
     return EC_OK;
 }
