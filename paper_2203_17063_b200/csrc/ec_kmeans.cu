@@ -25,6 +25,7 @@ constexpr int AS_THREADS = 256;
 constexpr int PT_THREADS = 256;
 constexpr int PT_WARPS = PT_THREADS / 32;
 constexpr size_t SMEM_BUDGET = 200 * 1024;
+constexpr size_t ASSIGN_SMEM_MAX = 64 * 1024;   // centroid chunk staged by the assignment kernels
 
 // ---------------------------------------------------------------------------------------------
 // assignment
@@ -386,18 +387,18 @@ int ec_kmeans_init(ec_kmeans_t** out, const float* points, size_t N, int D, int 
     const size_t stride = (size_t)D + 4;
     int rc = EC_OK;
     cudaError_t e = cudaSuccess;
-    if (km->assign_smem > 48 * 1024) {
-        switch (D) {
-            case 4: e = cudaFuncSetAttribute(assign_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)km->assign_smem); break;
-            case 8: e = cudaFuncSetAttribute(assign_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)km->assign_smem); break;
-            case 16: e = cudaFuncSetAttribute(assign_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)km->assign_smem); break;
-            case 32: e = cudaFuncSetAttribute(assign_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)km->assign_smem); break;
-            case 64: e = cudaFuncSetAttribute(assign_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)km->assign_smem); break;
-            default: e = cudaFuncSetAttribute(assign_generic_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)km->assign_smem);
-        }
+    // The dynamic shared memory limit is a property of the kernel, not of this context: always raise it to
+    // the largest size any shape can ask for, so that contexts of different shapes do not lower each other's.
+    switch (D) {
+        case 4: e = cudaFuncSetAttribute(assign_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ASSIGN_SMEM_MAX); break;
+        case 8: e = cudaFuncSetAttribute(assign_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ASSIGN_SMEM_MAX); break;
+        case 16: e = cudaFuncSetAttribute(assign_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ASSIGN_SMEM_MAX); break;
+        case 32: e = cudaFuncSetAttribute(assign_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ASSIGN_SMEM_MAX); break;
+        case 64: e = cudaFuncSetAttribute(assign_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ASSIGN_SMEM_MAX); break;
+        default: e = cudaFuncSetAttribute(assign_generic_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ASSIGN_SMEM_MAX);
     }
-    if (e == cudaSuccess && km->part_smem > 48 * 1024)
-        e = cudaFuncSetAttribute(partials_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)km->part_smem);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(partials_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BUDGET);
     if (e == cudaSuccess) e = cudaMemcpyAsync(km->centroids, init_centroids, (size_t)K * D * 4, cudaMemcpyDeviceToDevice, 0);
     if (e == cudaSuccess) e = cudaStreamSynchronize(0);
     if (e != cudaSuccess) rc = cuda_fail(e);
