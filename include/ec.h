@@ -221,6 +221,40 @@ int ec_kmeans_get(ec_kmeans_t* km, float* centroids, int32_t* labels, float* red
 
 int ec_kmeans_destroy(ec_kmeans_t* km);
 
+/* Per-rank partial sums for callers that are not allowed to allocate device
+ * memory.  (An addition of this library; the paper has no counterpart.)
+ *
+ * Some callers cannot call cudaMalloc at the point where they need this step:
+ * a serving process whose framework has claimed all device memory for its own
+ * pool at start-up, so that a later cudaMalloc simply fails; a latency-critical
+ * loop or a callback that must not block, while cudaMalloc and cudaFree
+ * synchronise the whole device and take a process-wide lock; a plug-in whose
+ * host forbids allocations outside its own allocator.  The context-based call
+ * above needs a workspace (someone has to allocate it); this one needs none.
+ *
+ * It computes exactly what ec_kmeans_partials computes (same kernels, same
+ * order of additions, same bits) from
+ *   points    device fp32 [N][D], 16-byte aligned
+ *   labels    device int32 [N]
+ *   partials  device fp32 [P][K][D+4], written
+ * with the same limits on N, D, K, P as the K-means driver.  The per-block
+ * partial sums that the workspace would hold go to a fixed 8 MiB array inside
+ * the library image (every GPU that loads the library holds those 8 MiB until
+ * the process ends).  Shapes whose per-block sums need more than 8 MiB are
+ * rejected with EC_ERR_CAPACITY before anything is launched (for the K-means
+ * workload of the benchmark they need 2.4 MB).
+ *
+ * The call itself allocates nothing: no cudaMalloc, no cudaFree, no allocating
+ * library routine.  The first call on each device looks up the device address
+ * of the array and raises the kernel's shared-memory limit; make that first
+ * call before starting any stream capture.
+ * All calls on a device share the one array.  A call overwrites every element
+ * it later reads, so no clearing is needed and nothing leaks from the previous
+ * call; but two calls that run on the GPU at the same time (different streams,
+ * different threads) race on it and give wrong sums - order them. */
+int ec_kmeans_partials_static(const float* points, const int32_t* labels, size_t N, int D, int K, int P,
+                              float* partials, ec_stream_t stream);
+
 /* ------------------------------------------------------------------------- */
 const char* ec_strerror(int code);
 /* The cudaError_t of the last failed CUDA call on this thread (0 if none). */

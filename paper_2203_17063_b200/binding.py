@@ -42,6 +42,7 @@ SYMBOLS = {
     "ec_kmeans_set_centroids": (_i, [_vp, _vp, _vp]),
     "ec_kmeans_get": (_i, [_vp, _vp, _vp, _vp, _vp, _vp]),
     "ec_kmeans_destroy": (_i, [_vp]),
+    "ec_kmeans_partials_static": (_i, [_vp, _vp, _sz, _i, _i, _i, _vp, _vp]),
     "ec_strerror": (C.c_char_p, [_i]),
     "ec_last_cuda_error": (_i, []),
     "ec_version": (_i, []),
@@ -199,3 +200,12 @@ class KMeans:
             self.destroy()
         except Exception:
             pass
+
+
+def kmeans_partials_static(points: torch.Tensor, labels: torch.Tensor, K: int, P: int, partials: torch.Tensor,
+                           stream=None) -> None:
+    """ec_kmeans_partials_static: the per-rank partial sums without a workspace, for callers that
+    must not allocate device memory (the per-block sums go to a fixed array inside the library)."""
+    N, D = points.shape
+    _check(lib().ec_kmeans_partials_static(_ptr(points), _ptr(labels), N, D, K, P, _ptr(partials), _stream(stream)),
+           "ec_kmeans_partials_static")

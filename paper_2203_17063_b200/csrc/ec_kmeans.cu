@@ -472,3 +472,69 @@ int ec_kmeans_destroy(ec_kmeans_t* km) {
 }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------------------------
+// Per-rank partial sums for callers that must not allocate device memory
+// ---------------------------------------------------------------------------------------------
+// Same two kernels as ec_kmeans_partials, but the per-block partial sums go to a fixed array that
+// is part of the library image instead of a workspace.  Every GPU that loads the library carries
+// these 8 MiB until the process exits, whether or not the entry point is ever called.
+namespace {
+
+constexpr size_t STATIC_SCRATCH_BYTES = 8u << 20;
+static __device__ __align__(256) unsigned char g_static_scratch[STATIC_SCRATCH_BYTES];
+
+constexpr int MAX_DEVICES = 64;
+struct StaticDeviceState {
+    bool ready;
+    float* scratch;   // device address of g_static_scratch on that device
+    int sms;
+};
+StaticDeviceState g_static_state[MAX_DEVICES];   // host side, indexed by device ordinal; zero-initialised
+
+// Once per device, with that device current.  In host code `g_static_scratch` is only a handle of
+// the symbol, not an address the GPU understands: the device address has to be asked for.
+int static_setup(int dev, StaticDeviceState** out) {
+    if (dev < 0 || dev >= MAX_DEVICES) return EC_ERR_CAPACITY;
+    StaticDeviceState* st = &g_static_state[dev];
+    if (!st->ready) {
+        void* addr = nullptr;
+        EC_CUDA(cudaGetSymbolAddress(&addr, g_static_scratch));
+        int sms = 0;
+        EC_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+        EC_CUDA(cudaFuncSetAttribute(partials_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BUDGET));
+        st->scratch = reinterpret_cast<float*>(addr);
+        st->sms = sms > 0 ? sms : 148;
+        st->ready = true;
+    }
+    *out = st;
+    return EC_OK;
+}
+
+}  // namespace
+
+extern "C" int ec_kmeans_partials_static(const float* points, const int32_t* labels, size_t N, int D, int K, int P,
+                                         float* partials, ec_stream_t stream) {
+    if (!points || !labels || !partials || km_bad_shape(N, D, K, P)) return EC_ERR_INVALID;
+    int dev = 0;
+    EC_CUDA(cudaGetDevice(&dev));
+    StaticDeviceState* st = nullptr;
+    const int rc = static_setup(dev, &st);
+    if (rc != EC_OK) return rc;
+    KmLayout L;
+    if (!km_plan(N, D, K, P, st->sms, &L)) return EC_ERR_CAPACITY;
+    const size_t row = (size_t)K * ((size_t)D + 4);
+    if (L.C > 1 && (size_t)P * L.C * row * sizeof(float) > STATIC_SCRATCH_BYTES) return EC_ERR_CAPACITY;
+    const size_t smem = (size_t)L.warps * ((size_t)K * D + K) * 4;
+    // Every element of the scratch that the fold reads was written by the first kernel of this
+    // same call, so nothing left over from an earlier call can leak in and nothing needs clearing.
+    float* first = L.C == 1 ? partials : st->scratch;
+    partials_kernel<<<(unsigned)(P * L.C), PT_THREADS, smem, stream>>>(points, labels, N, D, K, P, L.C, L.warps, first);
+    EC_CUDA(cudaGetLastError());
+    if (L.C > 1) {
+        const size_t total = row * P;
+        partials_fold_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(st->scratch, L.C, row, total, partials);
+        EC_CUDA(cudaGetLastError());
+    }
+    return EC_OK;
+}
