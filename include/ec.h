@@ -139,7 +139,7 @@ int ec_allreduce_apply(ec_ctx_t* ctx, const void* const* rank_bufs, int P, size_
 int ec_allreduce_reset(ec_ctx_t* ctx, ec_stream_t stream);
 
 /* Expert knob: elements of one segment handled per thread block (rounded to the
- * vector width) and threads per block (64..512, multiple of 32).  0 keeps the
+ * vector width) and threads per block (64..256, multiple of 32).  0 keeps the
  * current value.  Affects speed only, never results. */
 int ec_allreduce_set_tile(ec_ctx_t* ctx, int threads, size_t tile_elems);
 

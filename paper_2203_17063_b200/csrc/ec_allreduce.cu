@@ -145,6 +145,30 @@ struct ApplyArgs {
     int res_hint;                // reserved: cache policy of the result accesses
 };
 
+// Shape of the streaming loop, chosen by measurement on B200 (config 2 and 3 epochs): what counts
+// is resident threads, not loads per thread - 40 registers (6 blocks of 256 threads per SM) beat
+// 64 and 96 registers by 2 % and 20 %; spilling to reach 32 loses 10 %.
+#ifndef EC_MAXT
+#define EC_MAXT 256      // largest block size
+#endif
+#ifndef EC_MINB
+#define EC_MINB 6        // resident blocks of EC_MAXT threads the register allocation must allow
+#endif
+#ifndef EC_MAIN_RU
+#define EC_MAIN_RU 4     // first rounds: rank loads in flight per result vector
+#endif
+#ifndef EC_LATE_VPT
+#define EC_LATE_VPT 2    // late rounds with <= EC_LATE_RU new ranks: result vectors per thread
+#endif
+#ifndef EC_LATE_RU
+#define EC_LATE_RU 2
+#endif
+#ifndef EC_MID_VPT
+#define EC_MID_VPT 1
+#endif
+#ifndef EC_MID_RU
+#define EC_MID_RU 4
+#endif
 constexpr int RU = 8;        // rank buffers whose loads are issued together (independent loads, ordered adds)
 constexpr int MAX_W = EC_MAX_RANKS / 64;
 constexpr int TREE_LEVELS = 7;  // 1024 ranks / 8 per leaf block = 128 blocks = 2^7
@@ -204,7 +228,7 @@ __device__ __forceinline__ void fold_vectors(const char* const* s_ptr, int m, ty
 // the apply kernel
 // ---------------------------------------------------------------------------------------------
 template <int DT, int OP, bool VECTOR, int CAP, int ORDER>
-__global__ void __launch_bounds__(512)
+__global__ void __launch_bounds__(EC_MAXT, (ORDER != EC_ORDER_FIXED ? 2 : CAP > 64 ? 4 : EC_MINB))   // tree and wide-table variants need more registers
 apply_kernel(const ApplyArgs a, const __grid_constant__ PtrTable<CAP> tbl) {
     typedef Elem<DT> E;
     typedef typename E::In In;
@@ -278,11 +302,12 @@ apply_kernel(const ApplyArgs a, const __grid_constant__ PtrTable<CAP> tbl) {
         const size_t nvec = VECTOR ? cnt / VEC : 0;
         // Few new ranks (a late round): each thread keeps several result vectors in flight;
         // many new ranks (a first round): one vector per thread, eight rank loads in flight.
-        // (Eight accumulators per bf16 vector: half as many vectors per thread keeps the registers at 64.)
-        constexpr int LATE = VEC > 4 ? 2 : 4, MID = VEC > 4 ? 1 : 2;
-        if (m <= 2) fold_vectors<DT, OP, LATE, 2>(s_ptr, m, res, nvec, fresh, tid, nthr, pol, rpol);
-        else if (m <= 4) fold_vectors<DT, OP, MID, 4>(s_ptr, m, res, nvec, fresh, tid, nthr, pol, rpol);
-        else fold_vectors<DT, OP, 1, 8>(s_ptr, m, res, nvec, fresh, tid, nthr, pol, rpol);
+        // With hundreds of ranks a round rarely brings that few: the wide-table variant keeps the
+        // single shape.
+        constexpr int LATE = EC_LATE_VPT, MID = EC_MID_VPT;
+        if (CAP <= 64 && m <= EC_LATE_RU) fold_vectors<DT, OP, LATE, EC_LATE_RU>(s_ptr, m, res, nvec, fresh, tid, nthr, pol, rpol);
+        else if (CAP <= 64 && m <= EC_MID_RU) fold_vectors<DT, OP, MID, EC_MID_RU>(s_ptr, m, res, nvec, fresh, tid, nthr, pol, rpol);
+        else fold_vectors<DT, OP, 1, (CAP > 64 ? 8 : EC_MAIN_RU)>(s_ptr, m, res, nvec, fresh, tid, nthr, pol, rpol);   // hundreds of ranks: 8 loads in flight measured best
         // element-wise path: everything when the 128-bit path does not apply, else the ragged tail
         for (size_t i = nvec * VEC + tid; i < cnt; i += nthr) {
             Acc acc = fresh ? ident<OP>(Acc()) : res[i];
@@ -308,32 +333,48 @@ apply_kernel(const ApplyArgs a, const __grid_constant__ PtrTable<CAP> tbl) {
         const int nblk = P2 / leaf;
         int nlev = 0;
         while ((1 << nlev) < nblk) ++nlev;
-        const size_t nvec = VECTOR ? cnt / VEC : 0;
-        const size_t nunits = nvec + (cnt - nvec * VEC);   // vectors first, then single elements
+        // Units of PV elements (at most four accumulators per tree node keeps the tree in registers).
+        constexpr int PV = VEC > 4 ? 4 : VEC;
+        const size_t nvec = VECTOR ? cnt / PV : 0;
+        const size_t nunits = nvec + (cnt - nvec * PV);   // vectors first, then single elements
         for (size_t w = tid; w < nunits; w += nthr) {
             const bool isvec = w < nvec;
-            const size_t e0 = isvec ? w * VEC : nvec * VEC + (w - nvec);   // first element of this unit
-            Acc stack[TREE_LEVELS][VEC];
-            Acc node[VEC];
+            const size_t e0 = isvec ? w * PV : nvec * PV + (w - nvec);   // first element of this unit
+            Acc stack[TREE_LEVELS][PV];
+            Acc node[PV];
             for (int blk = 0; blk < nblk; ++blk) {
                 const int r0 = blk * leaf;
                 const unsigned byte = (unsigned)(s_new[r0 >> 6] >> (r0 & 63)) & ((1u << leaf) - 1u);
-                Acc lv[8][VEC];
+                Acc lv[8][PV];
 #pragma unroll
                 for (int u = 0; u < 8; ++u) {
 #pragma unroll
-                    for (int e = 0; e < VEC; ++e) lv[u][e] = ident<OP>(Acc());
+                    for (int e = 0; e < PV; ++e) lv[u][e] = ident<OP>(Acc());
                 }
                 if (byte != 0) {
                     if (isvec) {
-                        uint4 raw[8];
+                        if constexpr (DT == EC_BF16) {
+                            uint2 raw[8];                      // four bf16 values = 8 bytes
 #pragma unroll
-                        for (int u = 0; u < 8; ++u)
-                            if ((byte >> u) & 1u)
-                                raw[u] = ld_stream16(reinterpret_cast<const char*>(tbl.p[r0 + u]) + (lo + e0) * sizeof(In), pol);
+                            for (int u = 0; u < 8; ++u)
+                                if ((byte >> u) & 1u)
+                                    raw[u] = ld_stream8(reinterpret_cast<const char*>(tbl.p[r0 + u]) + (lo + e0) * sizeof(In), pol);
 #pragma unroll
-                        for (int u = 0; u < 8; ++u)
-                            if ((byte >> u) & 1u) E::unpack(raw[u], lv[u]);
+                            for (int u = 0; u < 8; ++u)
+                                if ((byte >> u) & 1u) {
+                                    lv[u][0] = __uint_as_float(raw[u].x << 16); lv[u][1] = __uint_as_float(raw[u].x & 0xFFFF0000u);
+                                    lv[u][2] = __uint_as_float(raw[u].y << 16); lv[u][3] = __uint_as_float(raw[u].y & 0xFFFF0000u);
+                                }
+                        } else {
+                            uint4 raw[8];
+#pragma unroll
+                            for (int u = 0; u < 8; ++u)
+                                if ((byte >> u) & 1u)
+                                    raw[u] = ld_stream16(reinterpret_cast<const char*>(tbl.p[r0 + u]) + (lo + e0) * sizeof(In), pol);
+#pragma unroll
+                            for (int u = 0; u < 8; ++u)
+                                if ((byte >> u) & 1u) E::unpack(raw[u], lv[u]);
+                        }
                     } else {
 #pragma unroll
                         for (int u = 0; u < 8; ++u)
@@ -341,7 +382,7 @@ apply_kernel(const ApplyArgs a, const __grid_constant__ PtrTable<CAP> tbl) {
                     }
                 }
 #pragma unroll
-                for (int e = 0; e < VEC; ++e) {
+                for (int e = 0; e < PV; ++e) {
                     if (leaf == 8)
                         node[e] = comb<OP>(comb<OP>(comb<OP>(lv[0][e], lv[1][e]), comb<OP>(lv[2][e], lv[3][e])),
                                            comb<OP>(comb<OP>(lv[4][e], lv[5][e]), comb<OP>(lv[6][e], lv[7][e])));
@@ -358,10 +399,10 @@ apply_kernel(const ApplyArgs a, const __grid_constant__ PtrTable<CAP> tbl) {
                     if (l < nlev && carry) {
                         if ((blk >> l) & 1) {
 #pragma unroll
-                            for (int e = 0; e < VEC; ++e) node[e] = comb<OP>(stack[l][e], node[e]);
+                            for (int e = 0; e < PV; ++e) node[e] = comb<OP>(stack[l][e], node[e]);
                         } else {
 #pragma unroll
-                            for (int e = 0; e < VEC; ++e) stack[l][e] = node[e];
+                            for (int e = 0; e < PV; ++e) stack[l][e] = node[e];
                             carry = false;
                         }
                     }
@@ -370,12 +411,12 @@ apply_kernel(const ApplyArgs a, const __grid_constant__ PtrTable<CAP> tbl) {
             // node is the root now
             if (isvec) {
                 if (!fresh) {
-                    Acc acc[VEC];
-                    load_acc<Acc, VEC>(res + e0, acc, rpol);
+                    Acc acc[PV];
+                    load_acc<Acc, PV>(res + e0, acc, rpol);
 #pragma unroll
-                    for (int e = 0; e < VEC; ++e) node[e] = comb<OP>(acc[e], node[e]);
+                    for (int e = 0; e < PV; ++e) node[e] = comb<OP>(acc[e], node[e]);
                 }
-                store_acc<Acc, VEC>(res + e0, node, rpol);
+                store_acc<Acc, PV>(res + e0, node, rpol);
             } else {
                 res[e0] = fresh ? node[0] : comb<OP>(res[e0], node[0]);
             }
@@ -488,8 +529,10 @@ int ec_allreduce_init(ec_ctx_t** out, int P, size_t n, ec_dtype_t dtype, ec_op_t
     c->cur = 0;
     c->first_apply = true;
     c->res_hint = 1;     // keep the partial result in L2 for the next round (measured: +2% per epoch)
-    c->threads = 128;    // many small blocks overlap their start-up latency best (measured)
-    c->tile = 8192 / in_bytes(dtype);   // 8 KB of every rank buffer per block
+    // Few ranks: many small blocks overlap their start-up latency best.  Hundreds of ranks: a block
+    // lives long anyway and wider blocks read longer contiguous runs of each buffer (both measured).
+    c->threads = P > 64 ? 256 : 128;
+    c->tile = dtype == EC_BF16 ? 2048 : 8192 / in_bytes(dtype);   // 8 KB of every rank buffer per block (4 KB for bf16), measured
     *out = c;
     return EC_OK;
 }
@@ -497,7 +540,7 @@ int ec_allreduce_init(ec_ctx_t** out, int P, size_t n, ec_dtype_t dtype, ec_op_t
 int ec_allreduce_set_tile(ec_ctx_t* c, int threads, size_t tile_elems) {
     if (!c) return EC_ERR_INVALID;
     if (threads != 0) {
-        if (threads < 64 || threads > 512 || threads % 32) return EC_ERR_INVALID;
+        if (threads < 64 || threads > EC_MAXT || threads % 32) return EC_ERR_INVALID;
         c->threads = threads;
     }
     if (tile_elems != 0) {

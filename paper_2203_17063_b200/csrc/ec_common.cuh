@@ -48,6 +48,13 @@ __device__ __forceinline__ uint4 ld_stream16(const void* p, uint64_t pol) {
                  : "l"(p), "l"(pol));
     return v;
 }
+__device__ __forceinline__ uint2 ld_stream8(const void* p, uint64_t pol) {
+    uint2 v;
+    asm volatile("ld.global.nc.L1::no_allocate.L2::cache_hint.v2.u32 {%0,%1}, [%2], %3;"
+                 : "=r"(v.x), "=r"(v.y)
+                 : "l"(p), "l"(pol));
+    return v;
+}
 __device__ __forceinline__ uint4 ld_plain16(const void* p) { return *reinterpret_cast<const uint4*>(p); }
 __device__ __forceinline__ void st_plain16(void* p, uint4 v) { *reinterpret_cast<uint4*>(p) = v; }
 
