@@ -505,11 +505,20 @@ def extras(args, dev, stream, peak):
                                           "bytes": gbytes, "note": "109 MB working set: L2-resident when repeated"}
     del db, d_out
 
-    # config 5: K-means iterations per second
+    out["config5_kmeans_N2^22_D32_K64_P64"] = kmeans_case(dev, stream, reps=5)
+    return out
+
+
+def kmeans_case(dev, stream, reps=5, iters=20, profile_only=False):
+    """Config 5: N = 2^22 points, D = 32, K = 64, P = 64 ranks, 20 Lloyd iterations with seeded masks."""
+    import torch
+    from paper_2203_17063_b200 import binding as ec
+    from paper_2203_17063_b200 import inputs
+    st = stream.cuda_stream
     N, D, K, P = 1 << 22, 32, 64, 64
     pts, comp, _ = inputs.kmeans_mixture(1005, N, D, K)
     init = inputs.kmeans_first_of_component(pts, comp, K)
-    masks = [torch.from_numpy(m.view(np.int64)).to(dev) for m in inputs.kmeans_masks(2005, 20, P, K, 0.75)]
+    masks = [torch.from_numpy(m.view(np.int64)).to(dev) for m in inputs.kmeans_masks(2005, iters, P, K, 0.75)]
     d_pts = torch.from_numpy(pts).to(dev)
     d_init = torch.from_numpy(init).to(dev)
     km = ec.KMeans(d_pts, K, P, d_init)
@@ -517,15 +526,18 @@ def extras(args, dev, stream, peak):
         for t in range(3):
             km.iterate_raw(masks[t].data_ptr(), st)
         runs = []
-        for rep in range(5):
+        for rep in range(reps):
             km.set_centroids(d_init, stream)
             a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             a.record(stream)
-            for t in range(20):
+            for t in range(iters):
                 km.iterate_raw(masks[t].data_ptr(), st)
             b.record(stream)
             torch.cuda.synchronize()
             runs.append(a.elapsed_time(b))
+        if profile_only:
+            km.destroy()
+            return {"ms_per_iteration": statistics.fmean(runs) / iters}
         lab = torch.empty(N, dtype=torch.int32, device=dev)
         ms_assign = time_calls(stream, lambda: km.assign(d_init, lab, stream), 10)
         part = torch.empty(P, K, D + 4, device=dev)
@@ -533,14 +545,14 @@ def extras(args, dev, stream, peak):
     m, ci = mean_ci(runs)
     sm_clock_ghz = 1.965
     alu_peak_lane_ops = 148 * 128 * sm_clock_ghz * 1e9
-    out["config5_kmeans_N2^22_D32_K64_P64"] = {
-        "iterations_per_s": round(20 / (m * 1e-3), 1), "ms_per_20_iterations": round(m, 3), "ci95": round(ci, 3),
+    res = {
+        "iterations_per_s": round(iters / (m * 1e-3), 1), "ms_per_20_iterations": round(m, 3), "ci95": round(ci, 3),
         "assign_ms": round(statistics.fmean(ms_assign), 4), "partials_ms": round(statistics.fmean(ms_part), 4),
         "assign_frac_of_fp32_alu_bound": round((2.0 * N * K * D / alu_peak_lane_ops) / (statistics.fmean(ms_assign) * 1e-3), 4),
         "note": "assign bound = 2*N*K*D lane-instructions (sub + fma) at 148 SMs x 128 lanes x 1.965 GHz",
     }
     km.destroy()
-    return out
+    return res
 
 
 # --------------------------------------------------------------------------------------------
@@ -590,6 +602,8 @@ def main():
     ap.add_argument("--profile-only", action="store_true", help="warm-up and timed steps only (for ncu captures)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-extras", action="store_true", help="headline workload only")
+    ap.add_argument("--workload", default="headline", choices=["headline", "kmeans"],
+                    help="kmeans: time only the K-means driver (config 5) and print its own JSON line")
     ap.add_argument("--cpu-seconds", type=float, default=15.0, help="time budget of the CPU baseline leg")
     ap.add_argument("--threads", type=int, default=0, help="expert: threads per block of the apply kernel")
     ap.add_argument("--tile", type=int, default=0, help="expert: elements per block of the apply kernel")
@@ -604,6 +618,13 @@ def main():
         return
     if world != args.gpus and world == 1 and args.gpus > 1:
         raise SystemExit("launch with torchrun for --gpus > 1")
+    if args.workload == "kmeans":
+        import torch
+        torch.cuda.set_device(local_rank)
+        dev = torch.device("cuda", local_rank)
+        print(json.dumps({"workload": "kmeans", **kmeans_case(dev, torch.cuda.Stream(device=dev), reps=max(1, min(args.steps, 5)),
+                                                               profile_only=args.profile_only)}))
+        return
     run_ours(args, rank, world, local_rank)
 
 

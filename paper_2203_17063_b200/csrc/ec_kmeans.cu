@@ -228,6 +228,227 @@ __global__ void update_kernel(const float* __restrict__ reduced, int D, int K, f
     if (pts > 0.0f) centroids[i] = __fdiv_rn(reduced[(size_t)k * (D + 4) + d], pts);
 }
 
+// ---------------------------------------------------------------------------------------------
+// fused assignment + partial sums (the path ec_kmeans_iterate takes)
+// ---------------------------------------------------------------------------------------------
+// Candidate search: argmin_k |x-c_k|^2 = argmin_k v_k with v_k = |c_k|^2 - 2 x.c_k, one FMA per
+// (point, centroid, coordinate) instead of a subtract and an FMA.  v_k cancels badly, so it only
+// *proposes*: the smallest and second smallest v are tracked, and whenever they are closer than a
+// bound on the rounding error of v (tau) the point is decided again by the exact form
+// sum_d (x-c)^2 over all centroids.  A point that is not re-decided has a winner that leads by more
+// than the error, hence is the winner of the exact form too.  Exact ties always re-decide, so the
+// lowest index wins them.  Two points per thread share each centroid value read from shared memory.
+//
+// Partial sums: the block's points pass through shared memory once more, transposed, and each warp
+// adds its 32 points one after the other into its own [K][D] slab with lane = coordinate: plain
+// read-add-write in a fixed order.  Block (r, c) covers the c-th of C runs of rank r's points and
+// writes one [K][D+4] row block of scratch; the rows of a rank are folded in order afterwards.
+constexpr int FU_THREADS = 256;
+constexpr int FU_PPT = 2;                       // points per thread
+constexpr int FU_TILE = FU_THREADS * FU_PPT;    // points per tile
+constexpr int FU_WARPS = FU_THREADS / 32;
+
+__host__ __device__ inline size_t fused_smem_floats(int D, int K, bool partials) {
+    size_t f = (size_t)K * D + (size_t)((K + 3) & ~3);                       // -2c and |c|^2
+    if (partials) f += (size_t)FU_THREADS * (D + 1) + FU_THREADS             // transposed points, labels
+                       + (size_t)FU_WARPS * K * D + (size_t)FU_WARPS * K;    // slabs and counts
+    return f;
+}
+
+template <int D>
+__device__ __forceinline__ void exact_argmin(const float (&x)[D], const float* s_c2, int K, int& kb) {
+    float best = __int_as_float(0x7f800000);
+    int bi = 0;
+    for (int k = 0; k < K; ++k) {
+        const float4* c = reinterpret_cast<const float4*>(s_c2 + (size_t)k * D);
+        float d0 = 0.0f;
+#pragma unroll
+        for (int q = 0; q < D / 4; ++q) {
+            const float4 a = c[q];                      // -2c: c = -0.5 * a exactly
+            float t;
+            t = x[4 * q] - (-0.5f * a.x); d0 = fmaf(t, t, d0);
+            t = x[4 * q + 1] - (-0.5f * a.y); d0 = fmaf(t, t, d0);
+            t = x[4 * q + 2] - (-0.5f * a.z); d0 = fmaf(t, t, d0);
+            t = x[4 * q + 3] - (-0.5f * a.w); d0 = fmaf(t, t, d0);
+        }
+        if (d0 < best) { best = d0; bi = k; }           // strict <: the lowest index wins a tie
+    }
+    kb = bi;
+}
+
+#define EC_TRACK(v, k, b1, b2, kb)                 \
+    do {                                           \
+        const bool lt__ = (v) < (b1);              \
+        (b2) = fminf((b2), lt__ ? (b1) : (v));     \
+        (kb) = lt__ ? (k) : (kb);                  \
+        (b1) = lt__ ? (v) : (b1);                  \
+    } while (0)
+
+template <int D, bool PARTIALS>
+__global__ void __launch_bounds__(FU_THREADS, 2)
+fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const float* __restrict__ centroids, int K,
+             int32_t* __restrict__ labels, float* __restrict__ scratch, float tau_scale) {
+    extern __shared__ __align__(16) float smem[];
+    float* s_c2 = smem;                                        // [K][D]   -2 c
+    float* s_cn = s_c2 + (size_t)K * D;                        // [K]      |c|^2
+    float* s_x = s_cn + ((K + 3) & ~3);                        // [256][D+1]
+    int* s_lab = reinterpret_cast<int*>(s_x + (size_t)FU_THREADS * (D + 1));
+    float* s_acc = reinterpret_cast<float*>(s_lab + FU_THREADS);          // [8][K][D]
+    int* s_cnt = reinterpret_cast<int*>(s_acc + (size_t)FU_WARPS * K * D);  // [8][K]
+    const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
+    const size_t KD = (size_t)K * D;
+
+    for (int i = tid; i < (int)KD; i += FU_THREADS) s_c2[i] = -2.0f * centroids[i];
+    for (int k = tid; k < K; k += FU_THREADS) {
+        float s = 0.0f;
+        for (int d = 0; d < D; ++d) s = fmaf(centroids[(size_t)k * D + d], centroids[(size_t)k * D + d], s);
+        s_cn[k] = s;
+    }
+    if (PARTIALS) {
+        for (size_t i = tid; i < (size_t)FU_WARPS * KD; i += FU_THREADS) s_acc[i] = 0.0f;
+        for (int i = tid; i < FU_WARPS * K; i += FU_THREADS) s_cnt[i] = 0;
+    }
+    __syncthreads();
+    float cmax = 0.0f;
+    for (int k = 0; k < K; ++k) cmax = fmaxf(cmax, s_cn[k]);
+
+    const int r = blockIdx.x / C, c = blockIdx.x - r * C;
+    const size_t j0 = (size_t)r * N / P, j1 = (size_t)(r + 1) * N / P;
+    const size_t len = j1 - j0;
+    const size_t b0 = j0 + len * c / C, b1 = j0 + len * (c + 1) / C;
+
+    for (size_t base = b0; base < b1; base += FU_TILE) {
+        float x[FU_PPT][D];
+        bool live[FU_PPT];
+        float xn[FU_PPT];
+#pragma unroll
+        for (int p = 0; p < FU_PPT; ++p) {
+            const size_t j = base + (size_t)p * FU_THREADS + tid;
+            live[p] = j < b1;
+            xn[p] = 0.0f;
+            if (live[p]) {
+                const float4* row = reinterpret_cast<const float4*>(points + j * D);
+#pragma unroll
+                for (int q = 0; q < D / 4; ++q) {
+                    const float4 v = __ldg(row + q);
+                    x[p][4 * q] = v.x; x[p][4 * q + 1] = v.y; x[p][4 * q + 2] = v.z; x[p][4 * q + 3] = v.w;
+                }
+#pragma unroll
+                for (int d = 0; d < D; ++d) xn[p] = fmaf(x[p][d], x[p][d], xn[p]);
+            } else {
+#pragma unroll
+                for (int d = 0; d < D; ++d) x[p][d] = 0.0f;
+            }
+        }
+        float m1[FU_PPT], m2[FU_PPT];
+        int kb[FU_PPT];
+#pragma unroll
+        for (int p = 0; p < FU_PPT; ++p) { m1[p] = __int_as_float(0x7f800000); m2[p] = m1[p]; kb[p] = 0; }
+        int k = 0;
+        for (; k + 4 <= K; k += 4) {                 // four centroids x two points: eight independent chains
+            float v[FU_PPT][4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const float cn = s_cn[k + u];
+#pragma unroll
+                for (int p = 0; p < FU_PPT; ++p) v[p][u] = cn;
+            }
+#pragma unroll
+            for (int q = 0; q < D / 4; ++q) {
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const float4 a = reinterpret_cast<const float4*>(s_c2 + (size_t)(k + u) * D)[q];
+#pragma unroll
+                    for (int p = 0; p < FU_PPT; ++p) {
+                        v[p][u] = fmaf(x[p][4 * q], a.x, v[p][u]);
+                        v[p][u] = fmaf(x[p][4 * q + 1], a.y, v[p][u]);
+                        v[p][u] = fmaf(x[p][4 * q + 2], a.z, v[p][u]);
+                        v[p][u] = fmaf(x[p][4 * q + 3], a.w, v[p][u]);
+                    }
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+#pragma unroll
+                for (int p = 0; p < FU_PPT; ++p) EC_TRACK(v[p][u], k + u, m1[p], m2[p], kb[p]);
+            }
+        }
+        for (; k < K; ++k) {
+            const float cn = s_cn[k];
+#pragma unroll
+            for (int p = 0; p < FU_PPT; ++p) {
+                float v = cn;
+#pragma unroll
+                for (int d = 0; d < D; ++d) v = fmaf(x[p][d], s_c2[(size_t)k * D + d], v);
+                EC_TRACK(v, k, m1[p], m2[p], kb[p]);
+            }
+        }
+#pragma unroll
+        for (int p = 0; p < FU_PPT; ++p) {
+            // |error of v| <= (D+3) u (|x| + |c|)^2 <= (D+3) u 2 (|x|^2 + |c|max^2); tau covers both candidates twice over
+            const float tau = tau_scale * (xn[p] + cmax);
+            if (live[p] && !(m2[p] - m1[p] > tau)) exact_argmin<D>(x[p], s_c2, K, kb[p]);
+            if (live[p]) labels[base + (size_t)p * FU_THREADS + tid] = kb[p];
+        }
+        if (PARTIALS) {
+#pragma unroll
+            for (int p = 0; p < FU_PPT; ++p) {
+                __syncthreads();                                   // the previous half has been consumed
+                s_lab[tid] = live[p] ? kb[p] : -1;
+#pragma unroll
+                for (int d = 0; d < D; ++d) s_x[(size_t)tid * (D + 1) + d] = x[p][d];
+                __syncthreads();
+                float* acc = s_acc + (size_t)w * KD;
+                int* cnt = s_cnt + w * K;
+                for (int jj = 0; jj < 32; jj += 4) {
+                    int lab[4];
+                    float xv[4][(D + 31) / 32];
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const int pt = w * 32 + jj + u;
+                        lab[u] = s_lab[pt];
+#pragma unroll
+                        for (int q = 0; q < (D + 31) / 32; ++q) {
+                            const int d = lane + 32 * q;
+                            xv[u][q] = d < D ? s_x[(size_t)pt * (D + 1) + d] : 0.0f;
+                        }
+                    }
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        if (lab[u] >= 0) {
+#pragma unroll
+                            for (int q = 0; q < (D + 31) / 32; ++q) {
+                                const int d = lane + 32 * q;
+                                if (d < D) acc[(size_t)lab[u] * D + d] = __fadd_rn(acc[(size_t)lab[u] * D + d], xv[u][q]);
+                            }
+                            if (lane == 0) cnt[lab[u]] += 1;
+                        }
+                    }
+                }
+            }
+        }
+    }
+    if (PARTIALS) {
+        __syncthreads();
+        const int stride = D + 4;
+        float* dst = scratch + ((size_t)r * C + c) * (size_t)K * stride;
+        for (size_t i = tid; i < (size_t)K * stride; i += FU_THREADS) {
+            const int kk = (int)(i / stride), d = (int)(i - (size_t)kk * stride);
+            float val = 0.0f;
+            if (d < D) {
+                val = s_acc[(size_t)kk * D + d];
+                for (int ww = 1; ww < FU_WARPS; ++ww) val = __fadd_rn(val, s_acc[(size_t)ww * KD + (size_t)kk * D + d]);
+            } else if (d == D) {
+                int n = 0;
+                for (int ww = 0; ww < FU_WARPS; ++ww) n += s_cnt[ww * K + kk];
+                val = (float)n;
+            }
+            dst[i] = val;
+        }
+    }
+}
+#undef EC_TRACK
+
 int sm_count_km() {
     int dev = 0, n = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return 148;
@@ -256,6 +477,8 @@ struct ec_kmeans {
     const void* bufs[EC_MAX_RANKS];
     int sms, C, warps, kc;
     size_t assign_smem, part_smem;
+    int Cf;                // runs per rank of the fused kernel; 0 = shape not covered by it
+    size_t fused_smem, fused_assign_smem;
 };
 
 using namespace ec;
@@ -265,7 +488,14 @@ namespace {
 struct KmLayout {
     size_t off_centroids, off_labels, off_partials, off_scratch, off_reduced, off_contrib, off_ar, total;
     int C, warps;
+    int Cf;   // runs per rank for the fused assignment+partials kernel, 0 if the shape is not covered
 };
+
+// Shapes the fused kernel is instantiated for and whose shared memory fits.
+bool fused_capable(int D, int K) {
+    if (D != 8 && D != 16 && D != 32 && D != 64) return false;
+    return fused_smem_floats(D, K, true) * 4 <= SMEM_BUDGET;
+}
 
 // Blocks per rank (C) and warps per block for the partials kernel, from the shape alone.
 bool km_plan(size_t N, int D, int K, int P, int sms, KmLayout* L) {
@@ -281,12 +511,18 @@ bool km_plan(size_t N, int D, int K, int P, int sms, KmLayout* L) {
     while (C > 1 && shard / (size_t)C < 256) --C;            // keep runs long enough to be worth a block
     L->C = C;
     L->warps = warps;
+    // fused kernel: runs of four tiles (2048 points); thousands of short blocks fill the SMs evenly
+    L->Cf = 0;
+    if (fused_capable(D, K)) {
+        size_t cf = shard / (4 * (size_t)FU_TILE);
+        L->Cf = (int)(cf < 1 ? 1 : cf > 64 ? 64 : cf);
+    }
     const size_t stride = (size_t)D + 4;
     size_t off = 0;
     L->off_centroids = off; off = align_up(off + KD * 4, 256);
     L->off_labels = off; off = align_up(off + N * 4, 256);
     L->off_partials = off; off = align_up(off + (size_t)P * K * stride * 4, 256);
-    L->off_scratch = off; off = align_up(off + (size_t)P * C * K * stride * 4, 256);
+    L->off_scratch = off; off = align_up(off + (size_t)P * (C > L->Cf ? C : L->Cf) * K * stride * 4, 256);
     L->off_reduced = off; off = align_up(off + (size_t)K * stride * 4, 256);
     L->off_contrib = off; off = align_up(off + (size_t)K * 4, 256);
     L->off_ar = off; off = align_up(off + ec_allreduce_workspace_bytes(P, (size_t)K * stride, stride), 256);
@@ -299,7 +535,44 @@ bool km_bad_shape(size_t N, int D, int K, int P) {
            (size_t)P > N;
 }
 
+float km_tau_scale(int D) { return 8.0f * (float)(D + 3) * 5.9604644775390625e-08f; }   // 8 (D+3) 2^-24
+
+template <int D>
+int km_fused_launch(ec_kmeans* km, bool partials, const float* centroids, int32_t* labels, cudaStream_t st) {
+    if (partials) {
+        fused_kernel<D, true><<<(unsigned)(km->P * km->Cf), FU_THREADS, km->fused_smem, st>>>(
+            km->points, km->N, km->P, km->Cf, centroids, km->K, labels, km->Cf == 1 ? km->partials : km->scratch,
+            km_tau_scale(D));
+    } else {
+        size_t runs = (km->N + 4 * FU_TILE - 1) / (4 * FU_TILE);
+        if (runs > 0x7fffffffull) return EC_ERR_CAPACITY;
+        fused_kernel<D, false><<<(unsigned)runs, FU_THREADS, km->fused_assign_smem, st>>>(
+            km->points, km->N, 1, (int)runs, centroids, km->K, labels, nullptr, km_tau_scale(D));
+    }
+    EC_CUDA(cudaGetLastError());
+    return EC_OK;
+}
+
+int km_fused(ec_kmeans* km, bool partials, const float* centroids, int32_t* labels, cudaStream_t st) {
+    switch (km->D) {
+        case 8: return km_fused_launch<8>(km, partials, centroids, labels, st);
+        case 16: return km_fused_launch<16>(km, partials, centroids, labels, st);
+        case 32: return km_fused_launch<32>(km, partials, centroids, labels, st);
+        case 64: return km_fused_launch<64>(km, partials, centroids, labels, st);
+    }
+    return EC_ERR_UNSUPPORTED;
+}
+
+template <int D>
+cudaError_t km_fused_attr() {
+    cudaError_t e = cudaFuncSetAttribute(fused_kernel<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BUDGET);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(fused_kernel<D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BUDGET);
+    return e;
+}
+
 int km_assign(ec_kmeans* km, const float* centroids, int32_t* labels, cudaStream_t st) {
+    if (km->Cf > 0) return km_fused(km, false, centroids, labels, st);
     const size_t tiles = (km->N + AS_THREADS - 1) / AS_THREADS;
     const size_t cap = (size_t)km->sms * 8;
     const unsigned grid = (unsigned)(tiles < cap ? tiles : cap);
@@ -376,6 +649,9 @@ int ec_kmeans_init(ec_kmeans_t** out, const float* points, size_t N, int D, int 
     km->contrib = reinterpret_cast<uint32_t*>(base + L.off_contrib);
     km->ar_ws = base + L.off_ar;
     km->sms = sms; km->C = L.C; km->warps = L.warps;
+    km->Cf = L.Cf;
+    km->fused_smem = fused_smem_floats(D, K, true) * 4;
+    km->fused_assign_smem = fused_smem_floats(D, K, false) * 4;
     // centroid chunk for the assignment: as many as fit in 64 KB, all of them if possible
     int kc = (int)((64 * 1024) / ((size_t)D * 4));
     if (kc > K) kc = K;
@@ -399,6 +675,8 @@ int ec_kmeans_init(ec_kmeans_t** out, const float* points, size_t N, int D, int 
     }
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(partials_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BUDGET);
+    if (e == cudaSuccess && km->Cf > 0)
+        e = D == 8 ? km_fused_attr<8>() : D == 16 ? km_fused_attr<16>() : D == 32 ? km_fused_attr<32>() : km_fused_attr<64>();
     if (e == cudaSuccess) e = cudaMemcpyAsync(km->centroids, init_centroids, (size_t)K * D * 4, cudaMemcpyDeviceToDevice, 0);
     if (e == cudaSuccess) e = cudaStreamSynchronize(0);
     if (e != cudaSuccess) rc = cuda_fail(e);
@@ -427,10 +705,23 @@ int ec_kmeans_partials(ec_kmeans_t* km, const int32_t* labels, float* partials, 
 
 int ec_kmeans_iterate(ec_kmeans_t* km, const uint64_t* arrival_mask, ec_stream_t stream) {
     if (!km) return EC_ERR_INVALID;
-    int rc = km_assign(km, km->centroids, km->labels, stream);
-    if (rc != EC_OK) return rc;
-    rc = km_partials(km, km->labels, km->partials, stream);
-    if (rc != EC_OK) return rc;
+    int rc;
+    if (km->Cf > 0) {
+        // assignment and per-block partial sums in one pass over the points, then the rows of a rank in order
+        rc = km_fused(km, true, km->centroids, km->labels, stream);
+        if (rc != EC_OK) return rc;
+        if (km->Cf > 1) {
+            const size_t row = (size_t)km->K * (km->D + 4), total = row * km->P;
+            partials_fold_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(km->scratch, km->Cf, row, total,
+                                                                                      km->partials);
+            EC_CUDA(cudaGetLastError());
+        }
+    } else {
+        rc = km_assign(km, km->centroids, km->labels, stream);
+        if (rc != EC_OK) return rc;
+        rc = km_partials(km, km->labels, km->partials, stream);
+        if (rc != EC_OK) return rc;
+    }
     rc = ec_allreduce_reset(km->ar, stream);
     if (rc != EC_OK) return rc;
     const size_t stride = (size_t)km->D + 4;
