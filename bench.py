@@ -190,16 +190,9 @@ def run_ours(args, rank, world, local_rank):
 
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist_mod
-        dist = dist_mod
-        dist.init_process_group("nccl", device_id=dev)
-
-    def barrier():
-        if dist is not None:
-            dist.barrier()
-        torch.cuda.synchronize()
+    from paper_2203_17063_b200.replicas import Replicas
+    rep = Replicas(backend="nccl", device=dev)     # N independent replicas; shared: barrier, max time, summed work
+    barrier = rep.barrier
 
     peak, peak_kind = measured_peaks()
     cfg, h_bufs, h_masks = make_headline_host()
@@ -293,14 +286,7 @@ def run_ours(args, rank, world, local_rank):
     e2e_ms = e0.elapsed_time(e1) / e2e_steps
     clock_info = clocks.stop(t_host0, t_host1)
 
-    # max over ranks
-    def max_over_ranks(x):
-        if dist is None:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
-
+    max_over_ranks = rep.max
     total_ms_max = max_over_ranks(total_ms)
     e2e_ms_max = max_over_ranks(e2e_ms)
     value = world * step_bytes * K / (total_ms_max * 1e-3) / 1e9
@@ -360,9 +346,7 @@ def run_ours(args, rank, world, local_rank):
             del h_bufs, pin_bufs, d_bufs
             ar.destroy()
             line["extras"] = extras(args, dev, stream, peak)
-    if dist is not None:
-        dist.barrier()
-        dist.destroy_process_group()
+    rep.close()
     if rank == 0:
         print(json.dumps(line))
 

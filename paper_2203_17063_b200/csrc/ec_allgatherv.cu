@@ -3,10 +3,12 @@
 //
 // Every rank owns a fixed slot (the placement rule of the ring's Allgather stage, Sec. IV-A, and
 // of the AlltoAll's one-target-per-writer, Sec. IV-B), so the displacements come from the counts
-// of all ranks.  Every block recomputes the scan of the (at most 1024) counts in shared memory -
-// 8 KB of reads that stay in L2 - which removes any ordering between blocks.  The flattened output
+// of all ranks.  Every block recomputes the scan of the (at most 1024) counts - a few KB that stay
+// in L2 - with warp shuffles, which removes any ordering between blocks.  The flattened output
 // range is cut into equal chunks; a block finds the first rank of its chunk by binary search in
 // the displacements and walks the ranks that overlap the chunk.
+
+#include <type_traits>
 
 #include "ec_common.cuh"
 
@@ -15,6 +17,7 @@ namespace {
 
 constexpr int GV_THREADS = 256;
 constexpr size_t GV_CHUNK_BYTES = 16384;
+constexpr int GV_BATCH = 4;            // loads in flight per thread before the stores
 
 struct GatherArgs {
     const int64_t* counts;
@@ -26,43 +29,98 @@ struct GatherArgs {
     int P, esize;              // element size in bytes
 };
 
+template <class T>
+__device__ __forceinline__ void copy_elems(T* __restrict__ dst, const T* __restrict__ src, size_t cnt, int tid) {
+    for (size_t i0 = tid; i0 < cnt; i0 += (size_t)GV_THREADS * GV_BATCH) {
+        T v[GV_BATCH];
+#pragma unroll
+        for (int b = 0; b < GV_BATCH; ++b) {
+            const size_t i = i0 + (size_t)b * GV_THREADS;
+            if (i < cnt) v[b] = src[i];
+        }
+#pragma unroll
+        for (int b = 0; b < GV_BATCH; ++b) {
+            const size_t i = i0 + (size_t)b * GV_THREADS;
+            if (i < cnt) dst[i] = v[b];
+        }
+    }
+}
+
+__device__ __forceinline__ void copy_vec16(char* __restrict__ dst, const char* __restrict__ src, size_t nvec, int tid,
+                                           uint64_t pol) {
+    for (size_t v0 = tid; v0 < nvec; v0 += (size_t)GV_THREADS * GV_BATCH) {
+        uint4 r[GV_BATCH];
+#pragma unroll
+        for (int b = 0; b < GV_BATCH; ++b) {
+            const size_t v = v0 + (size_t)b * GV_THREADS;
+            if (v < nvec) r[b] = ld_stream16(src + v * 16, pol);
+        }
+#pragma unroll
+        for (int b = 0; b < GV_BATCH; ++b) {
+            const size_t v = v0 + (size_t)b * GV_THREADS;
+            if (v < nvec) st_plain16(dst + v * 16, r[b]);
+        }
+    }
+}
+
+template <int ES>
+__device__ __forceinline__ void copy_small(char* dst, const char* src, size_t bytes, int tid) {
+    typedef typename std::conditional<ES == 8, uint64_t, typename std::conditional<ES == 4, uint32_t, uint16_t>::type>::type T;
+    copy_elems<T>(reinterpret_cast<T*>(dst), reinterpret_cast<const T*>(src), bytes / ES, tid);
+}
+
 template <int CAP>
 __global__ void __launch_bounds__(GV_THREADS)
 allgatherv_kernel(const GatherArgs a, const __grid_constant__ PtrTable<CAP> tbl) {
-    __shared__ long long s_scan[2][CAP];      // double-buffered inclusive scan
+    constexpr int ITEMS = CAP >= GV_THREADS ? CAP / GV_THREADS : 1;   // consecutive counts per thread
     __shared__ long long s_displs[CAP + 1];
-    __shared__ uint64_t s_arr[CAP / 64];
+    __shared__ long long s_warp[GV_THREADS / 32];
+    __shared__ uint64_t s_arr[(CAP + 63) / 64];
     __shared__ int s_bad;
-    const int tid = threadIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     const int P = a.P;
 
     if (tid == 0) s_bad = 0;
-    __syncthreads();
-    for (int r = tid; r < CAP; r += GV_THREADS) {
-        long long c = 0;
-        if (r < P) {
-            c = a.counts[r];
-            if (c < 0) { s_bad = 1; c = 0; }
-        }
-        s_scan[0][r] = c;
-    }
-    for (int w = tid; w < CAP / 64; w += GV_THREADS) {
+    for (int w = tid; w < (CAP + 63) / 64; w += GV_THREADS) {
         uint64_t word = 0;
         if (w * 64 < P) {
             word = a.arrival ? a.arrival[w] : ~0ull;
-            if (P - w * 64 < 64) word &= (1ull << (P - w * 64)) - 1;
+            if (P - w * 64 < 64) word &= (1ull << (P - w * 64)) - 1;       // bits >= P mean nothing
         }
         s_arr[w] = word;
     }
     __syncthreads();
-    int cur = 0;
-    for (int d = 1; d < CAP; d <<= 1) {          // Hillis-Steele inclusive scan
-        for (int r = tid; r < CAP; r += GV_THREADS)
-            s_scan[cur ^ 1][r] = s_scan[cur][r] + (r >= d ? s_scan[cur][r - d] : 0);
-        cur ^= 1;
-        __syncthreads();
+    // exclusive scan: thread-local prefix, warp shuffle scan of the thread totals, scan of the warp totals
+    long long cnt[ITEMS];
+    long long local = 0;
+    bool neg = false;
+#pragma unroll
+    for (int i = 0; i < ITEMS; ++i) {
+        const int r = tid * ITEMS + i;
+        long long c = (r < P && r < CAP) ? a.counts[r] : 0;
+        if (c < 0) { neg = true; c = 0; }
+        cnt[i] = c;
+        local += c;
     }
-    for (int r = tid; r <= P; r += GV_THREADS) s_displs[r] = r == 0 ? 0 : s_scan[cur][r - 1];
+    if (neg) s_bad = 1;
+    long long incl = local;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const long long y = __shfl_up_sync(0xffffffffu, incl, d);
+        if (lane >= d) incl += y;
+    }
+    if (lane == 31) s_warp[wid] = incl;
+    __syncthreads();
+    long long warp_off = 0;
+    for (int w = 0; w < wid; ++w) warp_off += s_warp[w];
+    long long run = warp_off + incl - local;                               // exclusive prefix of this thread's first item
+#pragma unroll
+    for (int i = 0; i < ITEMS; ++i) {
+        const int r = tid * ITEMS + i;
+        if (r <= P && r < CAP) s_displs[r] = run;
+        run += cnt[i];
+        if (r + 1 == P) s_displs[P] = run;                                 // the total
+    }
     __syncthreads();
     const long long total = s_displs[P];
     const bool bad = s_bad != 0 || (unsigned long long)total > (unsigned long long)a.capacity;
@@ -90,40 +148,28 @@ allgatherv_kernel(const GatherArgs a, const __grid_constant__ PtrTable<CAP> tbl)
             if (b >= e) continue;                                    // empty contribution
             const char* src = reinterpret_cast<const char*>(tbl.p[r]) + (size_t)(b - d0) * es;
             char* dst = a.out + (size_t)b * es;
-            size_t bytes = (size_t)(e - b) * es;
+            const size_t bytes = (size_t)(e - b) * es;
             if (((reinterpret_cast<uintptr_t>(src) ^ reinterpret_cast<uintptr_t>(dst)) & 15u) == 0) {
                 // same phase modulo 16: element-wise head up to the boundary, 128-bit body, element-wise tail
                 size_t head = (16 - (reinterpret_cast<uintptr_t>(dst) & 15u)) & 15u;
                 if (head > bytes) head = bytes;
                 const size_t body = (bytes - head) / 16;
                 const size_t tail0 = head + body * 16;
-                for (size_t o = (size_t)tid * es; o < head; o += (size_t)GV_THREADS * es) {
-                    if (es == 8) *reinterpret_cast<uint64_t*>(dst + o) = *reinterpret_cast<const uint64_t*>(src + o);
-                    else if (es == 4) *reinterpret_cast<uint32_t*>(dst + o) = *reinterpret_cast<const uint32_t*>(src + o);
-                    else *reinterpret_cast<uint16_t*>(dst + o) = *reinterpret_cast<const uint16_t*>(src + o);
+                if (head) {
+                    if (es == 8) copy_small<8>(dst, src, head, tid);
+                    else if (es == 4) copy_small<4>(dst, src, head, tid);
+                    else copy_small<2>(dst, src, head, tid);
                 }
-                for (size_t v = tid; v < body; v += GV_THREADS)
-                    st_plain16(dst + head + v * 16, ld_stream16(src + head + v * 16, pol));
-                for (size_t o = tail0 + (size_t)tid * es; o < bytes; o += (size_t)GV_THREADS * es) {
-                    if (es == 8) *reinterpret_cast<uint64_t*>(dst + o) = *reinterpret_cast<const uint64_t*>(src + o);
-                    else if (es == 4) *reinterpret_cast<uint32_t*>(dst + o) = *reinterpret_cast<const uint32_t*>(src + o);
-                    else *reinterpret_cast<uint16_t*>(dst + o) = *reinterpret_cast<const uint16_t*>(src + o);
+                copy_vec16(dst + head, src + head, body, tid, pol);
+                if (bytes > tail0) {
+                    if (es == 8) copy_small<8>(dst + tail0, src + tail0, bytes - tail0, tid);
+                    else if (es == 4) copy_small<4>(dst + tail0, src + tail0, bytes - tail0, tid);
+                    else copy_small<2>(dst + tail0, src + tail0, bytes - tail0, tid);
                 }
             } else {
-                const size_t cnt = (size_t)(e - b);
-                if (es == 8) {
-                    const uint64_t* s8 = reinterpret_cast<const uint64_t*>(src);
-                    uint64_t* d8 = reinterpret_cast<uint64_t*>(dst);
-                    for (size_t i = tid; i < cnt; i += GV_THREADS) d8[i] = s8[i];
-                } else if (es == 4) {
-                    const uint32_t* s4 = reinterpret_cast<const uint32_t*>(src);
-                    uint32_t* d4 = reinterpret_cast<uint32_t*>(dst);
-                    for (size_t i = tid; i < cnt; i += GV_THREADS) d4[i] = s4[i];
-                } else {
-                    const uint16_t* s2 = reinterpret_cast<const uint16_t*>(src);
-                    uint16_t* d2 = reinterpret_cast<uint16_t*>(dst);
-                    for (size_t i = tid; i < cnt; i += GV_THREADS) d2[i] = s2[i];
-                }
+                if (es == 8) copy_small<8>(dst, src, bytes, tid);
+                else if (es == 4) copy_small<4>(dst, src, bytes, tid);
+                else copy_small<2>(dst, src, bytes, tid);
             }
         }
     }
@@ -140,6 +186,13 @@ int sm_count() {
         cached_dev = dev;
     }
     return cached;
+}
+
+template <int CAP>
+void launch(const GatherArgs& a, const void* const* bufs, unsigned grid, cudaStream_t stream) {
+    PtrTable<CAP> tbl;
+    for (int r = 0; r < CAP; ++r) tbl.p[r] = r < a.P ? bufs[r] : nullptr;
+    allgatherv_kernel<CAP><<<grid, GV_THREADS, 0, stream>>>(a, tbl);
 }
 
 }  // namespace
@@ -162,20 +215,14 @@ extern "C" int ec_allgatherv(const void* const* bufs, const int64_t* counts, int
     GatherArgs a;
     a.counts = counts; a.arrival = arrival_mask; a.displs = displs; a.out = reinterpret_cast<char*>(out);
     a.status = status; a.capacity = out_capacity_elems; a.P = P; a.esize = es;
-    // enough blocks for every chunk the capacity allows, at most four per SM (the blocks loop)
+    // enough blocks for every chunk the capacity allows, at most eight per SM (the blocks loop)
     size_t chunks = (out_capacity_elems * (size_t)es + GV_CHUNK_BYTES - 1) / GV_CHUNK_BYTES;
     if (chunks < 1) chunks = 1;
-    const size_t cap_blocks = (size_t)sm_count() * 4;
+    const size_t cap_blocks = (size_t)sm_count() * 8;
     const unsigned grid = (unsigned)(chunks < cap_blocks ? chunks : cap_blocks);
-    if (P <= 64) {
-        PtrTable<64> tbl;
-        for (int r = 0; r < 64; ++r) tbl.p[r] = r < P ? bufs[r] : nullptr;
-        allgatherv_kernel<64><<<grid, GV_THREADS, 0, stream>>>(a, tbl);
-    } else {
-        PtrTable<EC_MAX_RANKS> tbl;
-        for (int r = 0; r < EC_MAX_RANKS; ++r) tbl.p[r] = r < P ? bufs[r] : nullptr;
-        allgatherv_kernel<EC_MAX_RANKS><<<grid, GV_THREADS, 0, stream>>>(a, tbl);
-    }
+    if (P <= 64) launch<64>(a, bufs, grid, stream);
+    else if (P <= 256) launch<256>(a, bufs, grid, stream);
+    else launch<EC_MAX_RANKS>(a, bufs, grid, stream);
     EC_CUDA(cudaGetLastError());
     return EC_OK;
 }

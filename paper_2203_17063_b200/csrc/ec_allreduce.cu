@@ -528,7 +528,14 @@ int ec_allreduce_init(ec_ctx_t** out, int P, size_t n, ec_dtype_t dtype, ec_op_t
     c->applied[1] = reinterpret_cast<uint64_t*>(reinterpret_cast<char*>(c->ws) + need / 2);
     c->cur = 0;
     c->first_apply = true;
-    c->res_hint = 1;     // keep the partial result in L2 for the next round (measured: +2% per epoch)
+    // A partial result that fits in L2 is kept there for the next round (evict-last: +2 % per epoch
+    // measured on 64 MiB); one that cannot fit is streamed through instead (evict-first).
+    {
+        int dev = 0, l2 = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&l2, cudaDevAttrL2CacheSize, dev) != cudaSuccess)
+            l2 = 0;
+        c->res_hint = (double)n * (double)out_bytes(dtype) <= 0.75 * (double)l2 ? 1 : 2;
+    }
     // Few ranks: many small blocks overlap their start-up latency best.  Hundreds of ranks: a block
     // lives long anyway and wider blocks read longer contiguous runs of each buffer (both measured).
     c->threads = P > 64 ? 256 : 128;
