@@ -219,6 +219,20 @@ int ec_kmeans_set_centroids(ec_kmeans_t* km, const float* centroids, ec_stream_t
 int ec_kmeans_get(ec_kmeans_t* km, float* centroids, int32_t* labels, float* reduced,
                   uint32_t* contrib_count, ec_stream_t stream);
 
+/* Expert knob: which kernel ec_kmeans_iterate / ec_kmeans_assign use.
+ *   0  automatic: the fastest one that covers the shape (default);
+ *   1  fp32 fused kernel: candidate search by one FMA per (point, centroid, coordinate);
+ *   2  tensor-core fused kernel: candidate search as a bf16 GEMM on tcgen05 (D in {16, 32, 64}, K <= 256).
+ * Both decide every point whose two best candidates lie within the error bound of the search again
+ * by the exact form sum_d (x-c)^2 in fp32, so labels do not depend on the choice; speed does.
+ * EC_ERR_UNSUPPORTED if the shape is not covered by the requested kernel. */
+int ec_kmeans_set_path(ec_kmeans_t* km, int path);
+
+/* Copies (device to device, on `stream`) the driver's health word to `device_out`: 0 = fine; nonzero =
+ * a bounded wait on the tensor core gave up at least once and the affected tiles were computed by the
+ * exact form instead (results are still correct). */
+int ec_kmeans_tc_status(ec_kmeans_t* km, uint32_t* device_out, ec_stream_t stream);
+
 int ec_kmeans_destroy(ec_kmeans_t* km);
 
 /* Per-rank partial sums for callers that are not allowed to allocate device

@@ -41,6 +41,8 @@ SYMBOLS = {
     "ec_kmeans_iterate": (_i, [_vp, _vp, _vp]),
     "ec_kmeans_set_centroids": (_i, [_vp, _vp, _vp]),
     "ec_kmeans_get": (_i, [_vp, _vp, _vp, _vp, _vp, _vp]),
+    "ec_kmeans_set_path": (_i, [_vp, _i]),
+    "ec_kmeans_tc_status": (_i, [_vp, _vp, _vp]),
     "ec_kmeans_destroy": (_i, [_vp]),
     "ec_kmeans_partials_static": (_i, [_vp, _vp, _sz, _i, _i, _i, _vp, _vp]),
     "ec_strerror": (C.c_char_p, [_i]),
@@ -189,6 +191,15 @@ class KMeans:
     def get(self, centroids=None, labels=None, reduced=None, contrib_count=None, stream=None) -> None:
         _check(lib().ec_kmeans_get(self._h, _ptr(centroids), _ptr(labels), _ptr(reduced), _ptr(contrib_count),
                                    _stream(stream)), "ec_kmeans_get")
+
+    def set_path(self, path: int) -> None:
+        """0 automatic, 1 fp32 fused kernel, 2 tensor-core fused kernel."""
+        _check(lib().ec_kmeans_set_path(self._h, path), "ec_kmeans_set_path")
+
+    def tc_status(self, stream=None) -> int:
+        out = torch.zeros(1, dtype=torch.int32, device=self.points.device)
+        _check(lib().ec_kmeans_tc_status(self._h, _ptr(out), _stream(stream)), "ec_kmeans_tc_status")
+        return int(out.item())
 
     def destroy(self) -> None:
         if getattr(self, "_h", None):

@@ -449,6 +449,14 @@ fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const flo
 }
 #undef EC_TRACK
 
+}  // namespace
+}  // namespace ec
+
+#include "ec_kmeans_tc.cuh"
+
+namespace ec {
+namespace {
+
 int sm_count_km() {
     int dev = 0, n = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return 148;
@@ -479,6 +487,10 @@ struct ec_kmeans {
     size_t assign_smem, part_smem;
     int Cf;                // runs per rank of the fused kernel; 0 = shape not covered by it
     size_t fused_smem, fused_assign_smem;
+    bool tc_ok;            // the tensor-core candidate search covers this shape
+    int path;              // 0 = automatic, 1 = fp32 fused kernel, 2 = tensor-core fused kernel
+    size_t tc_smem, tc_assign_smem;
+    uint32_t* tc_status;   // device word: nonzero if a wait on the tensor core ever gave up
 };
 
 using namespace ec;
@@ -495,6 +507,13 @@ struct KmLayout {
 bool fused_capable(int D, int K) {
     if (D != 8 && D != 16 && D != 32 && D != 64) return false;
     return fused_smem_floats(D, K, true) * 4 <= SMEM_BUDGET;
+}
+
+// Shapes the tensor-core kernel covers: accumulators of both point groups fit in tensor memory.
+bool tc_capable(int D, int K) {
+    if (D != 16 && D != 32 && D != 64) return false;
+    if (K > 256) return false;
+    return tc::layout_of(D, K, true).total <= SMEM_BUDGET;
 }
 
 // Blocks per rank (C) and warps per block for the partials kernel, from the shape alone.
@@ -524,7 +543,7 @@ bool km_plan(size_t N, int D, int K, int P, int sms, KmLayout* L) {
     L->off_partials = off; off = align_up(off + (size_t)P * K * stride * 4, 256);
     L->off_scratch = off; off = align_up(off + (size_t)P * (C > L->Cf ? C : L->Cf) * K * stride * 4, 256);
     L->off_reduced = off; off = align_up(off + (size_t)K * stride * 4, 256);
-    L->off_contrib = off; off = align_up(off + (size_t)K * 4, 256);
+    L->off_contrib = off; off = align_up(off + (size_t)K * 4 + 256, 256);   // + a status word
     L->off_ar = off; off = align_up(off + ec_allreduce_workspace_bytes(P, (size_t)K * stride, stride), 256);
     L->total = off;
     return true;
@@ -553,7 +572,39 @@ int km_fused_launch(ec_kmeans* km, bool partials, const float* centroids, int32_
     return EC_OK;
 }
 
+template <int D>
+int km_tc_launch(ec_kmeans* km, bool partials, const float* centroids, int32_t* labels, cudaStream_t st) {
+    const float tau_scale = 0.015625f;     // 2^-6: four times the bound 2^-8 (|x|^2 + |c|max^2) of one candidate's error
+    if (partials) {
+        tc::tc_fused_kernel<D, true><<<(unsigned)(km->P * km->Cf), tc::THREADS, km->tc_smem, st>>>(
+            km->points, km->N, km->P, km->Cf, centroids, km->K, labels, km->Cf == 1 ? km->partials : km->scratch,
+            tau_scale, km->tc_status);
+    } else {
+        size_t runs = (km->N + 8 * tc::TILE - 1) / (8 * tc::TILE);
+        if (runs > 0x7fffffffull) return EC_ERR_CAPACITY;
+        tc::tc_fused_kernel<D, false><<<(unsigned)runs, tc::THREADS, km->tc_assign_smem, st>>>(
+            km->points, km->N, 1, (int)runs, centroids, km->K, labels, nullptr, tau_scale, km->tc_status);
+    }
+    EC_CUDA(cudaGetLastError());
+    return EC_OK;
+}
+
+template <int D>
+cudaError_t km_tc_attr() {
+    cudaError_t e = cudaFuncSetAttribute(tc::tc_fused_kernel<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BUDGET);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(tc::tc_fused_kernel<D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BUDGET);
+    return e;
+}
+
 int km_fused(ec_kmeans* km, bool partials, const float* centroids, int32_t* labels, cudaStream_t st) {
+    if (km->tc_ok && km->path != 1) {
+        switch (km->D) {
+            case 16: return km_tc_launch<16>(km, partials, centroids, labels, st);
+            case 32: return km_tc_launch<32>(km, partials, centroids, labels, st);
+            case 64: return km_tc_launch<64>(km, partials, centroids, labels, st);
+        }
+    }
     switch (km->D) {
         case 8: return km_fused_launch<8>(km, partials, centroids, labels, st);
         case 16: return km_fused_launch<16>(km, partials, centroids, labels, st);
@@ -652,6 +703,11 @@ int ec_kmeans_init(ec_kmeans_t** out, const float* points, size_t N, int D, int 
     km->Cf = L.Cf;
     km->fused_smem = fused_smem_floats(D, K, true) * 4;
     km->fused_assign_smem = fused_smem_floats(D, K, false) * 4;
+    km->tc_ok = km->Cf > 0 && tc_capable(D, K);
+    km->path = 0;
+    km->tc_smem = tc::layout_of(D, K, true).total;
+    km->tc_assign_smem = tc::layout_of(D, K, false).total;
+    km->tc_status = reinterpret_cast<uint32_t*>(base + L.off_contrib + align_up((size_t)K * 4, 256));
     // centroid chunk for the assignment: as many as fit in 64 KB, all of them if possible
     int kc = (int)((64 * 1024) / ((size_t)D * 4));
     if (kc > K) kc = K;
@@ -677,6 +733,9 @@ int ec_kmeans_init(ec_kmeans_t** out, const float* points, size_t N, int D, int 
         e = cudaFuncSetAttribute(partials_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BUDGET);
     if (e == cudaSuccess && km->Cf > 0)
         e = D == 8 ? km_fused_attr<8>() : D == 16 ? km_fused_attr<16>() : D == 32 ? km_fused_attr<32>() : km_fused_attr<64>();
+    if (e == cudaSuccess && km->tc_ok)
+        e = D == 16 ? km_tc_attr<16>() : D == 32 ? km_tc_attr<32>() : km_tc_attr<64>();
+    if (e == cudaSuccess) e = cudaMemsetAsync(km->tc_status, 0, 4, 0);
     if (e == cudaSuccess) e = cudaMemcpyAsync(km->centroids, init_centroids, (size_t)K * D * 4, cudaMemcpyDeviceToDevice, 0);
     if (e == cudaSuccess) e = cudaStreamSynchronize(0);
     if (e != cudaSuccess) rc = cuda_fail(e);
@@ -747,6 +806,20 @@ int ec_kmeans_get(ec_kmeans_t* km, float* centroids, int32_t* labels, float* red
     if (labels) EC_CUDA(cudaMemcpyAsync(labels, km->labels, km->N * 4, cudaMemcpyDeviceToDevice, stream));
     if (reduced) EC_CUDA(cudaMemcpyAsync(reduced, km->reduced, (size_t)km->K * (km->D + 4) * 4, cudaMemcpyDeviceToDevice, stream));
     if (contrib_count) EC_CUDA(cudaMemcpyAsync(contrib_count, km->contrib, (size_t)km->K * 4, cudaMemcpyDeviceToDevice, stream));
+    return EC_OK;
+}
+
+int ec_kmeans_set_path(ec_kmeans_t* km, int path) {
+    if (!km || path < 0 || path > 2) return EC_ERR_INVALID;
+    if (path == 2 && !km->tc_ok) return EC_ERR_UNSUPPORTED;
+    if (path == 1 && km->Cf == 0) return EC_ERR_UNSUPPORTED;
+    km->path = path;
+    return EC_OK;
+}
+
+int ec_kmeans_tc_status(ec_kmeans_t* km, uint32_t* device_out, ec_stream_t stream) {
+    if (!km || !device_out) return EC_ERR_INVALID;
+    EC_CUDA(cudaMemcpyAsync(device_out, km->tc_status, 4, cudaMemcpyDeviceToDevice, stream));
     return EC_OK;
 }
 
