@@ -512,7 +512,7 @@ bool fused_capable(int D, int K) {
 // Shapes the tensor-core kernel covers: accumulators of both point groups fit in tensor memory.
 bool tc_capable(int D, int K) {
     if (D != 16 && D != 32 && D != 64) return false;
-    if (K > 256) return false;
+    if (tc::npad_of(K) > 256 || tc::GROUPS * tc::npad_of(K) > 512) return false;   // MMA width; accumulators fit in tensor memory
     return tc::layout_of(D, K, true).total <= SMEM_BUDGET;
 }
 
@@ -580,7 +580,7 @@ int km_tc_launch(ec_kmeans* km, bool partials, const float* centroids, int32_t* 
             km->points, km->N, km->P, km->Cf, centroids, km->K, labels, km->Cf == 1 ? km->partials : km->scratch,
             tau_scale, km->tc_status);
     } else {
-        size_t runs = (km->N + 8 * tc::TILE - 1) / (8 * tc::TILE);
+        size_t runs = (km->N + 2047) / 2048;
         if (runs > 0x7fffffffull) return EC_ERR_CAPACITY;
         tc::tc_fused_kernel<D, false><<<(unsigned)runs, tc::THREADS, km->tc_assign_smem, st>>>(
             km->points, km->N, 1, (int)runs, centroids, km->K, labels, nullptr, tau_scale, km->tc_status);

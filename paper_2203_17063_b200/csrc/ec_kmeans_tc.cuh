@@ -22,8 +22,15 @@
 namespace ec {
 namespace tc {
 
-constexpr int THREADS = 256;           // two groups of four warps; each group owns a 128-point accumulator
-constexpr int TILE = 256;              // points per tile
+#ifndef EC_TC_GROUPS
+#define EC_TC_GROUPS 1                 // groups of four warps per block; each group owns a 128-point accumulator
+#endif
+#ifndef EC_TC_MINB
+#define EC_TC_MINB 4                   // resident blocks the register allocation must allow
+#endif
+constexpr int GROUPS = EC_TC_GROUPS;
+constexpr int THREADS = 128 * GROUPS;
+constexpr int TILE = THREADS;          // points per tile, one per thread
 constexpr int WARPS = THREADS / 32;
 constexpr uint32_t WAIT_LIMIT = 1u << 20;
 
@@ -104,7 +111,7 @@ __host__ __device__ inline uint32_t instr_desc(int M, int N) {
 __host__ __device__ inline int npad_of(int K) { return (K + 31) & ~31; }             // accumulator columns per group
 __host__ __device__ inline int dpad_of(int D) { return (D + 15) & ~15; }             // K extent of the GEMM
 __host__ __device__ inline uint32_t tmem_cols_of(int K) {
-    uint32_t need = 2u * (uint32_t)npad_of(K), c = 32;
+    uint32_t need = (uint32_t)GROUPS * (uint32_t)npad_of(K), c = 32;
     while (c < need) c <<= 1;
     return c;
 }
@@ -162,7 +169,7 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 }
 
 template <int D, bool PARTIALS>
-__global__ void __launch_bounds__(THREADS, 2)
+__global__ void __launch_bounds__(THREADS, EC_TC_MINB)
 tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const float* __restrict__ centroids, int K,
                 int32_t* __restrict__ labels, float* __restrict__ scratch, float tau_scale, uint32_t* __restrict__ status) {
     constexpr int DPAD = (D + 15) & ~15;
@@ -264,7 +271,7 @@ tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const 
         if (tid == 0 && healthy) {
             fence_after_sync();
 #pragma unroll
-            for (int gg = 0; gg < 2; ++gg) {
+            for (int gg = 0; gg < GROUPS; ++gg) {
 #pragma unroll
                 for (int ks = 0; ks < DPAD / 16; ++ks) {
                     const uint64_t ad = smem_desc(a_base + gg * 128 * DPAD * 2 + ks * 2 * 128 * 16, 128 * 16, 128);
