@@ -512,7 +512,7 @@ bool fused_capable(int D, int K) {
 // Shapes the tensor-core kernel covers: accumulators of both point groups fit in tensor memory.
 bool tc_capable(int D, int K) {
     if (D != 16 && D != 32 && D != 64) return false;
-    if (tc::npad_of(K) > 256 || tc::GROUPS * tc::npad_of(K) > 512) return false;   // MMA width; accumulators fit in tensor memory
+    if (tc::npad_of(K) > 256) return false;   // MMA width; search and sums accumulators (2 x npad columns) fit in tensor memory
     return tc::layout_of(D, K, true).total <= SMEM_BUDGET;
 }
 

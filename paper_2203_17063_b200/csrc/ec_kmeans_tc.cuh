@@ -1,20 +1,28 @@
-// K-means assignment + partial sums with the candidate search on the 5th-generation tensor cores.
+// K-means assignment + partial sums on the 5th-generation tensor cores (tcgen05, tensor memory).
 //
-// The squared distance to centroid k is |x|^2 + v_k with v_k = |c_k|^2 - 2 x.c_k.  The inner products
-// x.c_k of a tile of points with all centroids are one small GEMM (128 points x NPAD centroids x D):
-// the points and centroids are rounded to bf16, staged in shared memory in the tensor core's
-// canonical K-major layout, multiplied by tcgen05.mma into an fp32 accumulator in tensor memory, and
-// read back with tcgen05.ld, one point per thread.  bf16 makes v_k approximate, so it only proposes:
-// the smallest and second smallest v are tracked and whenever they are closer than a bound on the
-// error of v (tau) the point is decided again in fp32 by the exact form sum_d (x-c)^2 over all
-// centroids - the same rule as the fp32 fused kernel, with a wider tau.  Labels are therefore those
-// of the exact form; only speed depends on how well separated the data is.
+// Candidate search.  The squared distance to centroid k is |x|^2 + v_k with v_k = |c_k|^2 - 2 x.c_k.
+// The inner products of a tile of 128 points with all centroids are one small GEMM: points and
+// centroids are rounded to bf16, staged in shared memory in the tensor core's canonical layout,
+// multiplied by tcgen05.mma into an fp32 accumulator in tensor memory and read back with tcgen05.ld,
+// one point per thread.  bf16 makes v_k approximate, so it only proposes: the smallest and second
+// smallest v are tracked and whenever they are closer than a bound on the error of v (tau) the point
+// is decided again in fp32 by the exact form sum_d (x-c)^2 over all centroids.  Labels are therefore
+// those of the exact form; only speed depends on how well separated the data is.
 //
-// Partial sums as in the fp32 fused kernel: points pass through shared memory transposed, each warp
-// adds its 32 points in order into its own [K][D] slab (lane = coordinate), fixed order, no atomics.
+// Partial sums.  sums[d][k] = sum_j x[j][d] onehot[j][k] is a GEMM too: the points, split into bf16
+// high and low parts (16 significand bits, relative error 2^-17 per coordinate, far inside the 1e-4
+// tolerance of the sums) and extended by a constant column of ones that yields the exact counts,
+// times the one-hot label matrix of the tile (exact in bf16).  The accumulator (row = coordinate,
+// column = centroid) stays in tensor memory over all tiles of the block and is written out once.
+// The shared-memory tile of the high parts serves both GEMMs: as the K-major A operand of the
+// search (row = point) and as the MN-major A operand here (row = coordinate) - both see the same
+// 8-point x 8-coordinate core matrices.  The sums MMA always works on 128 rows; rows beyond the
+// D + 16 real ones read whatever follows the tile in shared memory and are never looked at.
 //
-// Every wait on the tensor core is bounded; if one gives up the tile falls back to the exact form
-// (results stay correct) and a status word records it.
+// Block (r, c) covers the c-th of C runs of rank r's points and writes one [K][D+4] row block of
+// scratch; the rows of a rank are folded in order afterwards.  Every wait on the tensor core is
+// bounded; if one gives up, the block finishes in plain fp32 (exact form, atomic adds into its row
+// block) and a status word records it.
 #pragma once
 
 #include <cuda_bf16.h>
@@ -22,16 +30,12 @@
 namespace ec {
 namespace tc {
 
-#ifndef EC_TC_GROUPS
-#define EC_TC_GROUPS 1                 // groups of four warps per block; each group owns a 128-point accumulator
-#endif
 #ifndef EC_TC_MINB
 #define EC_TC_MINB 4                   // resident blocks the register allocation must allow
 #endif
-constexpr int GROUPS = EC_TC_GROUPS;
-constexpr int THREADS = 128 * GROUPS;
-constexpr int TILE = THREADS;          // points per tile, one per thread
-constexpr int WARPS = THREADS / 32;
+constexpr int THREADS = 128;           // four warps: one tensor-memory lane (= one point, one centroid row) per thread
+constexpr int TILE = THREADS;          // points per tile
+constexpr int MROWS = 128;             // rows of both accumulators
 constexpr uint32_t WAIT_LIMIT = 1u << 20;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -52,6 +56,11 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
+    for (uint32_t it = 0; it < WAIT_LIMIT; ++it)
+        if (mbar_try_wait(bar, parity)) return true;
+    return false;
+}
 __device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -63,7 +72,7 @@ __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.a
 __device__ __forceinline__ void fence_before_sync() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void fence_after_sync() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
-// D[tmem] (+)= A[smem] * B[smem]^T, bf16 inputs, fp32 accumulate, issued by one thread.
+// D[tmem] (+)= A[smem] * B[smem], bf16 inputs, fp32 accumulate, issued by one thread.
 __device__ __forceinline__ void mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
     asm volatile(
         "{\n"
@@ -77,7 +86,7 @@ __device__ __forceinline__ void mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint6
 __device__ __forceinline__ void mma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-// 32 consecutive fp32 columns of this thread's tensor-memory lane.
+// 32 / 16 consecutive fp32 columns of this thread's tensor-memory lane.
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
     asm volatile(
         "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
@@ -91,10 +100,21 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
         : "memory");
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
 
-// Shared-memory matrix descriptor, K-major, no swizzle: the operand is an array of 8-row x 16-byte
-// core matrices (rows 16 bytes apart); lbo = bytes between core matrices adjacent along K,
-// sbo = bytes between core matrices adjacent along the row dimension.
+// Shared-memory matrix descriptor without swizzle: the operand is an array of core matrices of
+// 8 x 16 bytes (eight 16-byte lines, 16 bytes apart).  lbo = bytes between core matrices adjacent
+// along the GEMM's K dimension, sbo = bytes between core matrices adjacent along the M/N dimension
+// (for K-major and for MN-major operands alike).
 __device__ __forceinline__ uint64_t smem_desc(uint32_t saddr, uint32_t lbo, uint32_t sbo) {
     uint64_t d = 0;
     d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
@@ -103,39 +123,39 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t saddr, uint32_t lbo, uint
     d |= 1ull << 46;                       // descriptor version of this architecture
     return d;                              // bits 61-63 = 0: no swizzle
 }
-// Instruction descriptor: fp32 accumulator, bf16 A and B, both K-major, M x N tile.
-__host__ __device__ inline uint32_t instr_desc(int M, int N) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+// Instruction descriptor: fp32 accumulator, bf16 A and B, M x N tile; mn_major = both operands MN-major.
+__host__ __device__ inline uint32_t instr_desc(int M, int N, bool mn_major) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | (mn_major ? (3u << 15) : 0u) | ((uint32_t)(N >> 3) << 17) |
+           ((uint32_t)(M >> 4) << 24);
 }
 
-__host__ __device__ inline int npad_of(int K) { return (K + 31) & ~31; }             // accumulator columns per group
-__host__ __device__ inline int dpad_of(int D) { return (D + 15) & ~15; }             // K extent of the GEMM
-__host__ __device__ inline uint32_t tmem_cols_of(int K) {
-    uint32_t need = (uint32_t)GROUPS * (uint32_t)npad_of(K), c = 32;
+__host__ __device__ inline int npad_of(int K) { return (K + 31) & ~31; }   // columns of the search accumulator
+__host__ __device__ inline int dpad_of(int D) { return (D + 15) & ~15; }   // K extent of the search GEMM
+__host__ __device__ inline uint32_t tmem_cols_of(int D, int K, bool partials) {
+    (void)D;
+    uint32_t need = (uint32_t)npad_of(K) * (partials ? 2u : 1u), c = 32;       // search accumulator + sums accumulator
     while (c < need) c <<= 1;
     return c;
 }
 
 struct Layout {   // byte offsets into dynamic shared memory
-    size_t cn, b, ax, lab, acc, cnt, bar, total;
+    size_t cn, b, xh, xl, oh, bar, total;
 };
 __host__ __device__ inline Layout layout_of(int D, int K, bool partials) {
     const size_t npad = npad_of(K), dpad = dpad_of(D);
     Layout L;
     size_t off = 0;
     L.cn = off; off += npad * 4;
-    off = (off + 1023) & ~(size_t)1023;
-    L.b = off; off += npad * dpad * 2;                                   // bf16 centroids
-    off = (off + 1023) & ~(size_t)1023;
-    const size_t a_bytes = (size_t)TILE * dpad * 2;                      // bf16 points of a tile
-    const size_t x_bytes = partials ? (size_t)TILE * (D + 1) * 4 : 0;    // transposed fp32 points (same storage, later)
-    L.ax = off; off += a_bytes > x_bytes ? a_bytes : x_bytes;
-    off = (off + 15) & ~(size_t)15;
-    L.lab = off; off += partials ? (size_t)TILE * 4 : 0;
-    L.acc = off; off += partials ? (size_t)WARPS * K * D * 4 : 0;
-    L.cnt = off; off += partials ? (size_t)WARPS * K * 4 : 0;
-    off = (off + 15) & ~(size_t)15;
-    L.bar = off; off += 16;                                              // mbarrier (8 bytes) + tensor-memory address
+    off = (off + 127) & ~(size_t)127;
+    L.b = off; off += npad * dpad * 2;                                        // bf16 centroids, K-major chunks
+    // The sums MMA reads 128 rows = 16 chunks starting at xl and at xh; every chunk it touches must lie
+    // inside this block's allocation.  Low parts first, then high parts, then the one-hot tile, then
+    // padding up to 16 chunks after xh.
+    L.xl = off; off += partials ? (size_t)(dpad / 8 + 2) * TILE * 16 : 0;     // low parts + two zero chunks
+    L.xh = off; off += (size_t)(dpad / 8 + 2) * TILE * 16;                    // high parts + ones chunk + zero chunk
+    L.oh = off; off += partials ? npad / 8 * (size_t)TILE * 16 : 0;           // one-hot labels
+    if (partials && off < L.xh + (size_t)(MROWS / 8) * TILE * 16) off = L.xh + (size_t)(MROWS / 8) * TILE * 16;
+    L.bar = off; off += 32;                                                   // two mbarriers + tensor-memory address
     L.total = off;
     return L;
 }
@@ -161,6 +181,16 @@ __device__ __forceinline__ int exact_argmin_global(const float (&x)[D], const fl
     return bi;
 }
 
+template <int D>
+__device__ __forceinline__ void load_point(const float* __restrict__ points, size_t j, float (&x)[D]) {
+    const float4* rowp = reinterpret_cast<const float4*>(points + j * D);
+#pragma unroll
+    for (int q = 0; q < D / 4; ++q) {
+        const float4 v = __ldg(rowp + q);
+        x[4 * q] = v.x; x[4 * q + 1] = v.y; x[4 * q + 2] = v.z; x[4 * q + 3] = v.w;
+    }
+}
+
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);   // .x = lo (low half), .y = hi
     uint32_t u;
@@ -173,28 +203,28 @@ __global__ void __launch_bounds__(THREADS, EC_TC_MINB)
 tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const float* __restrict__ centroids, int K,
                 int32_t* __restrict__ labels, float* __restrict__ scratch, float tau_scale, uint32_t* __restrict__ status) {
     constexpr int DPAD = (D + 15) & ~15;
-    constexpr int KCH = DPAD / 8;                        // 16-byte chunks along K per row
-    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    constexpr int KCH = DPAD / 8;                        // 16-byte chunks of coordinates per point
+    constexpr int NROWS = DPAD + 16;                     // live rows of the sums accumulator: coordinates, ones, zeros
+    constexpr uint32_t CHUNK = TILE * 16;                // bytes of one chunk column: 128 points x 16 bytes
+    extern __shared__ __align__(128) unsigned char smem_raw[];
     const int npad = npad_of(K);
     const Layout L = layout_of(D, K, PARTIALS);
     float* s_cn = reinterpret_cast<float*>(smem_raw + L.cn);
     unsigned char* s_b = smem_raw + L.b;
-    unsigned char* s_a = smem_raw + L.ax;                // bf16 operand tiles: group g at g * 128 * DPAD * 2
-    float* s_x = reinterpret_cast<float*>(smem_raw + L.ax);
-    int* s_lab = reinterpret_cast<int*>(smem_raw + L.lab);
-    float* s_acc = reinterpret_cast<float*>(smem_raw + L.acc);
-    int* s_cnt = reinterpret_cast<int*>(smem_raw + L.cnt);
+    unsigned char* s_xh = smem_raw + L.xh;
+    unsigned char* s_xl = smem_raw + L.xl;
+    unsigned char* s_oh = smem_raw + L.oh;
     uint64_t* s_bar = reinterpret_cast<uint64_t*>(smem_raw + L.bar);
-    uint32_t* s_tmem = reinterpret_cast<uint32_t*>(smem_raw + L.bar + 8);
+    uint32_t* s_tmem = reinterpret_cast<uint32_t*>(smem_raw + L.bar + 16);
 
-    const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5, g = tid >> 7, row = tid & 127;
-    const size_t KD = (size_t)K * D;
-    const uint32_t ncols = tmem_cols_of(K);
-    const uint32_t bar = smem_u32(s_bar);
+    const int tid = threadIdx.x, w = tid >> 5;
+    const uint32_t ncols = tmem_cols_of(D, K, PARTIALS);
+    const uint32_t bar1 = smem_u32(s_bar), bar2 = smem_u32(s_bar + 1);
 
     if (w == 0) tmem_alloc(smem_u32(s_tmem), ncols);
     if (tid == 0) {
-        mbar_init(bar, 1);
+        mbar_init(bar1, 1);
+        mbar_init(bar2, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     // |c|^2 (padding columns get a value that can never win) and the bf16 centroids in operand layout
@@ -214,159 +244,197 @@ tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const 
             const int d = kc * 8 + e;
             v[e] = (n < K && d < D) ? centroids[(size_t)n * D + d] : 0.0f;
         }
-        const uint4 q = make_uint4(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]), pack_bf16(v[4], v[5]), pack_bf16(v[6], v[7]));
-        *reinterpret_cast<uint4*>(s_b + (size_t)kc * npad * 16 + (size_t)n * 16) = q;
+        *reinterpret_cast<uint4*>(s_b + (size_t)kc * npad * 16 + (size_t)n * 16) =
+            make_uint4(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]), pack_bf16(v[4], v[5]), pack_bf16(v[6], v[7]));
     }
+    // constant chunks of the high tile: [1, 0, ..., 0] (its column sums are the counts) and zeros
+    *reinterpret_cast<uint4*>(s_xh + (size_t)KCH * CHUNK + (size_t)tid * 16) = make_uint4(0x00003F80u, 0u, 0u, 0u);
+    *reinterpret_cast<uint4*>(s_xh + (size_t)(KCH + 1) * CHUNK + (size_t)tid * 16) = make_uint4(0u, 0u, 0u, 0u);
     if (PARTIALS) {
-        for (size_t i = tid; i < (size_t)WARPS * KD; i += THREADS) s_acc[i] = 0.0f;
-        for (int i = tid; i < WARPS * K; i += THREADS) s_cnt[i] = 0;
+        *reinterpret_cast<uint4*>(s_xl + (size_t)KCH * CHUNK + (size_t)tid * 16) = make_uint4(0u, 0u, 0u, 0u);
+        *reinterpret_cast<uint4*>(s_xl + (size_t)(KCH + 1) * CHUNK + (size_t)tid * 16) = make_uint4(0u, 0u, 0u, 0u);
+        for (int ch = 0; ch < npad / 8; ++ch)
+            *reinterpret_cast<uint4*>(s_oh + (size_t)ch * CHUNK + (size_t)tid * 16) = make_uint4(0u, 0u, 0u, 0u);
     }
     fence_async_smem();
     fence_before_sync();
     __syncthreads();
     fence_after_sync();
     const uint32_t tmem_base = *s_tmem;
+    const uint32_t tmem_lane = tmem_base + ((uint32_t)(w * 32) << 16);   // this warp's 32 lanes
     float cmax = 0.0f;
     for (int k = 0; k < K; ++k) cmax = fmaxf(cmax, s_cn[k]);
-    const uint32_t idesc = instr_desc(128, npad);
-    const uint32_t a_base = smem_u32(s_a), b_base = smem_u32(s_b);
+    const uint32_t idesc_search = instr_desc(MROWS, npad, false);
+    const uint32_t idesc_sum = instr_desc(MROWS, npad, true);
+    const uint32_t b_base = smem_u32(s_b), xh_base = smem_u32(s_xh), xl_base = smem_u32(s_xl), oh_base = smem_u32(s_oh);
 
     const int r = blockIdx.x / C, c = blockIdx.x - r * C;
     const size_t j0 = (size_t)r * N / P, j1 = (size_t)(r + 1) * N / P;
     const size_t len = j1 - j0;
     const size_t b0 = j0 + len * c / C, b1 = j0 + len * (c + 1) / C;
-    uint32_t phase = 0;
-    bool healthy = true;             // false once a wait on the tensor core gave up: exact form from then on
+    const int stride = D + 4;
+    float* row_block = PARTIALS ? scratch + ((size_t)r * C + c) * (size_t)K * stride : nullptr;
+    if (PARTIALS)
+        for (int i = tid; i < K * stride; i += THREADS) row_block[i] = 0.0f;   // base of the by-hand adds, should they be needed
+    uint32_t phase1 = 0, phase2 = 0;
+    bool healthy = true;             // false once a wait on the tensor core gave up: plain fp32 from then on
+    bool sums_started = false;       // a sums MMA has been issued (the accumulator holds data)
+    bool sums_pending = false;       // ... and its completion has not been waited for yet
+    int prev_chunk = -1;             // one-hot chunk this thread set in the previous tile
 
     for (size_t base = b0; base < b1; base += TILE) {
         const size_t j = base + tid;
         const bool live = j < b1;
-        float x[D];
         float xn = 0.0f;
-        if (live) {
-            const float4* rowp = reinterpret_cast<const float4*>(points + j * D);
+        {
+            float x[D];
+            if (live) {
+                load_point<D>(points, j, x);
+            } else {
 #pragma unroll
-            for (int q = 0; q < D / 4; ++q) {
-                const float4 v = __ldg(rowp + q);
-                x[4 * q] = v.x; x[4 * q + 1] = v.y; x[4 * q + 2] = v.z; x[4 * q + 3] = v.w;
+                for (int d = 0; d < D; ++d) x[d] = 0.0f;
             }
 #pragma unroll
             for (int d = 0; d < D; ++d) xn = fmaf(x[d], x[d], xn);
-        } else {
+            if (PARTIALS && sums_pending) {
+                // the previous tile's sums MMA still reads the tiles: wait for it (its latency hid behind the loads)
+                const bool ok = mbar_wait_bounded(bar2, phase2);
+                phase2 ^= 1u;
+                sums_pending = false;
+                if (!ok) healthy = false;
+            }
+            if (PARTIALS && prev_chunk >= 0) {
+                *reinterpret_cast<uint4*>(s_oh + (size_t)prev_chunk * CHUNK + (size_t)tid * 16) = make_uint4(0u, 0u, 0u, 0u);
+                prev_chunk = -1;
+            }
+            // bf16 high parts (and low parts = bf16(x - high)) in chunk layout: chunk kc of point tid at kc*CHUNK + tid*16
 #pragma unroll
-            for (int d = 0; d < D; ++d) x[d] = 0.0f;
-        }
-        // bf16 operand: chunk kc of row `row` of group g at g*(128*DPAD*2) + kc*(128*16) + row*16
+            for (int kc = 0; kc < KCH; ++kc) {
+                uint32_t hw[4], lw[4];
 #pragma unroll
-        for (int kc = 0; kc < KCH; ++kc) {
-            float v[8];
-#pragma unroll
-            for (int e = 0; e < 8; ++e) v[e] = (kc * 8 + e < D) ? x[kc * 8 + e] : 0.0f;
-            const uint4 q = make_uint4(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]), pack_bf16(v[4], v[5]), pack_bf16(v[6], v[7]));
-            *reinterpret_cast<uint4*>(s_a + (size_t)g * 128 * DPAD * 2 + (size_t)kc * 128 * 16 + (size_t)row * 16) = q;
+                for (int e = 0; e < 4; ++e) {
+                    const int d = kc * 8 + 2 * e;
+                    const float a = d < D ? x[d < D ? d : 0] : 0.0f, b = d + 1 < D ? x[d + 1 < D ? d + 1 : 0] : 0.0f;
+                    hw[e] = pack_bf16(a, b);
+                    const float ah = __uint_as_float(hw[e] << 16), bh = __uint_as_float(hw[e] & 0xFFFF0000u);
+                    lw[e] = pack_bf16(a - ah, b - bh);
+                }
+                *reinterpret_cast<uint4*>(s_xh + (size_t)kc * CHUNK + (size_t)tid * 16) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
+                if (PARTIALS)
+                    *reinterpret_cast<uint4*>(s_xl + (size_t)kc * CHUNK + (size_t)tid * 16) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
+            }
         }
         fence_async_smem();          // the tensor core reads shared memory through the async proxy
         fence_before_sync();
-        __syncthreads();
+        healthy = __syncthreads_and(healthy) != 0;
         if (tid == 0 && healthy) {
             fence_after_sync();
 #pragma unroll
-            for (int gg = 0; gg < GROUPS; ++gg) {
-#pragma unroll
-                for (int ks = 0; ks < DPAD / 16; ++ks) {
-                    const uint64_t ad = smem_desc(a_base + gg * 128 * DPAD * 2 + ks * 2 * 128 * 16, 128 * 16, 128);
-                    const uint64_t bd = smem_desc(b_base + ks * 2 * npad * 16, npad * 16, 128);
-                    mma_bf16(tmem_base + (uint32_t)(gg * npad), ad, bd, idesc, ks > 0 ? 1u : 0u);
-                }
+            for (int ks = 0; ks < DPAD / 16; ++ks) {     // search: rows = points (K-major), columns = centroids
+                const uint64_t ad = smem_desc(xh_base + ks * 2 * CHUNK, CHUNK, 128);
+                const uint64_t bd = smem_desc(b_base + ks * 2 * npad * 16, npad * 16, 128);
+                mma_bf16(tmem_base, ad, bd, idesc_search, ks > 0 ? 1u : 0u);
             }
-            mma_commit(bar);         // the barrier completes when both accumulators are written
+            mma_commit(bar1);
         }
-        bool done = false;
-        if (healthy) {
-            for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
-                if (mbar_try_wait(bar, phase)) { done = true; break; }
-            }
-        }
+        bool done = healthy && mbar_wait_bounded(bar1, phase1);
+        phase1 ^= 1u;
         done = __syncthreads_and(done) != 0;     // all threads take the same path
         healthy = done;
-        phase ^= 1u;
         fence_after_sync();
         float m1 = __int_as_float(0x7f800000), m2 = m1;
         int kb = 0;
         if (done) {
             for (int ch = 0; ch < npad / 32; ++ch) {
                 uint32_t dot[32];
-                tmem_ld32(tmem_base + ((uint32_t)((w & 3) * 32) << 16) + (uint32_t)(g * npad + ch * 32), dot);
+                tmem_ld32(tmem_lane + (uint32_t)(ch * 32), dot);
 #pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    const int k = ch * 32 + i;
-                    const float v = fmaf(-2.0f, __uint_as_float(dot[i]), s_cn[k]);
-                    const bool lt = v < m1;
-                    m2 = fminf(m2, lt ? m1 : v);
-                    kb = lt ? k : kb;
-                    m1 = lt ? v : m1;
+                for (int q = 0; q < 8; ++q) {
+                    const float4 cn = *reinterpret_cast<const float4*>(s_cn + ch * 32 + q * 4);
+                    const float cnv[4] = {cn.x, cn.y, cn.z, cn.w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const int k = ch * 32 + q * 4 + e;
+                        const float v = fmaf(-2.0f, __uint_as_float(dot[q * 4 + e]), cnv[e]);
+                        const bool lt = v < m1;
+                        m2 = fminf(m2, lt ? m1 : v);
+                        kb = lt ? k : kb;
+                        m1 = lt ? v : m1;
+                    }
                 }
             }
         } else if (tid == 0 && status != nullptr) {
-            atomicOr(status, 1u);    // the tensor core did not answer in time: exact form from here on
+            atomicOr(status, 1u);    // the tensor core did not answer in time
         }
         fence_before_sync();         // accumulator reads are done before the next tile's MMA may overwrite it
         // rounding to bf16 perturbs v by at most 2^-7 |x||c| <= 2^-8 (|x|^2 + |c|max^2) per candidate
         const float tau = tau_scale * (xn + cmax);
-        if (live && (!done || !(m2 - m1 > tau))) kb = exact_argmin_global<D>(x, centroids, K);
-        if (live) labels[j] = kb;
-        if (PARTIALS) {
-            __syncthreads();                                   // (the operand tiles have been consumed: the MMA is complete)
-            s_lab[tid] = live ? kb : -1;
+        const bool redo = live && (!done || !(m2 - m1 > tau));
+        if (redo || (live && PARTIALS && !done)) {
+            float x[D];
+            load_point<D>(points, j, x);                 // rare: read the point again instead of keeping it in registers
+            if (redo) kb = exact_argmin_global<D>(x, centroids, K);
+            if (PARTIALS && !done) {                     // tensor core out of service: add this point by hand
 #pragma unroll
-            for (int d = 0; d < D; ++d) s_x[(size_t)tid * (D + 1) + d] = x[d];
-            __syncthreads();
-            float* acc = s_acc + (size_t)w * KD;
-            int* cnt = s_cnt + w * K;
-            for (int jj = 0; jj < 32; jj += 4) {
-                int lab[4];
-                float xv[4][(D + 31) / 32];
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const int pt = w * 32 + jj + u;
-                    lab[u] = s_lab[pt];
-#pragma unroll
-                    for (int q = 0; q < (D + 31) / 32; ++q) {
-                        const int d = lane + 32 * q;
-                        xv[u][q] = d < D ? s_x[(size_t)pt * (D + 1) + d] : 0.0f;
-                    }
-                }
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    if (lab[u] >= 0) {
-#pragma unroll
-                        for (int q = 0; q < (D + 31) / 32; ++q) {
-                            const int d = lane + 32 * q;
-                            if (d < D) acc[(size_t)lab[u] * D + d] = __fadd_rn(acc[(size_t)lab[u] * D + d], xv[u][q]);
-                        }
-                        if (lane == 0) cnt[lab[u]] += 1;
-                    }
-                }
+                for (int d = 0; d < D; ++d) atomicAdd(row_block + (size_t)kb * stride + d, x[d]);
+                atomicAdd(row_block + (size_t)kb * stride + D, 1.0f);
             }
-            __syncthreads();                                   // s_x is free again for the next tile's operands
+        }
+        if (live) labels[j] = kb;
+        if (PARTIALS && done) {
+            if (live) {
+                // one-hot row of this point: element kb of 128, i.e. 16-byte chunk kb/8, bf16 1.0 at position kb%8
+                uint32_t wv[4] = {0u, 0u, 0u, 0u};
+                wv[(kb & 7) >> 1] = 0x3F80u << (16 * (kb & 1));
+                prev_chunk = kb >> 3;
+                *reinterpret_cast<uint4*>(s_oh + (size_t)prev_chunk * CHUNK + (size_t)tid * 16) = make_uint4(wv[0], wv[1], wv[2], wv[3]);
+            }
+            fence_async_smem();
+            fence_before_sync();
+            __syncthreads();
+            if (tid == 0) {
+                fence_after_sync();
+                // sums[d][k] += sum_j x[j][d] * onehot[j][k]; 16 points per step; both operands MN-major:
+                // consecutive points are 16 bytes apart (K direction: 8 points = 128 bytes),
+                // consecutive chunks of 8 coordinates / 8 centroids are CHUNK bytes apart (M/N direction)
+#pragma unroll
+                for (int ks = 0; ks < TILE / 16; ++ks) {
+                    const uint64_t ah = smem_desc(xh_base + ks * 256, 128, CHUNK);
+                    const uint64_t al = smem_desc(xl_base + ks * 256, 128, CHUNK);
+                    const uint64_t bd = smem_desc(oh_base + ks * 256, 128, CHUNK);
+                    mma_bf16(tmem_base + (uint32_t)npad, ah, bd, idesc_sum, (sums_started || ks > 0) ? 1u : 0u);
+                    mma_bf16(tmem_base + (uint32_t)npad, al, bd, idesc_sum, 1u);
+                }
+                mma_commit(bar2);
+            }
+            sums_started = true;
+            sums_pending = true;
         }
     }
-    __syncthreads();
     if (PARTIALS) {
-        const int stride = D + 4;
-        float* dst = scratch + ((size_t)r * C + c) * (size_t)K * stride;
-        for (size_t i = tid; i < (size_t)K * stride; i += THREADS) {
-            const int kk = (int)(i / stride), d = (int)(i - (size_t)kk * stride);
-            float val = 0.0f;
-            if (d < D) {
-                val = s_acc[(size_t)kk * D + d];
-                for (int ww = 1; ww < WARPS; ++ww) val = __fadd_rn(val, s_acc[(size_t)ww * KD + (size_t)kk * D + d]);
-            } else if (d == D) {
-                int n = 0;
-                for (int ww = 0; ww < WARPS; ++ww) n += s_cnt[ww * K + kk];
-                val = (float)n;
+        bool ok = true;
+        if (sums_pending) ok = mbar_wait_bounded(bar2, phase2);
+        ok = __syncthreads_and(ok) != 0;
+        fence_after_sync();
+        if (!ok && tid == 0 && status != nullptr) atomicOr(status, 1u);
+        // this thread's tensor-memory lane is row tid of the accumulator: coordinate tid for tid < D,
+        // the counts at row DPAD, zeros in the three rows after it; columns are the centroids
+        const int col = tid < D ? tid : (tid >= DPAD && tid < DPAD + 4) ? D + (tid - DPAD) : -1;
+        if (ok && sums_started) {
+            for (int ch = 0; ch < npad / 32; ++ch) {
+                uint32_t v[32];
+                tmem_ld32(tmem_lane + (uint32_t)(npad + ch * 32), v);
+                if (col >= 0) {
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) {
+                        const int k = ch * 32 + e;
+                        if (k < K) {
+                            if (healthy) row_block[(size_t)k * stride + col] = __uint_as_float(v[e]);
+                            else atomicAdd(row_block + (size_t)k * stride + col, __uint_as_float(v[e]));   // some tiles were added by hand
+                        }
+                    }
+                }
             }
-            dst[i] = val;
         }
     }
     fence_before_sync();
