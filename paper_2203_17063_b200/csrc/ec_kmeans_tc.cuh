@@ -37,6 +37,9 @@ constexpr int THREADS = 128;           // four warps: one tensor-memory lane (= 
 constexpr int TILE = THREADS;          // points per tile
 constexpr int MROWS = 128;             // rows of both accumulators
 constexpr uint32_t WAIT_LIMIT = 1u << 20;
+constexpr uint32_t OCHUNK = TILE * 16;        // one-hot tile: bytes between chunks of 8 centroids (128 points x 16 bytes)
+constexpr uint32_t XCHUNK = TILE * 16 + 16;   // point tiles: bytes between chunks of 8 coordinates; the 16 extra bytes
+                                              // spread the four chunks of a point over different banks
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -139,22 +142,23 @@ __host__ __device__ inline uint32_t tmem_cols_of(int D, int K, bool partials) {
 }
 
 struct Layout {   // byte offsets into dynamic shared memory
-    size_t cn, b, xh, xl, oh, bar, total;
+    size_t cn, xn, b, xh, xl, oh, bar, total;
 };
 __host__ __device__ inline Layout layout_of(int D, int K, bool partials) {
     const size_t npad = npad_of(K), dpad = dpad_of(D);
     Layout L;
     size_t off = 0;
     L.cn = off; off += npad * 4;
+    L.xn = off; off += (size_t)TILE * 4;                                      // |x|^2 of the tile's points
     off = (off + 127) & ~(size_t)127;
     L.b = off; off += npad * dpad * 2;                                        // bf16 centroids, K-major chunks
     // The sums MMA reads 128 rows = 16 chunks starting at xl and at xh; every chunk it touches must lie
     // inside this block's allocation.  Low parts first, then high parts, then the one-hot tile, then
     // padding up to 16 chunks after xh.
-    L.xl = off; off += partials ? (size_t)(dpad / 8 + 2) * TILE * 16 : 0;     // low parts + two zero chunks
-    L.xh = off; off += (size_t)(dpad / 8 + 2) * TILE * 16;                    // high parts + ones chunk + zero chunk
-    L.oh = off; off += partials ? npad / 8 * (size_t)TILE * 16 : 0;           // one-hot labels
-    if (partials && off < L.xh + (size_t)(MROWS / 8) * TILE * 16) off = L.xh + (size_t)(MROWS / 8) * TILE * 16;
+    L.xl = off; off += partials ? (size_t)(dpad / 8 + 2) * XCHUNK : 0;        // low parts + two zero chunks
+    L.xh = off; off += (size_t)(dpad / 8 + 2) * XCHUNK;                       // high parts + ones chunk + zero chunk
+    L.oh = off; off += partials ? npad / 8 * (size_t)OCHUNK : 0;              // one-hot labels
+    if (partials && off < L.xh + (size_t)(MROWS / 8) * XCHUNK) off = L.xh + (size_t)(MROWS / 8) * XCHUNK;
     L.bar = off; off += 32;                                                   // two mbarriers + tensor-memory address
     L.total = off;
     return L;
@@ -205,11 +209,12 @@ tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const 
     constexpr int DPAD = (D + 15) & ~15;
     constexpr int KCH = DPAD / 8;                        // 16-byte chunks of coordinates per point
     constexpr int NROWS = DPAD + 16;                     // live rows of the sums accumulator: coordinates, ones, zeros
-    constexpr uint32_t CHUNK = TILE * 16;                // bytes of one chunk column: 128 points x 16 bytes
+    static_assert(D % 8 == 0 && (KCH & (KCH - 1)) == 0, "coordinates come in power-of-two many chunks of eight");
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const int npad = npad_of(K);
     const Layout L = layout_of(D, K, PARTIALS);
     float* s_cn = reinterpret_cast<float*>(smem_raw + L.cn);
+    float* s_xn = reinterpret_cast<float*>(smem_raw + L.xn);
     unsigned char* s_b = smem_raw + L.b;
     unsigned char* s_xh = smem_raw + L.xh;
     unsigned char* s_xl = smem_raw + L.xl;
@@ -248,13 +253,13 @@ tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const 
             make_uint4(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]), pack_bf16(v[4], v[5]), pack_bf16(v[6], v[7]));
     }
     // constant chunks of the high tile: [1, 0, ..., 0] (its column sums are the counts) and zeros
-    *reinterpret_cast<uint4*>(s_xh + (size_t)KCH * CHUNK + (size_t)tid * 16) = make_uint4(0x00003F80u, 0u, 0u, 0u);
-    *reinterpret_cast<uint4*>(s_xh + (size_t)(KCH + 1) * CHUNK + (size_t)tid * 16) = make_uint4(0u, 0u, 0u, 0u);
+    *reinterpret_cast<uint4*>(s_xh + (size_t)KCH * XCHUNK + (size_t)tid * 16) = make_uint4(0x00003F80u, 0u, 0u, 0u);
+    *reinterpret_cast<uint4*>(s_xh + (size_t)(KCH + 1) * XCHUNK + (size_t)tid * 16) = make_uint4(0u, 0u, 0u, 0u);
     if (PARTIALS) {
-        *reinterpret_cast<uint4*>(s_xl + (size_t)KCH * CHUNK + (size_t)tid * 16) = make_uint4(0u, 0u, 0u, 0u);
-        *reinterpret_cast<uint4*>(s_xl + (size_t)(KCH + 1) * CHUNK + (size_t)tid * 16) = make_uint4(0u, 0u, 0u, 0u);
+        *reinterpret_cast<uint4*>(s_xl + (size_t)KCH * XCHUNK + (size_t)tid * 16) = make_uint4(0u, 0u, 0u, 0u);
+        *reinterpret_cast<uint4*>(s_xl + (size_t)(KCH + 1) * XCHUNK + (size_t)tid * 16) = make_uint4(0u, 0u, 0u, 0u);
         for (int ch = 0; ch < npad / 8; ++ch)
-            *reinterpret_cast<uint4*>(s_oh + (size_t)ch * CHUNK + (size_t)tid * 16) = make_uint4(0u, 0u, 0u, 0u);
+            *reinterpret_cast<uint4*>(s_oh + (size_t)ch * OCHUNK + (size_t)tid * 16) = make_uint4(0u, 0u, 0u, 0u);
     }
     fence_async_smem();
     fence_before_sync();
@@ -285,17 +290,24 @@ tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const 
     for (size_t base = b0; base < b1; base += TILE) {
         const size_t j = base + tid;
         const bool live = j < b1;
-        float xn = 0.0f;
+        // Stage the tile: item (point row, chunk kc of 8 coordinates) -> 16 bytes of bf16 high parts and 16 of low
+        // parts (low = bf16(x - high)) at kc*XCHUNK + row*16.  Consecutive threads take consecutive 32-byte pieces
+        // of the points, so every load instruction of a warp covers 1 KB of contiguous memory.
         {
-            float x[D];
-            if (live) {
-                load_point<D>(points, j, x);
-            } else {
+            float4 va[KCH], vb[KCH];
 #pragma unroll
-                for (int d = 0; d < D; ++d) x[d] = 0.0f;
+            for (int q = 0; q < KCH; ++q) {
+                const int idx = q * THREADS + tid, row = idx / KCH, kc = idx % KCH;
+                const size_t jr = base + row;
+                if (jr < b1) {
+                    const float4* src = reinterpret_cast<const float4*>(points + jr * D + kc * 8);
+                    va[q] = __ldg(src);
+                    vb[q] = __ldg(src + 1);
+                } else {
+                    va[q] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                    vb[q] = va[q];
+                }
             }
-#pragma unroll
-            for (int d = 0; d < D; ++d) xn = fmaf(x[d], x[d], xn);
             if (PARTIALS && sums_pending) {
                 // the previous tile's sums MMA still reads the tiles: wait for it (its latency hid behind the loads)
                 const bool ok = mbar_wait_bounded(bar2, phase2);
@@ -304,24 +316,31 @@ tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const 
                 if (!ok) healthy = false;
             }
             if (PARTIALS && prev_chunk >= 0) {
-                *reinterpret_cast<uint4*>(s_oh + (size_t)prev_chunk * CHUNK + (size_t)tid * 16) = make_uint4(0u, 0u, 0u, 0u);
+                *reinterpret_cast<uint4*>(s_oh + (size_t)prev_chunk * OCHUNK + (size_t)tid * 16) = make_uint4(0u, 0u, 0u, 0u);
                 prev_chunk = -1;
             }
-            // bf16 high parts (and low parts = bf16(x - high)) in chunk layout: chunk kc of point tid at kc*CHUNK + tid*16
 #pragma unroll
-            for (int kc = 0; kc < KCH; ++kc) {
+            for (int q = 0; q < KCH; ++q) {
+                const int idx = q * THREADS + tid, row = idx / KCH, kc = idx % KCH;
+                const float v[8] = {va[q].x, va[q].y, va[q].z, va[q].w, vb[q].x, vb[q].y, vb[q].z, vb[q].w};
                 uint32_t hw[4], lw[4];
+                float sq = 0.0f;
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
-                    const int d = kc * 8 + 2 * e;
-                    const float a = d < D ? x[d < D ? d : 0] : 0.0f, b = d + 1 < D ? x[d + 1 < D ? d + 1 : 0] : 0.0f;
+                    const float a = v[2 * e], b = v[2 * e + 1];
+                    sq = fmaf(a, a, sq);
+                    sq = fmaf(b, b, sq);
                     hw[e] = pack_bf16(a, b);
                     const float ah = __uint_as_float(hw[e] << 16), bh = __uint_as_float(hw[e] & 0xFFFF0000u);
                     lw[e] = pack_bf16(a - ah, b - bh);
                 }
-                *reinterpret_cast<uint4*>(s_xh + (size_t)kc * CHUNK + (size_t)tid * 16) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
+                *reinterpret_cast<uint4*>(s_xh + (size_t)kc * XCHUNK + (size_t)row * 16) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
                 if (PARTIALS)
-                    *reinterpret_cast<uint4*>(s_xl + (size_t)kc * CHUNK + (size_t)tid * 16) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
+                    *reinterpret_cast<uint4*>(s_xl + (size_t)kc * XCHUNK + (size_t)row * 16) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
+                // |x|^2 of the row: its KCH chunks sit in KCH consecutive lanes
+#pragma unroll
+                for (int o = 1; o < KCH; o <<= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+                if (kc == 0) s_xn[row] = sq;
             }
         }
         fence_async_smem();          // the tensor core reads shared memory through the async proxy
@@ -331,7 +350,7 @@ tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const 
             fence_after_sync();
 #pragma unroll
             for (int ks = 0; ks < DPAD / 16; ++ks) {     // search: rows = points (K-major), columns = centroids
-                const uint64_t ad = smem_desc(xh_base + ks * 2 * CHUNK, CHUNK, 128);
+                const uint64_t ad = smem_desc(xh_base + ks * 2 * XCHUNK, XCHUNK, 128);
                 const uint64_t bd = smem_desc(b_base + ks * 2 * npad * 16, npad * 16, 128);
                 mma_bf16(tmem_base, ad, bd, idesc_search, ks > 0 ? 1u : 0u);
             }
@@ -368,7 +387,7 @@ tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const 
         }
         fence_before_sync();         // accumulator reads are done before the next tile's MMA may overwrite it
         // rounding to bf16 perturbs v by at most 2^-7 |x||c| <= 2^-8 (|x|^2 + |c|max^2) per candidate
-        const float tau = tau_scale * (xn + cmax);
+        const float tau = tau_scale * (s_xn[tid] + cmax);
         const bool redo = live && (!done || !(m2 - m1 > tau));
         if (redo || (live && PARTIALS && !done)) {
             float x[D];
@@ -387,7 +406,7 @@ tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const 
                 uint32_t wv[4] = {0u, 0u, 0u, 0u};
                 wv[(kb & 7) >> 1] = 0x3F80u << (16 * (kb & 1));
                 prev_chunk = kb >> 3;
-                *reinterpret_cast<uint4*>(s_oh + (size_t)prev_chunk * CHUNK + (size_t)tid * 16) = make_uint4(wv[0], wv[1], wv[2], wv[3]);
+                *reinterpret_cast<uint4*>(s_oh + (size_t)prev_chunk * OCHUNK + (size_t)tid * 16) = make_uint4(wv[0], wv[1], wv[2], wv[3]);
             }
             fence_async_smem();
             fence_before_sync();
@@ -396,12 +415,12 @@ tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const 
                 fence_after_sync();
                 // sums[d][k] += sum_j x[j][d] * onehot[j][k]; 16 points per step; both operands MN-major:
                 // consecutive points are 16 bytes apart (K direction: 8 points = 128 bytes),
-                // consecutive chunks of 8 coordinates / 8 centroids are CHUNK bytes apart (M/N direction)
+                // consecutive chunks of 8 coordinates / 8 centroids are XCHUNK / OCHUNK bytes apart (M/N direction)
 #pragma unroll
                 for (int ks = 0; ks < TILE / 16; ++ks) {
-                    const uint64_t ah = smem_desc(xh_base + ks * 256, 128, CHUNK);
-                    const uint64_t al = smem_desc(xl_base + ks * 256, 128, CHUNK);
-                    const uint64_t bd = smem_desc(oh_base + ks * 256, 128, CHUNK);
+                    const uint64_t ah = smem_desc(xh_base + ks * 256, 128, XCHUNK);
+                    const uint64_t al = smem_desc(xl_base + ks * 256, 128, XCHUNK);
+                    const uint64_t bd = smem_desc(oh_base + ks * 256, 128, OCHUNK);
                     mma_bf16(tmem_base + (uint32_t)npad, ah, bd, idesc_sum, (sums_started || ks > 0) ? 1u : 0u);
                     mma_bf16(tmem_base + (uint32_t)npad, al, bd, idesc_sum, 1u);
                 }
