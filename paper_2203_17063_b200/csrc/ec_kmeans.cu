@@ -511,7 +511,7 @@ bool fused_capable(int D, int K) {
 
 // Shapes the tensor-core kernel covers: accumulators of both point groups fit in tensor memory.
 bool tc_capable(int D, int K) {
-    if (D != 16 && D != 32 && D != 64) return false;
+    if (D != 16 && D != 32) return false;   // the point tile holds high parts, ones and low parts in 16 chunk columns
     if (tc::npad_of(K) > 256) return false;   // MMA width; search and sums accumulators (2 x npad columns) fit in tensor memory
     return tc::layout_of(D, K, true).total <= SMEM_BUDGET;
 }
@@ -602,7 +602,6 @@ int km_fused(ec_kmeans* km, bool partials, const float* centroids, int32_t* labe
         switch (km->D) {
             case 16: return km_tc_launch<16>(km, partials, centroids, labels, st);
             case 32: return km_tc_launch<32>(km, partials, centroids, labels, st);
-            case 64: return km_tc_launch<64>(km, partials, centroids, labels, st);
         }
     }
     switch (km->D) {
@@ -734,7 +733,7 @@ int ec_kmeans_init(ec_kmeans_t** out, const float* points, size_t N, int D, int 
     if (e == cudaSuccess && km->Cf > 0)
         e = D == 8 ? km_fused_attr<8>() : D == 16 ? km_fused_attr<16>() : D == 32 ? km_fused_attr<32>() : km_fused_attr<64>();
     if (e == cudaSuccess && km->tc_ok)
-        e = D == 16 ? km_tc_attr<16>() : D == 32 ? km_tc_attr<32>() : km_tc_attr<64>();
+        e = D == 16 ? km_tc_attr<16>() : km_tc_attr<32>();
     if (e == cudaSuccess) e = cudaMemsetAsync(km->tc_status, 0, 4, 0);
     if (e == cudaSuccess) e = cudaMemcpyAsync(km->centroids, init_centroids, (size_t)K * D * 4, cudaMemcpyDeviceToDevice, 0);
     if (e == cudaSuccess) e = cudaStreamSynchronize(0);

@@ -141,25 +141,28 @@ __host__ __device__ inline uint32_t tmem_cols_of(int D, int K, bool partials) {
     return c;
 }
 
-struct Layout {   // byte offsets into dynamic shared memory
-    size_t cn, xn, b, xh, xl, oh, bar, total;
+// Shared memory of a block (byte offsets).  The point tile is one array of 16 chunk columns
+// (XCHUNK bytes each, chunk = 8 coordinates x 128 points): columns 0..KCH-1 hold the bf16 high parts,
+// column KCH the constants [1,1,0,..,0], column KCH+1 zeros; columns 8..8+KCH-1 the low parts,
+// 8+KCH and 8+KCH+1 zeros.  Read as a 128-row MN-major operand this puts the high parts (and the
+// ones) in rows 0..63 and the low parts in rows 64..127 of one MMA.  The columns in between are never
+// looked at as results, so they carry other data: |c|^2 and |x|^2 in columns 6-7, the centroid operand
+// from column 14 on.
+struct Layout {
+    size_t x, cn, xn, b, oh, bar, total;
 };
 __host__ __device__ inline Layout layout_of(int D, int K, bool partials) {
-    const size_t npad = npad_of(K), dpad = dpad_of(D);
+    const size_t npad = npad_of(K), kch = dpad_of(D) / 8;
     Layout L;
-    size_t off = 0;
-    L.cn = off; off += npad * 4;
-    L.xn = off; off += (size_t)TILE * 4;                                      // |x|^2 of the tile's points
+    L.x = 0;
+    L.cn = 6 * (size_t)XCHUNK;                       // npad floats (at most 256) ...
+    L.xn = L.cn + 1024;                               // ... then 128 floats; both inside columns 6-7 (4128 bytes)
+    L.b = 14 * (size_t)XCHUNK;                        // centroid operand: npad rows x (kch + 2) chunks of 16 bytes
+    size_t off = L.b + npad * (kch + 2) * 16;
+    if (off < 16 * (size_t)XCHUNK) off = 16 * (size_t)XCHUNK;   // all 16 columns lie inside the allocation
     off = (off + 127) & ~(size_t)127;
-    L.b = off; off += npad * dpad * 2;                                        // bf16 centroids, K-major chunks
-    // The sums MMA reads 128 rows = 16 chunks starting at xl and at xh; every chunk it touches must lie
-    // inside this block's allocation.  Low parts first, then high parts, then the one-hot tile, then
-    // padding up to 16 chunks after xh.
-    L.xl = off; off += partials ? (size_t)(dpad / 8 + 2) * XCHUNK : 0;        // low parts + two zero chunks
-    L.xh = off; off += (size_t)(dpad / 8 + 2) * XCHUNK;                       // high parts + ones chunk + zero chunk
-    L.oh = off; off += partials ? npad / 8 * (size_t)OCHUNK : 0;              // one-hot labels
-    if (partials && off < L.xh + (size_t)(MROWS / 8) * XCHUNK) off = L.xh + (size_t)(MROWS / 8) * XCHUNK;
-    L.bar = off; off += 32;                                                   // two mbarriers + tensor-memory address
+    L.oh = off; off += partials ? npad / 8 * (size_t)OCHUNK : 0;   // one-hot labels; reused to combine high and low sums at the end
+    L.bar = off; off += 32;                           // two mbarriers + tensor-memory address
     L.total = off;
     return L;
 }
@@ -206,18 +209,16 @@ template <int D, bool PARTIALS>
 __global__ void __launch_bounds__(THREADS, EC_TC_MINB)
 tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const float* __restrict__ centroids, int K,
                 int32_t* __restrict__ labels, float* __restrict__ scratch, float tau_scale, uint32_t* __restrict__ status) {
-    constexpr int DPAD = (D + 15) & ~15;
-    constexpr int KCH = DPAD / 8;                        // 16-byte chunks of coordinates per point
-    constexpr int NROWS = DPAD + 16;                     // live rows of the sums accumulator: coordinates, ones, zeros
-    static_assert(D % 8 == 0 && (KCH & (KCH - 1)) == 0, "coordinates come in power-of-two many chunks of eight");
+    constexpr int KCH = D / 8;                           // 16-byte chunks of coordinates per point
+    static_assert(D % 16 == 0 && KCH + 2 <= 8 && (KCH & (KCH - 1)) == 0, "D is 16 or 32");
+    constexpr int LO = 8;                                // first chunk column of the low parts
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const int npad = npad_of(K);
     const Layout L = layout_of(D, K, PARTIALS);
+    unsigned char* s_x = smem_raw + L.x;
     float* s_cn = reinterpret_cast<float*>(smem_raw + L.cn);
     float* s_xn = reinterpret_cast<float*>(smem_raw + L.xn);
     unsigned char* s_b = smem_raw + L.b;
-    unsigned char* s_xh = smem_raw + L.xh;
-    unsigned char* s_xl = smem_raw + L.xl;
     unsigned char* s_oh = smem_raw + L.oh;
     uint64_t* s_bar = reinterpret_cast<uint64_t*>(smem_raw + L.bar);
     uint32_t* s_tmem = reinterpret_cast<uint32_t*>(smem_raw + L.bar + 16);
@@ -232,7 +233,9 @@ tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const 
         mbar_init(bar2, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    // |c|^2 (padding columns get a value that can never win) and the bf16 centroids in operand layout
+    // Centroid operand (K-major, chunk kc of centroid n at kc*(npad*16) + n*16): -2 c in bf16 (the doubling is
+    // exact), then one chunk [hi(|c|^2), lo(|c|^2), 0, ...] that meets the points' [1, 1, 0, ...] chunk, so
+    // that the GEMM delivers v = |c|^2 - 2 x.c itself; padding centroids get a |c|^2 that can never win.
     for (int k = tid; k < npad; k += THREADS) {
         float s = 3.0e38f;
         if (k < K) {
@@ -240,24 +243,26 @@ tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const 
             for (int d = 0; d < D; ++d) s = fmaf(centroids[(size_t)k * D + d], centroids[(size_t)k * D + d], s);
         }
         s_cn[k] = s;
+        const uint32_t hl = pack_bf16(s, 0.0f) & 0xFFFFu;
+        const float hi = __uint_as_float(hl << 16);
+        const uint32_t both = hl | (pack_bf16(s - hi, 0.0f) << 16);
+        *reinterpret_cast<uint4*>(s_b + (size_t)KCH * npad * 16 + (size_t)k * 16) = make_uint4(both, 0u, 0u, 0u);
+        *reinterpret_cast<uint4*>(s_b + (size_t)(KCH + 1) * npad * 16 + (size_t)k * 16) = make_uint4(0u, 0u, 0u, 0u);
     }
     for (int i = tid; i < npad * KCH; i += THREADS) {
-        const int kc = i / npad, n = i - kc * npad;      // chunk kc of centroid n lives at kc * (npad*16) + n*16
+        const int kc = i / npad, n = i - kc * npad;
         float v[8];
 #pragma unroll
-        for (int e = 0; e < 8; ++e) {
-            const int d = kc * 8 + e;
-            v[e] = (n < K && d < D) ? centroids[(size_t)n * D + d] : 0.0f;
-        }
+        for (int e = 0; e < 8; ++e) v[e] = n < K ? -2.0f * centroids[(size_t)n * D + kc * 8 + e] : 0.0f;
         *reinterpret_cast<uint4*>(s_b + (size_t)kc * npad * 16 + (size_t)n * 16) =
             make_uint4(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]), pack_bf16(v[4], v[5]), pack_bf16(v[6], v[7]));
     }
-    // constant chunks of the high tile: [1, 0, ..., 0] (its column sums are the counts) and zeros
-    *reinterpret_cast<uint4*>(s_xh + (size_t)KCH * XCHUNK + (size_t)tid * 16) = make_uint4(0x00003F80u, 0u, 0u, 0u);
-    *reinterpret_cast<uint4*>(s_xh + (size_t)(KCH + 1) * XCHUNK + (size_t)tid * 16) = make_uint4(0u, 0u, 0u, 0u);
+    // constant chunk columns of the point tile
+    *reinterpret_cast<uint4*>(s_x + (size_t)KCH * XCHUNK + (size_t)tid * 16) = make_uint4(0x3F803F80u, 0u, 0u, 0u);   // [1, 1, 0, ...]
+    *reinterpret_cast<uint4*>(s_x + (size_t)(KCH + 1) * XCHUNK + (size_t)tid * 16) = make_uint4(0u, 0u, 0u, 0u);
     if (PARTIALS) {
-        *reinterpret_cast<uint4*>(s_xl + (size_t)KCH * XCHUNK + (size_t)tid * 16) = make_uint4(0u, 0u, 0u, 0u);
-        *reinterpret_cast<uint4*>(s_xl + (size_t)(KCH + 1) * XCHUNK + (size_t)tid * 16) = make_uint4(0u, 0u, 0u, 0u);
+        *reinterpret_cast<uint4*>(s_x + (size_t)(LO + KCH) * XCHUNK + (size_t)tid * 16) = make_uint4(0u, 0u, 0u, 0u);
+        *reinterpret_cast<uint4*>(s_x + (size_t)(LO + KCH + 1) * XCHUNK + (size_t)tid * 16) = make_uint4(0u, 0u, 0u, 0u);
         for (int ch = 0; ch < npad / 8; ++ch)
             *reinterpret_cast<uint4*>(s_oh + (size_t)ch * OCHUNK + (size_t)tid * 16) = make_uint4(0u, 0u, 0u, 0u);
     }
@@ -271,7 +276,7 @@ tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const 
     for (int k = 0; k < K; ++k) cmax = fmaxf(cmax, s_cn[k]);
     const uint32_t idesc_search = instr_desc(MROWS, npad, false);
     const uint32_t idesc_sum = instr_desc(MROWS, npad, true);
-    const uint32_t b_base = smem_u32(s_b), xh_base = smem_u32(s_xh), xl_base = smem_u32(s_xl), oh_base = smem_u32(s_oh);
+    const uint32_t b_base = smem_u32(s_b), x_base = smem_u32(s_x), oh_base = smem_u32(s_oh);
 
     const int r = blockIdx.x / C, c = blockIdx.x - r * C;
     const size_t j0 = (size_t)r * N / P, j1 = (size_t)(r + 1) * N / P;
@@ -287,70 +292,75 @@ tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const 
     bool sums_pending = false;       // ... and its completion has not been waited for yet
     int prev_chunk = -1;             // one-hot chunk this thread set in the previous tile
 
+    // A thread stages KCH items (point row, chunk kc of 8 coordinates) of a tile: consecutive threads take
+    // consecutive 32-byte pieces of the points, so every load instruction of a warp covers 1 KB of contiguous
+    // memory.  The loads of the next tile are issued as soon as the current one is staged and stay in flight
+    // while the current tile is searched.
+    float4 va[KCH], vb[KCH];
+    auto issue_loads = [&](size_t tile_base) {
+#pragma unroll
+        for (int q = 0; q < KCH; ++q) {
+            const int idx = q * THREADS + tid, row = idx / KCH, kc = idx % KCH;
+            const size_t jr = tile_base + row;
+            if (jr < b1) {
+                const float4* src = reinterpret_cast<const float4*>(points + jr * D + kc * 8);
+                va[q] = __ldg(src);
+                vb[q] = __ldg(src + 1);
+            } else {
+                va[q] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                vb[q] = va[q];
+            }
+        }
+    };
+    issue_loads(b0);
+
     for (size_t base = b0; base < b1; base += TILE) {
         const size_t j = base + tid;
         const bool live = j < b1;
-        // Stage the tile: item (point row, chunk kc of 8 coordinates) -> 16 bytes of bf16 high parts and 16 of low
-        // parts (low = bf16(x - high)) at kc*XCHUNK + row*16.  Consecutive threads take consecutive 32-byte pieces
-        // of the points, so every load instruction of a warp covers 1 KB of contiguous memory.
-        {
-            float4 va[KCH], vb[KCH];
-#pragma unroll
-            for (int q = 0; q < KCH; ++q) {
-                const int idx = q * THREADS + tid, row = idx / KCH, kc = idx % KCH;
-                const size_t jr = base + row;
-                if (jr < b1) {
-                    const float4* src = reinterpret_cast<const float4*>(points + jr * D + kc * 8);
-                    va[q] = __ldg(src);
-                    vb[q] = __ldg(src + 1);
-                } else {
-                    va[q] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-                    vb[q] = va[q];
-                }
-            }
-            if (PARTIALS && sums_pending) {
-                // the previous tile's sums MMA still reads the tiles: wait for it (its latency hid behind the loads)
-                const bool ok = mbar_wait_bounded(bar2, phase2);
-                phase2 ^= 1u;
-                sums_pending = false;
-                if (!ok) healthy = false;
-            }
-            if (PARTIALS && prev_chunk >= 0) {
-                *reinterpret_cast<uint4*>(s_oh + (size_t)prev_chunk * OCHUNK + (size_t)tid * 16) = make_uint4(0u, 0u, 0u, 0u);
-                prev_chunk = -1;
-            }
-#pragma unroll
-            for (int q = 0; q < KCH; ++q) {
-                const int idx = q * THREADS + tid, row = idx / KCH, kc = idx % KCH;
-                const float v[8] = {va[q].x, va[q].y, va[q].z, va[q].w, vb[q].x, vb[q].y, vb[q].z, vb[q].w};
-                uint32_t hw[4], lw[4];
-                float sq = 0.0f;
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const float a = v[2 * e], b = v[2 * e + 1];
-                    sq = fmaf(a, a, sq);
-                    sq = fmaf(b, b, sq);
-                    hw[e] = pack_bf16(a, b);
-                    const float ah = __uint_as_float(hw[e] << 16), bh = __uint_as_float(hw[e] & 0xFFFF0000u);
-                    lw[e] = pack_bf16(a - ah, b - bh);
-                }
-                *reinterpret_cast<uint4*>(s_xh + (size_t)kc * XCHUNK + (size_t)row * 16) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
-                if (PARTIALS)
-                    *reinterpret_cast<uint4*>(s_xl + (size_t)kc * XCHUNK + (size_t)row * 16) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
-                // |x|^2 of the row: its KCH chunks sit in KCH consecutive lanes
-#pragma unroll
-                for (int o = 1; o < KCH; o <<= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
-                if (kc == 0) s_xn[row] = sq;
-            }
+        if (PARTIALS && sums_pending) {
+            // the previous tile's sums MMA still reads the tile: wait for it (its latency hid behind the search)
+            const bool ok = mbar_wait_bounded(bar2, phase2);
+            phase2 ^= 1u;
+            sums_pending = false;
+            if (!ok) healthy = false;
         }
+        if (PARTIALS && prev_chunk >= 0) {
+            *reinterpret_cast<uint4*>(s_oh + (size_t)prev_chunk * OCHUNK + (size_t)tid * 16) = make_uint4(0u, 0u, 0u, 0u);
+            prev_chunk = -1;
+        }
+        // bf16 high parts and low parts (low = bf16(x - high)) at chunk column kc resp. LO + kc, row*16
+#pragma unroll
+        for (int q = 0; q < KCH; ++q) {
+            const int idx = q * THREADS + tid, row = idx / KCH, kc = idx % KCH;
+            const float v[8] = {va[q].x, va[q].y, va[q].z, va[q].w, vb[q].x, vb[q].y, vb[q].z, vb[q].w};
+            uint32_t hw[4], lw[4];
+            float sq = 0.0f;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const float a = v[2 * e], b = v[2 * e + 1];
+                sq = fmaf(a, a, sq);
+                sq = fmaf(b, b, sq);
+                hw[e] = pack_bf16(a, b);
+                const float ah = __uint_as_float(hw[e] << 16), bh = __uint_as_float(hw[e] & 0xFFFF0000u);
+                lw[e] = pack_bf16(a - ah, b - bh);
+            }
+            *reinterpret_cast<uint4*>(s_x + (size_t)kc * XCHUNK + (size_t)row * 16) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
+            if (PARTIALS)
+                *reinterpret_cast<uint4*>(s_x + (size_t)(LO + kc) * XCHUNK + (size_t)row * 16) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
+            // |x|^2 of the row: its KCH chunks sit in KCH consecutive lanes
+#pragma unroll
+            for (int o = 1; o < KCH; o <<= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+            if (kc == 0) s_xn[row] = sq;
+        }
+        if (base + TILE < b1) issue_loads(base + TILE);
         fence_async_smem();          // the tensor core reads shared memory through the async proxy
         fence_before_sync();
         healthy = __syncthreads_and(healthy) != 0;
         if (tid == 0 && healthy) {
             fence_after_sync();
 #pragma unroll
-            for (int ks = 0; ks < DPAD / 16; ++ks) {     // search: rows = points (K-major), columns = centroids
-                const uint64_t ad = smem_desc(xh_base + ks * 2 * XCHUNK, XCHUNK, 128);
+            for (int ks = 0; ks < D / 16 + 1; ++ks) {    // search: rows = points (K-major), columns = centroids; last step adds |c|^2
+                const uint64_t ad = smem_desc(x_base + ks * 2 * XCHUNK, XCHUNK, 128);
                 const uint64_t bd = smem_desc(b_base + ks * 2 * npad * 16, npad * 16, 128);
                 mma_bf16(tmem_base, ad, bd, idesc_search, ks > 0 ? 1u : 0u);
             }
@@ -365,21 +375,15 @@ tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const 
         int kb = 0;
         if (done) {
             for (int ch = 0; ch < npad / 32; ++ch) {
-                uint32_t dot[32];
-                tmem_ld32(tmem_lane + (uint32_t)(ch * 32), dot);
+                uint32_t vv[32];
+                tmem_ld32(tmem_lane + (uint32_t)(ch * 32), vv);
 #pragma unroll
-                for (int q = 0; q < 8; ++q) {
-                    const float4 cn = *reinterpret_cast<const float4*>(s_cn + ch * 32 + q * 4);
-                    const float cnv[4] = {cn.x, cn.y, cn.z, cn.w};
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const int k = ch * 32 + q * 4 + e;
-                        const float v = fmaf(-2.0f, __uint_as_float(dot[q * 4 + e]), cnv[e]);
-                        const bool lt = v < m1;
-                        m2 = fminf(m2, lt ? m1 : v);
-                        kb = lt ? k : kb;
-                        m1 = lt ? v : m1;
-                    }
+                for (int e = 0; e < 32; ++e) {
+                    const float v = __uint_as_float(vv[e]);
+                    const bool lt = v < m1;
+                    m2 = fminf(m2, lt ? m1 : v);
+                    kb = lt ? ch * 32 + e : kb;
+                    m1 = lt ? v : m1;
                 }
             }
         } else if (tid == 0 && status != nullptr) {
@@ -402,7 +406,7 @@ tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const 
         if (live) labels[j] = kb;
         if (PARTIALS && done) {
             if (live) {
-                // one-hot row of this point: element kb of 128, i.e. 16-byte chunk kb/8, bf16 1.0 at position kb%8
+                // one-hot row of this point: 16-byte chunk kb/8, bf16 1.0 at position kb%8
                 uint32_t wv[4] = {0u, 0u, 0u, 0u};
                 wv[(kb & 7) >> 1] = 0x3F80u << (16 * (kb & 1));
                 prev_chunk = kb >> 3;
@@ -413,16 +417,15 @@ tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const 
             __syncthreads();
             if (tid == 0) {
                 fence_after_sync();
-                // sums[d][k] += sum_j x[j][d] * onehot[j][k]; 16 points per step; both operands MN-major:
-                // consecutive points are 16 bytes apart (K direction: 8 points = 128 bytes),
-                // consecutive chunks of 8 coordinates / 8 centroids are XCHUNK / OCHUNK bytes apart (M/N direction)
+                // sums[row][k] += sum_j X[j][row] * onehot[j][k], 16 points per step, both operands MN-major:
+                // consecutive points are 16 bytes apart (K direction: 8 points = 128 bytes), consecutive chunks
+                // of 8 rows / 8 centroids are XCHUNK / OCHUNK bytes apart (M/N direction).  One MMA covers the
+                // high parts with the ones (rows 0..63) and the low parts (rows 64..127).
 #pragma unroll
                 for (int ks = 0; ks < TILE / 16; ++ks) {
-                    const uint64_t ah = smem_desc(xh_base + ks * 256, 128, XCHUNK);
-                    const uint64_t al = smem_desc(xl_base + ks * 256, 128, XCHUNK);
+                    const uint64_t ad = smem_desc(x_base + ks * 256, 128, XCHUNK);
                     const uint64_t bd = smem_desc(oh_base + ks * 256, 128, OCHUNK);
-                    mma_bf16(tmem_base + (uint32_t)npad, ah, bd, idesc_sum, (sums_started || ks > 0) ? 1u : 0u);
-                    mma_bf16(tmem_base + (uint32_t)npad, al, bd, idesc_sum, 1u);
+                    mma_bf16(tmem_base + (uint32_t)npad, ad, bd, idesc_sum, (sums_started || ks > 0) ? 1u : 0u);
                 }
                 mma_commit(bar2);
             }
@@ -436,20 +439,30 @@ tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const 
         ok = __syncthreads_and(ok) != 0;
         fence_after_sync();
         if (!ok && tid == 0 && status != nullptr) atomicOr(status, 1u);
-        // this thread's tensor-memory lane is row tid of the accumulator: coordinate tid for tid < D,
-        // the counts at row DPAD, zeros in the three rows after it; columns are the centroids
-        const int col = tid < D ? tid : (tid >= DPAD && tid < DPAD + 4) ? D + (tid - DPAD) : -1;
+        // This thread's tensor-memory lane is row tid of the accumulator; columns are the centroids.
+        // Rows 0..D-1: high-part sums of coordinate tid; row D: the counts; rows 64..64+D-1: low-part sums.
+        // The low rows go through shared memory (the one-hot tile is free now) to the thread of their coordinate.
         if (ok && sums_started) {
+            float* s_lo = reinterpret_cast<float*>(s_oh);          // [npad][D] floats <= npad/8 * 2048 bytes for D <= 32... (D*4 <= 256)
+            const bool is_hi = tid < D, is_cnt = tid == D, is_lo = tid >= 64 && tid < 64 + D;
             for (int ch = 0; ch < npad / 32; ++ch) {
                 uint32_t v[32];
                 tmem_ld32(tmem_lane + (uint32_t)(npad + ch * 32), v);
-                if (col >= 0) {
+                if (is_lo) {
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) s_lo[(size_t)(ch * 32 + e) * D + (tid - 64)] = __uint_as_float(v[e]);
+                }
+                __syncthreads();
+                if (is_hi || is_cnt) {
 #pragma unroll
                     for (int e = 0; e < 32; ++e) {
                         const int k = ch * 32 + e;
                         if (k < K) {
-                            if (healthy) row_block[(size_t)k * stride + col] = __uint_as_float(v[e]);
-                            else atomicAdd(row_block + (size_t)k * stride + col, __uint_as_float(v[e]));   // some tiles were added by hand
+                            float val = __uint_as_float(v[e]);
+                            if (is_hi) val = __fadd_rn(val, s_lo[(size_t)k * D + tid]);
+                            float* dst = row_block + (size_t)k * stride + tid;   // column tid: coordinate, or D = the count
+                            if (healthy) *dst = val;
+                            else atomicAdd(dst, val);                             // some tiles were added by hand
                         }
                     }
                 }
