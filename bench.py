@@ -529,14 +529,32 @@ def kmeans_case(dev, stream, reps=5, iters=20, profile_only=False):
         ms_assign = time_calls(stream, lambda: km.assign(d_init, lab, stream), 10)
         part = torch.empty(P, K, D + 4, device=dev)
         ms_part = time_calls(stream, lambda: km.partials(lab, part, stream), 10)
+        # the same 20 iterations with the candidate search on the fp32 pipes instead of the tensor cores
+        km.set_path(1)
+        km.set_centroids(d_init, stream)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for t in range(iters):
+            km.iterate_raw(masks[t].data_ptr(), st)
+        b.record(stream)
+        torch.cuda.synchronize()
+        ms_fp32_path = a.elapsed_time(b)
+        km.set_path(0)
+        tc_status = km.tc_status(stream)
     m, ci = mean_ci(runs)
-    sm_clock_ghz = 1.965
-    alu_peak_lane_ops = 148 * 128 * sm_clock_ghz * 1e9
+    peak, _ = measured_peaks()
+    iter_bytes = N * D * 4 + N * 4            # the points once, the labels once (centroids and partial rows are < 1 %)
     res = {
         "iterations_per_s": round(iters / (m * 1e-3), 1), "ms_per_20_iterations": round(m, 3), "ci95": round(ci, 3),
-        "assign_ms": round(statistics.fmean(ms_assign), 4), "partials_ms": round(statistics.fmean(ms_part), 4),
-        "assign_frac_of_fp32_alu_bound": round((2.0 * N * K * D / alu_peak_lane_ops) / (statistics.fmean(ms_assign) * 1e-3), 4),
-        "note": "assign bound = 2*N*K*D lane-instructions (sub + fma) at 148 SMs x 128 lanes x 1.965 GHz",
+        "path": "tensor cores (tcgen05 bf16 candidate search + one-hot sums GEMM, exact fp32 re-decision)",
+        "tensor_core_status_word": tc_status,
+        "iteration_GBps": round(iter_bytes / (m / iters) / 1e6, 1),
+        "iteration_frac_of_hbm_measured": round(iter_bytes / (m / iters) / 1e6 / peak, 4),
+        "assign_only_ms": round(statistics.fmean(ms_assign), 4),
+        "standalone_partials_ms": round(statistics.fmean(ms_part), 4),
+        "fp32_path_iterations_per_s": round(iters / (ms_fp32_path * 1e-3), 1),
+        "note": "bound: HBM (537 MB of points + 17 MB of labels per iteration); the fp32 path is bound by the FMA pipe "
+                "(N*K*D fused multiply-adds = 0.23 ms at 148 SMs x 128 lanes x 1.965 GHz)",
     }
     km.destroy()
     return res
