@@ -54,6 +54,9 @@ def lib() -> C.CDLL:
         L.oracle_allreduce_ref64.restype = C.c_int
         L.oracle_allreduce_ref64.argtypes = [C.c_int, C.c_size_t, C.c_int, C.c_size_t, C.c_void_p,
                                              C.c_void_p, C.c_void_p, C.c_void_p]
+        L.oracle_allreduce_ssp.restype = C.c_int
+        L.oracle_allreduce_ssp.argtypes = [C.c_int, C.c_size_t, C.c_int, C.c_int, C.c_size_t, C.c_void_p, C.c_void_p,
+                                           C.c_uint32, C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.oracle_allgatherv.restype = C.c_int
         L.oracle_allgatherv.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_size_t, C.c_void_p,
                                         C.c_void_p, C.c_void_p, C.c_size_t]
@@ -151,6 +154,26 @@ def allreduce_ref64(bufs, dtype: int, segment_size: int, arrival_mask=None):
     if rc != 0:
         raise RuntimeError("oracle_allreduce_ref64 failed")
     return ref, mag
+
+
+def allreduce_ssp(bufs, dtype: int, op: int, segment_size: int, notif_clock: np.ndarray, clock: int, slack: int):
+    """Stale-synchronous allreduce: returns (result, contrib_count, seg_clock, wait_count).
+    notif_clock is uint32 [S][P]: the clock of the contribution each rank buffer holds, 0 = none."""
+    P = len(bufs)
+    keep, table = _ptr_table(bufs, _IN_NP[dtype])
+    n = keep[0].size
+    S = (n + segment_size - 1) // segment_size
+    notif_clock = np.ascontiguousarray(notif_clock, dtype=np.uint32)
+    assert notif_clock.shape == (S, P)
+    result = np.empty(n, dtype=_OUT_NP[dtype])
+    count = np.empty(S, dtype=np.uint32)
+    seg_clock = np.empty(S, dtype=np.uint32)
+    wait = np.empty(S, dtype=np.uint32)
+    rc = lib().oracle_allreduce_ssp(P, n, dtype, op, segment_size, table, _ptr(notif_clock), clock, slack,
+                                    _ptr(result), _ptr(count), _ptr(seg_clock), _ptr(wait))
+    if rc != 0:
+        raise RuntimeError("oracle_allreduce_ssp failed")
+    return result, count, seg_clock, wait
 
 
 def allgatherv(bufs, counts: np.ndarray, arrival_mask, out: np.ndarray):

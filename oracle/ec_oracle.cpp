@@ -302,6 +302,57 @@ int oracle_allreduce_ref64(int P, size_t n, int dtype, size_t seg, const void* c
 }
 
 // ---------------------------------------------------------------------------
+// Stale-synchronous allreduce (Sec. III-A, Algorithm 1), stateless.
+// Every rank buffer holds the last contribution that rank wrote for a segment, and
+// notif_clock[s][r] is the clock (iteration) in which it was computed; 0 = nothing
+// received yet.  As in the algorithm: min_clock_accepted = clock - slack; a received
+// contribution whose clock is below it is too stale - the paper's process would wait
+// for an update there; this sampled form leaves it out and counts it in wait_count.
+// The others are reduced in rank order starting from the identity.  The clock of a
+// reduction is the minimum of the clocks of what went into it (0 if nothing did).
+// ---------------------------------------------------------------------------
+int oracle_allreduce_ssp(int P, size_t n, int dtype, int op, size_t seg, const void* const* bufs,
+                         const uint32_t* notif_clock, uint32_t clock, uint32_t slack, void* result,
+                         uint32_t* contrib_count, uint32_t* seg_clock, uint32_t* wait_count) {
+    if (P < 1 || n == 0 || seg == 0 || !bufs || !notif_clock || !result || clock == 0) return -1;
+    const size_t S = (n + seg - 1) / seg;
+    const long long min_clock_accepted = (long long)clock - (long long)slack;
+    for (size_t s = 0; s < S; ++s) {
+        const size_t lo = s * seg;
+        const size_t hi = (lo + seg < n) ? lo + seg : n;
+        uint32_t used = 0, waits = 0, oldest = 0;
+        std::vector<int> order((size_t)P, -1);
+        for (int r = 0; r < P; ++r) {
+            const uint32_t rcv_clock = notif_clock[s * (size_t)P + (size_t)r];
+            if (rcv_clock == 0 || (long long)rcv_clock < min_clock_accepted) { ++waits; continue; }   // too stale: would wait
+            order[used++] = r;
+            if (oldest == 0 || rcv_clock < oldest) oldest = rcv_clock;
+        }
+        for (size_t i = lo; i < hi; ++i) {
+            switch (dtype) {
+                case DT_F32: { float acc = identity_of<float>(op);
+                    for (uint32_t j = 0; j < used; ++j) acc = combine(op, acc, ((const float*)bufs[order[j]])[i]);
+                    ((float*)result)[i] = acc; break; }
+                case DT_BF16: { float acc = identity_of<float>(op);
+                    for (uint32_t j = 0; j < used; ++j) acc = combine(op, acc, widen_bf16(((const uint16_t*)bufs[order[j]])[i]));
+                    ((float*)result)[i] = acc; break; }
+                case DT_I64: { int64_t acc = identity_of<int64_t>(op);
+                    for (uint32_t j = 0; j < used; ++j) acc = combine(op, acc, ((const int64_t*)bufs[order[j]])[i]);
+                    ((int64_t*)result)[i] = acc; break; }
+                case DT_F64: { double acc = identity_of<double>(op);
+                    for (uint32_t j = 0; j < used; ++j) acc = combine(op, acc, ((const double*)bufs[order[j]])[i]);
+                    ((double*)result)[i] = acc; break; }
+                default: return -1;
+            }
+        }
+        if (contrib_count) contrib_count[s] = used;
+        if (seg_clock) seg_clock[s] = oldest;
+        if (wait_count) wait_count[s] = waits;
+    }
+    return 0;
+}
+
+// ---------------------------------------------------------------------------
 // allgatherv: fixed slots from the counts of all ranks; notified ranks are copied,
 // the slots of the others are left as they were.
 // Returns 0, or 1 if the total exceeds out_capacity (then nothing is copied;
