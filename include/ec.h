@@ -133,6 +133,35 @@ int ec_allreduce_apply(ec_ctx_t* ctx, const void* const* rank_bufs, int P, size_
                        ec_op_t op, size_t segment_size, const uint64_t* arrival_mask, void* result,
                        uint32_t* contrib_count, ec_stream_t stream);
 
+/* Stale-synchronous apply (Sec. III-A, Algorithm 1 "allreduce_ssp").
+ *
+ * In the paper every process keeps, per communication step, the last contribution it received
+ * together with the logical clock (iteration number) in which that contribution was computed, and
+ * uses it instead of waiting as long as its clock is not below min_clock_accepted = clock - slack.
+ * Here rank r's buffer plays the part of that dedicated receive memory: it holds whatever rank r
+ * wrote last for a segment, and notif_clock says how old that is.
+ *
+ *   notif_clock    device uint32 [S][P]: clock of the contribution that rank_bufs[r] holds for
+ *                  segment s; 0 = nothing received yet.  Read on the device when the kernel runs.
+ *   clock, slack   the caller's current clock (>= 1) and the allowed staleness.
+ *   result         device, n output elements, written in full: per segment the reduction, in
+ *                  ascending rank order starting from the identity, of every contribution with
+ *                  notif_clock >= clock - slack (slack = 0 is the classic synchronous allreduce).
+ *   contrib_count  device uint32 [S] or NULL: number of contributions used.
+ *   seg_clock      device uint32 [S] or NULL: the clock of the reduction = the smallest clock among
+ *                  the contributions used (0 if none): "the result ... is associated with the
+ *                  minimum clock of both contributions".
+ *   wait_count     device uint32 [S] or NULL: contributions that were too stale (or absent).  The
+ *                  paper's process blocks on those; this call never waits - it reports them, and
+ *                  the caller applies again once they have been refreshed.
+ *
+ * The call keeps no state: it neither reads nor changes what ec_allreduce_apply has folded in.
+ * P, n, dtype, op, segment_size must equal the context's.  One kernel launch, no allocation. */
+int ec_allreduce_ssp_apply(ec_ctx_t* ctx, const void* const* rank_bufs, int P, size_t n, ec_dtype_t dtype,
+                           ec_op_t op, size_t segment_size, const uint32_t* notif_clock, uint32_t clock,
+                           uint32_t slack, void* result, uint32_t* contrib_count, uint32_t* seg_clock,
+                           uint32_t* wait_count, ec_stream_t stream);
+
 /* Start a new epoch: forget which contributions were folded in (the counterpart
  * of resetting notifications, Sec. II / Sec. IV-B).  `result` is not touched; the
  * next apply overwrites it. */

@@ -30,6 +30,7 @@ SYMBOLS = {
     "ec_allreduce_workspace_bytes": (_sz, [_i, _sz, _sz]),
     "ec_allreduce_init": (_i, [C.POINTER(_vp), _i, _sz, _i, _i, _sz, _i, _vp, _sz]),
     "ec_allreduce_apply": (_i, [_vp, _vp, _i, _sz, _i, _i, _sz, _vp, _vp, _vp, _vp]),
+    "ec_allreduce_ssp_apply": (_i, [_vp, _vp, _i, _sz, _i, _i, _sz, _vp, C.c_uint32, C.c_uint32, _vp, _vp, _vp, _vp, _vp]),
     "ec_allreduce_reset": (_i, [_vp, _vp]),
     "ec_allreduce_set_tile": (_i, [_vp, _i, _sz]),
     "ec_allreduce_destroy": (_i, [_vp]),
@@ -129,6 +130,14 @@ class Allreduce:
         """Same call with pre-marshalled arguments (for timing loops); returns the status code."""
         return lib().ec_allreduce_apply(self._h, table, self.P, self.n, self.dtype, self.op, self.seg,
                                         arrival_mask_ptr, result_ptr, count_ptr, stream_ptr)
+
+    def ssp_apply(self, rank_bufs, notif_clock, clock: int, slack: int, result, contrib_count=None, seg_clock=None,
+                  wait_count=None, stream=None) -> None:
+        """ec_allreduce_ssp_apply: stale-synchronous apply; notif_clock is a device uint32 [S][P] tensor."""
+        _check(lib().ec_allreduce_ssp_apply(self._h, _table(rank_bufs), len(rank_bufs), self.n, self.dtype, self.op,
+                                            self.seg, _ptr(notif_clock), clock, slack, _ptr(result),
+                                            _ptr(contrib_count), _ptr(seg_clock), _ptr(wait_count), _stream(stream)),
+               "ec_allreduce_ssp_apply")
 
     def reset(self, stream=None) -> None:
         _check(lib().ec_allreduce_reset(self._h, _stream(stream)), "ec_allreduce_reset")

@@ -143,6 +143,11 @@ struct ApplyArgs {
     unsigned tiles_per_seg;
     int P, W, first_apply;
     int res_hint;                // reserved: cache policy of the result accesses
+    // stale-synchronous mode: acceptance by clock instead of by notification bit (all nullptr / 0 otherwise)
+    const uint32_t* notif_clock; // [S][P] clock of the contribution each rank buffer holds; 0 = none
+    uint32_t min_clock;          // contributions with clock >= min_clock are accepted
+    uint32_t* seg_clock;         // [S] or nullptr: smallest clock among the accepted, 0 if none
+    uint32_t* wait_count;        // [S] or nullptr: ranks whose contribution is too stale
 };
 
 // Shape of the streaming loop, chosen by measurement on B200 (config 2 and 3 epochs): what counts
@@ -249,7 +254,31 @@ apply_kernel(const ApplyArgs a, const __grid_constant__ PtrTable<CAP> tbl) {
     if (threadIdx.x < 32) {
         const int lane = threadIdx.x;
         uint64_t nw = 0, old = 0;
-        if (lane < a.W) {
+        if (a.notif_clock != nullptr) {
+            // Stale-synchronous acceptance (Algorithm 1): a contribution takes part if its clock is not older
+            // than clock - slack.  32 ranks per step; the ballots of two steps make one 64-rank word.
+            uint32_t mn = 0xffffffffu;
+            int stale = 0;
+            for (int c = 0; c * 32 < a.P; ++c) {
+                const int r = c * 32 + lane;
+                const uint32_t ck = r < a.P ? a.notif_clock[(size_t)s * a.P + r] : 0u;
+                const bool ok = r < a.P && ck >= a.min_clock;
+                const unsigned bal = __ballot_sync(0xffffffffu, ok);
+                if (ok) mn = ck < mn ? ck : mn;
+                stale += (r < a.P && !ok) ? 1 : 0;
+                if (lane == (c >> 1)) nw |= (uint64_t)bal << ((c & 1) * 32);
+            }
+#pragma unroll
+            for (int d = 16; d > 0; d >>= 1) {
+                const uint32_t o = __shfl_xor_sync(0xffffffffu, mn, d);
+                mn = o < mn ? o : mn;
+                stale += __shfl_xor_sync(0xffffffffu, stale, d);
+            }
+            if (t == 0 && lane == 0) {
+                if (a.seg_clock) a.seg_clock[s] = mn == 0xffffffffu ? 0u : mn;   // the result is as old as its oldest input
+                if (a.wait_count) a.wait_count[s] = (uint32_t)stale;
+            }
+        } else if (lane < a.W) {
             uint64_t arr = a.arrival ? a.arrival[(size_t)s * a.W + lane] : ~0ull;
             if (lane == a.W - 1 && (a.P & 63)) arr &= (1ull << (a.P & 63)) - 1;   // bits >= P mean nothing
             // the first apply of an epoch starts from "nothing folded in": no need to clear the words
@@ -267,7 +296,7 @@ apply_kernel(const ApplyArgs a, const __grid_constant__ PtrTable<CAP> tbl) {
             total += __shfl_xor_sync(0xffffffffu, total, d);
         }
         if (t == 0) {
-            if (lane < a.W) a.applied_out[(size_t)s * a.W + lane] = old | nw;
+            if (lane < a.W && a.notif_clock == nullptr) a.applied_out[(size_t)s * a.W + lane] = old | nw;
             if (lane == 0 && a.contrib_count) a.contrib_count[s] = (uint32_t)total;
         }
         if (lane < MAX_W) s_new[lane] = nw;
@@ -557,9 +586,10 @@ int ec_allreduce_set_tile(ec_ctx_t* c, int threads, size_t tile_elems) {
     return EC_OK;
 }
 
-int ec_allreduce_apply(ec_ctx_t* c, const void* const* rank_bufs, int P, size_t n, ec_dtype_t dtype, ec_op_t op,
-                       size_t segment_size, const uint64_t* arrival_mask, void* result, uint32_t* contrib_count,
-                       ec_stream_t stream) {
+namespace {
+// Validation, tiling and launch shared by the notification-bit apply and the stale-synchronous apply.
+int apply_common(ec_ctx_t* c, const void* const* rank_bufs, int P, size_t n, ec_dtype_t dtype, ec_op_t op,
+                 size_t segment_size, void* result, ApplyArgs& a, ec_stream_t stream) {
     if (!c || !rank_bufs || !result) return EC_ERR_INVALID;
     if (P != c->P || n != c->n || (int)dtype != c->dtype || (int)op != c->op || segment_size != c->seg)
         return EC_ERR_INVALID;
@@ -571,29 +601,54 @@ int ec_allreduce_apply(ec_ctx_t* c, const void* const* rank_bufs, int P, size_t 
     const size_t seg_len = c->seg < c->n ? c->seg : c->n;
     const size_t tiles = (seg_len + c->tile - 1) / c->tile;
     if (tiles * c->S > 0x7fffffffull) return EC_ERR_CAPACITY;
-    ApplyArgs a;
     a.n = c->n; a.seg = c->seg; a.tile = c->tile;
+    a.result = result;
+    a.tiles_per_seg = (unsigned)tiles;
+    a.P = c->P; a.W = c->W;
+    a.res_hint = c->res_hint;
+    const unsigned grid = (unsigned)(tiles * c->S);
+    switch (c->dtype) {
+        case EC_F32: return launch_dt<EC_F32>(a, rank_bufs, c->op, vector, c->order, grid, c->threads, stream);
+        case EC_BF16: return launch_dt<EC_BF16>(a, rank_bufs, c->op, vector, c->order, grid, c->threads, stream);
+        case EC_I64: return launch_dt<EC_I64>(a, rank_bufs, c->op, vector, c->order, grid, c->threads, stream);
+        case EC_F64: return launch_dt<EC_F64>(a, rank_bufs, c->op, vector, c->order, grid, c->threads, stream);
+    }
+    return EC_ERR_INVALID;
+}
+}  // namespace
+
+int ec_allreduce_apply(ec_ctx_t* c, const void* const* rank_bufs, int P, size_t n, ec_dtype_t dtype, ec_op_t op,
+                       size_t segment_size, const uint64_t* arrival_mask, void* result, uint32_t* contrib_count,
+                       ec_stream_t stream) {
+    if (!c) return EC_ERR_INVALID;
+    ApplyArgs a = {};
     a.arrival = arrival_mask;
     a.applied_in = c->applied[c->cur];
     a.applied_out = c->applied[c->cur ^ 1];
-    a.result = result;
     a.contrib_count = contrib_count;
-    a.tiles_per_seg = (unsigned)tiles;
-    a.P = c->P; a.W = c->W; a.first_apply = c->first_apply ? 1 : 0;
-    a.res_hint = c->res_hint;
-    const unsigned grid = (unsigned)(tiles * c->S);
-    int rc;
-    switch (c->dtype) {
-        case EC_F32: rc = launch_dt<EC_F32>(a, rank_bufs, c->op, vector, c->order, grid, c->threads, stream); break;
-        case EC_BF16: rc = launch_dt<EC_BF16>(a, rank_bufs, c->op, vector, c->order, grid, c->threads, stream); break;
-        case EC_I64: rc = launch_dt<EC_I64>(a, rank_bufs, c->op, vector, c->order, grid, c->threads, stream); break;
-        case EC_F64: rc = launch_dt<EC_F64>(a, rank_bufs, c->op, vector, c->order, grid, c->threads, stream); break;
-        default: rc = EC_ERR_INVALID;
-    }
+    a.first_apply = c->first_apply ? 1 : 0;
+    const int rc = apply_common(c, rank_bufs, P, n, dtype, op, segment_size, result, a, stream);
     if (rc != EC_OK) return rc;
     c->cur ^= 1;
     c->first_apply = false;
     return EC_OK;
+}
+
+int ec_allreduce_ssp_apply(ec_ctx_t* c, const void* const* rank_bufs, int P, size_t n, ec_dtype_t dtype, ec_op_t op,
+                           size_t segment_size, const uint32_t* notif_clock, uint32_t clock, uint32_t slack,
+                           void* result, uint32_t* contrib_count, uint32_t* seg_clock, uint32_t* wait_count,
+                           ec_stream_t stream) {
+    if (!c || !notif_clock || clock == 0) return EC_ERR_INVALID;
+    ApplyArgs a = {};
+    a.applied_in = c->applied[c->cur];        // not used: this call keeps no state
+    a.applied_out = c->applied[c->cur ^ 1];
+    a.contrib_count = contrib_count;
+    a.first_apply = 1;                        // every segment is rebuilt from the identity
+    a.notif_clock = notif_clock;
+    a.min_clock = clock > slack ? clock - slack : 1u;   // clocks start at 1; 0 means "nothing received yet"
+    a.seg_clock = seg_clock;
+    a.wait_count = wait_count;
+    return apply_common(c, rank_bufs, P, n, dtype, op, segment_size, result, a, stream);
 }
 
 int ec_allreduce_reset(ec_ctx_t* c, ec_stream_t stream) {
