@@ -463,7 +463,38 @@ def extras(args, dev, stream, peak):
         ar.destroy()
         out[name] = entry
 
+    def ssp_case(name, P, n, seg, seed, sched_seed, p_first):
+        """Stale-synchronous apply on the config-2 shape: clocks 10 / 9 / 8 where the three-round schedule has
+        rounds 1 / 2 / 3; slack 0, 1, 2 accept about 70 %, 85 %, 100 % of the contributions."""
+        S = n // seg
+        h = inputs.rank_buffers("normal_f32", seed, P, n)
+        d = [torch.from_numpy(b).to(dev) for b in h]
+        del h
+        rounds = inputs.arrival_rounds(sched_seed, P, S, p_first)
+        clocks = (10 - (rounds.T - 1)).astype(np.uint32)
+        d_clocks = torch.from_numpy(clocks.view(np.int32)).to(dev)
+        res = torch.empty(n, dtype=torch.float32, device=dev)
+        cnt = torch.empty(S, dtype=torch.int32, device=dev)
+        clk = torch.empty(S, dtype=torch.int32, device=dev)
+        wait = torch.empty(S, dtype=torch.int32, device=dev)
+        ar = ec.Allreduce(P, n, ec.F32, ec.SUM, seg, device=dev)
+        table = (C.c_void_p * P)(*[t.data_ptr() for t in d])
+        entry = {}
+        for slack in (0, 1, 2):
+            accepted = int((clocks >= 10 - slack).sum())
+            nbytes = accepted * seg * 4 + n * 4 + S * P * 4 + 3 * S * 4
+            ms = time_calls(stream, lambda: L.ec_allreduce_ssp_apply(ar._h, table, P, n, ec.F32, ec.SUM, seg,
+                                                                     d_clocks.data_ptr(), 10, slack, res.data_ptr(),
+                                                                     cnt.data_ptr(), clk.data_ptr(), wait.data_ptr(), st), reps)
+            m, ci = mean_ci(ms)
+            entry[f"slack{slack}"] = {"ms": round(m, 5), "ci95": round(ci, 5), "GBps": round(nbytes / m / 1e6, 1),
+                                      "frac_measured": round(nbytes / m / 1e6 / peak, 4), "bytes": nbytes,
+                                      "accepted_fraction": round(accepted / (S * P), 4)}
+        ar.destroy()
+        out[name] = entry
+
     allreduce_case("config1_P4_f32_n2^20", 4, 1 << 20, 16384, ec.F32, "uniform_f32", 1001, 0, 1.0, 1)
+    ssp_case("ssp_apply_P16_f32_n2^24", 16, 1 << 24, 65536, 1002, 2002, 0.7)
     allreduce_case("config2_P16_f32_n2^24_all_at_once", 16, 1 << 24, 65536, ec.F32, "normal_f32", 1002, 2002, 0.7, 1)
     allreduce_case("config3_P32_bf16_n2^25", 32, 1 << 25, 131072, ec.BF16, "normal_bf16", 1003, 2003, 0.9, 3, sigma=1e-3)
     allreduce_case("config3_P32_bf16_n2^25_pairwise", 32, 1 << 25, 131072, ec.BF16, "normal_bf16", 1003, 2003, 0.9, 1,

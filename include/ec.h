@@ -298,6 +298,29 @@ int ec_kmeans_destroy(ec_kmeans_t* km);
 int ec_kmeans_partials_static(const float* points, const int32_t* labels, size_t N, int D, int K, int P,
                               float* partials, ec_stream_t stream);
 
+/* ------------------------------------------------------------------------- *
+ * Threshold variants of Reduce / Broadcast (Sec. III-B) as notification words,
+ * and the threshold test on the status output (Sec. III: "threshold" and
+ * "status" parameters).  host_mask is HOST memory, uint64 [S][W], written.
+ * ------------------------------------------------------------------------- */
+
+/* Strategy 1, "send less data": the first ceil(fraction * S) segments of every rank count as
+ * arrived, the others do not.  0 <= fraction <= 1. */
+int ec_mask_data_fraction(int P, size_t S, double fraction, uint64_t* host_mask);
+
+/* Strategy 2, "send all data but leave processes out": the binomial spanning tree works in stages
+ * that double the number of involved processes (stage k brings in ranks 2^k .. 2^(k+1)-1); whole
+ * stages are added until at least fraction * P processes take part.  Ranks 0 .. *ranks_included-1
+ * count as arrived for every segment.  The last stage alone adds half of the processes, so
+ * fractions 0.75 and 1.0 select the same set, as the paper observes.  ranks_included may be NULL. */
+int ec_mask_process_threshold(int P, size_t S, double fraction, uint64_t* host_mask, int* ranks_included);
+
+/* The threshold test: *ready_segments (device word, written) = number of segments whose
+ * contrib_count (device uint32 [S], as written by an apply) is at least `need`; the collective has
+ * reached a threshold theta when that equals S with need = ceil(theta * P).  One launch, one block. */
+int ec_threshold_segments(const uint32_t* contrib_count, size_t S, uint32_t need, uint32_t* ready_segments,
+                          ec_stream_t stream);
+
 /* ------------------------------------------------------------------------- */
 const char* ec_strerror(int code);
 /* The cudaError_t of the last failed CUDA call on this thread (0 if none). */

@@ -244,3 +244,63 @@ def kmeans_iterate(points: np.ndarray, centroids: np.ndarray, P: int, arrival_ma
     ar.apply([partials[r].reshape(-1) for r in range(P)], arrival_mask, reduced, count)
     reduced = reduced.reshape(K, D + 4)
     return kmeans_update(reduced, centroids), labels, reduced, count
+
+
+# ---------------------------------------------------------------------------
+# Threshold variants of Reduce / Broadcast (Sec. III-B), written out plainly.
+# ---------------------------------------------------------------------------
+def bst_stage_of_rank(rank: int) -> int:
+    """Stage of the binomial spanning tree in which a rank receives its data (root: -1).
+    The tree works in stages that double the number of involved processes: after stage k the
+    ranks 0 .. 2^(k+1)-1 are involved, so rank r > 0 joins in stage floor(log2 r)."""
+    if rank == 0:
+        return -1
+    stage = 0
+    while (1 << (stage + 1)) <= rank:
+        stage += 1
+    return stage
+
+
+def bst_parent(rank: int) -> int:
+    """Parent in the binomial tree: the children of p are p + 2^i for the stages i after p joined
+    (-1 for the root)."""
+    if rank == 0:
+        return -1
+    return rank - (1 << bst_stage_of_rank(rank))
+
+
+def process_threshold_ranks(P: int, fraction: float) -> int:
+    """Number of ranks involved when whole stages are added until at least fraction*P take part."""
+    involved = 1 if fraction > 0 else 0
+    stage = 0
+    while 0 < involved < P and involved < fraction * P:
+        involved = min(P, sum(1 for r in range(P) if bst_stage_of_rank(r) <= stage))
+        stage += 1
+    return involved
+
+
+def process_threshold_mask(P: int, S: int, fraction: float) -> np.ndarray:
+    arrived = np.zeros((P, S), dtype=bool)
+    arrived[:process_threshold_ranks(P, fraction)] = True
+    return _pack_words(arrived)
+
+
+def data_fraction_mask(P: int, S: int, fraction: float) -> np.ndarray:
+    import math
+    arrived = np.zeros((P, S), dtype=bool)
+    arrived[:, :min(S, math.ceil(fraction * S))] = True
+    return _pack_words(arrived)
+
+
+def _pack_words(arrived: np.ndarray) -> np.ndarray:
+    P, S = arrived.shape
+    out = np.zeros((S, (P + 63) // 64), dtype=np.uint64)
+    for s in range(S):
+        for r in range(P):
+            if arrived[r, s]:
+                out[s, r // 64] |= np.uint64(1 << (r % 64))
+    return out
+
+
+def threshold_segments(contrib_count: np.ndarray, need: int) -> int:
+    return int(sum(1 for c in contrib_count if c >= need))

@@ -46,6 +46,9 @@ SYMBOLS = {
     "ec_kmeans_tc_status": (_i, [_vp, _vp, _vp]),
     "ec_kmeans_destroy": (_i, [_vp]),
     "ec_kmeans_partials_static": (_i, [_vp, _vp, _sz, _i, _i, _i, _vp, _vp]),
+    "ec_mask_data_fraction": (_i, [_i, _sz, C.c_double, _vp]),
+    "ec_mask_process_threshold": (_i, [_i, _sz, C.c_double, _vp, C.POINTER(_i)]),
+    "ec_threshold_segments": (_i, [_vp, _sz, C.c_uint32, _vp, _vp]),
     "ec_strerror": (C.c_char_p, [_i]),
     "ec_last_cuda_error": (_i, []),
     "ec_version": (_i, []),
@@ -229,3 +232,26 @@ def kmeans_partials_static(points: torch.Tensor, labels: torch.Tensor, K: int, P
     N, D = points.shape
     _check(lib().ec_kmeans_partials_static(_ptr(points), _ptr(labels), N, D, K, P, _ptr(partials), _stream(stream)),
            "ec_kmeans_partials_static")
+
+
+def mask_data_fraction(P: int, S: int, fraction: float):
+    """ec_mask_data_fraction: host notification words (numpy uint64 [S][W]) with the first ceil(fraction*S) segments set."""
+    import numpy as np
+    out = np.zeros((S, (P + 63) // 64), dtype=np.uint64)
+    _check(lib().ec_mask_data_fraction(P, S, fraction, out.ctypes.data), "ec_mask_data_fraction")
+    return out
+
+
+def mask_process_threshold(P: int, S: int, fraction: float):
+    """ec_mask_process_threshold: (host notification words, number of ranks the binomial-tree stages bring in)."""
+    import numpy as np
+    out = np.zeros((S, (P + 63) // 64), dtype=np.uint64)
+    n = C.c_int(0)
+    _check(lib().ec_mask_process_threshold(P, S, fraction, out.ctypes.data, C.byref(n)), "ec_mask_process_threshold")
+    return out, n.value
+
+
+def threshold_segments(contrib_count, need: int, ready, stream=None) -> None:
+    """ec_threshold_segments: ready[0] = number of segments whose contributor count is at least `need` (device tensors)."""
+    _check(lib().ec_threshold_segments(_ptr(contrib_count), contrib_count.numel(), need, _ptr(ready), _stream(stream)),
+           "ec_threshold_segments")
