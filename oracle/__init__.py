@@ -18,7 +18,7 @@ _LIB = os.path.join(_HERE, "libec_oracle.so")
 
 F32, BF16, I64, F64 = 0, 1, 2, 3
 SUM, MAX, MIN = 0, 1, 2
-ORDER_FIXED, ORDER_PAIRWISE = 0, 1
+ORDER_FIXED, ORDER_PAIRWISE, ORDER_RING = 0, 1, 2
 
 _IN_NP = {F32: np.float32, BF16: np.uint16, I64: np.int64, F64: np.float64}
 _OUT_NP = {F32: np.float32, BF16: np.float32, I64: np.int64, F64: np.float64}

@@ -36,6 +36,8 @@
 //   int64 sum  wraps modulo 2^64;
 //   float max  acc = (x > acc) ? x : acc   (min: x < acc);
 //   bf16       raw bits widened exactly (bits << 16); arithmetic and output fp32;
+//   ring       the vector is cut into P chunks of ceil(n/P) elements; chunk c is folded over the ranks
+//              c, c+1, ..., c-1 (mod P), the order of the ring's Scatter-Reduce (Sec. IV-A);
 //   pairwise   balanced binary tree over the rank index, P padded to a power of
 //              two, absent ranks contribute the identity; a segment that already
 //              holds a partial result gets the tree's root added onto it.
@@ -62,7 +64,7 @@ namespace {
 
 enum { DT_F32 = 0, DT_BF16 = 1, DT_I64 = 2, DT_F64 = 3 };
 enum { OP_SUM = 0, OP_MAX = 1, OP_MIN = 2 };
-enum { ORDER_FIXED = 0, ORDER_PAIRWISE = 1 };
+enum { ORDER_FIXED = 0, ORDER_PAIRWISE = 1, ORDER_RING = 2 };
 
 inline bool notified(const uint64_t* mask, size_t W, size_t s, int r) {
     if (mask == nullptr) return true;  // no mask: every contribution has arrived
@@ -164,7 +166,20 @@ void apply_typed(AllreduceState* st, const void* const* bufs, const uint64_t* ma
         }
         // (3) fold the newly notified ranks
         if (has_new) {
-            if (order == ORDER_FIXED) {
+            if (order == ORDER_RING) {
+                // Scatter-Reduce of the segmented ring (Sec. IV-A): in step k node i sends chunk i-k and
+                // receives chunk i-k-1, reducing it into its own data.  Chunk c therefore starts at node c
+                // (step 0) and is reduced by nodes c+1, c+2, ... in turn: ranks c, c+1, ..., c-1 (mod P).
+                const size_t chunk_len = (st->n + (size_t)P - 1) / (size_t)P;
+                size_t c = lo / chunk_len;
+                if (c > (size_t)(P - 1)) c = (size_t)(P - 1);
+                for (int step = 0; step < P; ++step) {
+                    const int r = (int)((c + (size_t)step) % (size_t)P);
+                    if (!take[(size_t)r]) continue;
+                    const In* buf = (const In*)bufs[r];
+                    for (size_t i = lo; i < hi; ++i) result[i] = combine(st->op, result[i], T::widen(buf[i]));
+                }
+            } else if (order == ORDER_FIXED) {
                 for (int r = 0; r < P; ++r) {
                     if (!take[(size_t)r]) continue;
                     const In* buf = (const In*)bufs[r];
