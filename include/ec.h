@@ -55,7 +55,13 @@ typedef enum {
 
 typedef enum {
     EC_ORDER_FIXED = 0,   /* each apply folds its new ranks in ascending rank order: reproducible bits */
-    EC_ORDER_PAIRWISE = 1 /* balanced tree over the rank index (float sum only): smaller rounding error */
+    EC_ORDER_PAIRWISE = 1, /* balanced tree over the rank index (float sum only): smaller rounding error; for P a power
+                              of two this is the order of the hypercube allreduce of Sec. III-A (recursive doubling) */
+    EC_ORDER_RING = 2      /* the order of the segmented pipelined ring (Sec. IV-A, Scatter-Reduce): the vector is cut
+                              into P chunks of ceil(n/P) elements; chunk c is first sent by node c and reduced by nodes
+                              c+1, c+2, ... in turn, so its fold runs over the ranks c, c+1, ..., P-1, 0, ..., c-1
+                              (each apply folds its new ranks in that cyclic order).  segment_size must divide
+                              ceil(n/P) (EC_ERR_INVALID otherwise) */
 } ec_order_t;
 
 enum {

@@ -16,7 +16,7 @@ LIB_PATH = os.path.join(_HERE, "libec_b200.so")
 
 F32, BF16, I64, F64 = 0, 1, 2, 3
 SUM, MAX, MIN = 0, 1, 2
-ORDER_FIXED, ORDER_PAIRWISE = 0, 1
+ORDER_FIXED, ORDER_PAIRWISE, ORDER_RING = 0, 1, 2
 MAX_RANKS = 1024
 
 OK, ERR_INVALID, ERR_UNSUPPORTED, ERR_CUDA, ERR_STATE, ERR_CAPACITY = 0, -1, -2, -3, -4, -5

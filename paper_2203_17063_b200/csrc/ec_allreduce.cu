@@ -148,6 +148,7 @@ struct ApplyArgs {
     uint32_t min_clock;          // contributions with clock >= min_clock are accepted
     uint32_t* seg_clock;         // [S] or nullptr: smallest clock among the accepted, 0 if none
     uint32_t* wait_count;        // [S] or nullptr: ranks whose contribution is too stale
+    size_t ring_chunk;           // ring order: elements per 1/P chunk of the vector (0 = plain rank order)
 };
 
 // Shape of the streaming loop, chosen by measurement on B200 (config 2 and 3 epochs): what counts
@@ -300,12 +301,28 @@ apply_kernel(const ApplyArgs a, const __grid_constant__ PtrTable<CAP> tbl) {
             if (lane == 0 && a.contrib_count) a.contrib_count[s] = (uint32_t)total;
         }
         if (lane < MAX_W) s_new[lane] = nw;
+        // Ring order (Scatter-Reduce of the segmented ring, Sec. IV-A): chunk c of the vector is first sent by
+        // node c and reduced by nodes c+1, c+2, ... in turn, so its fold starts at rank c and wraps around.
+        // The ascending list is rotated: the j0 ranks below c go to the end.
+        const int m_all = __shfl_sync(0xffffffffu, incl, 31);
+        int j0 = 0;
+        if (a.ring_chunk != 0) {
+            size_t c = ((size_t)s * a.seg) / a.ring_chunk;
+            if (c > (size_t)(a.P - 1)) c = (size_t)(a.P - 1);
+            const int rel = (int)c - lane * 64;                       // ranks of this word below c
+            const uint64_t below = rel <= 0 ? 0ull : rel >= 64 ? ~0ull : (1ull << rel) - 1;
+            j0 = __popcll(nw & below);
+#pragma unroll
+            for (int d = 16; d > 0; d >>= 1) j0 += __shfl_xor_sync(0xffffffffu, j0, d);
+        }
         int j = incl - cnt_new;
         uint64_t bits = nw;
         while (bits) {
             const int b = __ffsll((long long)bits) - 1;
             bits &= bits - 1;
-            s_rank[j++] = (uint16_t)(lane * 64 + b);
+            const int pos = j >= j0 ? j - j0 : j + (m_all - j0);
+            s_rank[pos] = (uint16_t)(lane * 64 + b);
+            ++j;
         }
         if (lane == 31) s_m = incl;
         if (lane == 0) s_fresh = (any_old == 0) ? 1 : 0;
@@ -471,7 +488,7 @@ int launch_cap(const ApplyArgs& a, const void* const* bufs, unsigned grid, int t
 template <int DT, int OP>
 int launch_op(const ApplyArgs& a, const void* const* bufs, bool vector, int order, unsigned grid, int threads,
               cudaStream_t st) {
-    if (order == EC_ORDER_FIXED)
+    if (order == EC_ORDER_FIXED || order == EC_ORDER_RING)     // ring order = rank order rotated per chunk (a.ring_chunk)
         return vector ? launch_cap<DT, OP, true, EC_ORDER_FIXED>(a, bufs, grid, threads, st)
                       : launch_cap<DT, OP, false, EC_ORDER_FIXED>(a, bufs, grid, threads, st);
     if constexpr (OP == EC_SUM && DT != EC_I64)
@@ -532,7 +549,9 @@ int ec_allreduce_init(ec_ctx_t** out, int P, size_t n, ec_dtype_t dtype, ec_op_t
     *out = nullptr;
     if (bad_shape(P, n, segment_size)) return EC_ERR_INVALID;
     if ((int)dtype < 0 || (int)dtype > EC_F64 || (int)op < 0 || (int)op > EC_MIN) return EC_ERR_INVALID;
-    if ((int)order != EC_ORDER_FIXED && (int)order != EC_ORDER_PAIRWISE) return EC_ERR_INVALID;
+    if ((int)order != EC_ORDER_FIXED && (int)order != EC_ORDER_PAIRWISE && (int)order != EC_ORDER_RING) return EC_ERR_INVALID;
+    // ring order: the vector is cut into P chunks of ceil(n/P) elements; a segment must lie inside one chunk
+    if (order == EC_ORDER_RING && ((n + (size_t)P - 1) / (size_t)P) % segment_size != 0) return EC_ERR_INVALID;
     if (order == EC_ORDER_PAIRWISE && (op != EC_SUM || dtype == EC_I64)) return EC_ERR_UNSUPPORTED;
     const size_t need = ec_allreduce_workspace_bytes(P, n, segment_size);
     if (workspace && (workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 255u))) return EC_ERR_CAPACITY;
@@ -606,6 +625,7 @@ int apply_common(ec_ctx_t* c, const void* const* rank_bufs, int P, size_t n, ec_
     a.tiles_per_seg = (unsigned)tiles;
     a.P = c->P; a.W = c->W;
     a.res_hint = c->res_hint;
+    a.ring_chunk = c->order == EC_ORDER_RING ? (c->n + (size_t)c->P - 1) / (size_t)c->P : 0;
     const unsigned grid = (unsigned)(tiles * c->S);
     switch (c->dtype) {
         case EC_F32: return launch_dt<EC_F32>(a, rank_bufs, c->op, vector, c->order, grid, c->threads, stream);

@@ -290,3 +290,21 @@ def test_library_allocated_workspace():
     ref.apply(bufs, None, c, None)
     assert np.array_equal(bits(to_host(res)), bits(c))
     assert L.ec_allreduce_destroy(h) == ec.OK
+
+
+@pytest.mark.parametrize("P,n,seg", [(4, 1 << 16, 1024), (16, 1 << 20, 4096), (70, 70 * 3000, 1000), (5, 100, 10), (256, 256 * 512, 512)])
+def test_ring_order_matches_checker_bits(P, n, seg):
+    """EC_ORDER_RING: chunk c of the vector is folded over the ranks c, c+1, ..., c-1 (Scatter-Reduce of the ring)."""
+    S = (n + seg - 1) // seg
+    bufs = _bufs("normal_f32", 950 + P, P, n)
+    masks = inputs.cumulative_masks(inputs.arrival_rounds(951 + P, P, S, 0.6))
+    run_schedule(P, n, seg, ec.F32, ec.SUM, bufs, masks, order=ec.ORDER_RING)
+    run_schedule(P, n, seg, ec.F32, ec.SUM, bufs, [None], order=ec.ORDER_RING, tile=(64, 96))
+    b16 = _bufs("normal_bf16", 960 + P, P, n, sigma=1.0)
+    run_schedule(P, n, seg, ec.BF16, ec.SUM, b16, masks, order=ec.ORDER_RING)
+
+
+def test_ring_order_needs_segments_inside_chunks():
+    with pytest.raises(ec.EcError) as err:
+        ec.Allreduce(4, 1000, ec.F32, ec.SUM, 64, ec.ORDER_RING)        # ceil(1000/4) = 250 is not a multiple of 64
+    assert err.value.code == ec.ERR_INVALID
