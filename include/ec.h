@@ -208,6 +208,28 @@ int ec_allgatherv(const void* const* bufs, const int64_t* counts, int P, ec_dtyp
                   uint32_t* status, ec_stream_t stream);
 
 /* ------------------------------------------------------------------------- *
+ * Eventually consistent AlltoAll (Sec. IV-B): every rank writes its d-th block
+ * into rank d's receive memory, each write with a notification of its own; the
+ * receiver uses what has been notified and the collective is complete once all
+ * P blocks of every receiver have arrived.
+ *
+ *   send_bufs      HOST array of P DEVICE pointers: rank s's P blocks of
+ *                  block_bytes bytes, block d destined for rank d.
+ *   recv_bufs      HOST array of P DEVICE pointers: rank d's P slots of
+ *                  block_bytes bytes; slot s receives the block from rank s.
+ *                  No receive buffer may be a send buffer.
+ *   arrival_mask   device uint64 [P][W]: row d = destination, bit s = the block
+ *                  from rank s has arrived; NULL = all.  Slots whose bit is
+ *                  clear are left untouched (a late block is one more call with
+ *                  its bit set).
+ *   recv_count     device uint32 [P] or NULL: notified blocks per destination
+ *                  (= P when that rank's AlltoAll is complete).
+ * Stateless; one kernel launch; 128-bit copies when block_bytes and all pointers
+ * are multiples of 16, byte-wise otherwise. */
+int ec_alltoall(const void* const* send_bufs, void* const* recv_bufs, int P, size_t block_bytes,
+                const uint64_t* arrival_mask, uint32_t* recv_count, ec_stream_t stream);
+
+/* ------------------------------------------------------------------------- *
  * K-means driver: Lloyd iterations whose combine step is the allreduce above.
  * (The paper's iterative-convergent ML workload is a matrix factorisation on a
  * data set that is not available; K-means takes its place as the data-parallel

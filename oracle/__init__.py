@@ -57,6 +57,8 @@ def lib() -> C.CDLL:
         L.oracle_allreduce_ssp.restype = C.c_int
         L.oracle_allreduce_ssp.argtypes = [C.c_int, C.c_size_t, C.c_int, C.c_int, C.c_size_t, C.c_void_p, C.c_void_p,
                                            C.c_uint32, C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.oracle_alltoall.restype = C.c_int
+        L.oracle_alltoall.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_size_t, C.c_void_p, C.c_void_p]
         L.oracle_allgatherv.restype = C.c_int
         L.oracle_allgatherv.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_size_t, C.c_void_p,
                                         C.c_void_p, C.c_void_p, C.c_size_t]
@@ -191,6 +193,23 @@ def allgatherv(bufs, counts: np.ndarray, arrival_mask, out: np.ndarray):
     status = lib().oracle_allgatherv(table, _ptr(counts), P, out.dtype.itemsize, _ptr(arrival_mask),
                                      _ptr(displs), _ptr(out), out.size)
     return displs, int(status)
+
+
+def alltoall(send_bufs, recv_bufs, block_bytes: int, arrival_mask=None) -> np.ndarray:
+    """recv_bufs[d] block s <- send_bufs[s] block d for every notified (d, s), in place (uint8 arrays of
+    P * block_bytes bytes); returns recv_count uint32 [P]."""
+    P = len(send_bufs)
+    for b in list(send_bufs) + list(recv_bufs):
+        assert b.dtype == np.uint8 and b.flags.c_contiguous and b.size >= P * block_bytes
+    st = (C.c_void_p * P)(*[b.ctypes.data for b in send_bufs])
+    rt = (C.c_void_p * P)(*[b.ctypes.data for b in recv_bufs])
+    if arrival_mask is not None:
+        arrival_mask = np.ascontiguousarray(arrival_mask, dtype=np.uint64)
+    count = np.empty(P, dtype=np.uint32)
+    rc = lib().oracle_alltoall(st, rt, P, block_bytes, _ptr(arrival_mask), _ptr(count))
+    if rc != 0:
+        raise RuntimeError("oracle_alltoall failed")
+    return count
 
 
 def kmeans_assign(points: np.ndarray, centroids: np.ndarray, threads: int = 1):

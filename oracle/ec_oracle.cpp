@@ -394,6 +394,30 @@ int oracle_allgatherv(const void* const* bufs, const int64_t* counts, int P, siz
 }
 
 // ---------------------------------------------------------------------------
+// AlltoAll (Sec. IV-B): every rank writes its d-th block into rank d's memory, each write with its
+// own notification; the receiver uses what has been notified.  arrival_mask: uint64 [P][W], row d
+// = destination, bit s = the block from source s has arrived (NULL = all).  Blocks that have not
+// arrived are left as they were.  recv_count[d] = notified blocks of destination d.
+// ---------------------------------------------------------------------------
+int oracle_alltoall(const void* const* send_bufs, void* const* recv_bufs, int P, size_t block_bytes,
+                    const uint64_t* arrival_mask, uint32_t* recv_count) {
+    if (!send_bufs || !recv_bufs || P < 1 || block_bytes == 0) return -1;
+    const size_t W = (size_t)(P + 63) / 64;
+    for (int d = 0; d < P; ++d) {
+        uint32_t got = 0;
+        for (int s = 0; s < P; ++s) {
+            if (!notified(arrival_mask, W, (size_t)d, s)) continue;
+            ++got;
+            const unsigned char* src = (const unsigned char*)send_bufs[s] + (size_t)d * block_bytes;
+            unsigned char* dst = (unsigned char*)recv_bufs[d] + (size_t)s * block_bytes;
+            for (size_t b = 0; b < block_bytes; ++b) dst[b] = src[b];
+        }
+        if (recv_count) recv_count[d] = got;
+    }
+    return 0;
+}
+
+// ---------------------------------------------------------------------------
 // K-means (textbook Lloyd iteration; the data-parallel ML workload that stands
 // in for the paper's iterative-convergent solver).  Distances in double.
 // ---------------------------------------------------------------------------

@@ -46,6 +46,7 @@ SYMBOLS = {
     "ec_kmeans_tc_status": (_i, [_vp, _vp, _vp]),
     "ec_kmeans_destroy": (_i, [_vp]),
     "ec_kmeans_partials_static": (_i, [_vp, _vp, _sz, _i, _i, _i, _vp, _vp]),
+    "ec_alltoall": (_i, [_vp, _vp, _i, _sz, _vp, _vp, _vp]),
     "ec_mask_data_fraction": (_i, [_i, _sz, C.c_double, _vp]),
     "ec_mask_process_threshold": (_i, [_i, _sz, C.c_double, _vp, C.POINTER(_i)]),
     "ec_threshold_segments": (_i, [_vp, _sz, C.c_uint32, _vp, _vp]),
@@ -255,3 +256,9 @@ def threshold_segments(contrib_count, need: int, ready, stream=None) -> None:
     """ec_threshold_segments: ready[0] = number of segments whose contributor count is at least `need` (device tensors)."""
     _check(lib().ec_threshold_segments(_ptr(contrib_count), contrib_count.numel(), need, _ptr(ready), _stream(stream)),
            "ec_threshold_segments")
+
+
+def alltoall(send_bufs, recv_bufs, block_bytes: int, arrival_mask=None, recv_count=None, stream=None) -> None:
+    """ec_alltoall: recv[d] block s <- send[s] block d for every notified (d, s); device tensors."""
+    _check(lib().ec_alltoall(_table(send_bufs), _table(recv_bufs), len(send_bufs), block_bytes, _ptr(arrival_mask),
+                             _ptr(recv_count), _stream(stream)), "ec_alltoall")
