@@ -501,6 +501,27 @@ def extras(args, dev, stream, peak):
                    order=ec.ORDER_PAIRWISE, sigma=1e-3)
     allreduce_case("config4_P256_i64_n2^20", 256, 1 << 20, 8192, ec.I64, "int64_below", 1004, 2004, 0.8, 2, bound=1 << 20)
 
+    # AlltoAll at the paper's largest message size: 64 ranks (16 nodes x 4 processes), 32 KiB per block
+    P, B = 64, 32768
+    g = torch.Generator(device="cpu").manual_seed(77)
+    a_send = [torch.randint(0, 256, (P * B,), dtype=torch.uint8, generator=g).to(dev) for _ in range(P)]
+    a_recv = [torch.empty(P * B, dtype=torch.uint8, device=dev) for _ in range(P)]
+    a_cnt = torch.empty(P, dtype=torch.int32, device=dev)
+    a_mask = torch.from_numpy(inputs.pack_mask(inputs.bernoulli_mask(2006, 0, P, P, 0.8).T.copy()).view(np.int64)).to(dev)
+    st_tbl = (C.c_void_p * P)(*[t.data_ptr() for t in a_send])
+    rt_tbl = (C.c_void_p * P)(*[t.data_ptr() for t in a_recv])
+    entry = {}
+    for label, mptr, frac in (("all_arrived", None, 1.0), ("80pct_arrived", a_mask.data_ptr(), None)):
+        ms = time_calls(stream, lambda: L.ec_alltoall(st_tbl, rt_tbl, P, B, mptr, a_cnt.data_ptr(), st), reps)
+        m, ci = mean_ci(ms)
+        blocks = P * P if mptr is None else int(a_cnt.sum().item())
+        nbytes = 2 * blocks * B
+        entry[label] = {"ms": round(m, 5), "ci95": round(ci, 5), "GBps": round(nbytes / m / 1e6, 1),
+                        "frac_measured": round(nbytes / m / 1e6 / peak, 4), "bytes": nbytes}
+    entry["note"] = "read + write of every notified block; 2 x 128 MiB working set, partly L2-resident when repeated"
+    out["alltoall_P64_32KiB_blocks"] = entry
+    del a_send, a_recv
+
     # config 4 gather
     P = 256
     counts = inputs.gather_counts(1004, P)
