@@ -60,6 +60,50 @@ alltoall_kernel(const A2AArgs a, const __grid_constant__ A2ATables<CAP> t) {
     }
 }
 
+// Blocks of at least a few KB: one thread block copies one 8 KB piece of one (destination, source) block,
+// so the index arithmetic happens once per piece and every thread keeps two 128-bit loads in flight.
+constexpr size_t A2A_PIECE = 8192;
+
+template <int CAP>
+__global__ void __launch_bounds__(256)
+alltoall_piece_kernel(const A2AArgs a, const __grid_constant__ A2ATables<CAP> t) {
+    const int P = a.P;
+    if (blockIdx.x == 0 && a.recv_count != nullptr) {
+        for (int d = threadIdx.x; d < P; d += blockDim.x) {
+            unsigned c = 0;
+            for (int w = 0; w < a.W; ++w) {
+                uint64_t word = a.arrival ? a.arrival[(size_t)d * a.W + w] : ~0ull;
+                const int hi = P - w * 64;
+                if (hi < 64) word &= hi <= 0 ? 0ull : (1ull << hi) - 1;
+                c += (unsigned)__popcll(word);
+            }
+            a.recv_count[d] = c;
+        }
+    }
+    const uint64_t pol = evict_first_policy();
+    const size_t pieces = (a.block_bytes + A2A_PIECE - 1) / A2A_PIECE;
+    const size_t items = pieces * (size_t)P * (size_t)P;
+    for (size_t it = blockIdx.x; it < items; it += gridDim.x) {
+        const size_t pair = it / pieces, piece = it - pair * pieces;
+        const size_t d = pair / (size_t)P, s = pair - d * (size_t)P;
+        if (a.arrival) {
+            const uint64_t word = a.arrival[d * (size_t)a.W + (s >> 6)];
+            if (!((word >> (s & 63)) & 1ull)) continue;    // not notified: never read, block untouched
+        }
+        const size_t off = piece * A2A_PIECE;
+        const size_t len = a.block_bytes - off < A2A_PIECE ? a.block_bytes - off : A2A_PIECE;   // multiple of 16
+        const char* src = reinterpret_cast<const char*>(t.send[s]) + d * a.block_bytes + off;
+        char* dst = reinterpret_cast<char*>(t.recv[d]) + s * a.block_bytes + off;
+        const size_t nvec = len / 16;
+        const size_t v0 = threadIdx.x, v1 = threadIdx.x + 256;
+        uint4 r0, r1;
+        if (v0 < nvec) r0 = ld_stream16(src + v0 * 16, pol);
+        if (v1 < nvec) r1 = ld_stream16(src + v1 * 16, pol);
+        if (v0 < nvec) st_plain16(dst + v0 * 16, r0);
+        if (v1 < nvec) st_plain16(dst + v1 * 16, r1);
+    }
+}
+
 template <int CAP>
 int launch(const A2AArgs& a, const void* const* send, void* const* recv, bool vec, cudaStream_t st) {
     A2ATables<CAP> t;
@@ -74,7 +118,11 @@ int launch(const A2AArgs& a, const void* const* send, void* const* recv, bool ve
     const size_t cap = (size_t)sms * 16;
     if (blocks > cap) blocks = cap;
     if (blocks < 1) blocks = 1;
-    if (vec) alltoall_kernel<CAP, 16><<<(unsigned)blocks, 256, 0, st>>>(a, t);
+    if (vec && a.block_bytes >= 2048) {
+        const size_t items = ((a.block_bytes + A2A_PIECE - 1) / A2A_PIECE) * (size_t)a.P * (size_t)a.P;
+        size_t pb = items < (size_t)sms * 32 ? items : (size_t)sms * 32;
+        alltoall_piece_kernel<CAP><<<(unsigned)pb, 256, 0, st>>>(a, t);
+    } else if (vec) alltoall_kernel<CAP, 16><<<(unsigned)blocks, 256, 0, st>>>(a, t);
     else alltoall_kernel<CAP, 1><<<(unsigned)blocks, 256, 0, st>>>(a, t);
     EC_CUDA(cudaGetLastError());
     return EC_OK;
