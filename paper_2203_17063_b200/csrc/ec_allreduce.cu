@@ -183,7 +183,7 @@ constexpr int TREE_LEVELS = 7;  // 1024 ranks / 8 per leaf block = 128 blocks = 
 // Loads are independent and issued together; the adds of one vector stay in ascending rank order.
 template <int DT, int OP, int VPT, int RUN>
 __device__ __forceinline__ void fold_vectors(const char* const* s_ptr, int m, typename Elem<DT>::Acc* res, size_t nvec,
-                                             bool fresh, int tid, int nthr, uint64_t pol, uint64_t rpol) {
+                                             bool fresh, int tid, int nthr, uint64_t pol, uint64_t rpol_ld, uint64_t rpol_st) {
     typedef Elem<DT> E;
     typedef typename E::Acc Acc;
     constexpr int VEC = E::VEC;
@@ -196,7 +196,7 @@ __device__ __forceinline__ void fold_vectors(const char* const* s_ptr, int m, ty
 #pragma unroll
                 for (int e = 0; e < VEC; ++e) acc[p][e] = ident<OP>(Acc());
             } else {
-                load_acc<Acc, VEC>(res + v * VEC, acc[p], rpol);
+                load_acc<Acc, VEC>(res + v * VEC, acc[p], rpol_ld);
             }
         }
         for (int j = 0; j < m; j += RUN) {
@@ -225,7 +225,7 @@ __device__ __forceinline__ void fold_vectors(const char* const* s_ptr, int m, ty
 #pragma unroll
         for (int p = 0; p < VPT; ++p) {
             const size_t v = v0 + (size_t)p * nthr;
-            if (v < nvec) store_acc<Acc, VEC>(res + v * VEC, acc[p], rpol);
+            if (v < nvec) store_acc<Acc, VEC>(res + v * VEC, acc[p], rpol_st);
         }
     }
 }
@@ -339,7 +339,10 @@ apply_kernel(const ApplyArgs a, const __grid_constant__ PtrTable<CAP> tbl) {
     Acc* res = reinterpret_cast<Acc*>(a.result) + lo;
     const int tid = threadIdx.x, nthr = blockDim.x;
     const uint64_t pol = evict_first_policy();
-    const uint64_t rpol = result_policy(a.res_hint);
+    // Result accesses (measured on config 2 and 3 epochs): loads always keep the line in L2 (evict-last: the
+    // next round reads it again); stores keep it too when the whole result fits in L2, and let it go at once
+    // (evict-first) when it cannot fit anyway.
+    const uint64_t rpol_ld = result_policy(1), rpol_st = result_policy(a.res_hint == 2 ? 2 : 1);
 
     if (ORDER == EC_ORDER_FIXED) {
         for (int j = tid; j < m; j += nthr)
@@ -351,9 +354,9 @@ apply_kernel(const ApplyArgs a, const __grid_constant__ PtrTable<CAP> tbl) {
         // With hundreds of ranks a round rarely brings that few: the wide-table variant keeps the
         // single shape.
         constexpr int LATE = EC_LATE_VPT, MID = EC_MID_VPT;
-        if (CAP <= 64 && m <= EC_LATE_RU) fold_vectors<DT, OP, LATE, EC_LATE_RU>(s_ptr, m, res, nvec, fresh, tid, nthr, pol, rpol);
-        else if (CAP <= 64 && m <= EC_MID_RU) fold_vectors<DT, OP, MID, EC_MID_RU>(s_ptr, m, res, nvec, fresh, tid, nthr, pol, rpol);
-        else fold_vectors<DT, OP, 1, (CAP > 64 ? 8 : EC_MAIN_RU)>(s_ptr, m, res, nvec, fresh, tid, nthr, pol, rpol);   // hundreds of ranks: 8 loads in flight measured best
+        if (CAP <= 64 && m <= EC_LATE_RU) fold_vectors<DT, OP, LATE, EC_LATE_RU>(s_ptr, m, res, nvec, fresh, tid, nthr, pol, rpol_ld, rpol_st);
+        else if (CAP <= 64 && m <= EC_MID_RU) fold_vectors<DT, OP, MID, EC_MID_RU>(s_ptr, m, res, nvec, fresh, tid, nthr, pol, rpol_ld, rpol_st);
+        else fold_vectors<DT, OP, 1, (CAP > 64 ? 8 : EC_MAIN_RU)>(s_ptr, m, res, nvec, fresh, tid, nthr, pol, rpol_ld, rpol_st);   // hundreds of ranks: 8 loads in flight measured best
         // element-wise path: everything when the 128-bit path does not apply, else the ragged tail
         for (size_t i = nvec * VEC + tid; i < cnt; i += nthr) {
             Acc acc = fresh ? ident<OP>(Acc()) : res[i];
@@ -458,11 +461,11 @@ apply_kernel(const ApplyArgs a, const __grid_constant__ PtrTable<CAP> tbl) {
             if (isvec) {
                 if (!fresh) {
                     Acc acc[PV];
-                    load_acc<Acc, PV>(res + e0, acc, rpol);
+                    load_acc<Acc, PV>(res + e0, acc, rpol_ld);
 #pragma unroll
                     for (int e = 0; e < PV; ++e) node[e] = comb<OP>(acc[e], node[e]);
                 }
-                store_acc<Acc, PV>(res + e0, node, rpol);
+                store_acc<Acc, PV>(res + e0, node, rpol_st);
             } else {
                 res[e0] = fresh ? node[0] : comb<OP>(res[e0], node[0]);
             }
@@ -576,13 +579,11 @@ int ec_allreduce_init(ec_ctx_t** out, int P, size_t n, ec_dtype_t dtype, ec_op_t
     c->applied[1] = reinterpret_cast<uint64_t*>(reinterpret_cast<char*>(c->ws) + need / 2);
     c->cur = 0;
     c->first_apply = true;
-    // A partial result that fits in L2 is kept there for the next round (evict-last: +2 % per epoch
-    // measured on 64 MiB); one that cannot fit is streamed through instead (evict-first).
     {
         int dev = 0, l2 = 0;
         if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&l2, cudaDevAttrL2CacheSize, dev) != cudaSuccess)
             l2 = 0;
-        c->res_hint = (double)n * (double)out_bytes(dtype) <= 0.75 * (double)l2 ? 1 : 2;
+        c->res_hint = (double)n * (double)out_bytes(dtype) <= 0.75 * (double)l2 ? 1 : 2;   // does the result fit in L2?
     }
     // Few ranks: many small blocks overlap their start-up latency best.  Hundreds of ranks: a block
     // lives long anyway and wider blocks read longer contiguous runs of each buffer (both measured).
