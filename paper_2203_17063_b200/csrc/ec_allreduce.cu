@@ -142,7 +142,7 @@ struct ApplyArgs {
     uint32_t* contrib_count;     // [S] or nullptr
     unsigned tiles_per_seg;
     int P, W, first_apply;
-    int res_hint;                // reserved: cache policy of the result accesses
+    int res_hint;                // 1: the result fits in L2 (stores keep it there), 2: it does not (stores stream out)
     // stale-synchronous mode: acceptance by clock instead of by notification bit (all nullptr / 0 otherwise)
     const uint32_t* notif_clock; // [S][P] clock of the contribution each rank buffer holds; 0 = none
     uint32_t min_clock;          // contributions with clock >= min_clock are accepted

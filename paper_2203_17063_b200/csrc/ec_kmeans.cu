@@ -5,14 +5,20 @@
 // of points, forms per-centroid partial sums, and the partial sums are combined by one allreduce
 // epoch in which only the notified (rank, centroid-row) contributions take part.
 //
-// Kernels:
-//   assign    one thread per point, the point's coordinates in registers, centroids staged in
-//             shared memory and read as broadcasts; squared distance sum_d (x-c)^2 in fp32;
-//             bound by the fp32 pipes, not by memory.
-//   partials  one warp walks a contiguous run of points with lane = coordinate and keeps
-//             [K][D] running sums in its own shared-memory slab: plain read-add-write, no
-//             atomics, fixed order.  Warps, then blocks of a rank are folded in index order.
-//   update    centroid = sum / points where points > 0.
+// Kernels, fastest first (ec_kmeans_iterate takes the first that covers the shape):
+//   tc::tc_fused_kernel   (ec_kmeans_tc.cuh) assignment and partial sums as two small GEMMs on the
+//             tensor cores, exact fp32 re-decision of every point the bf16 search cannot separate;
+//             D in {16, 32}, K <= 256; bound by reading the points once.
+//   fused_kernel          the same two steps on the fp32 pipes: one FMA per (point, centroid,
+//             coordinate) proposes, the exact form decides inside the error bound; per-warp
+//             shared-memory slabs collect the sums in a fixed order; D in {8, 16, 32, 64}.
+//   assign_kernel / assign_generic_kernel, partials_kernel   one step each, any D that is a multiple
+//             of 4: squared distance sum_d (x-c)^2 in fp32 with the point in registers; one warp
+//             walks a run of points with lane = coordinate into its own [K][D] slab.  These also
+//             serve ec_kmeans_partials (and ec_kmeans_assign for shapes the fused kernels skip).
+//   partials_fold_kernel  folds the row blocks of a rank in index order;
+//   update_kernel         centroid = sum / points where points > 0.
+// No floating-point atomics on any of these paths: sums are the same bits run after run.
 
 #include <new>
 
