@@ -207,6 +207,15 @@ int ec_allgatherv(const void* const* bufs, const int64_t* counts, int P, ec_dtyp
                   const uint64_t* arrival_mask, int64_t* displs, void* out, size_t out_capacity_elems,
                   uint32_t* status, ec_stream_t stream);
 
+/* The other reading of "packed": only the ranks that have arrived get a slot, so the
+ * arrived contributions are contiguous from out[0] on.  displs is the exclusive prefix sum
+ * of (arrived ? counts[r] : 0); displs[P] = number of elements gathered.  Unlike the fixed-slot
+ * form above, a rank that arrives later moves every slot behind it, so a later call rewrites
+ * the whole output from the then-current notification word.  Same arguments and status rules. */
+int ec_allgatherv_compact(const void* const* bufs, const int64_t* counts, int P, ec_dtype_t dtype,
+                          const uint64_t* arrival_mask, int64_t* displs, void* out, size_t out_capacity_elems,
+                          uint32_t* status, ec_stream_t stream);
+
 /* ------------------------------------------------------------------------- *
  * Eventually consistent AlltoAll (Sec. IV-B): every rank writes its d-th block
  * into rank d's receive memory, each write with a notification of its own; the

@@ -57,6 +57,9 @@ def lib() -> C.CDLL:
         L.oracle_allreduce_ssp.restype = C.c_int
         L.oracle_allreduce_ssp.argtypes = [C.c_int, C.c_size_t, C.c_int, C.c_int, C.c_size_t, C.c_void_p, C.c_void_p,
                                            C.c_uint32, C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.oracle_allgatherv_compact.restype = C.c_int
+        L.oracle_allgatherv_compact.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_size_t, C.c_void_p,
+                                                C.c_void_p, C.c_void_p, C.c_size_t]
         L.oracle_alltoall.restype = C.c_int
         L.oracle_alltoall.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_size_t, C.c_void_p, C.c_void_p]
         L.oracle_allgatherv.restype = C.c_int
@@ -178,8 +181,9 @@ def allreduce_ssp(bufs, dtype: int, op: int, segment_size: int, notif_clock: np.
     return result, count, seg_clock, wait
 
 
-def allgatherv(bufs, counts: np.ndarray, arrival_mask, out: np.ndarray):
-    """Returns (displs int64 [P+1], status); copies notified ranks into ``out`` in place."""
+def allgatherv(bufs, counts: np.ndarray, arrival_mask, out: np.ndarray, compact: bool = False):
+    """Returns (displs int64 [P+1], status); copies notified ranks into ``out`` in place.
+    compact=False: fixed slots from the counts of all ranks; compact=True: only notified ranks get a slot."""
     P = len(bufs)
     counts = np.ascontiguousarray(counts, dtype=np.int64)
     keep = [np.ascontiguousarray(b) for b in bufs]
@@ -190,8 +194,8 @@ def allgatherv(bufs, counts: np.ndarray, arrival_mask, out: np.ndarray):
         arrival_mask = np.ascontiguousarray(arrival_mask, dtype=np.uint64)
     displs = np.empty(P + 1, dtype=np.int64)
     assert out.flags.c_contiguous
-    status = lib().oracle_allgatherv(table, _ptr(counts), P, out.dtype.itemsize, _ptr(arrival_mask),
-                                     _ptr(displs), _ptr(out), out.size)
+    fn = lib().oracle_allgatherv_compact if compact else lib().oracle_allgatherv
+    status = fn(table, _ptr(counts), P, out.dtype.itemsize, _ptr(arrival_mask), _ptr(displs), _ptr(out), out.size)
     return displs, int(status)
 
 

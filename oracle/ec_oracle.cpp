@@ -393,6 +393,26 @@ int oracle_allgatherv(const void* const* bufs, const int64_t* counts, int P, siz
     return 0;
 }
 
+// The compact reading of "packed": only notified ranks get a slot; the gathered contributions are
+// contiguous from out[0] on.  displs[r+1] - displs[r] = counts[r] if rank r is notified, else 0.
+int oracle_allgatherv_compact(const void* const* bufs, const int64_t* counts, int P, size_t elem_bytes,
+                              const uint64_t* arrival_mask, int64_t* displs, void* out, size_t out_capacity) {
+    int64_t running = 0;
+    for (int r = 0; r < P; ++r) {
+        displs[r] = running;
+        if (notified(arrival_mask, 1, 0, r)) running += counts[r];
+    }
+    displs[P] = running;
+    if ((uint64_t)running > (uint64_t)out_capacity) return 1;
+    unsigned char* o = (unsigned char*)out;
+    for (int r = 0; r < P; ++r) {
+        if (!notified(arrival_mask, 1, 0, r)) continue;
+        const unsigned char* src = (const unsigned char*)bufs[r];
+        for (size_t b = 0; b < (size_t)counts[r] * elem_bytes; ++b) o[(size_t)displs[r] * elem_bytes + b] = src[b];
+    }
+    return 0;
+}
+
 // ---------------------------------------------------------------------------
 // AlltoAll (Sec. IV-B): every rank writes its d-th block into rank d's memory, each write with its
 // own notification; the receiver uses what has been notified.  arrival_mask: uint64 [P][W], row d

@@ -46,6 +46,7 @@ SYMBOLS = {
     "ec_kmeans_tc_status": (_i, [_vp, _vp, _vp]),
     "ec_kmeans_destroy": (_i, [_vp]),
     "ec_kmeans_partials_static": (_i, [_vp, _vp, _sz, _i, _i, _i, _vp, _vp]),
+    "ec_allgatherv_compact": (_i, [_vp, _vp, _i, _i, _vp, _vp, _vp, _sz, _vp, _vp]),
     "ec_alltoall": (_i, [_vp, _vp, _i, _sz, _vp, _vp, _vp]),
     "ec_mask_data_fraction": (_i, [_i, _sz, C.c_double, _vp]),
     "ec_mask_process_threshold": (_i, [_i, _sz, C.c_double, _vp, C.POINTER(_i)]),
@@ -162,10 +163,12 @@ class Allreduce:
 
 
 def allgatherv(bufs, counts, dtype: int, arrival_mask, displs, out, status, stream=None,
-               out_capacity_elems: int | None = None) -> None:
-    """ec_allgatherv: counts/displs/out/status are device tensors, bufs a list of device tensors (or None)."""
+               out_capacity_elems: int | None = None, compact: bool = False) -> None:
+    """ec_allgatherv (fixed slots) or ec_allgatherv_compact (only arrived ranks get a slot):
+    counts/displs/out/status are device tensors, bufs a list of device tensors (or None)."""
     cap = out.numel() if out_capacity_elems is None else out_capacity_elems
-    _check(lib().ec_allgatherv(_table(bufs), _ptr(counts), len(bufs), dtype, _ptr(arrival_mask), _ptr(displs),
+    fn = lib().ec_allgatherv_compact if compact else lib().ec_allgatherv
+    _check(fn(_table(bufs), _ptr(counts), len(bufs), dtype, _ptr(arrival_mask), _ptr(displs),
                                _ptr(out), cap, _ptr(status), _stream(stream)), "ec_allgatherv")
 
 

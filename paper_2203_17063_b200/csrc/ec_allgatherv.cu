@@ -27,6 +27,7 @@ struct GatherArgs {
     uint32_t* status;
     size_t capacity;           // elements
     int P, esize;              // element size in bytes
+    int compact;               // 1: only the ranks that have arrived get a slot
 };
 
 template <class T>
@@ -98,6 +99,7 @@ allgatherv_kernel(const GatherArgs a, const __grid_constant__ PtrTable<CAP> tbl)
     for (int i = 0; i < ITEMS; ++i) {
         const int r = tid * ITEMS + i;
         long long c = (r < P && r < CAP) ? a.counts[r] : 0;
+        if (a.compact && r < P && !((s_arr[r >> 6] >> (r & 63)) & 1ull)) c = 0;   // compact reading: no slot for a missing rank
         if (c < 0) { neg = true; c = 0; }
         cnt[i] = c;
         local += c;
@@ -200,9 +202,9 @@ void launch(const GatherArgs& a, const void* const* bufs, unsigned grid, cudaStr
 
 using namespace ec;
 
-extern "C" int ec_allgatherv(const void* const* bufs, const int64_t* counts, int P, ec_dtype_t dtype,
-                             const uint64_t* arrival_mask, int64_t* displs, void* out, size_t out_capacity_elems,
-                             uint32_t* status, ec_stream_t stream) {
+namespace {
+int gather_common(const void* const* bufs, const int64_t* counts, int P, ec_dtype_t dtype, const uint64_t* arrival_mask,
+                  int64_t* displs, void* out, size_t out_capacity_elems, uint32_t* status, int compact, cudaStream_t stream) {
     if (!bufs || !counts || !displs || !status || P < 1 || P > EC_MAX_RANKS) return EC_ERR_INVALID;
     if ((int)dtype < 0 || (int)dtype > EC_F64) return EC_ERR_INVALID;
     if (!out && out_capacity_elems != 0) return EC_ERR_INVALID;
@@ -214,7 +216,7 @@ extern "C" int ec_allgatherv(const void* const* bufs, const int64_t* counts, int
     // device, so this cannot be checked here); the kernel dereferences neither.
     GatherArgs a;
     a.counts = counts; a.arrival = arrival_mask; a.displs = displs; a.out = reinterpret_cast<char*>(out);
-    a.status = status; a.capacity = out_capacity_elems; a.P = P; a.esize = es;
+    a.status = status; a.capacity = out_capacity_elems; a.P = P; a.esize = es; a.compact = compact;
     // enough blocks for every chunk the capacity allows, at most eight per SM (the blocks loop)
     size_t chunks = (out_capacity_elems * (size_t)es + GV_CHUNK_BYTES - 1) / GV_CHUNK_BYTES;
     if (chunks < 1) chunks = 1;
@@ -225,4 +227,17 @@ extern "C" int ec_allgatherv(const void* const* bufs, const int64_t* counts, int
     else launch<EC_MAX_RANKS>(a, bufs, grid, stream);
     EC_CUDA(cudaGetLastError());
     return EC_OK;
+}
+}  // namespace
+
+extern "C" int ec_allgatherv(const void* const* bufs, const int64_t* counts, int P, ec_dtype_t dtype,
+                             const uint64_t* arrival_mask, int64_t* displs, void* out, size_t out_capacity_elems,
+                             uint32_t* status, ec_stream_t stream) {
+    return gather_common(bufs, counts, P, dtype, arrival_mask, displs, out, out_capacity_elems, status, 0, stream);
+}
+
+extern "C" int ec_allgatherv_compact(const void* const* bufs, const int64_t* counts, int P, ec_dtype_t dtype,
+                                     const uint64_t* arrival_mask, int64_t* displs, void* out,
+                                     size_t out_capacity_elems, uint32_t* status, ec_stream_t stream) {
+    return gather_common(bufs, counts, P, dtype, arrival_mask, displs, out, out_capacity_elems, status, 1, stream);
 }

@@ -123,3 +123,23 @@ def test_large_contributions_span_many_chunks():
     bufs = inputs.gather_buffers(9, counts)
     g, gd, gs, c, cd, cs = gather_both(bufs, counts, ec.I64, [True, False, True])
     assert gs == 0 and np.array_equal(g, c)
+
+
+@pytest.mark.parametrize("P", [3, 64, 200])
+def test_compact_variant_matches_checker(P):
+    rng = np.random.default_rng(40 + P)
+    counts = rng.integers(0, 3000, size=P).astype(np.int64)
+    bufs = [rng.integers(-2 ** 63, 2 ** 63 - 1, size=int(c), dtype=np.int64) for c in counts]
+    arrived = rng.random(P) < 0.6
+    mask = inputs.pack_mask(arrived[:, None]).reshape(-1)
+    cap = int(counts.sum())
+    c_out = np.full(cap, SENT, dtype=np.int64)
+    c_displs, c_status = oracle.allgatherv(bufs, counts, mask, c_out, compact=True)
+    d_out = to_dev(np.full(cap, SENT, dtype=np.int64))
+    d_displs = torch.empty(P + 1, dtype=torch.int64, device="cuda")
+    d_status = torch.empty(1, dtype=torch.int32, device="cuda")
+    ec.allgatherv([to_dev(b) for b in bufs], to_dev(counts), ec.I64, to_dev(mask), d_displs, d_out, d_status, compact=True)
+    torch.cuda.synchronize()
+    assert int(d_status.item()) == 0 == c_status
+    assert np.array_equal(d_displs.cpu().numpy(), c_displs)
+    assert np.array_equal(to_host(d_out), c_out)

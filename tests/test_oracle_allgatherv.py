@@ -83,3 +83,24 @@ def test_other_element_sizes():
         out = np.zeros(8, dtype=dt)
         oracle.allgatherv(bufs, counts, None, out)
         assert np.array_equal(out, np.concatenate(bufs))
+
+
+def test_compact_reading_is_the_concatenation_of_the_arrived_ranks():
+    P = 70
+    rng = np.random.default_rng(8)
+    counts = rng.integers(0, 30, size=P).astype(np.int64)
+    bufs = [rng.integers(0, 1000, size=int(c), dtype=np.int64) for c in counts]
+    arrived = rng.random(P) < 0.6
+    total = int(counts[arrived].sum())
+    out = np.full(total + 3, SENT, dtype=np.int64)
+    displs, status = oracle.allgatherv(bufs, counts, mask_words(arrived), out, compact=True)
+    assert status == 0
+    assert np.array_equal(out[:total], np.concatenate([b for b, a in zip(bufs, arrived) if a]))
+    assert (out[total:] == SENT).all()
+    assert displs[0] == 0 and np.array_equal(np.diff(displs), np.where(arrived, counts, 0))
+    # with everything arrived both readings coincide
+    out2 = np.empty(int(counts.sum()), dtype=np.int64)
+    d1, _ = oracle.allgatherv(bufs, counts, None, out2, compact=True)
+    out3 = np.empty_like(out2)
+    d2, _ = oracle.allgatherv(bufs, counts, None, out3)
+    assert np.array_equal(d1, d2) and np.array_equal(out2, out3)
