@@ -276,6 +276,12 @@ int ec_kmeans_partials(ec_kmeans_t* km, const int32_t* labels, float* partials, 
  * uint64 [K][W] for this iteration, NULL = all arrived. */
 int ec_kmeans_iterate(ec_kmeans_t* km, const uint64_t* arrival_mask, ec_stream_t stream);
 
+/* The same iteration with the combine step spread over several rounds: one allreduce epoch with
+ * `rounds` applies (1..64) before the centroid update.  arrival_masks is a HOST array of `rounds`
+ * DEVICE pointers to cumulative notification words [K][W] (an entry may be NULL = all arrived);
+ * rows that are late in round 1 still count if a later round of the same iteration sees them. */
+int ec_kmeans_iterate_rounds(ec_kmeans_t* km, const uint64_t* const* arrival_masks, int rounds, ec_stream_t stream);
+
 /* Replace the context's centroids (device [K][D]); used for lock-step checks. */
 int ec_kmeans_set_centroids(ec_kmeans_t* km, const float* centroids, ec_stream_t stream);
 

@@ -264,7 +264,9 @@ def kmeans_iterate(points: np.ndarray, centroids: np.ndarray, P: int, arrival_ma
     ar = Allreduce(P, n, F32, SUM, D + 4)
     reduced = np.empty(n, dtype=np.float32)
     count = np.empty(K, dtype=np.uint32)
-    ar.apply([partials[r].reshape(-1) for r in range(P)], arrival_mask, reduced, count)
+    masks = arrival_mask if isinstance(arrival_mask, (list, tuple)) else [arrival_mask]
+    for m in masks:                       # several cumulative masks = several rounds of one epoch before the update
+        ar.apply([partials[r].reshape(-1) for r in range(P)], m, reduced, count)
     reduced = reduced.reshape(K, D + 4)
     return kmeans_update(reduced, centroids), labels, reduced, count
 

@@ -40,6 +40,7 @@ SYMBOLS = {
     "ec_kmeans_assign": (_i, [_vp, _vp, _vp, _vp]),
     "ec_kmeans_partials": (_i, [_vp, _vp, _vp, _vp]),
     "ec_kmeans_iterate": (_i, [_vp, _vp, _vp]),
+    "ec_kmeans_iterate_rounds": (_i, [_vp, _vp, _i, _vp]),
     "ec_kmeans_set_centroids": (_i, [_vp, _vp, _vp]),
     "ec_kmeans_get": (_i, [_vp, _vp, _vp, _vp, _vp, _vp]),
     "ec_kmeans_set_path": (_i, [_vp, _i]),
@@ -197,6 +198,11 @@ class KMeans:
 
     def iterate(self, arrival_mask=None, stream=None) -> None:
         _check(lib().ec_kmeans_iterate(self._h, _ptr(arrival_mask), _stream(stream)), "ec_kmeans_iterate")
+
+    def iterate_rounds(self, arrival_masks, stream=None) -> None:
+        """One iteration whose allreduce epoch has len(arrival_masks) applies (cumulative device masks)."""
+        _check(lib().ec_kmeans_iterate_rounds(self._h, _table(arrival_masks), len(arrival_masks), _stream(stream)),
+               "ec_kmeans_iterate_rounds")
 
     def iterate_raw(self, mask_ptr, stream_ptr) -> int:
         return lib().ec_kmeans_iterate(self._h, mask_ptr, stream_ptr)

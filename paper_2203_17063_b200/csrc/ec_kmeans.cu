@@ -767,8 +767,23 @@ int ec_kmeans_partials(ec_kmeans_t* km, const int32_t* labels, float* partials, 
     return km_partials(km, labels, partials, stream);
 }
 
+namespace {
+int km_iterate_rounds(ec_kmeans_t* km, const uint64_t* const* masks, int rounds, ec_stream_t stream);
+}
+
 int ec_kmeans_iterate(ec_kmeans_t* km, const uint64_t* arrival_mask, ec_stream_t stream) {
     if (!km) return EC_ERR_INVALID;
+    const uint64_t* one[1] = {arrival_mask};
+    return km_iterate_rounds(km, one, 1, stream);
+}
+
+int ec_kmeans_iterate_rounds(ec_kmeans_t* km, const uint64_t* const* arrival_masks, int rounds, ec_stream_t stream) {
+    if (!km || !arrival_masks || rounds < 1 || rounds > 64) return EC_ERR_INVALID;
+    return km_iterate_rounds(km, arrival_masks, rounds, stream);
+}
+
+namespace {
+int km_iterate_rounds(ec_kmeans_t* km, const uint64_t* const* masks, int rounds, ec_stream_t stream) {
     int rc;
     if (km->Cf > 0) {
         // assignment and per-block partial sums in one pass over the points, then the rows of a rank in order
@@ -789,14 +804,17 @@ int ec_kmeans_iterate(ec_kmeans_t* km, const uint64_t* arrival_mask, ec_stream_t
     rc = ec_allreduce_reset(km->ar, stream);
     if (rc != EC_OK) return rc;
     const size_t stride = (size_t)km->D + 4;
-    rc = ec_allreduce_apply(km->ar, km->bufs, km->P, (size_t)km->K * stride, EC_F32, EC_SUM, stride, arrival_mask,
-                            km->reduced, km->contrib, stream);
-    if (rc != EC_OK) return rc;
+    for (int t = 0; t < rounds; ++t) {     // one epoch: the first round builds the partial result, the others fold late rows in
+        rc = ec_allreduce_apply(km->ar, km->bufs, km->P, (size_t)km->K * stride, EC_F32, EC_SUM, stride, masks[t],
+                                km->reduced, km->contrib, stream);
+        if (rc != EC_OK) return rc;
+    }
     const int total = km->K * km->D;
     update_kernel<<<(total + 255) / 256, 256, 0, stream>>>(km->reduced, km->D, km->K, km->centroids);
     EC_CUDA(cudaGetLastError());
     return EC_OK;
 }
+}  // namespace
 
 int ec_kmeans_set_centroids(ec_kmeans_t* km, const float* centroids, ec_stream_t stream) {
     if (!km || !centroids) return EC_ERR_INVALID;

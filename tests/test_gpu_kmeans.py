@@ -154,3 +154,27 @@ def test_full_size_config5_one_iteration_sampled():
     mean = points[sel].astype(np.float64).mean(0)
     assert np.linalg.norm(to_host(d_cent)[k] - mean) <= 1e-4 * np.linalg.norm(mean)
     km.destroy()
+
+
+def test_iteration_with_two_rounds_matches_checker():
+    """Late rows of round 1 are folded in by round 2 of the same iteration, before the centroid update."""
+    N, D, K, P = 1 << 15, 32, 64, 64
+    points, comp, _ = inputs.kmeans_mixture(1005, N, D, K)
+    cents = inputs.kmeans_first_of_component(points, comp, K)
+    rounds = inputs.arrival_rounds(77, P, K, 0.75, last_round=2)             # [P][K] -> 1 or 2
+    masks = inputs.cumulative_masks(rounds)
+    km = ec.KMeans(to_dev(points), K, P, to_dev(cents))
+    km.iterate_rounds([to_dev(m) for m in masks])
+    d_cent = torch.empty(K, D, device="cuda")
+    d_red = torch.empty(K, D + 4, device="cuda")
+    d_cnt = torch.empty(K, dtype=torch.int32, device="cuda")
+    km.get(d_cent, None, d_red, d_cnt)
+    torch.cuda.synchronize()
+    new, labels, c_red, c_cnt = oracle.kmeans_iterate(points, cents, P, masks, 8)
+    assert (c_cnt == P).all() and np.array_equal(to_host(d_cnt).view(np.uint32), c_cnt)
+    assert np.array_equal(to_host(d_red)[:, D], c_red[:, D])
+    assert rows_close(to_host(d_cent), new)
+    # with both rounds every point counts: the centroids are the plain cluster means
+    means = np.stack([points[labels == k].astype(np.float64).mean(0) for k in range(K)])
+    assert rows_close(to_host(d_cent), means.astype(np.float32))
+    km.destroy()
