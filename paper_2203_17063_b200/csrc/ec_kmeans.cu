@@ -536,10 +536,16 @@ bool km_plan(size_t N, int D, int K, int P, int sms, KmLayout* L) {
     while (C > 1 && shard / (size_t)C < 256) --C;            // keep runs long enough to be worth a block
     L->C = C;
     L->warps = warps;
-    // fused kernel: runs of four tiles (2048 points); thousands of short blocks fill the SMs evenly
+    // fused kernels: runs of about 2048 points, their number rounded to whole waves of resident blocks
+    // (four per SM) so that the last wave is as full as the others
     L->Cf = 0;
     if (fused_capable(D, K)) {
-        size_t cf = shard / (4 * (size_t)FU_TILE);
+        const size_t slots = (size_t)sms * 4;
+        const size_t target = N / 2048 > 0 ? N / 2048 : 1;
+        size_t waves = (target + slots / 2) / slots;
+        if (waves < 1) waves = 1;
+        size_t cf = waves * slots / (size_t)P;
+        while (cf > 1 && shard / cf < 512) --cf;            // keep runs long enough to be worth a block
         L->Cf = (int)(cf < 1 ? 1 : cf > 64 ? 64 : cf);
     }
     const size_t stride = (size_t)D + 4;

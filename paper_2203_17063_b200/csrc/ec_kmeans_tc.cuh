@@ -273,13 +273,12 @@ tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const 
     const size_t b0 = j0 + len * c / C, b1 = j0 + len * (c + 1) / C;
     const int stride = D + 4;
     float* row_block = PARTIALS ? scratch + ((size_t)r * C + c) * (size_t)K * stride : nullptr;
-    if (PARTIALS)
-        for (int i = tid; i < K * stride; i += THREADS) row_block[i] = 0.0f;   // base of the by-hand adds, should they be needed
     uint32_t phase1 = 0, phase2 = 0;
     bool healthy = true;             // false once a wait on the tensor core gave up: plain fp32 from then on
     bool sums_started = false;       // a sums MMA has been issued (the accumulator holds data)
     bool sums_pending = false;       // ... and its completion has not been waited for yet
     int prev_chunk = -1;             // one-hot chunk this thread set in the previous tile
+    bool by_hand = false;            // some points were added to the row block with atomic adds
 
     // A thread stages KCH items (point row, chunk kc of 8 coordinates) of a tile: consecutive threads take
     // consecutive 32-byte pieces of the points, so every load instruction of a warp covers 1 KB of contiguous
@@ -343,7 +342,6 @@ tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const 
         }
         if (base + TILE < b1) issue_loads(base + TILE);
         fence_async_smem();          // the tensor core reads shared memory through the async proxy
-        fence_before_sync();
         healthy = __syncthreads_and(healthy) != 0;
         if (tid == 0 && healthy) {
             fence_after_sync();
@@ -358,6 +356,11 @@ tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const 
         bool done = healthy && mbar_wait_bounded(bar1, phase1);
         phase1 ^= 1u;
         done = __syncthreads_and(done) != 0;     // all threads take the same path
+        if (PARTIALS && !done && !by_hand) {     // first tile without the tensor core: clear the base of the by-hand adds
+            for (int i = tid; i < K * stride; i += THREADS) row_block[i] = 0.0f;
+            by_hand = true;
+            __syncthreads();
+        }
         healthy = done;
         fence_after_sync();
         float m1 = __int_as_float(0x7f800000), m2 = m1;
@@ -402,7 +405,6 @@ tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const 
                 *reinterpret_cast<uint4*>(s_oh + (size_t)prev_chunk * OCHUNK + (size_t)tid * 16) = make_uint4(wv[0], wv[1], wv[2], wv[3]);
             }
             fence_async_smem();
-            fence_before_sync();
             __syncthreads();
             if (tid == 0) {
                 fence_after_sync();
@@ -433,7 +435,7 @@ tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const 
         // The low rows go through shared memory (the one-hot tile is free now) to the thread of their coordinate.
         if (ok && sums_started) {
             float* s_lo = reinterpret_cast<float*>(s_oh);          // [npad][D] floats <= npad/8 * 2048 bytes for D <= 32... (D*4 <= 256)
-            const bool is_hi = tid < D, is_cnt = tid == D, is_lo = tid >= 64 && tid < 64 + D;
+            const bool is_hi = tid < D, is_cnt = tid == D, is_pad = tid > D && tid < D + 4, is_lo = tid >= 64 && tid < 64 + D;
             for (int ch = 0; ch < npad / 32; ++ch) {
                 uint32_t v[32];
                 tmem_ld32(tmem_lane + (uint32_t)(npad + ch * 32), v);
@@ -442,22 +444,24 @@ tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const 
                     for (int e = 0; e < 32; ++e) s_lo[(size_t)(ch * 32 + e) * D + (tid - 64)] = __uint_as_float(v[e]);
                 }
                 __syncthreads();
-                if (is_hi || is_cnt) {
+                if (is_hi || is_cnt || is_pad) {
 #pragma unroll
                     for (int e = 0; e < 32; ++e) {
                         const int k = ch * 32 + e;
                         if (k < K) {
-                            float val = __uint_as_float(v[e]);
+                            float val = is_pad ? 0.0f : __uint_as_float(v[e]);
                             if (is_hi) val = __fadd_rn(val, s_lo[(size_t)k * D + tid]);
-                            float* dst = row_block + (size_t)k * stride + tid;   // column tid: coordinate, or D = the count
-                            if (healthy) *dst = val;
-                            else atomicAdd(dst, val);                             // some tiles were added by hand
+                            float* dst = row_block + (size_t)k * stride + tid;   // column tid: coordinate, D = the count, then zeros
+                            if (!by_hand) *dst = val;
+                            else if (!is_pad) atomicAdd(dst, val);                // some tiles were added by hand
                         }
                     }
                 }
             }
         }
     }
+    if (PARTIALS && !sums_started && !by_hand)   // an empty run: its row block is all zeros
+        for (int i = tid; i < K * stride; i += THREADS) row_block[i] = 0.0f;
     fence_before_sync();
     __syncthreads();
     if (w == 0) tmem_dealloc(tmem_base, ncols);
