@@ -217,12 +217,14 @@ def run_ours(args, rank, world, local_rank):
     table = (C.c_void_p * P)(*[t.data_ptr() for t in d_bufs])
     L = ec.lib()
 
-    def epoch(events=None):
+    def epoch(events=None, res=None, cnt=None):
+        res = d_res if res is None else res
+        cnt = d_cnt if cnt is None else cnt
         L.ec_allreduce_reset(ar._h, st)
         for t in range(len(d_masks)):
             if events is not None:
                 events[t][0].record(stream)
-            rc = ar.apply_raw(table, d_masks[t].data_ptr(), d_res.data_ptr(), d_cnt.data_ptr(), st)
+            rc = ar.apply_raw(table, d_masks[t].data_ptr(), res.data_ptr(), cnt.data_ptr(), st)
             if events is not None:
                 events[t][1].record(stream)
             if rc != 0:
@@ -273,23 +275,45 @@ def run_ours(args, rank, world, local_rank):
     h2d = sum(t.numel() * t.element_size() for t in pin_bufs) + sum(m.numel() * 8 for m in d_masks)
     d2h = pin_res.numel() * 4 + pin_cnt.numel() * 4
     pin_masks = [torch.from_numpy(m.view(np.int64)).pin_memory() for m in h_masks]
-    with torch.cuda.stream(stream):
-        def e2e_epoch():
+    # Two result buffers alternate: the device-to-host read of one step's result runs on a second stream while the
+    # next step's host-to-device copies are already under way (PCIe carries both directions at once).
+    copy_stream = torch.cuda.Stream(device=dev)
+    res2 = [d_res, torch.empty_like(d_res)]
+    cnt2 = [d_cnt, torch.empty_like(d_cnt)]
+    pin_res2 = [pin_res, torch.empty_like(pin_res).pin_memory()]
+    pin_cnt2 = [pin_cnt, torch.empty_like(pin_cnt).pin_memory()]
+    done_ev = [torch.cuda.Event(), torch.cuda.Event()]       # the read-back of buffer i has finished
+    ready_ev = [torch.cuda.Event(), torch.cuda.Event()]      # the result in buffer i is complete
+
+    def e2e_epoch(i):
+        b = i & 1
+        with torch.cuda.stream(stream):
             for r in range(P):
                 d_bufs[r].copy_(pin_bufs[r], non_blocking=True)
             for t in range(len(d_masks)):
                 d_masks[t].copy_(pin_masks[t], non_blocking=True)
-            epoch()
-            pin_res.copy_(d_res, non_blocking=True)
-            pin_cnt.copy_(d_cnt, non_blocking=True)
-        e2e_epoch()
-        barrier()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(stream)
-        for _ in range(e2e_steps):
-            e2e_epoch()
-        e1.record(stream)
-        barrier()
+            stream.wait_event(done_ev[b])                    # buffer b was read back two steps ago
+            epoch(res=res2[b], cnt=cnt2[b])
+            ready_ev[b].record(stream)
+        with torch.cuda.stream(copy_stream):
+            copy_stream.wait_event(ready_ev[b])
+            pin_res2[b].copy_(res2[b], non_blocking=True)
+            pin_cnt2[b].copy_(cnt2[b], non_blocking=True)
+            done_ev[b].record(copy_stream)
+
+    for b in (0, 1):
+        done_ev[b].record(copy_stream)
+    e2e_epoch(0)
+    e2e_epoch(1)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for i in range(e2e_steps):
+        e2e_epoch(i)
+    stream.wait_event(done_ev[0])
+    stream.wait_event(done_ev[1])                            # the last results have reached the host
+    e1.record(stream)
+    barrier()
     e2e_ms = e0.elapsed_time(e1) / e2e_steps
     clock_info = clocks.stop(t_host0, t_host1)
 
