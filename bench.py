@@ -217,14 +217,12 @@ def run_ours(args, rank, world, local_rank):
     table = (C.c_void_p * P)(*[t.data_ptr() for t in d_bufs])
     L = ec.lib()
 
-    def epoch(events=None, res=None, cnt=None):
-        res = d_res if res is None else res
-        cnt = d_cnt if cnt is None else cnt
+    def epoch(events=None):
         L.ec_allreduce_reset(ar._h, st)
         for t in range(len(d_masks)):
             if events is not None:
                 events[t][0].record(stream)
-            rc = ar.apply_raw(table, d_masks[t].data_ptr(), res.data_ptr(), cnt.data_ptr(), st)
+            rc = ar.apply_raw(table, d_masks[t].data_ptr(), d_res.data_ptr(), d_cnt.data_ptr(), st)
             if events is not None:
                 events[t][1].record(stream)
             if rc != 0:
@@ -275,43 +273,47 @@ def run_ours(args, rank, world, local_rank):
     h2d = sum(t.numel() * t.element_size() for t in pin_bufs) + sum(m.numel() * 8 for m in d_masks)
     d2h = pin_res.numel() * 4 + pin_cnt.numel() * 4
     pin_masks = [torch.from_numpy(m.view(np.int64)).pin_memory() for m in h_masks]
-    # Two result buffers alternate: the device-to-host read of one step's result runs on a second stream while the
-    # next step's host-to-device copies are already under way (PCIe carries both directions at once).
-    copy_stream = torch.cuda.Stream(device=dev)
-    res2 = [d_res, torch.empty_like(d_res)]
-    cnt2 = [d_cnt, torch.empty_like(d_cnt)]
-    pin_res2 = [pin_res, torch.empty_like(pin_res).pin_memory()]
-    pin_cnt2 = [pin_cnt, torch.empty_like(pin_cnt).pin_memory()]
-    done_ev = [torch.cuda.Event(), torch.cuda.Event()]       # the read-back of buffer i has finished
-    ready_ev = [torch.cuda.Event(), torch.cuda.Event()]      # the result in buffer i is complete
+    # One ec_allreduce_epoch_host call per step: it uploads the P host buffers and the masks, runs the epoch and reads
+    # the result back, all on one stream.  Two streams (each with its context, staging area and host result) alternate,
+    # so that the read-back of one step runs while the next step's uploads are under way (PCIe carries both directions).
+    rounds = len(pin_masks)
+    lanes = []
+    for i in range(2):
+        a_i = ar if i == 0 else ec.Allreduce(P, n, ec.F32, ec.SUM, seg, device=dev)
+        if i and (args.threads or args.tile):
+            a_i.set_tile(args.threads, args.tile)
+        nbytes = a_i.host_staging_bytes(rounds)
+        lanes.append({
+            "ar": a_i, "stream": stream if i == 0 else torch.cuda.Stream(device=dev),
+            "staging": torch.empty(nbytes, dtype=torch.uint8, device=dev), "bytes": nbytes,
+            "res": pin_res if i == 0 else torch.empty_like(pin_res).pin_memory(),
+            "cnt": pin_cnt if i == 0 else torch.empty_like(pin_cnt).pin_memory(),
+            "done": torch.cuda.Event()})
+    host_table = (C.c_void_p * P)(*[t.data_ptr() for t in pin_bufs])
+    mask_table = (C.c_void_p * rounds)(*[t.data_ptr() for t in pin_masks])
 
     def e2e_epoch(i):
-        b = i & 1
-        with torch.cuda.stream(stream):
-            for r in range(P):
-                d_bufs[r].copy_(pin_bufs[r], non_blocking=True)
-            for t in range(len(d_masks)):
-                d_masks[t].copy_(pin_masks[t], non_blocking=True)
-            stream.wait_event(done_ev[b])                    # buffer b was read back two steps ago
-            epoch(res=res2[b], cnt=cnt2[b])
-            ready_ev[b].record(stream)
-        with torch.cuda.stream(copy_stream):
-            copy_stream.wait_event(ready_ev[b])
-            pin_res2[b].copy_(res2[b], non_blocking=True)
-            pin_cnt2[b].copy_(cnt2[b], non_blocking=True)
-            done_ev[b].record(copy_stream)
+        ln = lanes[i & 1]
+        rc = ln["ar"].epoch_host_raw(host_table, mask_table, rounds, ln["res"].data_ptr(), ln["cnt"].data_ptr(),
+                                     ln["staging"].data_ptr(), ln["bytes"], ln["stream"].cuda_stream)
+        if rc != 0:
+            raise ec.EcError(rc, "ec_allreduce_epoch_host")
+        ln["done"].record(ln["stream"])
 
-    for b in (0, 1):
-        done_ev[b].record(copy_stream)
+    torch.cuda.synchronize(dev)
     e2e_epoch(0)
     e2e_epoch(1)
+    torch.cuda.synchronize(dev)
+    if not (torch.equal(lanes[0]["res"], lanes[1]["res"]) and torch.equal(pin_res, d_res.cpu())):
+        raise RuntimeError("end-to-end result differs from the device-resident result")
     barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(stream)
+    lanes[1]["stream"].wait_event(e0)
     for i in range(e2e_steps):
         e2e_epoch(i)
-    stream.wait_event(done_ev[0])
-    stream.wait_event(done_ev[1])                            # the last results have reached the host
+    stream.wait_event(lanes[0]["done"])
+    stream.wait_event(lanes[1]["done"])                      # the last results have reached the host
     e1.record(stream)
     barrier()
     e2e_ms = e0.elapsed_time(e1) / e2e_steps

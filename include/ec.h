@@ -173,6 +173,29 @@ int ec_allreduce_ssp_apply(ec_ctx_t* ctx, const void* const* rank_bufs, int P, s
  * next apply overwrites it. */
 int ec_allreduce_reset(ec_ctx_t* ctx, ec_stream_t stream);
 
+/* One whole epoch from HOST memory (Sec. IV-B: a reset followed by an apply each
+ * time more contributions have come in, here `rounds` of them).
+ *
+ *   host_rank_bufs  HOST array of P HOST pointers, n elements of the context's
+ *                   dtype each; pinned memory makes the copies asynchronous.
+ *   host_masks      HOST array of `rounds` HOST pointers, each a cumulative
+ *                   notification mask uint64 [S][W] as in ec_allreduce_apply.
+ *   host_result     HOST, n elements of the accumulator type; written.
+ *   host_contrib_count  HOST uint32 [S] after the last round, or NULL.
+ *   staging         DEVICE scratch of at least ec_allreduce_host_staging_bytes
+ *                   (ctx, rounds) bytes, 256-byte aligned, owned by the caller;
+ *                   it holds the uploaded buffers, masks, the result and counts.
+ *
+ * Everything is enqueued on `stream` (P + rounds uploads, `rounds` applies, the
+ * read-back); the host arrays are valid once the stream has been synchronised.
+ * Two calls on two streams need two staging areas and two contexts.  Errors as
+ * in ec_allreduce_apply; EC_ERR_CAPACITY for a staging area that is too small or
+ * misaligned. */
+size_t ec_allreduce_host_staging_bytes(const ec_ctx_t* ctx, int rounds);
+int ec_allreduce_epoch_host(ec_ctx_t* ctx, const void* const* host_rank_bufs, const uint64_t* const* host_masks,
+                            int rounds, void* host_result, uint32_t* host_contrib_count, void* staging,
+                            size_t staging_bytes, ec_stream_t stream);
+
 /* Expert knob: elements of one segment handled per thread block (rounded to the
  * vector width) and threads per block (64..256, multiple of 32).  0 keeps the
  * current value.  Affects speed only, never results. */

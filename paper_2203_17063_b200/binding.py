@@ -32,6 +32,8 @@ SYMBOLS = {
     "ec_allreduce_apply": (_i, [_vp, _vp, _i, _sz, _i, _i, _sz, _vp, _vp, _vp, _vp]),
     "ec_allreduce_ssp_apply": (_i, [_vp, _vp, _i, _sz, _i, _i, _sz, _vp, C.c_uint32, C.c_uint32, _vp, _vp, _vp, _vp, _vp]),
     "ec_allreduce_reset": (_i, [_vp, _vp]),
+    "ec_allreduce_host_staging_bytes": (_sz, [_vp, _i]),
+    "ec_allreduce_epoch_host": (_i, [_vp, _vp, _vp, _i, _vp, _vp, _vp, _sz, _vp]),
     "ec_allreduce_set_tile": (_i, [_vp, _i, _sz]),
     "ec_allreduce_destroy": (_i, [_vp]),
     "ec_allgatherv": (_i, [_vp, _vp, _i, _i, _vp, _vp, _vp, _sz, _vp, _vp]),
@@ -147,6 +149,23 @@ class Allreduce:
 
     def reset(self, stream=None) -> None:
         _check(lib().ec_allreduce_reset(self._h, _stream(stream)), "ec_allreduce_reset")
+
+    def host_staging_bytes(self, rounds: int) -> int:
+        return lib().ec_allreduce_host_staging_bytes(self._h, rounds)
+
+    def epoch_host(self, host_rank_bufs, host_masks, host_result, host_contrib_count, staging, stream=None) -> None:
+        """ec_allreduce_epoch_host: a whole epoch from host tensors (pinned for asynchronous copies);
+        `staging` is a device uint8 tensor of at least host_staging_bytes(len(host_masks)) bytes."""
+        _check(lib().ec_allreduce_epoch_host(self._h, _table(host_rank_bufs), _table(host_masks), len(host_masks),
+                                             _ptr(host_result), _ptr(host_contrib_count), _ptr(staging),
+                                             staging.numel() * staging.element_size(), _stream(stream)),
+               "ec_allreduce_epoch_host")
+
+    def epoch_host_raw(self, buf_table, mask_table, rounds, result_ptr, count_ptr, staging_ptr, staging_bytes,
+                       stream_ptr) -> int:
+        """Same call with pre-marshalled arguments (for timing loops); returns the status code."""
+        return lib().ec_allreduce_epoch_host(self._h, buf_table, mask_table, rounds, result_ptr, count_ptr,
+                                             staging_ptr, staging_bytes, stream_ptr)
 
     def set_tile(self, threads: int = 0, tile_elems: int = 0) -> None:
         _check(lib().ec_allreduce_set_tile(self._h, threads, tile_elems), "ec_allreduce_set_tile")

@@ -679,6 +679,53 @@ int ec_allreduce_reset(ec_ctx_t* c, ec_stream_t stream) {
     return EC_OK;
 }
 
+size_t ec_allreduce_host_staging_bytes(const ec_ctx_t* c, int rounds) {
+    if (!c || rounds < 1) return 0;
+    const size_t buf = align_up(c->n * in_bytes(c->dtype), 256);
+    const size_t words = align_up(c->S * (size_t)c->W * sizeof(uint64_t), 256);
+    return (size_t)c->P * buf + (size_t)rounds * words + align_up(c->n * out_bytes(c->dtype), 256) +
+           align_up(c->S * sizeof(uint32_t), 256);
+}
+
+int ec_allreduce_epoch_host(ec_ctx_t* c, const void* const* host_rank_bufs, const uint64_t* const* host_masks,
+                            int rounds, void* host_result, uint32_t* host_contrib_count, void* staging,
+                            size_t staging_bytes, ec_stream_t stream) {
+    if (!c || !host_rank_bufs || !host_masks || !host_result || !staging || rounds < 1) return EC_ERR_INVALID;
+    if (staging_bytes < ec_allreduce_host_staging_bytes(c, rounds) || (reinterpret_cast<uintptr_t>(staging) & 255u))
+        return EC_ERR_CAPACITY;
+    for (int r = 0; r < c->P; ++r)
+        if (!host_rank_bufs[r]) return EC_ERR_INVALID;
+    for (int k = 0; k < rounds; ++k)
+        if (!host_masks[k]) return EC_ERR_INVALID;
+    const size_t in_b = c->n * in_bytes(c->dtype), out_b = c->n * out_bytes(c->dtype);
+    const size_t buf = align_up(in_b, 256);
+    const size_t words_b = c->S * (size_t)c->W * sizeof(uint64_t), words = align_up(words_b, 256);
+    char* p = static_cast<char*>(staging);
+    const void* dev_bufs[EC_MAX_RANKS];
+    for (int r = 0; r < c->P; ++r) {       // one plain copy per rank buffer; they queue behind one another on the stream
+        dev_bufs[r] = p;
+        EC_CUDA(cudaMemcpyAsync(p, host_rank_bufs[r], in_b, cudaMemcpyHostToDevice, stream));
+        p += buf;
+    }
+    const uint64_t* dev_masks = reinterpret_cast<const uint64_t*>(p);
+    for (int k = 0; k < rounds; ++k) {
+        EC_CUDA(cudaMemcpyAsync(p, host_masks[k], words_b, cudaMemcpyHostToDevice, stream));
+        p += words;
+    }
+    void* dev_result = p;
+    p += align_up(out_b, 256);
+    uint32_t* dev_count = reinterpret_cast<uint32_t*>(p);
+    int rc = ec_allreduce_reset(c, stream);
+    for (int k = 0; k < rounds && rc == EC_OK; ++k)
+        rc = ec_allreduce_apply(c, dev_bufs, c->P, c->n, (ec_dtype_t)c->dtype, (ec_op_t)c->op, c->seg,
+                                dev_masks + (size_t)k * (words / sizeof(uint64_t)), dev_result, dev_count, stream);
+    if (rc != EC_OK) return rc;
+    EC_CUDA(cudaMemcpyAsync(host_result, dev_result, out_b, cudaMemcpyDeviceToHost, stream));
+    if (host_contrib_count)
+        EC_CUDA(cudaMemcpyAsync(host_contrib_count, dev_count, c->S * sizeof(uint32_t), cudaMemcpyDeviceToHost, stream));
+    return EC_OK;
+}
+
 int ec_allreduce_destroy(ec_ctx_t* c) {
     if (!c) return EC_ERR_INVALID;
     int rc = EC_OK;

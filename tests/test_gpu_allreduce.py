@@ -308,3 +308,38 @@ def test_ring_order_needs_segments_inside_chunks():
     with pytest.raises(ec.EcError) as err:
         ec.Allreduce(4, 1000, ec.F32, ec.SUM, 64, ec.ORDER_RING)        # ceil(1000/4) = 250 is not a multiple of 64
     assert err.value.code == ec.ERR_INVALID
+
+
+# ---------------------------------------------------------------------------
+# the whole epoch from host memory in one call (uploads, reset, applies, read-back)
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("dtype,kind,kw", [(ec.F32, "normal_f32", {}), (ec.BF16, "normal_bf16", {"sigma": 1.0})],
+                         ids=["f32", "bf16"])
+def test_epoch_from_host_buffers_matches_round_by_round_checker(dtype, kind, kw):
+    P, n, seg = 16, (1 << 18) + 24, 8192
+    S = (n + seg - 1) // seg
+    bufs = _bufs(kind, 1010, P, n, **kw)
+    rounds = inputs.arrival_rounds(2010, P, S, 0.6)
+    masks = inputs.cumulative_masks(rounds)
+    ref = oracle.Allreduce(P, n, dtype, ec.SUM, seg)
+    c_res = sentinel(NP_OUT[dtype], n)
+    c_cnt = np.zeros(S, dtype=np.uint32)
+    for m in masks:
+        ref.apply(bufs, m, c_res, c_cnt)
+    ar = ec.Allreduce(P, n, dtype, ec.SUM, seg)
+    h_bufs = [torch.from_numpy(b.view(np.int16) if b.dtype == np.uint16 else b).pin_memory() for b in bufs]
+    h_masks = [torch.from_numpy(np.ascontiguousarray(m, dtype=np.uint64).view(np.int64)).pin_memory() for m in masks]
+    h_res = torch.from_numpy(sentinel(NP_OUT[dtype], n)).pin_memory()
+    h_cnt = torch.full((S,), -1, dtype=torch.int32).pin_memory()
+    staging = torch.empty(ar.host_staging_bytes(len(masks)), dtype=torch.uint8, device="cuda")
+    for _ in range(2):                                   # a second epoch on the same context and staging area
+        h_res.fill_(float("nan"))
+        ar.epoch_host(h_bufs, h_masks, h_res, h_cnt, staging)
+        torch.cuda.synchronize()
+        assert np.array_equal(h_cnt.numpy().view(np.uint32), c_cnt)
+        assert np.array_equal(bits(h_res.numpy()), bits(c_res))
+    small = torch.empty(ar.host_staging_bytes(len(masks)) - 256, dtype=torch.uint8, device="cuda")
+    with pytest.raises(ec.EcError) as err:
+        ar.epoch_host(h_bufs, h_masks, h_res, h_cnt, small)
+    assert err.value.code == ec.ERR_CAPACITY
+    ar.destroy()
