@@ -36,9 +36,10 @@ HEADLINE = dict(P=16, n=1 << 24, seg=65536, p_first=0.7, seed=1002, seed_sched=2
 NOMINAL_HBM_GBS = 8000.0
 
 # dram__bytes_read.sum + dram__bytes_write.sum of the three apply launches of one headline epoch, from one
-# ncu capture (profiles/apply_kernel_config2_epoch.md): reads 750.5 + 214.7 + 233.1 MB, writes 9.7 + 8.0 + 8.5 MB.
-# Below the algorithmic bytes because result writes stay in L2 as dirty lines while the kernel runs.
-NCU_TRAFFIC_BYTES_PER_EPOCH = 1_224_616_192
+# one-pass ncu capture that leaves the caches alone (profiles/apply_kernel_config2_epoch.md): reads 750.5 + 191.4 +
+# 211.0 MB, writes 44.0 + 31.5 + 33.9 MB.  Below the algorithmic bytes because about half of the 64 MiB result is
+# found in L2 by the next round.
+NCU_TRAFFIC_BYTES_PER_EPOCH = 1_262_126_720
 
 
 def measured_peaks():
