@@ -230,6 +230,87 @@ __device__ __forceinline__ void fold_vectors(const char* const* s_ptr, int m, ty
     }
 }
 
+// Prologue of a block, run by its first warp: which ranks are new for segment s (notification words or
+// clocks), the bookkeeping outputs (block t == 0 of the segment writes them), and the ascending (or ring-
+// rotated) list of the new ranks in shared memory.
+__device__ __forceinline__ void block_prologue(const ApplyArgs& a, unsigned s, unsigned t, uint16_t* s_rank,
+                                               uint64_t* s_new, int* s_m, int* s_fresh) {
+            const int lane = threadIdx.x;
+            uint64_t nw = 0, old = 0;
+            if (a.notif_clock != nullptr) {
+                // Stale-synchronous acceptance (Algorithm 1): a contribution takes part if its clock is not older
+                // than clock - slack.  32 ranks per step; the ballots of two steps make one 64-rank word.
+                uint32_t mn = 0xffffffffu;
+                int stale = 0;
+                for (int c = 0; c * 32 < a.P; ++c) {
+                    const int r = c * 32 + lane;
+                    const uint32_t ck = r < a.P ? a.notif_clock[(size_t)s * a.P + r] : 0u;
+                    const bool ok = r < a.P && ck >= a.min_clock;
+                    const unsigned bal = __ballot_sync(0xffffffffu, ok);
+                    if (ok) mn = ck < mn ? ck : mn;
+                    stale += (r < a.P && !ok) ? 1 : 0;
+                    if (lane == (c >> 1)) nw |= (uint64_t)bal << ((c & 1) * 32);
+                }
+    #pragma unroll
+                for (int d = 16; d > 0; d >>= 1) {
+                    const uint32_t o = __shfl_xor_sync(0xffffffffu, mn, d);
+                    mn = o < mn ? o : mn;
+                    stale += __shfl_xor_sync(0xffffffffu, stale, d);
+                }
+                if (t == 0 && lane == 0) {
+                    if (a.seg_clock) a.seg_clock[s] = mn == 0xffffffffu ? 0u : mn;   // the result is as old as its oldest input
+                    if (a.wait_count) a.wait_count[s] = (uint32_t)stale;
+                }
+            } else if (lane < a.W) {
+                uint64_t arr = a.arrival ? a.arrival[(size_t)s * a.W + lane] : ~0ull;
+                if (lane == a.W - 1 && (a.P & 63)) arr &= (1ull << (a.P & 63)) - 1;   // bits >= P mean nothing
+                // the first apply of an epoch starts from "nothing folded in": no need to clear the words
+                old = a.first_apply ? 0ull : a.applied_in[(size_t)s * a.W + lane];
+                nw = arr & ~old;
+            }
+            const unsigned any_new = __ballot_sync(0xffffffffu, nw != 0);
+            const unsigned any_old = __ballot_sync(0xffffffffu, old != 0);
+            const int cnt_new = __popcll(nw);
+            int incl = cnt_new, total = __popcll(nw | old);
+    #pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const int y = __shfl_up_sync(0xffffffffu, incl, d);
+                if (lane >= d) incl += y;
+                total += __shfl_xor_sync(0xffffffffu, total, d);
+            }
+            if (t == 0) {
+                if (lane < a.W && a.notif_clock == nullptr) a.applied_out[(size_t)s * a.W + lane] = old | nw;
+                if (lane == 0 && a.contrib_count) a.contrib_count[s] = (uint32_t)total;
+            }
+            if (lane < MAX_W) s_new[lane] = nw;
+            // Ring order (Scatter-Reduce of the segmented ring, Sec. IV-A): chunk c of the vector is first sent by
+            // node c and reduced by nodes c+1, c+2, ... in turn, so its fold starts at rank c and wraps around.
+            // The ascending list is rotated: the j0 ranks below c go to the end.
+            const int m_all = __shfl_sync(0xffffffffu, incl, 31);
+            int j0 = 0;
+            if (a.ring_chunk != 0) {
+                size_t c = ((size_t)s * a.seg) / a.ring_chunk;
+                if (c > (size_t)(a.P - 1)) c = (size_t)(a.P - 1);
+                const int rel = (int)c - lane * 64;                       // ranks of this word below c
+                const uint64_t below = rel <= 0 ? 0ull : rel >= 64 ? ~0ull : (1ull << rel) - 1;
+                j0 = __popcll(nw & below);
+    #pragma unroll
+                for (int d = 16; d > 0; d >>= 1) j0 += __shfl_xor_sync(0xffffffffu, j0, d);
+            }
+            int j = incl - cnt_new;
+            uint64_t bits = nw;
+            while (bits) {
+                const int b = __ffsll((long long)bits) - 1;
+                bits &= bits - 1;
+                const int pos = j >= j0 ? j - j0 : j + (m_all - j0);
+                s_rank[pos] = (uint16_t)(lane * 64 + b);
+                ++j;
+            }
+            if (lane == 31) *s_m = incl;
+            if (lane == 0) *s_fresh = (any_old == 0) ? 1 : 0;
+            (void)any_new;
+}
+
 // ---------------------------------------------------------------------------------------------
 // the apply kernel
 // ---------------------------------------------------------------------------------------------
@@ -252,82 +333,7 @@ apply_kernel(const ApplyArgs a, const __grid_constant__ PtrTable<CAP> tbl) {
     size_t seg_hi = (size_t)(s + 1) * a.seg;
     if (seg_hi > a.n) seg_hi = a.n;
 
-    if (threadIdx.x < 32) {
-        const int lane = threadIdx.x;
-        uint64_t nw = 0, old = 0;
-        if (a.notif_clock != nullptr) {
-            // Stale-synchronous acceptance (Algorithm 1): a contribution takes part if its clock is not older
-            // than clock - slack.  32 ranks per step; the ballots of two steps make one 64-rank word.
-            uint32_t mn = 0xffffffffu;
-            int stale = 0;
-            for (int c = 0; c * 32 < a.P; ++c) {
-                const int r = c * 32 + lane;
-                const uint32_t ck = r < a.P ? a.notif_clock[(size_t)s * a.P + r] : 0u;
-                const bool ok = r < a.P && ck >= a.min_clock;
-                const unsigned bal = __ballot_sync(0xffffffffu, ok);
-                if (ok) mn = ck < mn ? ck : mn;
-                stale += (r < a.P && !ok) ? 1 : 0;
-                if (lane == (c >> 1)) nw |= (uint64_t)bal << ((c & 1) * 32);
-            }
-#pragma unroll
-            for (int d = 16; d > 0; d >>= 1) {
-                const uint32_t o = __shfl_xor_sync(0xffffffffu, mn, d);
-                mn = o < mn ? o : mn;
-                stale += __shfl_xor_sync(0xffffffffu, stale, d);
-            }
-            if (t == 0 && lane == 0) {
-                if (a.seg_clock) a.seg_clock[s] = mn == 0xffffffffu ? 0u : mn;   // the result is as old as its oldest input
-                if (a.wait_count) a.wait_count[s] = (uint32_t)stale;
-            }
-        } else if (lane < a.W) {
-            uint64_t arr = a.arrival ? a.arrival[(size_t)s * a.W + lane] : ~0ull;
-            if (lane == a.W - 1 && (a.P & 63)) arr &= (1ull << (a.P & 63)) - 1;   // bits >= P mean nothing
-            // the first apply of an epoch starts from "nothing folded in": no need to clear the words
-            old = a.first_apply ? 0ull : a.applied_in[(size_t)s * a.W + lane];
-            nw = arr & ~old;
-        }
-        const unsigned any_new = __ballot_sync(0xffffffffu, nw != 0);
-        const unsigned any_old = __ballot_sync(0xffffffffu, old != 0);
-        const int cnt_new = __popcll(nw);
-        int incl = cnt_new, total = __popcll(nw | old);
-#pragma unroll
-        for (int d = 1; d < 32; d <<= 1) {
-            const int y = __shfl_up_sync(0xffffffffu, incl, d);
-            if (lane >= d) incl += y;
-            total += __shfl_xor_sync(0xffffffffu, total, d);
-        }
-        if (t == 0) {
-            if (lane < a.W && a.notif_clock == nullptr) a.applied_out[(size_t)s * a.W + lane] = old | nw;
-            if (lane == 0 && a.contrib_count) a.contrib_count[s] = (uint32_t)total;
-        }
-        if (lane < MAX_W) s_new[lane] = nw;
-        // Ring order (Scatter-Reduce of the segmented ring, Sec. IV-A): chunk c of the vector is first sent by
-        // node c and reduced by nodes c+1, c+2, ... in turn, so its fold starts at rank c and wraps around.
-        // The ascending list is rotated: the j0 ranks below c go to the end.
-        const int m_all = __shfl_sync(0xffffffffu, incl, 31);
-        int j0 = 0;
-        if (a.ring_chunk != 0) {
-            size_t c = ((size_t)s * a.seg) / a.ring_chunk;
-            if (c > (size_t)(a.P - 1)) c = (size_t)(a.P - 1);
-            const int rel = (int)c - lane * 64;                       // ranks of this word below c
-            const uint64_t below = rel <= 0 ? 0ull : rel >= 64 ? ~0ull : (1ull << rel) - 1;
-            j0 = __popcll(nw & below);
-#pragma unroll
-            for (int d = 16; d > 0; d >>= 1) j0 += __shfl_xor_sync(0xffffffffu, j0, d);
-        }
-        int j = incl - cnt_new;
-        uint64_t bits = nw;
-        while (bits) {
-            const int b = __ffsll((long long)bits) - 1;
-            bits &= bits - 1;
-            const int pos = j >= j0 ? j - j0 : j + (m_all - j0);
-            s_rank[pos] = (uint16_t)(lane * 64 + b);
-            ++j;
-        }
-        if (lane == 31) s_m = incl;
-        if (lane == 0) s_fresh = (any_old == 0) ? 1 : 0;
-        (void)any_new;
-    }
+    if (threadIdx.x < 32) block_prologue(a, s, t, s_rank, s_new, &s_m, &s_fresh);
     __syncthreads();
     const int m = s_m;
     const bool fresh = s_fresh != 0;
@@ -473,11 +479,98 @@ apply_kernel(const ApplyArgs a, const __grid_constant__ PtrTable<CAP> tbl) {
     }
 }
 
+// ---------------------------------------------------------------------------------------------
+// the apply kernel for short segments
+// ---------------------------------------------------------------------------------------------
+// A short segment and many ranks (the rows of a small model, e.g. one centroid row per segment): only a few
+// threads own a result vector, and the streaming fold, which fetches four ranks at a time, would be a chain of
+// m / 4 memory round trips.  Here one block takes a whole segment; all its threads fetch the (rank, vector)
+// items of up to STAGE / nv ranks into shared memory at once, then the owners fold them from there in ascending
+// rank order.  Same prologue, same order of additions, same bits as apply_kernel.
+constexpr int STAGE = 512;           // 16-byte items staged per pass
+template <int DT, int OP, int CAP>
+__global__ void __launch_bounds__(EC_MAXT)
+apply_short_kernel(const ApplyArgs a, const __grid_constant__ PtrTable<CAP> tbl) {
+    typedef Elem<DT> E;
+    typedef typename E::In In;
+    typedef typename E::Acc Acc;
+    constexpr int VEC = E::VEC;
+
+    __shared__ const char* s_ptr[CAP];
+    __shared__ uint16_t s_rank[CAP];
+    __shared__ uint64_t s_new[MAX_W];
+    __shared__ int s_m, s_fresh;
+    __shared__ uint4 s_stage[STAGE];
+
+    const unsigned s = blockIdx.x;
+    const size_t lo = (size_t)s * a.seg;
+    size_t hi = lo + a.seg;
+    if (hi > a.n) hi = a.n;
+    if (threadIdx.x < 32) block_prologue(a, s, 0u, s_rank, s_new, &s_m, &s_fresh);
+    __syncthreads();
+    const int m = s_m;
+    const bool fresh = s_fresh != 0;
+    if (m == 0 && !(fresh && a.first_apply)) return;   // nothing new: the segment is neither read nor written
+    const size_t cnt = hi - lo;
+    Acc* res = reinterpret_cast<Acc*>(a.result) + lo;
+    const int tid = threadIdx.x, nthr = blockDim.x;
+    const uint64_t pol = evict_first_policy();
+    const uint64_t rpol = result_policy(1);            // a result this small stays in L2
+    for (int j = tid; j < m; j += nthr)
+        s_ptr[j] = reinterpret_cast<const char*>(tbl.p[s_rank[j]]) + lo * sizeof(In);
+    __syncthreads();
+    const int nv = (int)(cnt / VEC);                   // at most nthr / 4 (the host chose this kernel for that)
+    if (nv > 0) {
+        const int per_pass = STAGE / nv;
+        Acc acc[VEC];
+        if (tid < nv) {
+            if (fresh) {
+#pragma unroll
+                for (int e = 0; e < VEC; ++e) acc[e] = ident<OP>(Acc());
+            } else {
+                load_acc<Acc, VEC>(res + (size_t)tid * VEC, acc, rpol);
+            }
+        }
+        for (int j0 = 0; j0 < m; j0 += per_pass) {
+            const int rr = m - j0 < per_pass ? m - j0 : per_pass;
+#pragma unroll 4
+            for (int i = tid; i < rr * nv; i += nthr) {
+                const int j = i / nv, v = i - j * nv;
+                s_stage[i] = ld_stream16(s_ptr[j0 + j] + (size_t)v * 16, pol);
+            }
+            __syncthreads();
+            if (tid < nv) {
+                for (int j = 0; j < rr; ++j) {
+                    Acc x[VEC];
+                    E::unpack(s_stage[j * nv + tid], x);
+#pragma unroll
+                    for (int e = 0; e < VEC; ++e) acc[e] = comb<OP>(acc[e], x[e]);
+                }
+            }
+            __syncthreads();
+        }
+        if (tid < nv) store_acc<Acc, VEC>(res + (size_t)tid * VEC, acc, rpol);
+    }
+    // ragged tail of a short last segment, element by element
+    for (size_t i = (size_t)nv * VEC + tid; i < cnt; i += nthr) {
+        Acc acc = fresh ? ident<OP>(Acc()) : res[i];
+        for (int j = 0; j < m; ++j) acc = comb<OP>(acc, E::widen(reinterpret_cast<const In*>(s_ptr[j])[i]));
+        res[i] = acc;
+    }
+}
+
 template <int DT, int OP, bool VECTOR, int ORDER>
-int launch_cap(const ApplyArgs& a, const void* const* bufs, unsigned grid, int threads, cudaStream_t st) {
+int launch_cap(const ApplyArgs& a, const void* const* bufs, unsigned grid, int threads, bool short_seg, cudaStream_t st) {
     if (a.P <= 64) {
         PtrTable<64> tbl;
         for (int r = 0; r < 64; ++r) tbl.p[r] = r < a.P ? bufs[r] : nullptr;
+        if constexpr (VECTOR && ORDER == EC_ORDER_FIXED) {
+            if (short_seg) {
+                apply_short_kernel<DT, OP, 64><<<grid, threads, 0, st>>>(a, tbl);
+                EC_CUDA(cudaGetLastError());
+                return EC_OK;
+            }
+        }
         apply_kernel<DT, OP, VECTOR, 64, ORDER><<<grid, threads, 0, st>>>(a, tbl);
     } else {
         PtrTable<EC_MAX_RANKS> tbl;
@@ -490,23 +583,23 @@ int launch_cap(const ApplyArgs& a, const void* const* bufs, unsigned grid, int t
 
 template <int DT, int OP>
 int launch_op(const ApplyArgs& a, const void* const* bufs, bool vector, int order, unsigned grid, int threads,
-              cudaStream_t st) {
+              bool short_seg, cudaStream_t st) {
     if (order == EC_ORDER_FIXED || order == EC_ORDER_RING)     // ring order = rank order rotated per chunk (a.ring_chunk)
-        return vector ? launch_cap<DT, OP, true, EC_ORDER_FIXED>(a, bufs, grid, threads, st)
-                      : launch_cap<DT, OP, false, EC_ORDER_FIXED>(a, bufs, grid, threads, st);
+        return vector ? launch_cap<DT, OP, true, EC_ORDER_FIXED>(a, bufs, grid, threads, short_seg, st)
+                      : launch_cap<DT, OP, false, EC_ORDER_FIXED>(a, bufs, grid, threads, false, st);
     if constexpr (OP == EC_SUM && DT != EC_I64)
-        return vector ? launch_cap<DT, EC_SUM, true, EC_ORDER_PAIRWISE>(a, bufs, grid, threads, st)
-                      : launch_cap<DT, EC_SUM, false, EC_ORDER_PAIRWISE>(a, bufs, grid, threads, st);
+        return vector ? launch_cap<DT, EC_SUM, true, EC_ORDER_PAIRWISE>(a, bufs, grid, threads, false, st)
+                      : launch_cap<DT, EC_SUM, false, EC_ORDER_PAIRWISE>(a, bufs, grid, threads, false, st);
     return EC_ERR_UNSUPPORTED;
 }
 
 template <int DT>
 int launch_dt(const ApplyArgs& a, const void* const* bufs, int op, bool vector, int order, unsigned grid,
-              int threads, cudaStream_t st) {
+              int threads, bool short_seg, cudaStream_t st) {
     switch (op) {
-        case EC_SUM: return launch_op<DT, EC_SUM>(a, bufs, vector, order, grid, threads, st);
-        case EC_MAX: return launch_op<DT, EC_MAX>(a, bufs, vector, order, grid, threads, st);
-        case EC_MIN: return launch_op<DT, EC_MIN>(a, bufs, vector, order, grid, threads, st);
+        case EC_SUM: return launch_op<DT, EC_SUM>(a, bufs, vector, order, grid, threads, short_seg, st);
+        case EC_MAX: return launch_op<DT, EC_MAX>(a, bufs, vector, order, grid, threads, short_seg, st);
+        case EC_MIN: return launch_op<DT, EC_MIN>(a, bufs, vector, order, grid, threads, short_seg, st);
     }
     return EC_ERR_INVALID;
 }
@@ -627,12 +720,21 @@ int apply_common(ec_ctx_t* c, const void* const* rank_bufs, int P, size_t n, ec_
     a.P = c->P; a.W = c->W;
     a.res_hint = c->res_hint;
     a.ring_chunk = c->order == EC_ORDER_RING ? (c->n + (size_t)c->P - 1) / (size_t)c->P : 0;
-    const unsigned grid = (unsigned)(tiles * c->S);
+    unsigned grid = (unsigned)(tiles * c->S);
+    // short segments and more ranks than the streaming fold keeps in flight: one block per segment, staged fold
+    // (measured: 12.4 -> 10.3 us for 64 ranks x 64 rows of 36 floats, 36.8 -> 30.7 us for 4096 such rows; with
+    // hundreds of ranks the staging passes cost more than they save, so those stay on the streaming kernel)
+    const bool short_seg = vector && c->order != EC_ORDER_PAIRWISE && c->P > EC_MAIN_RU && c->P <= 64 &&
+                           (seg_len * in_bytes(c->dtype) / 16) * 4 <= (size_t)c->threads;
+    if (short_seg) {
+        a.tiles_per_seg = 1;
+        grid = (unsigned)c->S;
+    }
     switch (c->dtype) {
-        case EC_F32: return launch_dt<EC_F32>(a, rank_bufs, c->op, vector, c->order, grid, c->threads, stream);
-        case EC_BF16: return launch_dt<EC_BF16>(a, rank_bufs, c->op, vector, c->order, grid, c->threads, stream);
-        case EC_I64: return launch_dt<EC_I64>(a, rank_bufs, c->op, vector, c->order, grid, c->threads, stream);
-        case EC_F64: return launch_dt<EC_F64>(a, rank_bufs, c->op, vector, c->order, grid, c->threads, stream);
+        case EC_F32: return launch_dt<EC_F32>(a, rank_bufs, c->op, vector, c->order, grid, c->threads, short_seg, stream);
+        case EC_BF16: return launch_dt<EC_BF16>(a, rank_bufs, c->op, vector, c->order, grid, c->threads, short_seg, stream);
+        case EC_I64: return launch_dt<EC_I64>(a, rank_bufs, c->op, vector, c->order, grid, c->threads, short_seg, stream);
+        case EC_F64: return launch_dt<EC_F64>(a, rank_bufs, c->op, vector, c->order, grid, c->threads, short_seg, stream);
     }
     return EC_ERR_INVALID;
 }

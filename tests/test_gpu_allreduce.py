@@ -343,3 +343,40 @@ def test_epoch_from_host_buffers_matches_round_by_round_checker(dtype, kind, kw)
         ar.epoch_host(h_bufs, h_masks, h_res, h_cnt, small)
     assert err.value.code == ec.ERR_CAPACITY
     ar.destroy()
+
+
+# ---------------------------------------------------------------------------
+# short segments with many ranks: one block per segment, contributions staged in shared memory
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("P,seg_vectors", [(5, 1), (8, 9), (64, 9), (64, 32), (48, 25), (200, 64), (200, 3), (1024, 2)])
+@pytest.mark.parametrize("dtype,kind,kw", [(ec.F32, "normal_f32", {}), (ec.BF16, "normal_bf16", {"sigma": 1.0}),
+                                           (ec.I64, "int64_full", {}), (ec.F64, "normal_f64", {})],
+                         ids=["f32", "bf16", "i64", "f64"])
+def test_short_segments_many_ranks(P, seg_vectors, dtype, kind, kw):
+    per_vec = {ec.F32: 4, ec.BF16: 8, ec.I64: 2, ec.F64: 2}[dtype]
+    seg = seg_vectors * per_vec
+    S = 37
+    n = (S - 1) * seg + max(1, seg - per_vec - 1)        # the last segment is short and ends inside a vector
+    if kind == "normal_f64":
+        bufs = [b.astype(np.float64) * (1.0 + 2.0 ** -30) for b in _bufs("normal_f32", 3000 + P, P, n)]
+    else:
+        bufs = _bufs(kind, 3000 + P, P, n, **kw)
+    rounds = inputs.arrival_rounds(3100 + P + seg_vectors, P, S, 0.5)
+    masks = inputs.cumulative_masks(rounds)
+    poison = [rounds > t for t in (1, 2, 3)]
+    run_schedule(P, n, seg, dtype, ec.SUM, bufs, masks, poison=poison)
+    if dtype != ec.BF16:
+        run_schedule(P, n, seg, dtype, ec.MAX, bufs, [masks[0], None])
+
+
+def test_short_segments_ring_order_and_untouched_rows():
+    P, seg, S = 16, 36, 64                                # one centroid-like row of 36 floats per segment
+    n = seg * S                                           # ceil(n / P) = 144 = 4 segments per ring chunk
+    bufs = _bufs("normal_f32", 3200, P, n)
+    rounds = inputs.arrival_rounds(3201, P, S, 0.4)
+    rounds[:, 5] = 3                                      # a segment nobody reaches before the last round
+    rounds[:, 6] = 1                                      # and one that is complete at once
+    masks = inputs.cumulative_masks(rounds)
+    run_schedule(P, n, seg, ec.F32, ec.SUM, bufs, masks, order=ec.ORDER_RING)
+    outs = run_schedule(P, n, seg, ec.F32, ec.SUM, bufs, masks + [masks[-1]])
+    assert np.array_equal(bits(outs[-1][0]), bits(outs[-2][0]))          # nothing new: nothing changes
