@@ -38,8 +38,10 @@ constexpr int TILE = THREADS;          // points per tile
 constexpr int MROWS = 128;             // rows of both accumulators
 constexpr uint32_t WAIT_LIMIT = 1u << 20;
 constexpr uint32_t OCHUNK = TILE * 16;        // one-hot tile: bytes between chunks of 8 centroids (128 points x 16 bytes)
-constexpr uint32_t XCHUNK = TILE * 16 + 16;   // point tiles: bytes between chunks of 8 coordinates; the 16 extra bytes
-                                              // spread the four chunks of a point over different banks
+// Point tiles: bytes between chunks of 8 coordinates.  Eight consecutive threads store one quarter-warp's 16-byte
+// items: D/8 chunks of 8/(D/8) consecutive points.  The padding of 1024/D bytes puts them on all 32 banks
+// (D = 32: chunks 32 bytes apart modulo 128, points 16 bytes apart; D = 16: chunks 64 bytes apart).
+__host__ __device__ constexpr uint32_t xchunk_of(int D) { return TILE * 16 + 1024u / (uint32_t)D; }
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -142,10 +144,11 @@ struct Layout {
 };
 __host__ __device__ inline Layout layout_of(int D, int K, bool partials) {
     const size_t npad = npad_of(K), kch = dpad_of(D) / 8;
+    const size_t XCHUNK = xchunk_of(D);
     Layout L;
     L.x = 0;
     L.cn = 6 * (size_t)XCHUNK;                       // npad floats (at most 256) ...
-    L.xn = L.cn + 1024;                               // ... then 128 floats; both inside columns 6-7 (4128 bytes)
+    L.xn = L.cn + 1024;                               // ... then 128 floats; both inside columns 6-7 (at least 4160 bytes)
     L.b = 14 * (size_t)XCHUNK;                        // centroid operand: npad rows x (kch + 2) chunks of 16 bytes
     size_t off = L.b + npad * (kch + 2) * 16;
     if (off < 16 * (size_t)XCHUNK) off = 16 * (size_t)XCHUNK;   // all 16 columns lie inside the allocation
@@ -201,6 +204,7 @@ tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const 
     constexpr int KCH = D / 8;                           // 16-byte chunks of coordinates per point
     static_assert(D % 16 == 0 && KCH + 2 <= 8 && (KCH & (KCH - 1)) == 0, "D is 16 or 32");
     constexpr int LO = 8;                                // first chunk column of the low parts
+    constexpr uint32_t XCHUNK = xchunk_of(D);
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const int npad = npad_of(K);
     const Layout L = layout_of(D, K, PARTIALS);
