@@ -15,9 +15,15 @@
 namespace ec {
 namespace {
 
+#ifndef EC_GV_BATCH
+#define EC_GV_BATCH 4
+#endif
+#ifndef EC_GV_CHUNK
+#define EC_GV_CHUNK 16384
+#endif
 constexpr int GV_THREADS = 256;
-constexpr size_t GV_CHUNK_BYTES = 16384;
-constexpr int GV_BATCH = 4;            // loads in flight per thread before the stores
+constexpr size_t GV_CHUNK_BYTES = EC_GV_CHUNK;
+constexpr int GV_BATCH = EC_GV_BATCH;  // loads in flight per thread before the stores
 
 struct GatherArgs {
     const int64_t* counts;
@@ -190,8 +196,28 @@ int sm_count() {
     return cached;
 }
 
+// Resident blocks of the kernel on the whole device (the blocks loop over the chunks, so more would only repeat
+// the scan in a second wave).
+template <int CAP>
+unsigned resident_blocks() {
+    static thread_local int cached_dev = -1;
+    static thread_local unsigned cached = 0;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 148 * 4;
+    if (dev != cached_dev) {
+        int per_sm = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, allgatherv_kernel<CAP>, GV_THREADS, 0) != cudaSuccess || per_sm < 1)
+            per_sm = 1;
+        cached = (unsigned)(sm_count() * per_sm);
+        cached_dev = dev;
+    }
+    return cached;
+}
+
 template <int CAP>
 void launch(const GatherArgs& a, const void* const* bufs, unsigned grid, cudaStream_t stream) {
+    const unsigned cap_blocks = resident_blocks<CAP>();
+    if (grid > cap_blocks) grid = cap_blocks;
     PtrTable<CAP> tbl;
     for (int r = 0; r < CAP; ++r) tbl.p[r] = r < a.P ? bufs[r] : nullptr;
     allgatherv_kernel<CAP><<<grid, GV_THREADS, 0, stream>>>(a, tbl);
@@ -217,11 +243,10 @@ int gather_common(const void* const* bufs, const int64_t* counts, int P, ec_dtyp
     GatherArgs a;
     a.counts = counts; a.arrival = arrival_mask; a.displs = displs; a.out = reinterpret_cast<char*>(out);
     a.status = status; a.capacity = out_capacity_elems; a.P = P; a.esize = es; a.compact = compact;
-    // enough blocks for every chunk the capacity allows, at most eight per SM (the blocks loop)
+    // enough blocks for every chunk the capacity allows, at most one wave of resident blocks (the blocks loop)
     size_t chunks = (out_capacity_elems * (size_t)es + GV_CHUNK_BYTES - 1) / GV_CHUNK_BYTES;
     if (chunks < 1) chunks = 1;
-    const size_t cap_blocks = (size_t)sm_count() * 8;
-    const unsigned grid = (unsigned)(chunks < cap_blocks ? chunks : cap_blocks);
+    const unsigned grid = (unsigned)(chunks < 0x7fffffffull ? chunks : 0x7fffffffull);
     if (P <= 64) launch<64>(a, bufs, grid, stream);
     else if (P <= 256) launch<256>(a, bufs, grid, stream);
     else launch<EC_MAX_RANKS>(a, bufs, grid, stream);
