@@ -314,8 +314,11 @@ __device__ __forceinline__ void block_prologue(const ApplyArgs& a, unsigned s, u
 // ---------------------------------------------------------------------------------------------
 // the apply kernel
 // ---------------------------------------------------------------------------------------------
+#ifndef EC_PW_MINB
+#define EC_PW_MINB 2
+#endif
 template <int DT, int OP, bool VECTOR, int CAP, int ORDER>
-__global__ void __launch_bounds__(EC_MAXT, (ORDER != EC_ORDER_FIXED ? 2 : CAP > 64 ? 4 : EC_MINB))   // tree and wide-table variants need more registers
+__global__ void __launch_bounds__(EC_MAXT, (ORDER != EC_ORDER_FIXED ? (CAP > 64 ? 2 : EC_PW_MINB) : CAP > 64 ? 4 : EC_MINB))   // tree and wide-table variants need more registers
 apply_kernel(const ApplyArgs a, const __grid_constant__ PtrTable<CAP> tbl) {
     typedef Elem<DT> E;
     typedef typename E::In In;
@@ -395,8 +398,23 @@ apply_kernel(const ApplyArgs a, const __grid_constant__ PtrTable<CAP> tbl) {
         for (size_t w = tid; w < nunits; w += nthr) {
             const bool isvec = w < nvec;
             const size_t e0 = isvec ? w * PV : nvec * PV + (w - nvec);   // first element of this unit
-            Acc stack[TREE_LEVELS][PV];
+            constexpr int LEVELS = CAP <= 64 ? 3 : TREE_LEVELS;     // 64 ranks / 8 per leaf block = 2^3 blocks
+            Acc stack[LEVELS][PV];
             Acc node[PV];
+            // bf16 moves only 8 bytes per rank and thread: the loads of the next leaf block are issued before
+            // the current one is reduced, so that twice as many bytes are in flight
+            uint2 pre[8];
+            auto fetch8 = [&](int blk_i) {
+                const int q0 = blk_i * leaf;
+                const unsigned bt = (unsigned)(s_new[q0 >> 6] >> (q0 & 63)) & ((1u << leaf) - 1u);
+#pragma unroll
+                for (int u = 0; u < 8; ++u)
+                    if ((bt >> u) & 1u)
+                        pre[u] = ld_stream8(reinterpret_cast<const char*>(tbl.p[q0 + u]) + (lo + e0) * sizeof(In), pol);
+            };
+            if constexpr (DT == EC_BF16) {
+                if (isvec) fetch8(0);
+            }
             for (int blk = 0; blk < nblk; ++blk) {
                 const int r0 = blk * leaf;
                 const unsigned byte = (unsigned)(s_new[r0 >> 6] >> (r0 & 63)) & ((1u << leaf) - 1u);
@@ -406,14 +424,17 @@ apply_kernel(const ApplyArgs a, const __grid_constant__ PtrTable<CAP> tbl) {
 #pragma unroll
                     for (int e = 0; e < PV; ++e) lv[u][e] = ident<OP>(Acc());
                 }
+                uint2 raw[8];                                  // bf16: four values = 8 bytes per rank
+                if constexpr (DT == EC_BF16) {
+                    if (isvec) {
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) raw[u] = pre[u];
+                        if (blk + 1 < nblk) fetch8(blk + 1);
+                    }
+                }
                 if (byte != 0) {
                     if (isvec) {
                         if constexpr (DT == EC_BF16) {
-                            uint2 raw[8];                      // four bf16 values = 8 bytes
-#pragma unroll
-                            for (int u = 0; u < 8; ++u)
-                                if ((byte >> u) & 1u)
-                                    raw[u] = ld_stream8(reinterpret_cast<const char*>(tbl.p[r0 + u]) + (lo + e0) * sizeof(In), pol);
 #pragma unroll
                             for (int u = 0; u < 8; ++u)
                                 if ((byte >> u) & 1u) {
@@ -450,7 +471,7 @@ apply_kernel(const ApplyArgs a, const __grid_constant__ PtrTable<CAP> tbl) {
                 }
                 bool carry = true;
 #pragma unroll
-                for (int l = 0; l < TREE_LEVELS; ++l) {
+                for (int l = 0; l < LEVELS; ++l) {
                     if (l < nlev && carry) {
                         if ((blk >> l) & 1) {
 #pragma unroll
