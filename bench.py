@@ -557,6 +557,24 @@ def extras(args, dev, stream, peak):
     out["alltoall_P64_32KiB_blocks"] = entry
     del a_send, a_recv
 
+    # Broadcast with the paper's data thresholds (a quarter, half, three quarters, all of the vector): 16 ranks, 64 MiB
+    P, n, seg = 16, 1 << 24, 65536
+    b_src = torch.randn(n, device=dev)
+    b_dst = [b_src if r == 0 else torch.empty(n, device=dev) for r in range(P)]
+    b_words = torch.empty(n // seg, dtype=torch.int64, device=dev)
+    b_tbl = (C.c_void_p * P)(*[t.data_ptr() for t in b_dst])
+    entry = {}
+    for frac in (0.25, 0.5, 0.75, 1.0):
+        ms = time_calls(stream, lambda: L.ec_bcast(b_src.data_ptr(), b_tbl, P, 0, n, ec.F32, seg, frac,
+                                                   b_words.data_ptr(), st), reps)
+        m, ci = mean_ci(ms)
+        nbytes = int(frac * n) * 4 * P                      # read once, written P - 1 times
+        entry[f"threshold_{int(frac * 100)}"] = {"ms": round(m, 5), "ci95": round(ci, 5), "GBps": round(nbytes / m / 1e6, 1),
+                                                 "frac_measured": round(nbytes / m / 1e6 / peak, 4), "bytes": nbytes}
+    entry["note"] = "root in place; bytes = delivered prefix read once + written to 15 receive buffers"
+    out["bcast_P16_f32_n2^24"] = entry
+    del b_src, b_dst
+
     # config 4 gather
     P = 256
     counts = inputs.gather_counts(1004, P)

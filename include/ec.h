@@ -370,6 +370,25 @@ int ec_kmeans_partials_static(const float* points, const int32_t* labels, size_t
  * "status" parameters).  host_mask is HOST memory, uint64 [S][W], written.
  * ------------------------------------------------------------------------- */
 
+/* Eventually consistent Broadcast (Sec. III-B): the root ships only the leading share of its
+ * vector that the threshold `data_fraction` names, i.e. the first ceil(data_fraction * S) segments
+ * (the rule of ec_mask_data_fraction), into the receive buffer of every rank; the rest of every
+ * receive buffer is not touched.  On one device the binomial tree of the paper collapses into one
+ * pass that reads each delivered byte once and writes it P times.
+ *
+ *   src            device, n elements of `dtype`: the root's data.
+ *   dst_bufs       HOST array of P DEVICE pointers (n elements each).  NULL = that rank receives
+ *                  nothing.  dst_bufs[root] may be NULL or equal to src (nothing is copied for it);
+ *                  no other buffer may overlap src (EC_ERR_INVALID).
+ *   notify         device uint64 [S][W], written in full, or NULL: bit r of segment s is 1 iff
+ *                  s was delivered and (dst_bufs[r] != NULL or r == root) - ready to be used as
+ *                  the arrival mask of a consumer.
+ *
+ * 16-byte aligned pointers take the 128-bit path, anything else a byte-wise one.  One launch, no
+ * allocation, stateless. */
+int ec_bcast(const void* src, void* const* dst_bufs, int P, int root, size_t n, ec_dtype_t dtype,
+             size_t segment_size, double data_fraction, uint64_t* notify, ec_stream_t stream);
+
 /* Strategy 1, "send less data": the first ceil(fraction * S) segments of every rank count as
  * arrived, the others do not.  0 <= fraction <= 1. */
 int ec_mask_data_fraction(int P, size_t S, double fraction, uint64_t* host_mask);

@@ -317,6 +317,28 @@ def data_fraction_mask(P: int, S: int, fraction: float) -> np.ndarray:
     return _pack_words(arrived)
 
 
+def bcast(src: np.ndarray, dst_bufs, root: int, segment_size: int, data_fraction: float):
+    """Broadcast with a data threshold (Sec. III-B): the first ceil(fraction * S) segments of the root's
+    vector are written into every receive buffer that exists (entries of dst_bufs may be None, and the
+    root's own entry may be the source itself); nothing else is touched.  Works in place on dst_bufs and
+    returns the notification words uint64 [S][W]: bit r of segment s = rank r now holds segment s."""
+    import math
+    n, P = src.size, len(dst_bufs)
+    S = (n + segment_size - 1) // segment_size
+    keep = min(S, math.ceil(data_fraction * S))
+    holds = np.zeros((P, S), dtype=bool)
+    for r in range(P):
+        if dst_bufs[r] is None and r != root:
+            continue
+        for s in range(keep):
+            lo, hi = s * segment_size, min(n, (s + 1) * segment_size)
+            if dst_bufs[r] is not None and dst_bufs[r] is not src:
+                for i in range(lo, hi):
+                    dst_bufs[r][i] = src[i]
+            holds[r, s] = True
+    return _pack_words(holds)
+
+
 def _pack_words(arrived: np.ndarray) -> np.ndarray:
     P, S = arrived.shape
     out = np.zeros((S, (P + 63) // 64), dtype=np.uint64)

@@ -51,6 +51,7 @@ SYMBOLS = {
     "ec_kmeans_partials_static": (_i, [_vp, _vp, _sz, _i, _i, _i, _vp, _vp]),
     "ec_allgatherv_compact": (_i, [_vp, _vp, _i, _i, _vp, _vp, _vp, _sz, _vp, _vp]),
     "ec_alltoall": (_i, [_vp, _vp, _i, _sz, _vp, _vp, _vp]),
+    "ec_bcast": (_i, [_vp, _vp, _i, _i, _sz, _i, _sz, C.c_double, _vp, _vp]),
     "ec_mask_data_fraction": (_i, [_i, _sz, C.c_double, _vp]),
     "ec_mask_process_threshold": (_i, [_i, _sz, C.c_double, _vp, C.POINTER(_i)]),
     "ec_threshold_segments": (_i, [_vp, _sz, C.c_uint32, _vp, _vp]),
@@ -190,6 +191,13 @@ def allgatherv(bufs, counts, dtype: int, arrival_mask, displs, out, status, stre
     fn = lib().ec_allgatherv_compact if compact else lib().ec_allgatherv
     _check(fn(_table(bufs), _ptr(counts), len(bufs), dtype, _ptr(arrival_mask), _ptr(displs),
                                _ptr(out), cap, _ptr(status), _stream(stream)), "ec_allgatherv")
+
+
+def bcast(src, dst_bufs, root: int, dtype: int, segment_size: int, data_fraction: float, notify=None,
+          stream=None) -> None:
+    """ec_bcast: src and the entries of dst_bufs are device tensors (entries may be None)."""
+    _check(lib().ec_bcast(_ptr(src), _table(dst_bufs), len(dst_bufs), root, src.numel(), dtype, segment_size,
+                          data_fraction, _ptr(notify), _stream(stream)), "ec_bcast")
 
 
 class KMeans:
