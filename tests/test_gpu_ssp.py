@@ -102,3 +102,34 @@ def test_config2_shape_with_clocks_and_state_is_untouched():
         ref.apply(bufs, m, c, None, threads=8)
     assert np.array_equal(bits(to_host(d_res)), bits(c))
     ar.destroy()
+
+
+@pytest.mark.parametrize("order,P,n,seg", [(ec.ORDER_PAIRWISE, 8, 5000, 500), (ec.ORDER_PAIRWISE, 16, 1 << 16, 4096),
+                                           (ec.ORDER_PAIRWISE, 100, 3000, 256), (ec.ORDER_RING, 16, 1 << 16, 1024),
+                                           (ec.ORDER_RING, 6, 6 * 700, 100)])
+def test_stale_synchronous_apply_in_hypercube_and_ring_order(order, P, n, seg):
+    """Algorithm 1 is a hypercube allreduce: with the pairwise order the accepted contributions are summed as the
+    recursive-doubling tree sums them (an excluded process contributes the identity).  The checker composes its
+    own pieces: acceptance by clock gives a mask, the mask goes through its order-aware apply."""
+    S = (n + seg - 1) // seg
+    bufs = inputs.rank_buffers("normal_f32", 300 + P, P, n)
+    clocks = np.random.default_rng(P).integers(0, 8, size=(S, P)).astype(np.uint32)
+    clock, slack = 7, 2
+    accepted = (clocks >= clock - slack) & (clocks > 0)                       # [S][P]
+    ref = oracle.Allreduce(P, n, oracle.F32, oracle.SUM, seg)
+    want = np.full(n, np.nan, dtype=np.float32)
+    want_cnt = np.zeros(S, dtype=np.uint32)
+    ref.apply(bufs, inputs.pack_mask(accepted.T.copy()), want, want_cnt, order=order)
+    ar = ec.Allreduce(P, n, ec.F32, ec.SUM, seg, order)
+    d_res = torch.full((n,), float("nan"), device="cuda")
+    d_cnt = torch.zeros(S, dtype=torch.int32, device="cuda")
+    d_clk = torch.zeros(S, dtype=torch.int32, device="cuda")
+    d_wait = torch.zeros(S, dtype=torch.int32, device="cuda")
+    ar.ssp_apply([to_dev(b) for b in bufs], to_dev(clocks), clock, slack, d_res, d_cnt, d_clk, d_wait)
+    torch.cuda.synchronize()
+    assert np.array_equal(bits(to_host(d_res)), bits(want))
+    assert np.array_equal(d_cnt.cpu().numpy().view(np.uint32), want_cnt)
+    masked = np.where(accepted, clocks, np.uint32(0xFFFFFFFF)).min(axis=1)
+    assert np.array_equal(d_clk.cpu().numpy().view(np.uint32), np.where(accepted.any(axis=1), masked, 0).astype(np.uint32))
+    assert np.array_equal(d_wait.cpu().numpy().view(np.uint32), (P - accepted.sum(axis=1)).astype(np.uint32))
+    ar.destroy()
