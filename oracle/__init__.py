@@ -351,3 +351,94 @@ def _pack_words(arrived: np.ndarray) -> np.ndarray:
 
 def threshold_segments(contrib_count: np.ndarray, need: int) -> int:
     return int(sum(1 for c in contrib_count if c >= need))
+
+
+# ---------------------------------------------------------------------------------------------
+# Matrix factorisation trained by gradient steps whose item gradients go through the
+# stale-synchronous allreduce (the paper's experiment with allreduce_SSP, Sec. V; the paper names the
+# model and the collective, not the update rule: what follows is the textbook rule).
+#
+#   model      r_ui ~ <p_u, q_i>;  e_ui = r_ui - <p_u, q_i>
+#   rank r     owns the users [r*U/P, (r+1)*U/P) with all their ratings; user factors are local
+#   shared     the item factors; every rank contributes G_r[i] = sum over its ratings of e_ui * p_u
+#   one iteration at clock t (all errors e are taken at the factors the iteration starts from)
+#     1. contribution (r, s) - s an item segment of `segment_rows` rows - is recomputed if its bit in
+#        `refresh` is set, if it was never computed, or if it is older than t - slack (Algorithm 1:
+#        a contribution that is too stale is waited for); then its clock becomes t.  Otherwise the
+#        rank's buffer keeps the gradient it delivered earlier.
+#     2. R = sum over ranks of G_r in rank order (all clocks are now >= t - slack);
+#        seg_clock[s] = min over ranks of the clocks (the age of the result, Sec. III-A)
+#     3. p_u += lr * (sum_i e_ui * q_i - lam * p_u)        for every user
+#     4. q_i += lr * (R_i - lam * q_i)                       for every item
+#   sse = sum of e_ui^2 over all ratings at the start of the iteration.
+# ---------------------------------------------------------------------------------------------
+class MatrixFactorization:
+    def __init__(self, data: dict, user_factors: np.ndarray, item_factors: np.ndarray, lr: float, lam: float,
+                 segment_rows: int):
+        self.d = data
+        self.U, self.I, self.P = data["n_users"], data["n_items"], data["P"]
+        self.k = user_factors.shape[1]
+        self.pu = user_factors.astype(np.float64)
+        self.qi = item_factors.astype(np.float64)
+        self.lr, self.lam, self.seg = float(lr), float(lam), int(segment_rows)
+        self.S = (self.I + self.seg - 1) // self.seg
+        self.clock = 0
+        self.grad = np.zeros((self.P, self.I, self.k), dtype=np.float64)      # what each rank delivered last
+        self.notif_clock = np.zeros((self.S, self.P), dtype=np.uint32)
+
+    def rank_item_gradient(self, r: int) -> np.ndarray:
+        """G_r[i] = sum over rank r's ratings (u, i) of e_ui * p_u, at the current factors."""
+        d = self.d
+        out = np.zeros((self.I, self.k), dtype=np.float64)
+        for i in range(self.I):
+            for j in range(int(d["rank_item_ptr"][r, i]), int(d["rank_item_ptr"][r, i + 1])):
+                u = int(d["item_user"][j])
+                e = float(d["item_val"][j]) - float(np.dot(self.pu[u], self.qi[i]))
+                out[i] += e * self.pu[u]
+        return out
+
+    def user_gradient(self):
+        """(g_u = sum_i e_ui * q_i for every user, sum of e^2), at the current factors."""
+        d = self.d
+        g = np.zeros((self.U, self.k), dtype=np.float64)
+        sse = 0.0
+        for u in range(self.U):
+            for j in range(int(d["user_ptr"][u]), int(d["user_ptr"][u + 1])):
+                i = int(d["user_item"][j])
+                e = float(d["user_val"][j]) - float(np.dot(self.pu[u], self.qi[i]))
+                g[u] += e * self.qi[i]
+                sse += e * e
+        return g, sse
+
+    def iterate(self, refresh: np.ndarray | None, slack: int):
+        """One iteration; refresh is bool [P][S] or None (= everything fresh).
+        Returns (sse at the start of the iteration, seg_clock uint32 [S], refreshed bool [P][S])."""
+        self.clock += 1
+        t = self.clock
+        min_ok = t - slack if t > slack else 1
+        refreshed = np.zeros((self.P, self.S), dtype=bool)
+        for r in range(self.P):
+            fresh = None
+            for s in range(self.S):
+                want = refresh is None or bool(refresh[r, s])
+                c = int(self.notif_clock[s, r])
+                if want or c == 0 or c < min_ok:
+                    if fresh is None:
+                        fresh = self.rank_item_gradient(r)
+                    lo, hi = s * self.seg, min(self.I, (s + 1) * self.seg)
+                    self.grad[r, lo:hi] = fresh[lo:hi]
+                    self.notif_clock[s, r] = t
+                    refreshed[r, s] = True
+        reduced = np.zeros((self.I, self.k), dtype=np.float64)
+        for r in range(self.P):
+            reduced += self.grad[r]
+        seg_clock = self.notif_clock.min(axis=1).astype(np.uint32)
+        g_user, sse = self.user_gradient()
+        self.pu = self.pu + self.lr * (g_user - self.lam * self.pu)
+        self.qi = self.qi + self.lr * (reduced - self.lam * self.qi)
+        return sse, seg_clock, refreshed
+
+    def loss(self) -> float:
+        """0.5 * sum e^2 + 0.5 * lam * (|P|^2 + |Q|^2): the function whose gradient the steps follow."""
+        _, sse = self.user_gradient()
+        return 0.5 * sse + 0.5 * self.lam * (float((self.pu ** 2).sum()) + float((self.qi ** 2).sum()))

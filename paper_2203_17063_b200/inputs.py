@@ -28,6 +28,7 @@ _STREAM_COUNTS = 2 << 20
 _STREAM_KM_CENTRES = 3 << 20
 _STREAM_KM_POINTS = 4 << 20   # + chunk
 _STREAM_KM_MASK = 5 << 20     # + iteration
+_STREAM_MF = 6 << 20          # + purpose / iteration
 
 
 def _rng(seed: int, stream: int) -> np.random.Generator:
@@ -230,3 +231,63 @@ def kmeans_masks(seed: int, iters: int, P: int, K: int, p: float) -> list[np.nda
     """Per iteration the packed notification words [K][W]: contribution
     (rank, centroid row) has arrived with probability p."""
     return [pack_mask(_rng(seed, _STREAM_KM_MASK + t).random((P, K)) < p) for t in range(iters)]
+
+
+# --------------------------------------------------------------------------
+# Matrix-factorisation ratings (stand-in for the paper's MovieLens experiment)
+# --------------------------------------------------------------------------
+def mf_ratings(seed: int, n_users: int, n_items: int, k_true: int, nnz: int, P: int, noise: float = 0.1) -> dict:
+    """A sparse low-rank rating matrix, stored twice as such data usually is: by user
+    (CSR over all users; rank r owns the users [r*U/P, (r+1)*U/P) and so a contiguous
+    range of the ratings) and, inside every rank's share, by item.
+
+    Users are drawn uniformly, items with a popularity that falls off like a power law
+    (item = floor(I * x^2), x uniform), ratings are the inner product of two hidden
+    factor vectors with N(0, 1/k_true) entries plus N(0, noise^2).  Returns a dict with
+        user_ptr  int64 [U+1], user_item int32 [nnz], user_val fp32 [nnz]       (by user)
+        rank_item_ptr int64 [P][I+1] (offsets into the next two), item_user int32 [nnz],
+        item_val fp32 [nnz]                                                     (by rank, then item)
+    """
+    g = _rng(seed, _STREAM_MF)
+    users = np.sort(g.integers(0, n_users, size=nnz, dtype=np.int64))
+    items = np.minimum((n_items * g.random(nnz) ** 2).astype(np.int64), n_items - 1)
+    a = _rng(seed, _STREAM_MF + 1).standard_normal((n_users, k_true)).astype(np.float32) / np.float32(np.sqrt(k_true))
+    b = _rng(seed, _STREAM_MF + 2).standard_normal((n_items, k_true)).astype(np.float32) / np.float32(np.sqrt(k_true))
+    val = np.empty(nnz, dtype=np.float32)
+    chunk = 1 << 20
+    for lo in range(0, nnz, chunk):
+        hi = min(nnz, lo + chunk)
+        clean = np.einsum("jk,jk->j", a[users[lo:hi]], b[items[lo:hi]])
+        val[lo:hi] = clean + np.float32(noise) * _rng(seed, _STREAM_MF + 16 + lo // chunk).standard_normal(hi - lo, dtype=np.float32)
+    # inside one user the ratings are ordered by item
+    order = np.lexsort((items, users))
+    users, items, val = users[order], items[order], val[order]
+    user_ptr = np.zeros(n_users + 1, dtype=np.int64)
+    np.cumsum(np.bincount(users, minlength=n_users), out=user_ptr[1:])
+    rank_item_ptr = np.zeros((P, n_items + 1), dtype=np.int64)
+    item_user = np.empty(nnz, dtype=np.int32)
+    item_val = np.empty(nnz, dtype=np.float32)
+    for r in range(P):
+        lo, hi = int(user_ptr[r * n_users // P]), int(user_ptr[(r + 1) * n_users // P])
+        by_item = np.argsort(items[lo:hi], kind="stable")
+        item_user[lo:hi] = users[lo:hi][by_item]
+        item_val[lo:hi] = val[lo:hi][by_item]
+        rank_item_ptr[r, 0] = lo
+        np.cumsum(np.bincount(items[lo:hi], minlength=n_items), out=rank_item_ptr[r, 1:])
+        rank_item_ptr[r, 1:] += lo
+    return {"user_ptr": user_ptr, "user_item": items.astype(np.int32), "user_val": val,
+            "rank_item_ptr": rank_item_ptr, "item_user": item_user, "item_val": item_val,
+            "n_users": n_users, "n_items": n_items, "nnz": nnz, "P": P}
+
+
+def mf_init_factors(seed: int, n_users: int, n_items: int, k: int, scale: float = 0.1) -> tuple[np.ndarray, np.ndarray]:
+    """Starting factors: small normal values, fp32 [U][k] and [I][k]."""
+    pu = (scale * _rng(seed, _STREAM_MF + 3).standard_normal((n_users, k))).astype(np.float32)
+    qi = (scale * _rng(seed, _STREAM_MF + 4).standard_normal((n_items, k))).astype(np.float32)
+    return pu, qi
+
+
+def mf_refresh_masks(seed: int, iters: int, P: int, S: int, p: float) -> list[np.ndarray]:
+    """Per iteration the packed words [S][W]: the gradient of (rank, item segment) is delivered fresh
+    with probability p (the others keep what they sent last)."""
+    return [pack_mask(_rng(seed, _STREAM_MF + 1024 + t).random((P, S)) < p) for t in range(iters)]
