@@ -598,6 +598,49 @@ def extras(args, dev, stream, peak):
     del db, d_out
 
     out["config5_kmeans_N2^22_D32_K64_P64"] = kmeans_case(dev, stream, reps=5)
+    out["mf_ssp_U2^17_I2^14_k32_nnz2^23_P16"] = mf_case(dev, stream)
+    return out
+
+
+def mf_case(dev, stream, iters=20):
+    """Matrix factorisation over the stale-synchronous allreduce (stands in for the paper's MovieLens experiment):
+    2^17 users, 2^14 items, 32 factors, 2^23 synthetic ratings, 16 ranks, item segments of 64 rows; each
+    contribution is delivered fresh with probability 0.5, otherwise reused until it is older than the slack."""
+    import torch
+    from paper_2203_17063_b200 import binding as ec
+    from paper_2203_17063_b200 import inputs
+    U, I, k, nnz, P, seg_rows = 1 << 17, 1 << 14, 32, 1 << 23, 16, 64
+    d = inputs.mf_ratings(1006, U, I, 16, nnz, P)
+    pu, qi = inputs.mf_init_factors(1006, U, I, k, 0.3)
+    dd = {key: torch.from_numpy(d[key]).to(dev) for key in ("user_ptr", "user_item", "user_val", "rank_item_ptr",
+                                                             "item_user", "item_val")}
+    d_pu, d_qi = torch.from_numpy(pu).to(dev), torch.from_numpy(qi).to(dev)
+    S = (I + seg_rows - 1) // seg_rows
+    masks = [torch.from_numpy(m.view(np.int64)).to(dev) for m in inputs.mf_refresh_masks(2006, iters + 2, P, S, 0.5)]
+    sse = torch.empty(1, dtype=torch.float64, device=dev)
+    out = {}
+    for label, slack, use_masks in (("synchronous", 0, False), ("slack1_half_fresh", 1, True), ("slack2_half_fresh", 2, True)):
+        mf = ec.MatrixFactorization(dd, U, I, P, d_pu, d_qi, 1e-3, 0.05, seg_rows)
+        with torch.cuda.stream(stream):
+            for t in range(2):
+                mf.iterate(masks[t] if use_masks else None, slack, stream)
+            mf.get(sse=sse, stream=stream)
+            torch.cuda.synchronize()
+            mse0 = float(sse.item()) / nnz
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            for t in range(iters):
+                mf.iterate(masks[t + 2] if use_masks else None, slack, stream)
+            b.record(stream)
+            mf.get(sse=sse, stream=stream)
+            torch.cuda.synchronize()
+        ms = a.elapsed_time(b)
+        out[label] = {"iterations_per_s": round(iters / (ms * 1e-3), 1), "ms_per_iteration": round(ms / iters, 4),
+                      "mse_before": round(mse0, 5), "mse_after_20_iterations": round(float(sse.item()) / nnz, 5)}
+        mf.destroy()
+    out["note"] = ("5 launches per iteration: refresh decision, item gradients of the refreshed (rank, segment) pairs, "
+                   "ec_allreduce_ssp_apply over 16 x 2 MiB, user step, item step; mse = mean squared error at the start "
+                   "of the last iteration")
     return out
 
 

@@ -365,6 +365,64 @@ int ec_kmeans_partials_static(const float* points, const int32_t* labels, size_t
                               float* partials, ec_stream_t stream);
 
 /* ------------------------------------------------------------------------- *
+ * Matrix factorisation whose item gradients go through the stale-synchronous
+ * allreduce (the experiment of Sec. V; the paper names the model and the
+ * collective, the update rule here is the textbook one).
+ *
+ * r_ui ~ <p_u, q_i>, k = 32 or 64 factors.  Rank r owns the users
+ * [r*U/P, (r+1)*U/P) with all their ratings; user factors are updated locally,
+ * item factors are shared.  The ratings are given twice: by user (CSR over all
+ * users: user_ptr int64 [U+1], user_item int32 [nnz], user_val fp32 [nnz]) and,
+ * inside every rank's share, by item (rank_item_ptr int64 [P][I+1] = offsets
+ * into item_user int32 [nnz] / item_val fp32 [nnz]).  All six arrays are DEVICE
+ * memory owned by the caller and must stay valid until destroy.
+ *
+ * One ec_mf_iterate at clock t (the clock starts at 0 and is raised first; all
+ * errors e_ui = r_ui - <p_u, q_i> are taken at the factors the call starts from):
+ *   1. the contribution G_r[i] = sum over rank r's ratings of e_ui * p_u of a
+ *      (rank, item segment) pair is recomputed if its bit in refresh_mask is set
+ *      (device uint64 [S][W], S = ceil(I / segment_rows); NULL = all), if it was
+ *      never computed, or if its clock is below t - slack (Algorithm 1: a
+ *      contribution that is too stale is waited for); its clock becomes t.
+ *      Otherwise the rank's buffer keeps what it delivered before.
+ *   2. R = ec_allreduce_ssp_apply over the P buffers (sum, rank order).
+ *   3. p_u += lr * (sum_i e_ui * q_i - lambda * p_u) for every user.
+ *   4. q_i += lr * (R_i - lambda * q_i) for every item.
+ * Sums run in storage order with a fixed shape, so results repeat bit for bit.
+ * ------------------------------------------------------------------------- */
+typedef struct ec_mf ec_mf_t;
+
+/* Bytes of device workspace (factors, P gradient buffers, clocks, the allreduce's
+ * words).  0 on invalid arguments (k other than 32 or 64, P > n_users, ...). */
+size_t ec_mf_workspace_bytes(int n_users, int n_items, int k, int P, size_t segment_rows);
+
+/* user_factors fp32 [U][k] and item_factors fp32 [I][k] (device) are copied.
+ * workspace as in ec_allreduce_init (NULL: the library allocates it).  Must not
+ * be called during stream capture (it synchronises the legacy default stream). */
+int ec_mf_init(ec_mf_t** mf, int n_users, int n_items, int k, int P, const int64_t* user_ptr, const int32_t* user_item,
+               const float* user_val, const int64_t* rank_item_ptr, const int32_t* item_user, const float* item_val,
+               const float* user_factors, const float* item_factors, float lr, float lambda, size_t segment_rows,
+               void* workspace, size_t workspace_bytes);
+
+/* One iteration as described above: five launches on `stream`, no allocation. */
+int ec_mf_iterate(ec_mf_t* mf, const uint64_t* refresh_mask, uint32_t slack, ec_stream_t stream);
+
+/* Replace the factors (device to device copies on `stream`); clocks and the
+ * delivered gradients are kept. */
+int ec_mf_set_factors(ec_mf_t* mf, const float* user_factors, const float* item_factors, ec_stream_t stream);
+
+/* Copy out (device pointers, any may be NULL): the factors, sse = sum of e_ui^2
+ * over all ratings at the start of the last iteration (one double), the clock of
+ * each segment of the last reduction uint32 [S] (the minimum over the ranks,
+ * Sec. III-A), the clocks of all contributions uint32 [S][P], and the number of
+ * contributions the last reduction found too stale uint32 [S] (always 0 here,
+ * since step 1 refreshes them). */
+int ec_mf_get(ec_mf_t* mf, float* user_factors, float* item_factors, double* sse, uint32_t* seg_clock,
+              uint32_t* notif_clock, uint32_t* wait_count, ec_stream_t stream);
+
+int ec_mf_destroy(ec_mf_t* mf);
+
+/* ------------------------------------------------------------------------- *
  * Threshold variants of Reduce / Broadcast (Sec. III-B) as notification words,
  * and the threshold test on the status output (Sec. III: "threshold" and
  * "status" parameters).  host_mask is HOST memory, uint64 [S][W], written.

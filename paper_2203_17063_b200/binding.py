@@ -51,6 +51,12 @@ SYMBOLS = {
     "ec_kmeans_partials_static": (_i, [_vp, _vp, _sz, _i, _i, _i, _vp, _vp]),
     "ec_allgatherv_compact": (_i, [_vp, _vp, _i, _i, _vp, _vp, _vp, _sz, _vp, _vp]),
     "ec_alltoall": (_i, [_vp, _vp, _i, _sz, _vp, _vp, _vp]),
+    "ec_mf_workspace_bytes": (_sz, [_i, _i, _i, _i, _sz]),
+    "ec_mf_init": (_i, [C.POINTER(_vp), _i, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, C.c_float, C.c_float, _sz, _vp, _sz]),
+    "ec_mf_iterate": (_i, [_vp, _vp, C.c_uint32, _vp]),
+    "ec_mf_set_factors": (_i, [_vp, _vp, _vp, _vp]),
+    "ec_mf_get": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "ec_mf_destroy": (_i, [_vp]),
     "ec_bcast": (_i, [_vp, _vp, _i, _i, _sz, _i, _sz, C.c_double, _vp, _vp]),
     "ec_mask_data_fraction": (_i, [_i, _sz, C.c_double, _vp]),
     "ec_mask_process_threshold": (_i, [_i, _sz, C.c_double, _vp, C.POINTER(_i)]),
@@ -298,3 +304,45 @@ def alltoall(send_bufs, recv_bufs, block_bytes: int, arrival_mask=None, recv_cou
     """ec_alltoall: recv[d] block s <- send[s] block d for every notified (d, s); device tensors."""
     _check(lib().ec_alltoall(_table(send_bufs), _table(recv_bufs), len(send_bufs), block_bytes, _ptr(arrival_mask),
                              _ptr(recv_count), _stream(stream)), "ec_alltoall")
+
+
+class MatrixFactorization:
+    """ec_mf_*: data is a dict of device tensors (user_ptr, user_item, user_val, rank_item_ptr, item_user,
+    item_val) laid out as inputs.mf_ratings describes; the factors are device fp32 tensors."""
+
+    def __init__(self, data: dict, n_users: int, n_items: int, P: int, user_factors: torch.Tensor,
+                 item_factors: torch.Tensor, lr: float, lam: float, segment_rows: int):
+        L = lib()
+        self.data = data                                   # keep alive: the library does not copy the ratings
+        self.U, self.I, self.P, self.k = n_users, n_items, P, user_factors.shape[1]
+        self.S = (n_items + segment_rows - 1) // segment_rows
+        need = L.ec_mf_workspace_bytes(n_users, n_items, self.k, P, segment_rows)
+        self._ws = torch.empty(max(need, 256), dtype=torch.uint8, device=user_factors.device)
+        h = C.c_void_p()
+        _check(L.ec_mf_init(C.byref(h), n_users, n_items, self.k, P, _ptr(data["user_ptr"]), _ptr(data["user_item"]),
+                            _ptr(data["user_val"]), _ptr(data["rank_item_ptr"]), _ptr(data["item_user"]),
+                            _ptr(data["item_val"]), _ptr(user_factors), _ptr(item_factors), lr, lam, segment_rows,
+                            _ptr(self._ws), need), "ec_mf_init")
+        self._h = h
+
+    def iterate(self, refresh_mask=None, slack: int = 0, stream=None) -> None:
+        _check(lib().ec_mf_iterate(self._h, _ptr(refresh_mask), slack, _stream(stream)), "ec_mf_iterate")
+
+    def set_factors(self, user_factors, item_factors, stream=None) -> None:
+        _check(lib().ec_mf_set_factors(self._h, _ptr(user_factors), _ptr(item_factors), _stream(stream)), "ec_mf_set_factors")
+
+    def get(self, user_factors=None, item_factors=None, sse=None, seg_clock=None, notif_clock=None, wait_count=None,
+            stream=None) -> None:
+        _check(lib().ec_mf_get(self._h, _ptr(user_factors), _ptr(item_factors), _ptr(sse), _ptr(seg_clock),
+                               _ptr(notif_clock), _ptr(wait_count), _stream(stream)), "ec_mf_get")
+
+    def destroy(self) -> None:
+        if getattr(self, "_h", None):
+            lib().ec_mf_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass

@@ -17,7 +17,7 @@ INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libec_b200.so")
 OBJDIR = os.path.join(HERE, "build")
 
-SOURCES = ["ec_allreduce.cu", "ec_allgatherv.cu", "ec_kmeans.cu", "ec_threshold.cu", "ec_alltoall.cu", "ec_bcast.cu"]
+SOURCES = ["ec_allreduce.cu", "ec_allgatherv.cu", "ec_kmeans.cu", "ec_threshold.cu", "ec_alltoall.cu", "ec_bcast.cu", "ec_mf.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "--fmad=true",          # contraction is irrelevant to the ordered sums (explicit __fadd_rn) and wanted in the distance loop

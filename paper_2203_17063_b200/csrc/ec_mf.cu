@@ -1,0 +1,326 @@
+// Matrix factorisation trained by gradient steps whose item gradients are combined by the
+// stale-synchronous allreduce (the experiment of Sec. V: allreduce_SSP inside an ML solver).
+//
+// r_ui ~ <p_u, q_i>.  Rank r owns a contiguous block of users with all their ratings, so user factors
+// are updated locally; the item factors are shared, and every rank contributes the gradient
+// G_r[i] = sum over its ratings of e_ui * p_u.  The P gradients live as rank buffers in device memory
+// with one logical clock per (item segment, rank); an iteration recomputes only the contributions that
+// are delivered fresh (or have become too stale: Algorithm 1's wait), reduces all buffers with
+// ec_allreduce_ssp_apply and takes the step.  One warp owns one row (an item of one rank, or a user):
+// it walks the row's ratings in storage order, 32 at a time, with the factor vector spread over the
+// lanes, so every sum has a fixed order and results repeat bit for bit from run to run.
+
+#include <new>
+
+#include "ec_common.cuh"
+
+namespace ec {
+namespace {
+
+constexpr int MF_THREADS = 256;
+constexpr int MF_WARPS = MF_THREADS / 32;
+
+struct MfArgs {
+    const int64_t* user_ptr; const int32_t* user_item; const float* user_val;
+    const int64_t* rank_item_ptr; const int32_t* item_user; const float* item_val;
+    float* pu; float* qi; float* grad; const float* reduced;
+    uint32_t* notif_clock; uint8_t* refreshed; const uint64_t* refresh;
+    double* sse_partial; double* sse;
+    size_t seg_rows, S;
+    int U, I, P, W;
+    uint32_t clock, min_ok;
+    float lr, lam;
+    int sse_blocks;
+};
+
+__device__ __forceinline__ float warp_sum(float x) {
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) x += __shfl_xor_sync(0xffffffffu, x, d);
+    return x;
+}
+
+// which contributions are recomputed in this iteration, and their new clocks
+__global__ void mf_decide_kernel(const MfArgs a) {
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= a.S * (size_t)a.P) return;
+    const size_t s = i / (size_t)a.P;
+    const int r = (int)(i - s * (size_t)a.P);
+    bool want = true;
+    if (a.refresh != nullptr) want = (a.refresh[s * (size_t)a.W + (r >> 6)] >> (r & 63)) & 1ull;
+    const uint32_t c = a.notif_clock[i];
+    const bool fresh = want || c == 0u || c < a.min_ok;      // never delivered, or too stale: it is waited for
+    a.refreshed[i] = fresh ? 1 : 0;
+    if (fresh) a.notif_clock[i] = a.clock;
+}
+
+// One warp per row.  SIDE 0: row = (rank r, item i), other = users, writes G_r[i].
+//                    SIDE 1: row = user u, other = items, takes the user step in place and adds up e^2.
+// KPL = factor entries per lane (k = 32 * KPL).
+template <int KPL, int SIDE>
+__global__ void __launch_bounds__(MF_THREADS) mf_row_kernel(const MfArgs a) {
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    const size_t row = (size_t)blockIdx.x * MF_WARPS + wid;
+    const size_t rows = SIDE == 0 ? (size_t)a.P * a.I : (size_t)a.U;
+    __shared__ float s_sse[MF_WARPS];
+    float sse = 0.0f;
+    if (row < rows) {
+        const int k = 32 * KPL;
+        int r = 0;
+        size_t self = row;                       // index of the row's own factor vector
+        bool active = true;
+        if (SIDE == 0) {
+            r = (int)(row / (size_t)a.I);
+            self = row - (size_t)r * a.I;
+            active = a.refreshed[(self / a.seg_rows) * (size_t)a.P + r] != 0;
+        }
+        if (active) {
+            const int64_t beg = SIDE == 0 ? a.rank_item_ptr[(size_t)r * (a.I + 1) + self] : a.user_ptr[self];
+            const int64_t end = SIDE == 0 ? a.rank_item_ptr[(size_t)r * (a.I + 1) + self + 1] : a.user_ptr[self + 1];
+            const int32_t* idx = SIDE == 0 ? a.item_user : a.user_item;
+            const float* val = SIDE == 0 ? a.item_val : a.user_val;
+            const float* own = SIDE == 0 ? a.qi : a.pu;          // the row's factors
+            const float* oth = SIDE == 0 ? a.pu : a.qi;          // the factors its ratings point at
+            float mine[KPL], g[KPL];
+#pragma unroll
+            for (int c = 0; c < KPL; ++c) {
+                mine[c] = own[self * k + c * 32 + lane];
+                g[c] = 0.0f;
+            }
+            for (int64_t j0 = beg; j0 < end; j0 += 32) {
+                const int cnt = end - j0 < 32 ? (int)(end - j0) : 32;
+                const int my_i = lane < cnt ? idx[j0 + lane] : 0;
+                const float my_v = lane < cnt ? val[j0 + lane] : 0.0f;
+                for (int t0 = 0; t0 < cnt; t0 += 4) {
+                    float x[4][KPL], dot[4];
+#pragma unroll
+                    for (int t = 0; t < 4; ++t) {
+                        const int o = __shfl_sync(0xffffffffu, my_i, (t0 + t) & 31);
+                        dot[t] = 0.0f;
+#pragma unroll
+                        for (int c = 0; c < KPL; ++c) {
+                            x[t][c] = t0 + t < cnt ? __ldg(oth + (size_t)o * k + c * 32 + lane) : 0.0f;
+                            dot[t] = fmaf(x[t][c], mine[c], dot[t]);
+                        }
+                    }
+#pragma unroll
+                    for (int t = 0; t < 4; ++t) dot[t] = warp_sum(dot[t]);
+#pragma unroll
+                    for (int t = 0; t < 4; ++t) {
+                        const float v = __shfl_sync(0xffffffffu, my_v, (t0 + t) & 31);
+                        const float e = t0 + t < cnt ? v - dot[t] : 0.0f;
+#pragma unroll
+                        for (int c = 0; c < KPL; ++c) g[c] = fmaf(e, x[t][c], g[c]);
+                        if (SIDE == 1) sse = fmaf(e, e, sse);
+                    }
+                }
+            }
+#pragma unroll
+            for (int c = 0; c < KPL; ++c) {
+                if (SIDE == 0) a.grad[((size_t)r * a.I + self) * k + c * 32 + lane] = g[c];
+                else a.pu[self * k + c * 32 + lane] = mine[c] + a.lr * (g[c] - a.lam * mine[c]);
+            }
+        }
+    }
+    if (SIDE == 1) {
+        if (lane == 0) s_sse[wid] = sse;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            double t = 0.0;
+            for (int w = 0; w < MF_WARPS; ++w) t += (double)s_sse[w];
+            a.sse_partial[blockIdx.x] = t;
+        }
+    }
+}
+
+// q_i += lr * (R_i - lam * q_i); the first block also adds up the per-block error sums in a fixed order
+__global__ void __launch_bounds__(MF_THREADS) mf_item_step_kernel(const MfArgs a, size_t n) {
+    const size_t i = (size_t)blockIdx.x * MF_THREADS + threadIdx.x;
+    if (i < n) {
+        const float q = a.qi[i];
+        a.qi[i] = q + a.lr * (a.reduced[i] - a.lam * q);
+    }
+    if (blockIdx.x == 0) {
+        __shared__ double s[MF_THREADS];
+        double t = 0.0;
+        for (int b = threadIdx.x; b < a.sse_blocks; b += MF_THREADS) t += a.sse_partial[b];
+        s[threadIdx.x] = t;
+        __syncthreads();
+        for (int d = MF_THREADS / 2; d > 0; d >>= 1) {
+            if (threadIdx.x < d) s[threadIdx.x] += s[threadIdx.x + d];
+            __syncthreads();
+        }
+        if (threadIdx.x == 0) *a.sse = s[0];
+    }
+}
+
+struct MfLayout {
+    size_t pu, qi, grad, reduced, notif, seg_clock, count, wait, refreshed, sse_partial, sse, ar, total;
+    int sse_blocks;
+};
+
+bool mf_plan(int U, int I, int k, int P, size_t seg_rows, MfLayout* L) {
+    if (U < 1 || I < 1 || P < 1 || P > EC_MAX_RANKS || P > U || seg_rows == 0 || (k != 32 && k != 64)) return false;
+    const size_t S = ((size_t)I + seg_rows - 1) / seg_rows;
+    size_t off = 0;
+    L->pu = off; off = align_up(off + (size_t)U * k * 4, 256);
+    L->qi = off; off = align_up(off + (size_t)I * k * 4, 256);
+    L->grad = off; off = align_up(off + (size_t)P * I * k * 4, 256);
+    L->reduced = off; off = align_up(off + (size_t)I * k * 4, 256);
+    L->notif = off; off = align_up(off + S * P * 4, 256);
+    L->seg_clock = off; off = align_up(off + S * 4, 256);
+    L->count = off; off = align_up(off + S * 4, 256);
+    L->wait = off; off = align_up(off + S * 4, 256);
+    L->refreshed = off; off = align_up(off + S * P, 256);
+    L->sse_blocks = (U + MF_WARPS - 1) / MF_WARPS;
+    L->sse_partial = off; off = align_up(off + (size_t)L->sse_blocks * 8, 256);
+    L->sse = off; off = align_up(off + 8, 256);
+    L->ar = off; off = align_up(off + ec_allreduce_workspace_bytes(P, (size_t)I * k, seg_rows * k), 256);
+    L->total = off;
+    return true;
+}
+
+}  // namespace
+}  // namespace ec
+
+using namespace ec;
+
+struct ec_mf {
+    MfArgs a;
+    MfLayout L;
+    int k;
+    void* ws;
+    bool own_ws;
+    ec_ctx_t* ar;
+    uint32_t* seg_clock; uint32_t* count; uint32_t* wait;
+    const void* bufs[EC_MAX_RANKS];
+};
+
+extern "C" {
+
+size_t ec_mf_workspace_bytes(int n_users, int n_items, int k, int P, size_t segment_rows) {
+    MfLayout L;
+    if (!mf_plan(n_users, n_items, k, P, segment_rows, &L)) return 0;
+    return L.total;
+}
+
+int ec_mf_init(ec_mf_t** out, int n_users, int n_items, int k, int P, const int64_t* user_ptr, const int32_t* user_item,
+               const float* user_val, const int64_t* rank_item_ptr, const int32_t* item_user, const float* item_val,
+               const float* user_factors, const float* item_factors, float lr, float lambda, size_t segment_rows,
+               void* workspace, size_t workspace_bytes) {
+    if (!out) return EC_ERR_INVALID;
+    *out = nullptr;
+    if (!user_ptr || !user_item || !user_val || !rank_item_ptr || !item_user || !item_val || !user_factors || !item_factors)
+        return EC_ERR_INVALID;
+    if (n_users < 1 || n_items < 1 || P < 1 || P > EC_MAX_RANKS || P > n_users || segment_rows == 0) return EC_ERR_INVALID;
+    if (k != 32 && k != 64) return EC_ERR_UNSUPPORTED;
+    MfLayout L;
+    if (!mf_plan(n_users, n_items, k, P, segment_rows, &L)) return EC_ERR_INVALID;
+    if (workspace && (workspace_bytes < L.total || (reinterpret_cast<uintptr_t>(workspace) & 255u))) return EC_ERR_CAPACITY;
+    ec_mf* m = new (std::nothrow) ec_mf();
+    if (!m) return EC_ERR_INVALID;
+    m->own_ws = workspace == nullptr;
+    m->ws = workspace;
+    if (m->own_ws) {
+        cudaError_t e = cudaMalloc(&m->ws, L.total);
+        if (e != cudaSuccess) { delete m; return cuda_fail(e); }
+    }
+    char* base = static_cast<char*>(m->ws);
+    m->L = L;
+    m->k = k;
+    MfArgs& a = m->a;
+    a.user_ptr = user_ptr; a.user_item = user_item; a.user_val = user_val;
+    a.rank_item_ptr = rank_item_ptr; a.item_user = item_user; a.item_val = item_val;
+    a.pu = reinterpret_cast<float*>(base + L.pu);
+    a.qi = reinterpret_cast<float*>(base + L.qi);
+    a.grad = reinterpret_cast<float*>(base + L.grad);
+    a.reduced = reinterpret_cast<float*>(base + L.reduced);
+    a.notif_clock = reinterpret_cast<uint32_t*>(base + L.notif);
+    a.refreshed = reinterpret_cast<uint8_t*>(base + L.refreshed);
+    a.refresh = nullptr;
+    a.sse_partial = reinterpret_cast<double*>(base + L.sse_partial);
+    a.sse = reinterpret_cast<double*>(base + L.sse);
+    a.seg_rows = segment_rows;
+    a.S = ((size_t)n_items + segment_rows - 1) / segment_rows;
+    a.U = n_users; a.I = n_items; a.P = P; a.W = (P + 63) / 64;
+    a.clock = 0; a.min_ok = 1;
+    a.lr = lr; a.lam = lambda;
+    a.sse_blocks = L.sse_blocks;
+    m->seg_clock = reinterpret_cast<uint32_t*>(base + L.seg_clock);
+    m->count = reinterpret_cast<uint32_t*>(base + L.count);
+    m->wait = reinterpret_cast<uint32_t*>(base + L.wait);
+    for (int r = 0; r < P; ++r) m->bufs[r] = a.grad + (size_t)r * n_items * k;
+    // clocks 0 = nothing delivered yet; gradients and sums start at zero
+    cudaError_t e = cudaMemsetAsync(base + L.grad, 0, L.ar - L.grad, 0);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(a.pu, user_factors, (size_t)n_users * k * 4, cudaMemcpyDeviceToDevice, 0);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(a.qi, item_factors, (size_t)n_items * k * 4, cudaMemcpyDeviceToDevice, 0);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(0);
+    int rc = e == cudaSuccess ? EC_OK : cuda_fail(e);
+    if (rc == EC_OK)
+        rc = ec_allreduce_init(&m->ar, P, (size_t)n_items * k, EC_F32, EC_SUM, segment_rows * k, EC_ORDER_FIXED, base + L.ar,
+                               L.total - L.ar);
+    if (rc != EC_OK) {
+        if (m->own_ws) cudaFree(m->ws);
+        delete m;
+        return rc;
+    }
+    *out = m;
+    return EC_OK;
+}
+
+int ec_mf_iterate(ec_mf_t* m, const uint64_t* refresh_mask, uint32_t slack, ec_stream_t stream) {
+    if (!m) return EC_ERR_INVALID;
+    MfArgs& a = m->a;
+    a.clock += 1;
+    a.min_ok = a.clock > slack ? a.clock - slack : 1u;
+    a.refresh = refresh_mask;
+    const size_t pairs = a.S * (size_t)a.P;
+    mf_decide_kernel<<<(unsigned)((pairs + 255) / 256), 256, 0, stream>>>(a);
+    const size_t item_rows = (size_t)a.P * a.I;
+    const unsigned gi = (unsigned)((item_rows + MF_WARPS - 1) / MF_WARPS), gu = (unsigned)a.sse_blocks;
+    if (m->k == 32) mf_row_kernel<1, 0><<<gi, MF_THREADS, 0, stream>>>(a);
+    else mf_row_kernel<2, 0><<<gi, MF_THREADS, 0, stream>>>(a);
+    EC_CUDA(cudaGetLastError());
+    const size_t n = (size_t)a.I * m->k;
+    int rc = ec_allreduce_ssp_apply(m->ar, m->bufs, a.P, n, EC_F32, EC_SUM, a.seg_rows * m->k, a.notif_clock, a.clock, slack,
+                                    const_cast<float*>(a.reduced), m->count, m->seg_clock, m->wait, stream);
+    if (rc != EC_OK) return rc;
+    if (m->k == 32) mf_row_kernel<1, 1><<<gu, MF_THREADS, 0, stream>>>(a);
+    else mf_row_kernel<2, 1><<<gu, MF_THREADS, 0, stream>>>(a);
+    mf_item_step_kernel<<<(unsigned)((n + MF_THREADS - 1) / MF_THREADS), MF_THREADS, 0, stream>>>(a, n);
+    EC_CUDA(cudaGetLastError());
+    return EC_OK;
+}
+
+int ec_mf_set_factors(ec_mf_t* m, const float* user_factors, const float* item_factors, ec_stream_t stream) {
+    if (!m || !user_factors || !item_factors) return EC_ERR_INVALID;
+    EC_CUDA(cudaMemcpyAsync(m->a.pu, user_factors, (size_t)m->a.U * m->k * 4, cudaMemcpyDeviceToDevice, stream));
+    EC_CUDA(cudaMemcpyAsync(m->a.qi, item_factors, (size_t)m->a.I * m->k * 4, cudaMemcpyDeviceToDevice, stream));
+    return EC_OK;
+}
+
+int ec_mf_get(ec_mf_t* m, float* user_factors, float* item_factors, double* sse, uint32_t* seg_clock, uint32_t* notif_clock,
+              uint32_t* wait_count, ec_stream_t stream) {
+    if (!m) return EC_ERR_INVALID;
+    const MfArgs& a = m->a;
+    if (user_factors) EC_CUDA(cudaMemcpyAsync(user_factors, a.pu, (size_t)a.U * m->k * 4, cudaMemcpyDeviceToDevice, stream));
+    if (item_factors) EC_CUDA(cudaMemcpyAsync(item_factors, a.qi, (size_t)a.I * m->k * 4, cudaMemcpyDeviceToDevice, stream));
+    if (sse) EC_CUDA(cudaMemcpyAsync(sse, a.sse, 8, cudaMemcpyDeviceToDevice, stream));
+    if (seg_clock) EC_CUDA(cudaMemcpyAsync(seg_clock, m->seg_clock, a.S * 4, cudaMemcpyDeviceToDevice, stream));
+    if (notif_clock) EC_CUDA(cudaMemcpyAsync(notif_clock, a.notif_clock, a.S * a.P * 4, cudaMemcpyDeviceToDevice, stream));
+    if (wait_count) EC_CUDA(cudaMemcpyAsync(wait_count, m->wait, a.S * 4, cudaMemcpyDeviceToDevice, stream));
+    return EC_OK;
+}
+
+int ec_mf_destroy(ec_mf_t* m) {
+    if (!m) return EC_ERR_INVALID;
+    int rc = EC_OK;
+    if (m->ar) rc = ec_allreduce_destroy(m->ar);
+    if (m->own_ws && m->ws) {
+        cudaError_t e = cudaFree(m->ws);
+        if (e != cudaSuccess) rc = cuda_fail(e);
+    }
+    delete m;
+    return rc;
+}
+
+}  // extern "C"
