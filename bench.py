@@ -617,6 +617,7 @@ def mf_case(dev, stream, iters=20):
     d_pu, d_qi = torch.from_numpy(pu).to(dev), torch.from_numpy(qi).to(dev)
     S = (I + seg_rows - 1) // seg_rows
     masks = [torch.from_numpy(m.view(np.int64)).to(dev) for m in inputs.mf_refresh_masks(2006, iters + 2, P, S, 0.5)]
+    key_after = f"mse_after_{iters}_iterations"
     sse = torch.empty(1, dtype=torch.float64, device=dev)
     out = {}
     for label, slack, use_masks in (("synchronous", 0, False), ("slack1_half_fresh", 1, True), ("slack2_half_fresh", 2, True)):
@@ -636,7 +637,7 @@ def mf_case(dev, stream, iters=20):
             torch.cuda.synchronize()
         ms = a.elapsed_time(b)
         out[label] = {"iterations_per_s": round(iters / (ms * 1e-3), 1), "ms_per_iteration": round(ms / iters, 4),
-                      "mse_before": round(mse0, 5), "mse_after_20_iterations": round(float(sse.item()) / nnz, 5)}
+                      "mse_before": round(mse0, 5), key_after: round(float(sse.item()) / nnz, 5)}
         mf.destroy()
     out["note"] = ("5 launches per iteration: refresh decision, item gradients of the refreshed (rank, segment) pairs, "
                    "ec_allreduce_ssp_apply over 16 x 2 MiB, user step, item step; mse = mean squared error at the start "
@@ -755,7 +756,7 @@ def main():
     ap.add_argument("--profile-only", action="store_true", help="warm-up and timed steps only (for ncu captures)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-extras", action="store_true", help="headline workload only")
-    ap.add_argument("--workload", default="headline", choices=["headline", "kmeans"],
+    ap.add_argument("--workload", default="headline", choices=["headline", "kmeans", "mf"],
                     help="kmeans: time only the K-means driver (config 5) and print its own JSON line")
     ap.add_argument("--cpu-seconds", type=float, default=15.0, help="time budget of the CPU baseline leg")
     ap.add_argument("--threads", type=int, default=0, help="expert: threads per block of the apply kernel")
@@ -777,6 +778,12 @@ def main():
         dev = torch.device("cuda", local_rank)
         print(json.dumps({"workload": "kmeans", **kmeans_case(dev, torch.cuda.Stream(device=dev), reps=max(1, min(args.steps, 5)),
                                                                profile_only=args.profile_only)}))
+        return
+    if args.workload == "mf":
+        import torch
+        torch.cuda.set_device(local_rank)
+        dev = torch.device("cuda", local_rank)
+        print(json.dumps({"workload": "mf", **mf_case(dev, torch.cuda.Stream(device=dev), iters=max(1, min(args.steps, 20)))}))
         return
     run_ours(args, rank, world, local_rank)
 

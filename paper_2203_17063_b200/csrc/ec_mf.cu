@@ -7,8 +7,9 @@
 // with one logical clock per (item segment, rank); an iteration recomputes only the contributions that
 // are delivered fresh (or have become too stale: Algorithm 1's wait), reduces all buffers with
 // ec_allreduce_ssp_apply and takes the step.  One warp owns one row (an item of one rank, or a user):
-// it walks the row's ratings in storage order, 32 at a time, with the factor vector spread over the
-// lanes, so every sum has a fixed order and results repeat bit for bit from run to run.
+// it walks the row's ratings in storage order, four groups of eight lanes taking one rating each with
+// the factor vector spread over the group's lanes, so every sum has a fixed shape and results repeat bit
+// for bit from run to run.
 
 #include <new>
 
@@ -33,12 +34,6 @@ struct MfArgs {
     int sse_blocks;
 };
 
-__device__ __forceinline__ float warp_sum(float x) {
-#pragma unroll
-    for (int d = 16; d > 0; d >>= 1) x += __shfl_xor_sync(0xffffffffu, x, d);
-    return x;
-}
-
 // which contributions are recomputed in this iteration, and their new clocks
 __global__ void mf_decide_kernel(const MfArgs a) {
     const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -55,16 +50,21 @@ __global__ void mf_decide_kernel(const MfArgs a) {
 
 // One warp per row.  SIDE 0: row = (rank r, item i), other = users, writes G_r[i].
 //                    SIDE 1: row = user u, other = items, takes the user step in place and adds up e^2.
-// KPL = factor entries per lane (k = 32 * KPL).
-template <int KPL, int SIDE>
+// The warp works as four groups of eight lanes: a group takes one rating at a time (ratings t, t+4, t+8, ... of
+// the row go to group t mod 4), each of its lanes holds V = k/8 entries of the factor vectors, so one 128-bit
+// load per lane fetches the 128-byte factor row of the rating and the inner product needs three shuffle steps.
+// The four partial gradients are added at the end of the row ((g0+g1)+(g2+g3)): a fixed shape, the same bits
+// every run.  V4 = float4 per lane (k = 32 * V4).
+template <int V4, int SIDE>
 __global__ void __launch_bounds__(MF_THREADS) mf_row_kernel(const MfArgs a) {
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    const int grp = lane >> 3, sub = lane & 7;
     const size_t row = (size_t)blockIdx.x * MF_WARPS + wid;
     const size_t rows = SIDE == 0 ? (size_t)a.P * a.I : (size_t)a.U;
     __shared__ float s_sse[MF_WARPS];
     float sse = 0.0f;
     if (row < rows) {
-        const int k = 32 * KPL;
+        constexpr int k = 32 * V4;
         int r = 0;
         size_t self = row;                       // index of the row's own factor vector
         bool active = true;
@@ -80,44 +80,83 @@ __global__ void __launch_bounds__(MF_THREADS) mf_row_kernel(const MfArgs a) {
             const float* val = SIDE == 0 ? a.item_val : a.user_val;
             const float* own = SIDE == 0 ? a.qi : a.pu;          // the row's factors
             const float* oth = SIDE == 0 ? a.pu : a.qi;          // the factors its ratings point at
-            float mine[KPL], g[KPL];
+            // lane `sub` of every group holds entries [c*32 + sub*4, +4) of a factor vector, c < V4
+            float4 mine[V4], g[V4];
 #pragma unroll
-            for (int c = 0; c < KPL; ++c) {
-                mine[c] = own[self * k + c * 32 + lane];
-                g[c] = 0.0f;
+            for (int c = 0; c < V4; ++c) {
+                mine[c] = *reinterpret_cast<const float4*>(own + self * k + c * 32 + sub * 4);
+                g[c] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
             }
             for (int64_t j0 = beg; j0 < end; j0 += 32) {
                 const int cnt = end - j0 < 32 ? (int)(end - j0) : 32;
                 const int my_i = lane < cnt ? idx[j0 + lane] : 0;
                 const float my_v = lane < cnt ? val[j0 + lane] : 0.0f;
-                for (int t0 = 0; t0 < cnt; t0 += 4) {
-                    float x[4][KPL], dot[4];
+                for (int t0 = 0; t0 < cnt; t0 += 8) {            // two ratings per group in flight
+                    float4 x[2][V4];
+                    float dot[2], v[2];
+                    bool ok[2];
 #pragma unroll
-                    for (int t = 0; t < 4; ++t) {
-                        const int o = __shfl_sync(0xffffffffu, my_i, (t0 + t) & 31);
-                        dot[t] = 0.0f;
+                    for (int h = 0; h < 2; ++h) {
+                        const int t = t0 + h * 4 + grp;
+                        ok[h] = t < cnt;
+                        const int o = __shfl_sync(0xffffffffu, my_i, t & 31);
+                        v[h] = __shfl_sync(0xffffffffu, my_v, t & 31);
+                        dot[h] = 0.0f;
 #pragma unroll
-                        for (int c = 0; c < KPL; ++c) {
-                            x[t][c] = t0 + t < cnt ? __ldg(oth + (size_t)o * k + c * 32 + lane) : 0.0f;
-                            dot[t] = fmaf(x[t][c], mine[c], dot[t]);
+                        for (int c = 0; c < V4; ++c) {
+                            x[h][c] = ok[h] ? __ldg(reinterpret_cast<const float4*>(oth + (size_t)o * k + c * 32 + sub * 4))
+                                            : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                            dot[h] = fmaf(x[h][c].x, mine[c].x, dot[h]);
+                            dot[h] = fmaf(x[h][c].y, mine[c].y, dot[h]);
+                            dot[h] = fmaf(x[h][c].z, mine[c].z, dot[h]);
+                            dot[h] = fmaf(x[h][c].w, mine[c].w, dot[h]);
                         }
                     }
 #pragma unroll
-                    for (int t = 0; t < 4; ++t) dot[t] = warp_sum(dot[t]);
+                    for (int d = 1; d < 8; d <<= 1) {
+                        dot[0] += __shfl_xor_sync(0xffffffffu, dot[0], d);
+                        dot[1] += __shfl_xor_sync(0xffffffffu, dot[1], d);
+                    }
 #pragma unroll
-                    for (int t = 0; t < 4; ++t) {
-                        const float v = __shfl_sync(0xffffffffu, my_v, (t0 + t) & 31);
-                        const float e = t0 + t < cnt ? v - dot[t] : 0.0f;
+                    for (int h = 0; h < 2; ++h) {
+                        const float e = ok[h] ? v[h] - dot[h] : 0.0f;
 #pragma unroll
-                        for (int c = 0; c < KPL; ++c) g[c] = fmaf(e, x[t][c], g[c]);
+                        for (int c = 0; c < V4; ++c) {
+                            g[c].x = fmaf(e, x[h][c].x, g[c].x);
+                            g[c].y = fmaf(e, x[h][c].y, g[c].y);
+                            g[c].z = fmaf(e, x[h][c].z, g[c].z);
+                            g[c].w = fmaf(e, x[h][c].w, g[c].w);
+                        }
                         if (SIDE == 1) sse = fmaf(e, e, sse);
                     }
                 }
             }
+            // the four groups' partial sums: (g0 + g1) + (g2 + g3), the same in every lane
 #pragma unroll
-            for (int c = 0; c < KPL; ++c) {
-                if (SIDE == 0) a.grad[((size_t)r * a.I + self) * k + c * 32 + lane] = g[c];
-                else a.pu[self * k + c * 32 + lane] = mine[c] + a.lr * (g[c] - a.lam * mine[c]);
+            for (int d = 8; d < 32; d <<= 1) {
+#pragma unroll
+                for (int c = 0; c < V4; ++c) {
+                    g[c].x += __shfl_xor_sync(0xffffffffu, g[c].x, d);
+                    g[c].y += __shfl_xor_sync(0xffffffffu, g[c].y, d);
+                    g[c].z += __shfl_xor_sync(0xffffffffu, g[c].z, d);
+                    g[c].w += __shfl_xor_sync(0xffffffffu, g[c].w, d);
+                }
+                if (SIDE == 1) sse += __shfl_xor_sync(0xffffffffu, sse, d);
+            }
+            if (grp == 0) {
+#pragma unroll
+                for (int c = 0; c < V4; ++c) {
+                    if (SIDE == 0) {
+                        *reinterpret_cast<float4*>(a.grad + ((size_t)r * a.I + self) * k + c * 32 + sub * 4) = g[c];
+                    } else {
+                        float4 p = mine[c];
+                        p.x += a.lr * (g[c].x - a.lam * p.x);
+                        p.y += a.lr * (g[c].y - a.lam * p.y);
+                        p.z += a.lr * (g[c].z - a.lam * p.z);
+                        p.w += a.lr * (g[c].w - a.lam * p.w);
+                        *reinterpret_cast<float4*>(a.pu + self * k + c * 32 + sub * 4) = p;
+                    }
+                }
             }
         }
     }
