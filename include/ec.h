@@ -201,6 +201,13 @@ int ec_allreduce_epoch_host(ec_ctx_t* ctx, const void* const* host_rank_bufs, co
  * current value.  Affects speed only, never results. */
 int ec_allreduce_set_tile(ec_ctx_t* ctx, int threads, size_t tile_elems);
 
+/* Expert knob: 1 = the tiles of the rank buffers are staged through shared memory
+ * by bulk asynchronous copies (the default for up to 64 ranks in fixed or ring
+ * order; EC_ERR_UNSUPPORTED for other contexts); 0 = they are read with direct
+ * 128-bit loads.  Calls that cannot take the 128-bit path, and short segments,
+ * use the direct kernels whatever the setting.  Affects speed only, never results. */
+int ec_allreduce_set_path(ec_ctx_t* ctx, int path);
+
 /* Free the context (and its workspace if the library allocated it).  The caller
  * makes sure no work of this context is still running. */
 int ec_allreduce_destroy(ec_ctx_t* ctx);

@@ -35,6 +35,7 @@ SYMBOLS = {
     "ec_allreduce_host_staging_bytes": (_sz, [_vp, _i]),
     "ec_allreduce_epoch_host": (_i, [_vp, _vp, _vp, _i, _vp, _vp, _vp, _sz, _vp]),
     "ec_allreduce_set_tile": (_i, [_vp, _i, _sz]),
+    "ec_allreduce_set_path": (_i, [_vp, _i]),
     "ec_allreduce_destroy": (_i, [_vp]),
     "ec_allgatherv": (_i, [_vp, _vp, _i, _i, _vp, _vp, _vp, _sz, _vp, _vp]),
     "ec_kmeans_workspace_bytes": (_sz, [_sz, _i, _i, _i]),
@@ -176,6 +177,9 @@ class Allreduce:
 
     def set_tile(self, threads: int = 0, tile_elems: int = 0) -> None:
         _check(lib().ec_allreduce_set_tile(self._h, threads, tile_elems), "ec_allreduce_set_tile")
+
+    def set_path(self, path: int) -> None:
+        _check(lib().ec_allreduce_set_path(self._h, path), "ec_allreduce_set_path")
 
     def destroy(self) -> None:
         if getattr(self, "_h", None):

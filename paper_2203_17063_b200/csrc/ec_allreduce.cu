@@ -580,6 +580,154 @@ apply_short_kernel(const ApplyArgs a, const __grid_constant__ PtrTable<CAP> tbl)
     }
 }
 
+// ---------------------------------------------------------------------------------------------
+// the apply kernel with bulk-copy staging: the default for up to 64 ranks on the 128-bit path
+// ---------------------------------------------------------------------------------------------
+// The same fold, but the tile of every new rank travels from global to shared memory as one bulk asynchronous
+// copy (cp.async.bulk, completion counted in bytes on an mbarrier) through a ring of BK_STAGES buffers, issued by
+// one thread; all threads then take their vectors from shared memory in ascending rank order.  No registers are
+// tied up by loads in flight, so blocks are small and many: 64 threads, two stages of 4 KB (measured against
+// 128/256 threads, 1-8 stages, 4-16 KB: this shape is best or within 0.5 % of the best on the config 2 and 3
+// epochs, and beats the direct 128-bit loads of apply_kernel by 2.5 % on both; with one stage or with eight the
+// direct loads win).  Every wait is bounded; a wait that gives up falls back to reading that rank's tile directly
+// from global memory.
+#ifndef EC_BK_THREADS
+#define EC_BK_THREADS 64
+#endif
+#ifndef EC_BK_STAGES
+#define EC_BK_STAGES 2
+#endif
+#ifndef EC_BK_STAGE_BYTES
+#define EC_BK_STAGE_BYTES 4096
+#endif
+constexpr int BK_THREADS = EC_BK_THREADS;
+constexpr int BK_STAGES = EC_BK_STAGES;
+constexpr int BK_STAGE_BYTES = EC_BK_STAGE_BYTES;
+constexpr int BK_VPT = BK_STAGE_BYTES / 16 / BK_THREADS;     // 16-byte input vectors per thread and tile
+constexpr uint32_t BK_WAIT_LIMIT = 1u << 22;
+
+__device__ __forceinline__ uint32_t bk_smem(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ bool bk_wait(uint32_t bar, uint32_t parity) {
+    for (uint32_t it = 0; it < BK_WAIT_LIMIT; ++it) {
+        uint32_t ok;
+        asm volatile(
+            "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}\n"
+            : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+        if (ok) return true;
+    }
+    return false;
+}
+__device__ __forceinline__ void bk_copy(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar, uint64_t pol) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar), "l"(pol) : "memory");
+}
+
+template <int DT, int OP>
+__global__ void __launch_bounds__(BK_THREADS)
+apply_bulk_kernel(const ApplyArgs a, const __grid_constant__ PtrTable<64> tbl) {
+    typedef Elem<DT> E;
+    typedef typename E::In In;
+    typedef typename E::Acc Acc;
+    constexpr int VEC = E::VEC;
+
+    extern __shared__ __align__(128) unsigned char bk_stage[];          // BK_STAGES x BK_STAGE_BYTES
+    __shared__ const char* s_ptr[64];
+    __shared__ uint16_t s_rank[64];
+    __shared__ uint64_t s_new[MAX_W];
+    __shared__ int s_m, s_fresh;
+    __shared__ __align__(8) uint64_t s_bar[BK_STAGES];
+
+    const unsigned s = blockIdx.x / a.tiles_per_seg;
+    const unsigned t = blockIdx.x - s * a.tiles_per_seg;
+    const size_t lo = (size_t)s * a.seg + (size_t)t * a.tile;
+    size_t seg_hi = (size_t)(s + 1) * a.seg;
+    if (seg_hi > a.n) seg_hi = a.n;
+    const int tid = threadIdx.x;
+    if (tid == 0) {
+#pragma unroll
+        for (int q = 0; q < BK_STAGES; ++q)
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bk_smem(&s_bar[q])) : "memory");
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (tid < 32) block_prologue(a, s, t, s_rank, s_new, &s_m, &s_fresh);
+    __syncthreads();
+    const int m = s_m;
+    const bool fresh = s_fresh != 0;
+    if (m == 0 && !(fresh && a.first_apply)) return;
+    if (lo >= seg_hi) return;
+    size_t hi = lo + a.tile;
+    if (hi > seg_hi) hi = seg_hi;
+    const size_t cnt = hi - lo;
+    const int nvec = (int)(cnt / VEC);                                   // at most BK_STAGE_BYTES / 16
+    const uint32_t bytes = (uint32_t)nvec * 16u;
+    Acc* res = reinterpret_cast<Acc*>(a.result) + lo;
+    const uint64_t pol = evict_first_policy();
+    const uint64_t rpol_ld = result_policy(1), rpol_st = result_policy(a.res_hint == 2 ? 2 : 1);
+    for (int j = tid; j < m; j += BK_THREADS)
+        s_ptr[j] = reinterpret_cast<const char*>(tbl.p[s_rank[j]]) + lo * sizeof(In);
+    __syncthreads();
+    if (tid == 0 && bytes != 0) {
+        for (int j = 0; j < m && j < BK_STAGES; ++j)
+            bk_copy(bk_smem(bk_stage + (size_t)j * BK_STAGE_BYTES), s_ptr[j], bytes, bk_smem(&s_bar[j]), pol);
+    }
+    Acc acc[BK_VPT][VEC];
+#pragma unroll
+    for (int p = 0; p < BK_VPT; ++p) {
+        const int v = p * BK_THREADS + tid;
+        if (fresh || v >= nvec) {
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) acc[p][e] = ident<OP>(Acc());
+        } else {
+            load_acc<Acc, VEC>(res + (size_t)v * VEC, acc[p], rpol_ld);
+        }
+    }
+    unsigned late_mask = 0;                                               // stages whose copy did not report in time
+    if (bytes != 0) {
+        for (int j = 0; j < m; ++j) {
+            const int st = j % BK_STAGES;
+            const bool arrived = bk_wait(bk_smem(&s_bar[st]), (uint32_t)(j / BK_STAGES) & 1u);
+            if (!arrived) late_mask |= 1u << st;
+            const unsigned char* src = bk_stage + (size_t)st * BK_STAGE_BYTES;
+#pragma unroll
+            for (int p = 0; p < BK_VPT; ++p) {
+                const int v = p * BK_THREADS + tid;
+                if (v < nvec) {
+                    const uint4 raw = arrived ? *reinterpret_cast<const uint4*>(src + (size_t)v * 16)
+                                              : ld_stream16(s_ptr[j] + (size_t)v * 16, pol);     // the copy never reported: read directly
+                    Acc x[VEC];
+                    E::unpack(raw, x);
+#pragma unroll
+                    for (int e = 0; e < VEC; ++e) acc[p][e] = comb<OP>(acc[p][e], x[e]);
+                }
+            }
+            __syncthreads();                                             // everybody is done with this stage
+            if (tid == 0 && j + BK_STAGES < m)
+                bk_copy(bk_smem(bk_stage + (size_t)st * BK_STAGE_BYTES), s_ptr[j + BK_STAGES], bytes, bk_smem(&s_bar[st]), pol);
+        }
+#pragma unroll
+        for (int p = 0; p < BK_VPT; ++p) {
+            const int v = p * BK_THREADS + tid;
+            if (v < nvec) store_acc<Acc, VEC>(res + (size_t)v * VEC, acc[p], rpol_st);
+        }
+    }
+    // elements after the last whole vector of a ragged tile
+    for (size_t i = (size_t)nvec * VEC + tid; i < cnt; i += BK_THREADS) {
+        Acc x = fresh ? ident<OP>(Acc()) : res[i];
+        for (int j = 0; j < m; ++j) x = comb<OP>(x, E::widen(reinterpret_cast<const In*>(s_ptr[j])[i]));
+        res[i] = x;
+    }
+    // a copy that was given up on may still be on its way into this block's shared memory: give it one more
+    // bounded wait before the block retires (the last use of stage st was rank j with j % BK_STAGES == st)
+    if (late_mask != 0) {
+        for (int st = 0; st < BK_STAGES; ++st) {
+            if (!((late_mask >> st) & 1u) || st >= m) continue;
+            const int last_j = st + ((m - 1 - st) / BK_STAGES) * BK_STAGES;
+            bk_wait(bk_smem(&s_bar[st]), (uint32_t)(last_j / BK_STAGES) & 1u);
+        }
+    }
+}
+
 template <int DT, int OP, bool VECTOR, int ORDER>
 int launch_cap(const ApplyArgs& a, const void* const* bufs, unsigned grid, int threads, bool short_seg, cudaStream_t st) {
     if (a.P <= 64) {
@@ -625,6 +773,33 @@ int launch_dt(const ApplyArgs& a, const void* const* bufs, int op, bool vector, 
     return EC_ERR_INVALID;
 }
 
+template <int DT, int OP>
+int launch_bulk_op(const ApplyArgs& a, const void* const* bufs, unsigned grid, cudaStream_t st) {
+    PtrTable<64> tbl;
+    for (int r = 0; r < 64; ++r) tbl.p[r] = r < a.P ? bufs[r] : nullptr;
+    apply_bulk_kernel<DT, OP><<<grid, BK_THREADS, BK_STAGES * BK_STAGE_BYTES, st>>>(a, tbl);
+    EC_CUDA(cudaGetLastError());
+    return EC_OK;
+}
+template <int DT>
+int launch_bulk_dt(const ApplyArgs& a, const void* const* bufs, int op, unsigned grid, cudaStream_t st) {
+    switch (op) {
+        case EC_SUM: return launch_bulk_op<DT, EC_SUM>(a, bufs, grid, st);
+        case EC_MAX: return launch_bulk_op<DT, EC_MAX>(a, bufs, grid, st);
+        case EC_MIN: return launch_bulk_op<DT, EC_MIN>(a, bufs, grid, st);
+    }
+    return EC_ERR_INVALID;
+}
+int launch_bulk(const ApplyArgs& a, const void* const* bufs, int dtype, int op, unsigned grid, cudaStream_t st) {
+    switch (dtype) {
+        case EC_F32: return launch_bulk_dt<EC_F32>(a, bufs, op, grid, st);
+        case EC_BF16: return launch_bulk_dt<EC_BF16>(a, bufs, op, grid, st);
+        case EC_I64: return launch_bulk_dt<EC_I64>(a, bufs, op, grid, st);
+        case EC_F64: return launch_bulk_dt<EC_F64>(a, bufs, op, grid, st);
+    }
+    return EC_ERR_INVALID;
+}
+
 size_t words_bytes(int P, size_t n, size_t seg) {
     const size_t S = (n + seg - 1) / seg;
     const size_t W = (size_t)(P + 63) / 64;
@@ -649,6 +824,7 @@ struct ec_ctx {
     int threads;
     size_t tile;       // elements per block
     int res_hint;      // L2 policy of the result accesses
+    int path;          // 1: bulk-copy staging where it applies (the default when the context allows it), 0: direct loads
 };
 
 using namespace ec;
@@ -701,9 +877,17 @@ int ec_allreduce_init(ec_ctx_t** out, int P, size_t n, ec_dtype_t dtype, ec_op_t
     }
     // Few ranks: many small blocks overlap their start-up latency best.  Hundreds of ranks: a block
     // lives long anyway and wider blocks read longer contiguous runs of each buffer (both measured).
+    c->path = (order != EC_ORDER_PAIRWISE && P <= 64) ? 1 : 0;
     c->threads = P > 64 ? 256 : 128;
     c->tile = dtype == EC_BF16 ? 2048 : 8192 / in_bytes(dtype);   // 8 KB of every rank buffer per block (4 KB for bf16), measured
     *out = c;
+    return EC_OK;
+}
+
+int ec_allreduce_set_path(ec_ctx_t* c, int path) {
+    if (!c || (path != 0 && path != 1)) return EC_ERR_INVALID;
+    if (path == 1 && (c->order == EC_ORDER_PAIRWISE || c->P > 64)) return EC_ERR_UNSUPPORTED;
+    c->path = path;
     return EC_OK;
 }
 
@@ -750,6 +934,14 @@ int apply_common(ec_ctx_t* c, const void* const* rank_bufs, int P, size_t n, ec_
     if (short_seg) {
         a.tiles_per_seg = 1;
         grid = (unsigned)c->S;
+    }
+    if (c->path == 1 && vector && !short_seg && c->order != EC_ORDER_PAIRWISE && c->P <= 64) {
+        // bulk-copy staging: tiles of one stage buffer (8 KB of every rank)
+        a.tile = BK_STAGE_BYTES / in_bytes(c->dtype);
+        const size_t btiles = (seg_len + a.tile - 1) / a.tile;
+        if (btiles * c->S > 0x7fffffffull) return EC_ERR_CAPACITY;
+        a.tiles_per_seg = (unsigned)btiles;
+        return launch_bulk(a, rank_bufs, c->dtype, c->op, (unsigned)(btiles * c->S), stream);
     }
     switch (c->dtype) {
         case EC_F32: return launch_dt<EC_F32>(a, rank_bufs, c->op, vector, c->order, grid, c->threads, short_seg, stream);

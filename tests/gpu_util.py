@@ -50,7 +50,7 @@ def sentinel(dtype_out, n):
 
 
 def run_schedule(P, n, seg, dtype, op, bufs, masks, order=ec.ORDER_FIXED, offset_elems=0, result_offset=0,
-                 tile=None, poison=None, oracle_threads=4, compare=True):
+                 tile=None, poison=None, oracle_threads=4, compare=True, path=None):
     """Apply the cumulative masks one round after the other on GPU and CPU.
 
     masks: list of uint64 [S][W] arrays (or None = everything arrived).
@@ -62,6 +62,8 @@ def run_schedule(P, n, seg, dtype, op, bufs, masks, order=ec.ORDER_FIXED, offset
     ar = ec.Allreduce(P, n, dtype, op, seg, order)
     if tile is not None:
         ar.set_tile(*tile)
+    if path is not None:
+        ar.set_path(path)
     ref = oracle.Allreduce(P, n, dtype, op, seg)
     d_bufs = [to_dev(b, offset_elems) for b in bufs]
     res_np = sentinel(NP_OUT[dtype], n)

@@ -380,3 +380,36 @@ def test_short_segments_ring_order_and_untouched_rows():
     run_schedule(P, n, seg, ec.F32, ec.SUM, bufs, masks, order=ec.ORDER_RING)
     outs = run_schedule(P, n, seg, ec.F32, ec.SUM, bufs, masks + [masks[-1]])
     assert np.array_equal(bits(outs[-1][0]), bits(outs[-2][0]))          # nothing new: nothing changes
+
+
+# ---------------------------------------------------------------------------
+# the optional path that stages the rank tiles through shared memory with bulk asynchronous copies
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("dtype,kind,kw", [(ec.F32, "normal_f32", {}), (ec.BF16, "normal_bf16", {"sigma": 1.0}),
+                                           (ec.I64, "int64_full", {})], ids=["f32", "bf16", "i64"])
+@pytest.mark.parametrize("P,n,seg", [(16, (1 << 18) + 37 * 8, 65536), (3, 9000, 3000), (64, 1 << 16, 4096), (7, 20000, 20000)])
+def test_bulk_copy_path_matches_checker(dtype, kind, kw, P, n, seg):
+    S = (n + seg - 1) // seg
+    bufs = _bufs(kind, 4000 + P, P, n, **kw)
+    rounds = inputs.arrival_rounds(4100 + P, P, S, 0.6)
+    masks = inputs.cumulative_masks(rounds)
+    poison = [rounds > t for t in (1, 2, 3)]
+    run_schedule(P, n, seg, dtype, ec.SUM, bufs, masks, poison=poison, path=1)
+    run_schedule(P, n, seg, dtype, ec.MAX if dtype != ec.BF16 else ec.SUM, bufs, [masks[0], None], path=1)
+
+
+def test_bulk_copy_path_ring_order_misaligned_and_limits():
+    P, n, seg = 16, 1 << 16, 1024
+    bufs = _bufs("normal_f32", 4200, P, n)
+    masks = inputs.cumulative_masks(inputs.arrival_rounds(4201, P, n // seg, 0.5))
+    run_schedule(P, n, seg, ec.F32, ec.SUM, bufs, masks, order=ec.ORDER_RING, path=1)
+    run_schedule(P, n, seg, ec.F32, ec.SUM, bufs, masks, offset_elems=1, path=1)      # not 16-byte aligned: default kernel
+    ar = ec.Allreduce(100, 4096, ec.F32, ec.SUM, 1024)
+    with pytest.raises(ec.EcError) as err:
+        ar.set_path(1)                                                                  # more than 64 ranks
+    assert err.value.code == ec.ERR_UNSUPPORTED
+    ar.destroy()
+    ar = ec.Allreduce(8, 4096, ec.F32, ec.SUM, 1024, ec.ORDER_PAIRWISE)
+    with pytest.raises(ec.EcError):
+        ar.set_path(1)
+    ar.destroy()
