@@ -36,10 +36,10 @@ HEADLINE = dict(P=16, n=1 << 24, seg=65536, p_first=0.7, seed=1002, seed_sched=2
 NOMINAL_HBM_GBS = 8000.0
 
 # dram__bytes_read.sum + dram__bytes_write.sum of the three apply launches of one headline epoch, from one
-# one-pass ncu capture that leaves the caches alone (profiles/apply_kernel_config2_epoch.md): reads 750.5 + 191.4 +
-# 211.0 MB, writes 44.0 + 31.5 + 33.9 MB.  Below the algorithmic bytes because about half of the 64 MiB result is
+# one-pass ncu capture that leaves the caches alone (profiles/apply_kernel_config2_epoch.md): reads 750.4 + 192.2 +
+# 212.9 MB, writes 66.5 + 36.2 + 38.7 MB.  Below the algorithmic bytes because about half of the 64 MiB result is
 # found in L2 by the next round.
-NCU_TRAFFIC_BYTES_PER_EPOCH = 1_262_126_720
+NCU_TRAFFIC_BYTES_PER_EPOCH = 1_296_705_920
 
 
 def measured_peaks():
@@ -215,6 +215,8 @@ def run_ours(args, rank, world, local_rank):
     ar = ec.Allreduce(P, n, ec.F32, ec.SUM, seg, device=dev)
     if args.threads or args.tile:
         ar.set_tile(args.threads, args.tile)
+    if args.apply_path == "direct":
+        ar.set_path(0)
     table = (C.c_void_p * P)(*[t.data_ptr() for t in d_bufs])
     L = ec.lib()
 
@@ -283,6 +285,8 @@ def run_ours(args, rank, world, local_rank):
         a_i = ar if i == 0 else ec.Allreduce(P, n, ec.F32, ec.SUM, seg, device=dev)
         if i and (args.threads or args.tile):
             a_i.set_tile(args.threads, args.tile)
+        if i and args.apply_path == "direct":
+            a_i.set_path(0)
         nbytes = a_i.host_staging_bytes(rounds)
         lanes.append({
             "ar": a_i, "stream": stream if i == 0 else torch.cuda.Stream(device=dev),
@@ -358,7 +362,7 @@ def run_ours(args, rank, world, local_rank):
         },
         "roofline": {
             "bound": "hbm",
-            "kernel": "apply_kernel<f32,sum,vector,64,fixed> (all three launches of an epoch)",
+            "kernel": "apply_bulk_kernel<f32,sum> (all three launches of an epoch)",
             "achieved": round(achieved, 1),
             "peak": peak,
             "peak_kind": f"of {peak_kind}",
@@ -464,6 +468,8 @@ def extras(args, dev, stream, peak):
         ar = ec.Allreduce(P, n, dtype, ec.SUM, seg, order, device=dev)
         if args.threads or args.tile:
             ar.set_tile(args.threads, args.tile)
+        if args.apply_path == "direct":
+            ar.set_path(0)
         table = (C.c_void_p * P)(*[t.data_ptr() for t in d])
         cfgd = dict(P=P, n=n, seg=seg)
         rb = epoch_bytes(cfgd, masks, in_b, out_b) if masks[0] is not None else [apply_bytes(None, None, P, n, seg, in_b, out_b, True)]
@@ -756,6 +762,8 @@ def main():
     ap.add_argument("--profile-only", action="store_true", help="warm-up and timed steps only (for ncu captures)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-extras", action="store_true", help="headline workload only")
+    ap.add_argument("--apply-path", default="default", choices=["default", "direct"],
+                    help="direct: force the direct-load apply kernel (ec_allreduce_set_path(0)) where bulk staging is the default")
     ap.add_argument("--workload", default="headline", choices=["headline", "kmeans", "mf"],
                     help="kmeans: time only the K-means driver (config 5) and print its own JSON line")
     ap.add_argument("--cpu-seconds", type=float, default=15.0, help="time budget of the CPU baseline leg")
