@@ -303,7 +303,13 @@ int ec_kmeans_assign(ec_kmeans_t* km, const float* centroids, int32_t* labels, e
 int ec_kmeans_partials(ec_kmeans_t* km, const int32_t* labels, float* partials, ec_stream_t stream);
 
 /* One full iteration on the context's own centroids.  arrival_mask: device
- * uint64 [K][W] for this iteration, NULL = all arrived. */
+ * uint64 [K][W] for this iteration, NULL = all arrived.
+ * The context keeps the labels and the per-rank sums between iterations; on the
+ * tensor-core path (D = 16 or 32, K <= 256) an iteration after the first adds to
+ * the sums only what changed - +x for the cluster a point joins, -x for the one
+ * it leaves - and every 32nd iteration sums everything afresh, which bounds the
+ * rounding the running sums collect (about 2^-24 of a sum per iteration; counts
+ * stay exact).  Results repeat bit for bit from run to run either way. */
 int ec_kmeans_iterate(ec_kmeans_t* km, const uint64_t* arrival_mask, ec_stream_t stream);
 
 /* The same iteration with the combine step spread over several rounds: one allreduce epoch with

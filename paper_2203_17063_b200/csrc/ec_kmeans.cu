@@ -31,6 +31,7 @@ constexpr int AS_THREADS = 256;
 constexpr int PT_THREADS = 256;
 constexpr int PT_WARPS = PT_THREADS / 32;
 constexpr size_t SMEM_BUDGET = 200 * 1024;
+constexpr int KM_REFRESH = 32;                  // iterations that sum only changes before a full pass
 constexpr size_t ASSIGN_SMEM_MAX = 64 * 1024;   // centroid chunk staged by the assignment kernels
 
 // ---------------------------------------------------------------------------------------------
@@ -215,14 +216,28 @@ partials_kernel(const float* __restrict__ points, const int32_t* __restrict__ la
 }
 
 // partials[r][k][d] = scratch[r][0][k][d] + scratch[r][1][k][d] + ... in index order
+// (accumulate: the row blocks hold changes, which are added to what partials holds)
 __global__ void partials_fold_kernel(const float* __restrict__ scratch, int C, size_t row_elems, size_t total,
-                                     float* __restrict__ partials) {
+                                     float* __restrict__ partials, int accumulate = 0,
+                                     const uint32_t* __restrict__ dirty = nullptr) {
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
         const size_t r = i / row_elems, e = i - r * row_elems;
         const float* src = scratch + r * (size_t)C * row_elems + e;
-        float v = src[0];
-        for (int c = 1; c < C; ++c) v = __fadd_rn(v, src[(size_t)c * row_elems]);
-        partials[i] = v;
+        if (accumulate) {                        // only the row blocks that hold changes (dirty) were written
+            float v = partials[i];
+            bool any = false;
+            for (int c = 0; c < C; ++c) {
+                if (dirty[r * (size_t)C + c]) {
+                    v = __fadd_rn(v, src[(size_t)c * row_elems]);
+                    any = true;
+                }
+            }
+            if (any) partials[i] = v;
+        } else {
+            float v = src[0];
+            for (int c = 1; c < C; ++c) v = __fadd_rn(v, src[(size_t)c * row_elems]);
+            partials[i] = v;
+        }
     }
 }
 
@@ -497,6 +512,9 @@ struct ec_kmeans {
     int path;              // 0 = automatic, 1 = fp32 fused kernel, 2 = tensor-core fused kernel
     size_t tc_smem, tc_assign_smem;
     uint32_t* tc_status;   // device word: nonzero if a wait on the tensor core ever gave up
+    uint32_t* dirty;       // [P][Cf]: delta mode, which row blocks of scratch hold changes
+    bool state_valid;      // labels and partials belong together (an iteration has run): changes can be summed
+    int since_full;        // iterations since everything was summed afresh
 };
 
 using namespace ec;
@@ -504,7 +522,7 @@ using namespace ec;
 namespace {
 
 struct KmLayout {
-    size_t off_centroids, off_labels, off_partials, off_scratch, off_reduced, off_contrib, off_ar, total;
+    size_t off_centroids, off_labels, off_partials, off_scratch, off_reduced, off_contrib, off_dirty, off_ar, total;
     int C, warps;
     int Cf;   // runs per rank for the fused assignment+partials kernel, 0 if the shape is not covered
 };
@@ -556,6 +574,7 @@ bool km_plan(size_t N, int D, int K, int P, int sms, KmLayout* L) {
     L->off_scratch = off; off = align_up(off + (size_t)P * (C > L->Cf ? C : L->Cf) * K * stride * 4, 256);
     L->off_reduced = off; off = align_up(off + (size_t)K * stride * 4, 256);
     L->off_contrib = off; off = align_up(off + (size_t)K * 4 + 256, 256);   // + a status word
+    L->off_dirty = off; off = align_up(off + (size_t)P * (L->Cf > 0 ? L->Cf : 1) * 4, 256);   // change flags of the row blocks
     L->off_ar = off; off = align_up(off + ec_allreduce_workspace_bytes(P, (size_t)K * stride, stride), 256);
     L->total = off;
     return true;
@@ -585,17 +604,17 @@ int km_fused_launch(ec_kmeans* km, bool partials, const float* centroids, int32_
 }
 
 template <int D>
-int km_tc_launch(ec_kmeans* km, bool partials, const float* centroids, int32_t* labels, cudaStream_t st) {
+int km_tc_launch(ec_kmeans* km, bool partials, const float* centroids, int32_t* labels, cudaStream_t st, bool delta) {
     const float tau_scale = 0.015625f;     // 2^-6: four times the bound 2^-8 (|x|^2 + |c|max^2) of one candidate's error
     if (partials) {
         tc::tc_fused_kernel<D, true><<<(unsigned)(km->P * km->Cf), tc::THREADS, km->tc_smem, st>>>(
-            km->points, km->N, km->P, km->Cf, centroids, km->K, labels, km->Cf == 1 ? km->partials : km->scratch,
-            tau_scale, km->tc_status);
+            km->points, km->N, km->P, km->Cf, centroids, km->K, labels, (km->Cf == 1 && !delta) ? km->partials : km->scratch,
+            tau_scale, km->tc_status, delta ? 1 : 0, km->dirty);
     } else {
         size_t runs = (km->N + 2047) / 2048;
         if (runs > 0x7fffffffull) return EC_ERR_CAPACITY;
         tc::tc_fused_kernel<D, false><<<(unsigned)runs, tc::THREADS, km->tc_assign_smem, st>>>(
-            km->points, km->N, 1, (int)runs, centroids, km->K, labels, nullptr, tau_scale, km->tc_status);
+            km->points, km->N, 1, (int)runs, centroids, km->K, labels, nullptr, tau_scale, km->tc_status, 0, nullptr);
     }
     EC_CUDA(cudaGetLastError());
     return EC_OK;
@@ -609,11 +628,11 @@ cudaError_t km_tc_attr() {
     return e;
 }
 
-int km_fused(ec_kmeans* km, bool partials, const float* centroids, int32_t* labels, cudaStream_t st) {
+int km_fused(ec_kmeans* km, bool partials, const float* centroids, int32_t* labels, cudaStream_t st, bool delta = false) {
     if (km->tc_ok && km->path != 1) {
         switch (km->D) {
-            case 16: return km_tc_launch<16>(km, partials, centroids, labels, st);
-            case 32: return km_tc_launch<32>(km, partials, centroids, labels, st);
+            case 16: return km_tc_launch<16>(km, partials, centroids, labels, st, delta);
+            case 32: return km_tc_launch<32>(km, partials, centroids, labels, st, delta);
         }
     }
     switch (km->D) {
@@ -716,9 +735,12 @@ int ec_kmeans_init(ec_kmeans_t** out, const float* points, size_t N, int D, int 
     km->fused_assign_smem = fused_smem_floats(D, K, false) * 4;
     km->tc_ok = km->Cf > 0 && tc_capable(D, K);
     km->path = 0;
+    km->state_valid = false;
+    km->since_full = 0;
     km->tc_smem = tc::layout_of(D, K, true).total;
     km->tc_assign_smem = tc::layout_of(D, K, false).total;
     km->tc_status = reinterpret_cast<uint32_t*>(base + L.off_contrib + align_up((size_t)K * 4, 256));
+    km->dirty = reinterpret_cast<uint32_t*>(base + L.off_dirty);
     // centroid chunk for the assignment: as many as fit in 64 KB, all of them if possible
     int kc = (int)((64 * 1024) / ((size_t)D * 4));
     if (kc > K) kc = K;
@@ -793,14 +815,20 @@ int km_iterate_rounds(ec_kmeans_t* km, const uint64_t* const* masks, int rounds,
     int rc;
     if (km->Cf > 0) {
         // assignment and per-block partial sums in one pass over the points, then the rows of a rank in order
-        rc = km_fused(km, true, km->centroids, km->labels, stream);
+        // On the tensor-core path only the changes since the last iteration are summed (labels and per-rank sums
+        // are kept between iterations); every KM_REFRESH-th iteration sums everything afresh, which bounds the
+        // rounding that the running sums collect.
+        const bool delta = km->tc_ok && km->path != 1 && km->state_valid && km->since_full < KM_REFRESH;
+        rc = km_fused(km, true, km->centroids, km->labels, stream, delta);
         if (rc != EC_OK) return rc;
-        if (km->Cf > 1) {
+        if (km->Cf > 1 || delta) {
             const size_t row = (size_t)km->K * (km->D + 4), total = row * km->P;
             partials_fold_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(km->scratch, km->Cf, row, total,
-                                                                                      km->partials);
+                                                                                      km->partials, delta ? 1 : 0, km->dirty);
             EC_CUDA(cudaGetLastError());
         }
+        km->state_valid = true;
+        km->since_full = delta ? km->since_full + 1 : 0;
     } else {
         rc = km_assign(km, km->centroids, km->labels, stream);
         if (rc != EC_OK) return rc;
@@ -843,6 +871,7 @@ int ec_kmeans_set_path(ec_kmeans_t* km, int path) {
     if (path == 2 && !km->tc_ok) return EC_ERR_UNSUPPORTED;
     if (path == 1 && km->Cf == 0) return EC_ERR_UNSUPPORTED;
     km->path = path;
+    km->state_valid = false;        // the next iteration sums everything afresh
     return EC_OK;
 }
 

@@ -19,6 +19,13 @@
 // 8-point x 8-coordinate core matrices.  The sums MMA always works on 128 rows; rows beyond the
 // D + 16 real ones read whatever follows the tile in shared memory and are never looked at.
 //
+// Delta mode (iterations after the first): the labels of the previous iteration are read back, a point that
+// keeps its label contributes nothing, one that moves puts +1 in the one-hot column of its new cluster and
+// -1 in that of its old one, so the accumulator collects the change of the sums; a tile without a move
+// issues no sums MMA at all (and the low parts, needed only by that MMA, are staged on demand from L2), a
+// block without one leaves its row block unwritten and says so in a flag.  Once the clustering has settled
+// an iteration is the search alone.
+//
 // Block (r, c) covers the c-th of C runs of rank r's points and writes one [K][D+4] row block of
 // scratch; the rows of a rank are folded in order afterwards.  Every wait on the tensor core is
 // bounded; if one gives up, the block finishes in plain fp32 (exact form, atomic adds into its row
@@ -200,7 +207,8 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 template <int D, bool PARTIALS>
 __global__ void __launch_bounds__(THREADS, EC_TC_MINB)
 tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const float* __restrict__ centroids, int K,
-                int32_t* __restrict__ labels, float* __restrict__ scratch, float tau_scale, uint32_t* __restrict__ status) {
+                int32_t* __restrict__ labels, float* __restrict__ scratch, float tau_scale, uint32_t* __restrict__ status,
+                int delta, uint32_t* __restrict__ dirty) {
     constexpr int KCH = D / 8;                           // 16-byte chunks of coordinates per point
     static_assert(D % 16 == 0 && KCH + 2 <= 8 && (KCH & (KCH - 1)) == 0, "D is 16 or 32");
     constexpr int LO = 8;                                // first chunk column of the low parts
@@ -282,6 +290,7 @@ tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const 
     bool sums_started = false;       // a sums MMA has been issued (the accumulator holds data)
     bool sums_pending = false;       // ... and its completion has not been waited for yet
     int prev_chunk = -1;             // one-hot chunk this thread set in the previous tile
+    int prev_chunk2 = -1;            // ... and a second one (delta mode: the chunk of the label the point left)
     bool by_hand = false;            // some points were added to the row block with atomic adds
 
     // A thread stages KCH items (point row, chunk kc of 8 coordinates) of a tile: consecutive threads take
@@ -309,6 +318,7 @@ tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const 
     for (size_t base = b0; base < b1; base += TILE) {
         const size_t j = base + tid;
         const bool live = j < b1;
+        const int old = (delta && live) ? labels[j] : -1;   // delta mode: the label this point had (asked for early: used after the search)
         if (PARTIALS && sums_pending) {
             // the previous tile's sums MMA still reads the tile: wait for it (its latency hid behind the search)
             const bool ok = mbar_wait_bounded(bar2, phase2);
@@ -319,6 +329,10 @@ tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const 
         if (PARTIALS && prev_chunk >= 0) {
             *reinterpret_cast<uint4*>(s_oh + (size_t)prev_chunk * OCHUNK + (size_t)tid * 16) = make_uint4(0u, 0u, 0u, 0u);
             prev_chunk = -1;
+        }
+        if (PARTIALS && prev_chunk2 >= 0) {
+            *reinterpret_cast<uint4*>(s_oh + (size_t)prev_chunk2 * OCHUNK + (size_t)tid * 16) = make_uint4(0u, 0u, 0u, 0u);
+            prev_chunk2 = -1;
         }
         // bf16 high parts and low parts (low = bf16(x - high)) at chunk column kc resp. LO + kc, row*16
 #pragma unroll
@@ -333,12 +347,16 @@ tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const 
                 sq = fmaf(a, a, sq);
                 sq = fmaf(b, b, sq);
                 hw[e] = pack_bf16(a, b);
-                const float ah = __uint_as_float(hw[e] << 16), bh = __uint_as_float(hw[e] & 0xFFFF0000u);
-                lw[e] = pack_bf16(a - ah, b - bh);
             }
             *reinterpret_cast<uint4*>(s_x + (size_t)kc * XCHUNK + (size_t)row * 16) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
-            if (PARTIALS)
+            if (PARTIALS && !delta) {    // delta mode: the low parts are made only for a tile that turns out to hold a change
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const float ah = __uint_as_float(hw[e] << 16), bh = __uint_as_float(hw[e] & 0xFFFF0000u);
+                    lw[e] = pack_bf16(v[2 * e] - ah, v[2 * e + 1] - bh);
+                }
                 *reinterpret_cast<uint4*>(s_x + (size_t)(LO + kc) * XCHUNK + (size_t)row * 16) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
+            }
             // |x|^2 of the row: its KCH chunks sit in KCH consecutive lanes
 #pragma unroll
             for (int o = 1; o < KCH; o <<= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
@@ -389,33 +407,75 @@ tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const 
         // rounding to bf16 perturbs v by at most 2^-7 |x||c| <= 2^-8 (|x|^2 + |c|max^2) per candidate
         const float tau = tau_scale * (s_xn[tid] + cmax);
         const bool redo = live && (!done || !(m2 - m1 > tau));
+        // Delta mode: the row block receives only what changed since the labels were written last: +x for the
+        // cluster a point joins, -x for the one it leaves (old label < 0: it was in none).  A tile in which no
+        // label changed needs no sums MMA at all.  Otherwise every live point joins its cluster.
         if (redo || (live && PARTIALS && !done)) {
             float x[D];
             load_point<D>(points, j, x);                 // rare: read the point again instead of keeping it in registers
             if (redo) kb = exact_argmin_global<D>(x, centroids, K);
-            if (PARTIALS && !done) {                     // tensor core out of service: add this point by hand
+            if (PARTIALS && !done && !(delta && old == kb)) {   // tensor core out of service: add this point by hand
 #pragma unroll
                 for (int d = 0; d < D; ++d) atomicAdd(row_block + (size_t)kb * stride + d, x[d]);
                 atomicAdd(row_block + (size_t)kb * stride + D, 1.0f);
+                if (old >= 0) {
+#pragma unroll
+                    for (int d = 0; d < D; ++d) atomicAdd(row_block + (size_t)old * stride + d, -x[d]);
+                    atomicAdd(row_block + (size_t)old * stride + D, -1.0f);
+                }
             }
         }
-        if (live) labels[j] = kb;
+        const bool changed = live && !(delta && old == kb);
+        if (changed) labels[j] = kb;
         if (PARTIALS && done) {
-            if (live) {
-                // one-hot row of this point: 16-byte chunk kb/8, bf16 1.0 at position kb%8
+            if (changed) {
+                // one-hot row of this point: 16-byte chunk kb/8, bf16 1.0 at position kb%8 (and -1.0 for the old label)
                 uint32_t wv[4] = {0u, 0u, 0u, 0u};
                 wv[(kb & 7) >> 1] = 0x3F80u << (16 * (kb & 1));
                 prev_chunk = kb >> 3;
+                if (old >= 0 && (old >> 3) == prev_chunk) wv[(old & 7) >> 1] |= 0xBF80u << (16 * (old & 1));
                 *reinterpret_cast<uint4*>(s_oh + (size_t)prev_chunk * OCHUNK + (size_t)tid * 16) = make_uint4(wv[0], wv[1], wv[2], wv[3]);
+                if (old >= 0 && (old >> 3) != prev_chunk) {
+                    uint32_t wo[4] = {0u, 0u, 0u, 0u};
+                    wo[(old & 7) >> 1] = 0xBF80u << (16 * (old & 1));
+                    prev_chunk2 = old >> 3;
+                    *reinterpret_cast<uint4*>(s_oh + (size_t)prev_chunk2 * OCHUNK + (size_t)tid * 16) = make_uint4(wo[0], wo[1], wo[2], wo[3]);
+                }
             }
             fence_async_smem();
-            __syncthreads();
-            if (tid == 0) {
+            const bool any_changed = __syncthreads_or(changed ? 1 : 0) != 0;
+            if (any_changed && delta) {
+                // rare once the labels have settled: read the tile again (it is still in L2) and stage the low parts
+#pragma unroll
+                for (int q = 0; q < KCH; ++q) {
+                    const int idx = q * THREADS + tid, row = idx / KCH, kc = idx % KCH;
+                    const size_t jr = base + row;
+                    float4 ta = make_float4(0.0f, 0.0f, 0.0f, 0.0f), tb = ta;
+                    if (jr < b1) {
+                        const float4* src = reinterpret_cast<const float4*>(points + jr * D + kc * 8);
+                        ta = __ldg(src);
+                        tb = __ldg(src + 1);
+                    }
+                    const float v[8] = {ta.x, ta.y, ta.z, ta.w, tb.x, tb.y, tb.z, tb.w};
+                    uint32_t lw[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float a = v[2 * e], b = v[2 * e + 1];
+                        const uint32_t h = pack_bf16(a, b);
+                        lw[e] = pack_bf16(a - __uint_as_float(h << 16), b - __uint_as_float(h & 0xFFFF0000u));
+                    }
+                    *reinterpret_cast<uint4*>(s_x + (size_t)(LO + kc) * XCHUNK + (size_t)row * 16) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
+                }
+                fence_async_smem();
+                __syncthreads();
+            }
+            if (any_changed && tid == 0) {
                 fence_after_sync();
                 // sums[row][k] += sum_j X[j][row] * onehot[j][k], 16 points per step, both operands MN-major:
                 // consecutive points are 16 bytes apart (K direction: 8 points = 128 bytes), consecutive chunks
                 // of 8 rows / 8 centroids are XCHUNK / OCHUNK bytes apart (M/N direction).  One MMA covers the
                 // high parts with the ones (rows 0..63) and the low parts (rows 64..127).
+#pragma unroll
 #pragma unroll
                 for (int ks = 0; ks < TILE / 16; ++ks) {
                     const uint64_t ad = smem_desc(x_base + ks * 256, 128, XCHUNK);
@@ -424,8 +484,10 @@ tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const 
                 }
                 mma_commit(bar2);
             }
-            sums_started = true;
-            sums_pending = true;
+            if (any_changed) {
+                sums_started = true;
+                sums_pending = true;
+            }
         }
     }
     if (PARTIALS) {
@@ -464,8 +526,11 @@ tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const 
             }
         }
     }
-    if (PARTIALS && !sums_started && !by_hand)   // an empty run: its row block is all zeros
+    if (PARTIALS && delta) {                     // delta mode: a block without changes leaves its row block alone and says so
+        if (tid == 0) dirty[blockIdx.x] = (sums_started || by_hand) ? 1u : 0u;
+    } else if (PARTIALS && !sums_started && !by_hand) {   // an empty run: its row block is all zeros
         for (int i = tid; i < K * stride; i += THREADS) row_block[i] = 0.0f;
+    }
     fence_before_sync();
     __syncthreads();
     if (w == 0) tmem_dealloc(tmem_base, ncols);

@@ -178,3 +178,36 @@ def test_iteration_with_two_rounds_matches_checker():
     means = np.stack([points[labels == k].astype(np.float64).mean(0) for k in range(K)])
     assert rows_close(to_host(d_cent), means.astype(np.float32))
     km.destroy()
+
+
+def test_running_sums_follow_label_changes_over_many_iterations():
+    """The tensor-core path sums only what changed since the previous iteration (+x into the cluster a point joins,
+    -x out of the one it leaves) and sums everything afresh every 32nd iteration.  With overlapping clusters and
+    centroids that are pushed around before every iteration many points change hands each time; after each of 40
+    iterations the reduced sums and counts must still be those of the labels (counts exactly)."""
+    N, D, K, P = 30000, 32, 16, 8
+    points, comp, _ = inputs.kmeans_mixture(77, N, D, K, sigma=6.0)          # heavily overlapping components
+    cents = inputs.kmeans_first_of_component(points, comp, K)
+    rng = np.random.default_rng(78)
+    km = ec.KMeans(to_dev(points), K, P, to_dev(cents))
+    d_labels = torch.empty(N, dtype=torch.int32, device="cuda")
+    d_red = torch.empty(K, D + 4, device="cuda")
+    prev = None
+    moved = 0
+    for t in range(40):
+        cents = (cents + rng.normal(0.0, 0.8, size=cents.shape)).astype(np.float32)
+        km.set_centroids(to_dev(cents))
+        km.iterate(None)
+        km.get(labels=d_labels, reduced=d_red)
+        torch.cuda.synchronize()
+        g_labels = to_host(d_labels)
+        check_labels(g_labels, points, cents)
+        if prev is not None:
+            moved += int((g_labels != prev).sum())
+        prev = g_labels.copy()
+        want = oracle.kmeans_partials(points, g_labels, K, P, 4).astype(np.float64).sum(axis=0)      # [K][D+4]
+        got = to_host(d_red)
+        assert np.array_equal(got[:, D], want[:, D].astype(np.float32)), f"iteration {t}: counts"
+        assert rows_close(got[:, :D], want[:, :D]), f"iteration {t}: sums"
+    assert moved > 20 * N // 10                                                   # the test did exercise the changes
+    km.destroy()
