@@ -701,7 +701,7 @@ def kmeans_case(dev, stream, reps=5, iters=20, profile_only=False):
     iter_bytes = N * D * 4 + N * 4            # the points once, the labels once (centroids and partial rows are < 1 %)
     res = {
         "iterations_per_s": round(iters / (m * 1e-3), 1), "ms_per_20_iterations": round(m, 3), "ci95": round(ci, 3),
-        "path": "tensor cores (tcgen05 bf16 candidate search + one-hot sums GEMM, exact fp32 re-decision)",
+        "path": "tensor cores (tcgen05 bf16 candidate search + one-hot sums GEMM, exact fp32 re-decision); iterations after the first sum only the points whose label changed",
         "tensor_core_status_word": tc_status,
         "iteration_GBps": round(iter_bytes / (m / iters) / 1e6, 1),
         "iteration_frac_of_hbm_measured": round(iter_bytes / (m / iters) / 1e6 / peak, 4),
