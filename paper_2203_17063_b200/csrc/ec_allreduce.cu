@@ -4,8 +4,12 @@
 // warp reads the segment's notification words and the "already folded in" words,
 // takes the difference (what is new), and - by ballot - decides whether the
 // segment has news at all and whether it ever had a contributor.  The block then
-// streams the tile of every new rank with 128-bit loads, folds in ascending rank
-// order (or as a pairwise tree) and writes the result tile.  The block of tile 0
+// brings in the tile of every new rank - by bulk asynchronous copies through a
+// small ring of shared-memory stages (apply_bulk_kernel: up to 64 ranks, 128-bit
+// aligned calls), by direct 128-bit loads (apply_kernel: wide rank tables, the
+// pairwise tree, unaligned calls), or all at once for short segments
+// (apply_short_kernel) - folds in ascending rank order (or as a pairwise tree)
+// and writes the result tile.  The block of tile 0
 // also writes the segment's updated words and its contributor count.  The folded
 // words are double buffered (read one copy, write the other) so that no block can
 // see another block's update: there is no inter-block dependency and no wait.

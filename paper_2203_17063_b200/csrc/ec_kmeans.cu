@@ -8,7 +8,9 @@
 // Kernels, fastest first (ec_kmeans_iterate takes the first that covers the shape):
 //   tc::tc_fused_kernel   (ec_kmeans_tc.cuh) assignment and partial sums as two small GEMMs on the
 //             tensor cores, exact fp32 re-decision of every point the bf16 search cannot separate;
-//             D in {16, 32}, K <= 256; bound by reading the points once.
+//             D in {16, 32}, K <= 256.  After the first iteration it adds to the per-rank sums only
+//             what changed since the labels were last written (every KM_REFRESH-th iteration sums
+//             everything afresh).
 //   fused_kernel          the same two steps on the fp32 pipes: one FMA per (point, centroid,
 //             coordinate) proposes, the exact form decides inside the error bound; per-warp
 //             shared-memory slabs collect the sums in a fixed order; D in {8, 16, 32, 64}.
