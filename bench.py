@@ -684,6 +684,17 @@ def kmeans_case(dev, stream, reps=5, iters=20, profile_only=False):
         ms_assign = time_calls(stream, lambda: km.assign(d_init, lab, stream), 10)
         part = torch.empty(P, K, D + 4, device=dev)
         ms_part = time_calls(stream, lambda: km.partials(lab, part, stream), 10)
+        # the same 20 iterations with every iteration summing all points (the running sums switched off)
+        km.set_refresh(1)
+        km.set_centroids(d_init, stream)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for t in range(iters):
+            km.iterate_raw(masks[t].data_ptr(), st)
+        b.record(stream)
+        torch.cuda.synchronize()
+        ms_full_sums = a.elapsed_time(b)
+        km.set_refresh(32)
         # the same 20 iterations with the candidate search on the fp32 pipes instead of the tensor cores
         km.set_path(1)
         km.set_centroids(d_init, stream)
@@ -705,6 +716,7 @@ def kmeans_case(dev, stream, reps=5, iters=20, profile_only=False):
         "tensor_core_status_word": tc_status,
         "iteration_GBps": round(iter_bytes / (m / iters) / 1e6, 1),
         "iteration_frac_of_hbm_measured": round(iter_bytes / (m / iters) / 1e6 / peak, 4),
+        "iterations_per_s_all_points_summed_every_iteration": round(iters / (ms_full_sums * 1e-3), 1),
         "assign_only_ms": round(statistics.fmean(ms_assign), 4),
         "standalone_partials_ms": round(statistics.fmean(ms_part), 4),
         "fp32_path_iterations_per_s": round(iters / (ms_fp32_path * 1e-3), 1),

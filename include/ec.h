@@ -327,6 +327,12 @@ int ec_kmeans_set_centroids(ec_kmeans_t* km, const float* centroids, ec_stream_t
 int ec_kmeans_get(ec_kmeans_t* km, float* centroids, int32_t* labels, float* reduced,
                   uint32_t* contrib_count, ec_stream_t stream);
 
+/* Expert knob: on the tensor-core path every `every`-th iteration sums all points
+ * afresh and the iterations in between only what changed (default 32; 1 = every
+ * iteration sums everything, the running sums are not used).  The next iteration
+ * after this call is a full one.  EC_ERR_INVALID for every < 1. */
+int ec_kmeans_set_refresh(ec_kmeans_t* km, int every);
+
 /* Expert knob: which kernel ec_kmeans_iterate / ec_kmeans_assign use.
  *   0  automatic: the fastest one that covers the shape (default);
  *   1  fp32 fused kernel: candidate search by one FMA per (point, centroid, coordinate);

@@ -47,6 +47,7 @@ SYMBOLS = {
     "ec_kmeans_set_centroids": (_i, [_vp, _vp, _vp]),
     "ec_kmeans_get": (_i, [_vp, _vp, _vp, _vp, _vp, _vp]),
     "ec_kmeans_set_path": (_i, [_vp, _i]),
+    "ec_kmeans_set_refresh": (_i, [_vp, _i]),
     "ec_kmeans_tc_status": (_i, [_vp, _vp, _vp]),
     "ec_kmeans_destroy": (_i, [_vp]),
     "ec_kmeans_partials_static": (_i, [_vp, _vp, _sz, _i, _i, _i, _vp, _vp]),
@@ -250,6 +251,10 @@ class KMeans:
     def get(self, centroids=None, labels=None, reduced=None, contrib_count=None, stream=None) -> None:
         _check(lib().ec_kmeans_get(self._h, _ptr(centroids), _ptr(labels), _ptr(reduced), _ptr(contrib_count),
                                    _stream(stream)), "ec_kmeans_get")
+
+    def set_refresh(self, every: int) -> None:
+        """Every `every`-th iteration sums all points afresh (1 = each one does; default 32)."""
+        _check(lib().ec_kmeans_set_refresh(self._h, every), "ec_kmeans_set_refresh")
 
     def set_path(self, path: int) -> None:
         """0 automatic, 1 fp32 fused kernel, 2 tensor-core fused kernel."""

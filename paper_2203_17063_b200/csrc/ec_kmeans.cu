@@ -517,6 +517,7 @@ struct ec_kmeans {
     uint32_t* dirty;       // [P][Cf]: delta mode, which row blocks of scratch hold changes
     bool state_valid;      // labels and partials belong together (an iteration has run): changes can be summed
     int since_full;        // iterations since everything was summed afresh
+    int refresh;           // every refresh-th iteration sums everything afresh (1: every iteration)
 };
 
 using namespace ec;
@@ -609,14 +610,18 @@ template <int D>
 int km_tc_launch(ec_kmeans* km, bool partials, const float* centroids, int32_t* labels, cudaStream_t st, bool delta) {
     const float tau_scale = 0.015625f;     // 2^-6: four times the bound 2^-8 (|x|^2 + |c|max^2) of one candidate's error
     if (partials) {
-        tc::tc_fused_kernel<D, true><<<(unsigned)(km->P * km->Cf), tc::THREADS, km->tc_smem, st>>>(
-            km->points, km->N, km->P, km->Cf, centroids, km->K, labels, (km->Cf == 1 && !delta) ? km->partials : km->scratch,
-            tau_scale, km->tc_status, delta ? 1 : 0, km->dirty);
+        if (delta)
+            tc::tc_fused_kernel<D, true, true><<<(unsigned)(km->P * km->Cf), tc::THREADS, km->tc_smem, st>>>(
+                km->points, km->N, km->P, km->Cf, centroids, km->K, labels, km->scratch, tau_scale, km->tc_status, km->dirty);
+        else
+            tc::tc_fused_kernel<D, true, false><<<(unsigned)(km->P * km->Cf), tc::THREADS, km->tc_smem, st>>>(
+                km->points, km->N, km->P, km->Cf, centroids, km->K, labels, km->Cf == 1 ? km->partials : km->scratch,
+                tau_scale, km->tc_status, km->dirty);
     } else {
         size_t runs = (km->N + 2047) / 2048;
         if (runs > 0x7fffffffull) return EC_ERR_CAPACITY;
-        tc::tc_fused_kernel<D, false><<<(unsigned)runs, tc::THREADS, km->tc_assign_smem, st>>>(
-            km->points, km->N, 1, (int)runs, centroids, km->K, labels, nullptr, tau_scale, km->tc_status, 0, nullptr);
+        tc::tc_fused_kernel<D, false, false><<<(unsigned)runs, tc::THREADS, km->tc_assign_smem, st>>>(
+            km->points, km->N, 1, (int)runs, centroids, km->K, labels, nullptr, tau_scale, km->tc_status, nullptr);
     }
     EC_CUDA(cudaGetLastError());
     return EC_OK;
@@ -624,9 +629,11 @@ int km_tc_launch(ec_kmeans* km, bool partials, const float* centroids, int32_t* 
 
 template <int D>
 cudaError_t km_tc_attr() {
-    cudaError_t e = cudaFuncSetAttribute(tc::tc_fused_kernel<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BUDGET);
+    cudaError_t e = cudaFuncSetAttribute(tc::tc_fused_kernel<D, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BUDGET);
     if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(tc::tc_fused_kernel<D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BUDGET);
+        e = cudaFuncSetAttribute(tc::tc_fused_kernel<D, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BUDGET);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(tc::tc_fused_kernel<D, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BUDGET);
     return e;
 }
 
@@ -739,6 +746,7 @@ int ec_kmeans_init(ec_kmeans_t** out, const float* points, size_t N, int D, int 
     km->path = 0;
     km->state_valid = false;
     km->since_full = 0;
+    km->refresh = KM_REFRESH;
     km->tc_smem = tc::layout_of(D, K, true).total;
     km->tc_assign_smem = tc::layout_of(D, K, false).total;
     km->tc_status = reinterpret_cast<uint32_t*>(base + L.off_contrib + align_up((size_t)K * 4, 256));
@@ -820,7 +828,7 @@ int km_iterate_rounds(ec_kmeans_t* km, const uint64_t* const* masks, int rounds,
         // On the tensor-core path only the changes since the last iteration are summed (labels and per-rank sums
         // are kept between iterations); every KM_REFRESH-th iteration sums everything afresh, which bounds the
         // rounding that the running sums collect.
-        const bool delta = km->tc_ok && km->path != 1 && km->state_valid && km->since_full < KM_REFRESH;
+        const bool delta = km->tc_ok && km->path != 1 && km->state_valid && km->since_full + 1 < km->refresh;
         rc = km_fused(km, true, km->centroids, km->labels, stream, delta);
         if (rc != EC_OK) return rc;
         if (km->Cf > 1 || delta) {
@@ -865,6 +873,13 @@ int ec_kmeans_get(ec_kmeans_t* km, float* centroids, int32_t* labels, float* red
     if (labels) EC_CUDA(cudaMemcpyAsync(labels, km->labels, km->N * 4, cudaMemcpyDeviceToDevice, stream));
     if (reduced) EC_CUDA(cudaMemcpyAsync(reduced, km->reduced, (size_t)km->K * (km->D + 4) * 4, cudaMemcpyDeviceToDevice, stream));
     if (contrib_count) EC_CUDA(cudaMemcpyAsync(contrib_count, km->contrib, (size_t)km->K * 4, cudaMemcpyDeviceToDevice, stream));
+    return EC_OK;
+}
+
+int ec_kmeans_set_refresh(ec_kmeans_t* km, int every) {
+    if (!km || every < 1) return EC_ERR_INVALID;
+    km->refresh = every;
+    km->state_valid = false;        // the next iteration sums everything afresh
     return EC_OK;
 }
 

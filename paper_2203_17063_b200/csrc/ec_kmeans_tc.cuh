@@ -204,11 +204,12 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     return u;
 }
 
-template <int D, bool PARTIALS>
+template <int D, bool PARTIALS, bool DELTA>
 __global__ void __launch_bounds__(THREADS, EC_TC_MINB)
 tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const float* __restrict__ centroids, int K,
                 int32_t* __restrict__ labels, float* __restrict__ scratch, float tau_scale, uint32_t* __restrict__ status,
-                int delta, uint32_t* __restrict__ dirty) {
+                uint32_t* __restrict__ dirty) {
+    constexpr bool delta = DELTA;                        // sum only what changed since the labels were written last
     constexpr int KCH = D / 8;                           // 16-byte chunks of coordinates per point
     static_assert(D % 16 == 0 && KCH + 2 <= 8 && (KCH & (KCH - 1)) == 0, "D is 16 or 32");
     constexpr int LO = 8;                                // first chunk column of the low parts

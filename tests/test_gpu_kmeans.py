@@ -190,8 +190,11 @@ def test_running_sums_follow_label_changes_over_many_iterations():
     cents = inputs.kmeans_first_of_component(points, comp, K)
     rng = np.random.default_rng(78)
     km = ec.KMeans(to_dev(points), K, P, to_dev(cents))
+    full = ec.KMeans(to_dev(points), K, P, to_dev(cents))
+    full.set_refresh(1)                                                         # sums all points in every iteration
     d_labels = torch.empty(N, dtype=torch.int32, device="cuda")
     d_red = torch.empty(K, D + 4, device="cuda")
+    d_red_full = torch.empty(K, D + 4, device="cuda")
     prev = None
     moved = 0
     for t in range(40):
@@ -199,7 +202,12 @@ def test_running_sums_follow_label_changes_over_many_iterations():
         km.set_centroids(to_dev(cents))
         km.iterate(None)
         km.get(labels=d_labels, reduced=d_red)
+        full.set_centroids(to_dev(cents))
+        full.iterate(None)
+        full.get(reduced=d_red_full)
         torch.cuda.synchronize()
+        assert torch.equal(d_red[:, D], d_red_full[:, D])                       # counts: running = summed afresh
+        assert rows_close(to_host(d_red)[:, :D], to_host(d_red_full)[:, :D], rel=1e-5)
         g_labels = to_host(d_labels)
         check_labels(g_labels, points, cents)
         if prev is not None:
@@ -211,3 +219,4 @@ def test_running_sums_follow_label_changes_over_many_iterations():
         assert rows_close(got[:, :D], want[:, :D]), f"iteration {t}: sums"
     assert moved > 20 * N // 10                                                   # the test did exercise the changes
     km.destroy()
+    full.destroy()
