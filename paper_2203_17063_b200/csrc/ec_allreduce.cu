@@ -301,14 +301,24 @@ __device__ __forceinline__ void block_prologue(const ApplyArgs& a, unsigned s, u
     #pragma unroll
                 for (int d = 16; d > 0; d >>= 1) j0 += __shfl_xor_sync(0xffffffffu, j0, d);
             }
-            int j = incl - cnt_new;
-            uint64_t bits = nw;
-            while (bits) {
-                const int b = __ffsll((long long)bits) - 1;
-                bits &= bits - 1;
-                const int pos = j >= j0 ? j - j0 : j + (m_all - j0);
-                s_rank[pos] = (uint16_t)(lane * 64 + b);
-                ++j;
+            // The list of new ranks, ascending (rotated for the ring order): word by word, every lane places
+            // the two ranks it owns in the word at the position the popcount of the lower bits gives.
+            const int excl = incl - cnt_new;                              // new ranks in the words before this lane's
+            for (int wd = 0; wd < a.W; ++wd) {
+                const uint32_t lo32 = __shfl_sync(0xffffffffu, (uint32_t)nw, wd);
+                const uint32_t hi32 = __shfl_sync(0xffffffffu, (uint32_t)(nw >> 32), wd);
+                const int base = __shfl_sync(0xffffffffu, excl, wd);
+                const uint64_t word = ((uint64_t)hi32 << 32) | lo32;
+                if (word == 0) continue;
+    #pragma unroll
+                for (int half = 0; half < 2; ++half) {
+                    const int b = half * 32 + lane;
+                    if ((word >> b) & 1ull) {
+                        const int j = base + __popcll(word & ((1ull << b) - 1ull));
+                        const int pos = j >= j0 ? j - j0 : j + (m_all - j0);
+                        s_rank[pos] = (uint16_t)(wd * 64 + b);
+                    }
+                }
             }
             if (lane == 31) *s_m = incl;
             if (lane == 0) *s_fresh = (any_old == 0) ? 1 : 0;
