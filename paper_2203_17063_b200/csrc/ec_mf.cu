@@ -24,6 +24,10 @@ constexpr int MF_WARPS = MF_THREADS / 32;
 #define EC_MF_INFLIGHT 4     // measured: 1, 2, 4, 8 in flight give 2363, 2389, 2507, 1572 iterations per second
 #endif
 constexpr int MF_INFLIGHT = EC_MF_INFLIGHT;   // ratings a group of eight lanes keeps in flight
+#ifndef EC_MF_ROWS
+#define EC_MF_ROWS 1         // measured: 1, 2, 4, 8 rows per warp give 2680, 2161, 2011, 1741 iterations per second
+#endif
+constexpr int MF_ROWS = EC_MF_ROWS;           // consecutive rows a warp works through (at most 32)
 
 struct MfArgs {
     const int64_t* user_ptr; const int32_t* user_item; const float* user_val;
@@ -52,8 +56,12 @@ __global__ void mf_decide_kernel(const MfArgs a) {
     if (fresh) a.notif_clock[i] = a.clock;
 }
 
-// One warp per row.  SIDE 0: row = (rank r, item i), other = users, writes G_r[i].
-//                    SIDE 1: row = user u, other = items, takes the user step in place and adds up e^2.
+// A warp works through MF_ROWS consecutive rows (one by default).  SIDE 0: row = (rank r, item i), other = users,
+// writes G_r[i].  SIDE 1: row = user u, other = items, takes the user step in place and adds up e^2.
+// Rows are short (tens of ratings), so a row is a chain of dependent loads (extent -> ratings -> factor rows).
+// With several rows per warp the extents of all of them are read at once and the first ratings and the factor
+// vector of the next row while the current one is computed; that measured slower than one row per warp and
+// more warps, so it is off.
 // The warp works as four groups of eight lanes: a group takes one rating at a time (ratings t, t+4, t+8, ... of
 // the row go to group t mod 4), each of its lanes holds V = k/8 entries of the factor vectors, so one 128-bit
 // load per lane fetches the 128-byte factor row of the rating and the inner product needs three shuffle steps.
@@ -63,108 +71,150 @@ template <int V4, int SIDE>
 __global__ void __launch_bounds__(MF_THREADS) mf_row_kernel(const MfArgs a) {
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     const int grp = lane >> 3, sub = lane & 7;
-    const size_t row = (size_t)blockIdx.x * MF_WARPS + wid;
+    constexpr int k = 32 * V4;
     const size_t rows = SIDE == 0 ? (size_t)a.P * a.I : (size_t)a.U;
+    const size_t first = ((size_t)blockIdx.x * MF_WARPS + wid) * MF_ROWS;      // the warp's rows: first .. first + MF_ROWS - 1
+    const int32_t* idx = SIDE == 0 ? a.item_user : a.user_item;
+    const float* val = SIDE == 0 ? a.item_val : a.user_val;
+    const float* own = SIDE == 0 ? a.qi : a.pu;          // the rows' factors
+    const float* oth = SIDE == 0 ? a.pu : a.qi;          // the factors their ratings point at
     __shared__ float s_sse[MF_WARPS];
     float sse = 0.0f;
-    if (row < rows) {
-        constexpr int k = 32 * V4;
-        int r = 0;
+    // Lane l < MF_ROWS looks up row first + l (its extent in the rating arrays, whether it is to be computed), so
+    // the warp pays the latency of these dependent loads once for all its rows.
+    long long l_beg = 0, l_end = 0, l_self = 0;
+    int l_r = 0, l_active = 0;
+    if (lane < MF_ROWS && first + lane < rows) {
+        const size_t row = first + lane;
         size_t self = row;                       // index of the row's own factor vector
         bool active = true;
         if (SIDE == 0) {
-            r = (int)(row / (size_t)a.I);
-            self = row - (size_t)r * a.I;
-            active = a.refreshed[(self / a.seg_rows) * (size_t)a.P + r] != 0;
+            l_r = (int)(row / (size_t)a.I);
+            self = row - (size_t)l_r * a.I;
+            active = a.refreshed[(self / a.seg_rows) * (size_t)a.P + l_r] != 0;
         }
+        l_self = (long long)self;
+        l_active = active ? 1 : 0;
         if (active) {
-            const int64_t beg = SIDE == 0 ? a.rank_item_ptr[(size_t)r * (a.I + 1) + self] : a.user_ptr[self];
-            const int64_t end = SIDE == 0 ? a.rank_item_ptr[(size_t)r * (a.I + 1) + self + 1] : a.user_ptr[self + 1];
-            const int32_t* idx = SIDE == 0 ? a.item_user : a.user_item;
-            const float* val = SIDE == 0 ? a.item_val : a.user_val;
-            const float* own = SIDE == 0 ? a.qi : a.pu;          // the row's factors
-            const float* oth = SIDE == 0 ? a.pu : a.qi;          // the factors its ratings point at
-            // lane `sub` of every group holds entries [c*32 + sub*4, +4) of a factor vector, c < V4
-            float4 mine[V4], g[V4];
+            const int64_t* ptr = SIDE == 0 ? a.rank_item_ptr + (size_t)l_r * (a.I + 1) + self : a.user_ptr + self;
+            l_beg = ptr[0];
+            l_end = ptr[1];
+        }
+    }
+    // The first 32 ratings and the factor vector of the next row are fetched while the current row is computed.
+    int nxt_i = 0;
+    float nxt_v = 0.0f;
+    float4 nxt_mine[V4];
+    auto prefetch = [&](int rr) {
+        const long long beg = __shfl_sync(0xffffffffu, l_beg, rr), end = __shfl_sync(0xffffffffu, l_end, rr);
+        const long long self = __shfl_sync(0xffffffffu, l_self, rr);
+        const int active = __shfl_sync(0xffffffffu, l_active, rr);
+        nxt_i = 0;
+        nxt_v = 0.0f;
+        if (active) {
+            if (beg + lane < end) {
+                nxt_i = idx[beg + lane];
+                nxt_v = val[beg + lane];
+            }
+#pragma unroll
+            for (int c = 0; c < V4; ++c) nxt_mine[c] = *reinterpret_cast<const float4*>(own + (size_t)self * k + c * 32 + sub * 4);
+        }
+    };
+    prefetch(0);
+#pragma unroll 1
+    for (int rr = 0; rr < MF_ROWS; ++rr) {
+        const long long beg = __shfl_sync(0xffffffffu, l_beg, rr), end = __shfl_sync(0xffffffffu, l_end, rr);
+        const size_t self = (size_t)__shfl_sync(0xffffffffu, l_self, rr);
+        const int r = __shfl_sync(0xffffffffu, l_r, rr);
+        const bool active = __shfl_sync(0xffffffffu, l_active, rr) != 0;
+        int my_i = nxt_i;
+        float my_v = nxt_v;
+        // lane `sub` of every group holds entries [c*32 + sub*4, +4) of a factor vector, c < V4
+        float4 mine[V4], g[V4];
+#pragma unroll
+        for (int c = 0; c < V4; ++c) {
+            mine[c] = nxt_mine[c];
+            g[c] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+        }
+        if (rr + 1 < MF_ROWS) prefetch(rr + 1);
+        if (!active) continue;                   // warp-uniform: a row that is not recomputed, or past the last one
+        for (long long j0 = beg; j0 < end; j0 += 32) {
+            const int cnt = end - j0 < 32 ? (int)(end - j0) : 32;
+            if (j0 != beg) {
+                my_i = lane < cnt ? idx[j0 + lane] : 0;
+                my_v = lane < cnt ? val[j0 + lane] : 0.0f;
+            }
+            for (int t0 = 0; t0 < cnt; t0 += 4 * MF_INFLIGHT) {   // MF_INFLIGHT ratings per group in flight
+                float4 x[MF_INFLIGHT][V4];
+                float dot[MF_INFLIGHT], v[MF_INFLIGHT];
+                bool ok[MF_INFLIGHT];
+#pragma unroll
+                for (int h = 0; h < MF_INFLIGHT; ++h) {
+                    const int t = t0 + h * 4 + grp;
+                    ok[h] = t < cnt;
+                    const int o = __shfl_sync(0xffffffffu, my_i, t & 31);
+                    v[h] = __shfl_sync(0xffffffffu, my_v, t & 31);
+                    dot[h] = 0.0f;
+#pragma unroll
+                    for (int c = 0; c < V4; ++c) {
+                        x[h][c] = ok[h] ? __ldg(reinterpret_cast<const float4*>(oth + (size_t)o * k + c * 32 + sub * 4))
+                                        : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                        dot[h] = fmaf(x[h][c].x, mine[c].x, dot[h]);
+                        dot[h] = fmaf(x[h][c].y, mine[c].y, dot[h]);
+                        dot[h] = fmaf(x[h][c].z, mine[c].z, dot[h]);
+                        dot[h] = fmaf(x[h][c].w, mine[c].w, dot[h]);
+                    }
+                }
+#pragma unroll
+                for (int d = 1; d < 8; d <<= 1) {
+#pragma unroll
+                    for (int h = 0; h < MF_INFLIGHT; ++h) dot[h] += __shfl_xor_sync(0xffffffffu, dot[h], d);
+                }
+#pragma unroll
+                for (int h = 0; h < MF_INFLIGHT; ++h) {
+                    const float e = ok[h] ? v[h] - dot[h] : 0.0f;
+#pragma unroll
+                    for (int c = 0; c < V4; ++c) {
+                        g[c].x = fmaf(e, x[h][c].x, g[c].x);
+                        g[c].y = fmaf(e, x[h][c].y, g[c].y);
+                        g[c].z = fmaf(e, x[h][c].z, g[c].z);
+                        g[c].w = fmaf(e, x[h][c].w, g[c].w);
+                    }
+                    if (SIDE == 1) sse = fmaf(e, e, sse);
+                }
+            }
+        }
+        // the four groups' partial sums: (g0 + g1) + (g2 + g3), the same in every lane
+#pragma unroll
+        for (int d = 8; d < 32; d <<= 1) {
 #pragma unroll
             for (int c = 0; c < V4; ++c) {
-                mine[c] = *reinterpret_cast<const float4*>(own + self * k + c * 32 + sub * 4);
-                g[c] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                g[c].x += __shfl_xor_sync(0xffffffffu, g[c].x, d);
+                g[c].y += __shfl_xor_sync(0xffffffffu, g[c].y, d);
+                g[c].z += __shfl_xor_sync(0xffffffffu, g[c].z, d);
+                g[c].w += __shfl_xor_sync(0xffffffffu, g[c].w, d);
             }
-            for (int64_t j0 = beg; j0 < end; j0 += 32) {
-                const int cnt = end - j0 < 32 ? (int)(end - j0) : 32;
-                const int my_i = lane < cnt ? idx[j0 + lane] : 0;
-                const float my_v = lane < cnt ? val[j0 + lane] : 0.0f;
-                for (int t0 = 0; t0 < cnt; t0 += 4 * MF_INFLIGHT) {   // MF_INFLIGHT ratings per group in flight
-                    float4 x[MF_INFLIGHT][V4];
-                    float dot[MF_INFLIGHT], v[MF_INFLIGHT];
-                    bool ok[MF_INFLIGHT];
+        }
+        if (grp == 0) {
 #pragma unroll
-                    for (int h = 0; h < MF_INFLIGHT; ++h) {
-                        const int t = t0 + h * 4 + grp;
-                        ok[h] = t < cnt;
-                        const int o = __shfl_sync(0xffffffffu, my_i, t & 31);
-                        v[h] = __shfl_sync(0xffffffffu, my_v, t & 31);
-                        dot[h] = 0.0f;
-#pragma unroll
-                        for (int c = 0; c < V4; ++c) {
-                            x[h][c] = ok[h] ? __ldg(reinterpret_cast<const float4*>(oth + (size_t)o * k + c * 32 + sub * 4))
-                                            : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-                            dot[h] = fmaf(x[h][c].x, mine[c].x, dot[h]);
-                            dot[h] = fmaf(x[h][c].y, mine[c].y, dot[h]);
-                            dot[h] = fmaf(x[h][c].z, mine[c].z, dot[h]);
-                            dot[h] = fmaf(x[h][c].w, mine[c].w, dot[h]);
-                        }
-                    }
-#pragma unroll
-                    for (int d = 1; d < 8; d <<= 1) {
-#pragma unroll
-                        for (int h = 0; h < MF_INFLIGHT; ++h) dot[h] += __shfl_xor_sync(0xffffffffu, dot[h], d);
-                    }
-#pragma unroll
-                    for (int h = 0; h < MF_INFLIGHT; ++h) {
-                        const float e = ok[h] ? v[h] - dot[h] : 0.0f;
-#pragma unroll
-                        for (int c = 0; c < V4; ++c) {
-                            g[c].x = fmaf(e, x[h][c].x, g[c].x);
-                            g[c].y = fmaf(e, x[h][c].y, g[c].y);
-                            g[c].z = fmaf(e, x[h][c].z, g[c].z);
-                            g[c].w = fmaf(e, x[h][c].w, g[c].w);
-                        }
-                        if (SIDE == 1) sse = fmaf(e, e, sse);
-                    }
-                }
-            }
-            // the four groups' partial sums: (g0 + g1) + (g2 + g3), the same in every lane
-#pragma unroll
-            for (int d = 8; d < 32; d <<= 1) {
-#pragma unroll
-                for (int c = 0; c < V4; ++c) {
-                    g[c].x += __shfl_xor_sync(0xffffffffu, g[c].x, d);
-                    g[c].y += __shfl_xor_sync(0xffffffffu, g[c].y, d);
-                    g[c].z += __shfl_xor_sync(0xffffffffu, g[c].z, d);
-                    g[c].w += __shfl_xor_sync(0xffffffffu, g[c].w, d);
-                }
-                if (SIDE == 1) sse += __shfl_xor_sync(0xffffffffu, sse, d);
-            }
-            if (grp == 0) {
-#pragma unroll
-                for (int c = 0; c < V4; ++c) {
-                    if (SIDE == 0) {
-                        *reinterpret_cast<float4*>(a.grad + ((size_t)r * a.I + self) * k + c * 32 + sub * 4) = g[c];
-                    } else {
-                        float4 p = mine[c];
-                        p.x += a.lr * (g[c].x - a.lam * p.x);
-                        p.y += a.lr * (g[c].y - a.lam * p.y);
-                        p.z += a.lr * (g[c].z - a.lam * p.z);
-                        p.w += a.lr * (g[c].w - a.lam * p.w);
-                        *reinterpret_cast<float4*>(a.pu + self * k + c * 32 + sub * 4) = p;
-                    }
+            for (int c = 0; c < V4; ++c) {
+                if (SIDE == 0) {
+                    *reinterpret_cast<float4*>(a.grad + ((size_t)r * a.I + self) * k + c * 32 + sub * 4) = g[c];
+                } else {
+                    float4 p = mine[c];
+                    p.x += a.lr * (g[c].x - a.lam * p.x);
+                    p.y += a.lr * (g[c].y - a.lam * p.y);
+                    p.z += a.lr * (g[c].z - a.lam * p.z);
+                    p.w += a.lr * (g[c].w - a.lam * p.w);
+                    *reinterpret_cast<float4*>(a.pu + self * k + c * 32 + sub * 4) = p;
                 }
             }
         }
     }
     if (SIDE == 1) {
+        // e^2 of the warp's rows: every group added up its own ratings; (s0 + s1) + (s2 + s3), then the warps in order
+#pragma unroll
+        for (int d = 8; d < 32; d <<= 1) sse += __shfl_xor_sync(0xffffffffu, sse, d);
         if (lane == 0) s_sse[wid] = sse;
         __syncthreads();
         if (threadIdx.x == 0) {
@@ -214,7 +264,7 @@ bool mf_plan(int U, int I, int k, int P, size_t seg_rows, MfLayout* L) {
     L->count = off; off = align_up(off + S * 4, 256);
     L->wait = off; off = align_up(off + S * 4, 256);
     L->refreshed = off; off = align_up(off + S * P, 256);
-    L->sse_blocks = (U + MF_WARPS - 1) / MF_WARPS;
+    L->sse_blocks = (U + MF_WARPS * MF_ROWS - 1) / (MF_WARPS * MF_ROWS);
     L->sse_partial = off; off = align_up(off + (size_t)L->sse_blocks * 8, 256);
     L->sse = off; off = align_up(off + 8, 256);
     L->ar = off; off = align_up(off + ec_allreduce_workspace_bytes(P, (size_t)I * k, seg_rows * k), 256);
@@ -319,7 +369,7 @@ int ec_mf_iterate(ec_mf_t* m, const uint64_t* refresh_mask, uint32_t slack, ec_s
     const size_t pairs = a.S * (size_t)a.P;
     mf_decide_kernel<<<(unsigned)((pairs + 255) / 256), 256, 0, stream>>>(a);
     const size_t item_rows = (size_t)a.P * a.I;
-    const unsigned gi = (unsigned)((item_rows + MF_WARPS - 1) / MF_WARPS), gu = (unsigned)a.sse_blocks;
+    const unsigned gi = (unsigned)((item_rows + MF_WARPS * MF_ROWS - 1) / (MF_WARPS * MF_ROWS)), gu = (unsigned)a.sse_blocks;
     if (m->k == 32) mf_row_kernel<1, 0><<<gi, MF_THREADS, 0, stream>>>(a);
     else mf_row_kernel<2, 0><<<gi, MF_THREADS, 0, stream>>>(a);
     EC_CUDA(cudaGetLastError());
