@@ -95,11 +95,10 @@ __global__ void __launch_bounds__(MF_THREADS) mf_row_kernel(const MfArgs a) {
         }
         l_self = (long long)self;
         l_active = active ? 1 : 0;
-        if (active) {
-            const int64_t* ptr = SIDE == 0 ? a.rank_item_ptr + (size_t)l_r * (a.I + 1) + self : a.user_ptr + self;
-            l_beg = ptr[0];
-            l_end = ptr[1];
-        }
+        // the extent is read whether or not the row is recomputed: the two loads then do not wait for the flag
+        const int64_t* ptr = SIDE == 0 ? a.rank_item_ptr + (size_t)l_r * (a.I + 1) + self : a.user_ptr + self;
+        l_beg = ptr[0];
+        l_end = ptr[1];
     }
     // The first 32 ratings and the factor vector of the next row are fetched while the current row is computed.
     int nxt_i = 0;
