@@ -355,6 +355,7 @@ def run_ours(args, rank, world, local_rank):
             "input_elements_per_s": round(world * P * n * K / (total_ms_max * 1e-3), 1),
             "l2": "rank buffers (1 GiB) exceed L2 every step; the 64 MiB result is carried between rounds as in the workload",
             "ms_per_step_mean_ci95": [round(m_step, 5), round(ci_step, 5)],
+            "ms_per_step_median_min": [round(statistics.median(steps_ms), 5), round(min(steps_ms), 5)],
             "timing": f"value: two events around all {K} steps; per-launch and per-step events on every {SAMPLE}th step",
             "ms_per_round_mean": [round(statistics.fmean(r[t] for r in round_ms), 5) for t in range(len(d_masks))],
             "GBps_per_round": [round(per_round_bytes[t] / (statistics.fmean(r[t] for r in round_ms) * 1e-3) / 1e9, 1)
