@@ -99,3 +99,65 @@ def test_allgatherv_beyond_2_32_bytes(cuda_device):
             assert torch.equal(slot, bufs[r]), f"rank {r}"
         else:
             assert bool((slot == -7).all())
+
+
+def _byte_pattern(nbytes, salt):
+    """bytes[i] = low byte of (i * 2654435761 + salt) >> 11, filled on the device in pieces."""
+    out = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    step = 1 << 27
+    for lo in range(0, nbytes, step):
+        hi = min(nbytes, lo + step)
+        i = torch.arange(lo, hi, dtype=torch.int64, device="cuda")
+        out[lo:hi] = (((i * 2654435761 + salt) >> 11) & 255).to(torch.uint8)
+    return out
+
+
+def test_alltoall_rank_buffers_beyond_2_32_bytes(cuda_device):
+    free, _ = torch.cuda.mem_get_info()
+    P = 3
+    block = (3 << 29) + 48                                # 1.5 GiB blocks: a rank's buffer is 4.5 GiB
+    if free < 2 * P * P * block + (6 << 30):
+        pytest.skip("not enough free device memory")
+    send = [_byte_pattern(P * block, 1000003 * (s + 1)) for s in range(P)]
+    recv = [torch.full((P * block,), 0xA5, dtype=torch.uint8, device="cuda") for _ in range(P)]
+    arrived = np.ones((P, P), dtype=bool)
+    arrived[2, 0] = False                                 # the block from rank 0 to rank 2 is late
+    words = np.zeros((P, 1), dtype=np.uint64)
+    for d in range(P):
+        for s in range(P):
+            if arrived[d, s]:
+                words[d, 0] |= np.uint64(1) << np.uint64(s)
+    d_mask = torch.from_numpy(words.view(np.int64)).cuda()
+    cnt = torch.zeros(P, dtype=torch.int32, device="cuda")
+    ec.alltoall(send, recv, block, d_mask, cnt)
+    torch.cuda.synchronize()
+    assert cnt.cpu().tolist() == [3, 3, 2]
+    for d in range(P):
+        for s in range(P):
+            slot = recv[d][s * block:(s + 1) * block]
+            if arrived[d, s]:
+                assert torch.equal(slot, send[s][d * block:(d + 1) * block]), f"block {s} -> {d}"   # the transpose rule of Sec. IV-B
+            else:
+                assert bool((slot == 0xA5).all())
+
+
+def test_bcast_prefix_beyond_2_32_bytes(cuda_device):
+    free, _ = torch.cuda.mem_get_info()
+    n = (3 << 29) + 5                                     # 6.4 GB of fp32; three quarters of it are delivered
+    seg = (1 << 22) + 64
+    if free < 3 * n * 4 + (6 << 30):
+        pytest.skip("not enough free device memory")
+    S = (n + seg - 1) // seg
+    keep = -(-3 * S // 4)                                 # ceil(0.75 S) segments
+    src = _byte_pattern(n * 4, 77).view(torch.float32)
+    dst = [src, torch.full((n,), -3.0, device="cuda"), torch.full((n,), -3.0, device="cuda")]   # the root receives in place
+    notify = torch.zeros(S, dtype=torch.int64, device="cuda")
+    ec.bcast(src, dst, 0, ec.F32, seg, 0.75, notify)
+    torch.cuda.synchronize()
+    got = notify.cpu().numpy().view(np.uint64)
+    assert (got[:keep] == 7).all() and (got[keep:] == 0).all()
+    edge = min(n, keep * seg)
+    assert edge * 4 > 1 << 32
+    for r in (1, 2):
+        assert torch.equal(dst[r][:edge].view(torch.int32), src[:edge].view(torch.int32)), f"receiver {r}"
+        assert bool((dst[r][edge:] == -3.0).all())
