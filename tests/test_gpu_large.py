@@ -161,3 +161,43 @@ def test_bcast_prefix_beyond_2_32_bytes(cuda_device):
     for r in (1, 2):
         assert torch.equal(dst[r][:edge].view(torch.int32), src[:edge].view(torch.int32)), f"receiver {r}"
         assert bool((dst[r][edge:] == -3.0).all())
+
+
+def test_kmeans_points_beyond_2_31_elements(cuda_device):
+    """N * D > 2^31: point j sits within 0.5 of centre j mod K (centres 20 apart), so the labels, the counts and,
+    to rounding, the centroids of one iteration are known in closed form at any size."""
+    free, _ = torch.cuda.mem_get_info()
+    N, D, K, P = (1 << 26) + 777, 32, 8, 3
+    if free < N * D * 4 + (8 << 30):
+        pytest.skip("not enough free device memory")
+    g = torch.Generator(device="cuda").manual_seed(4242)
+    centres = torch.zeros(K, D, device="cuda")
+    centres[torch.arange(K), torch.arange(K)] = 20.0                      # centre k = 20 e_k
+    pts = torch.empty(N, D, device="cuda")
+    sums = torch.zeros(K, D, dtype=torch.float64, device="cuda")
+    step = 1 << 22
+    for lo in range(0, N, step):
+        hi = min(N, lo + step)
+        lab = torch.arange(lo, hi, device="cuda") % K
+        blockp = centres[lab] + (torch.rand(hi - lo, D, device="cuda", generator=g) - 0.5)
+        pts[lo:hi] = blockp
+        sums.index_add_(0, lab, blockp.double())
+    init = centres + 0.25                                                 # start off the centres: still the nearest by far
+    km = ec.KMeans(pts, K, P, init.contiguous())
+    km.iterate(None)
+    cents = torch.empty(K, D, device="cuda")
+    labels = torch.empty(N, dtype=torch.int32, device="cuda")
+    reduced = torch.empty(K, D + 4, device="cuda")
+    contrib = torch.empty(K, dtype=torch.int32, device="cuda")
+    km.get(cents, labels, reduced, contrib)
+    torch.cuda.synchronize()
+    for lo in range(0, N, step):
+        hi = min(N, lo + step)
+        assert torch.equal(labels[lo:hi].long(), torch.arange(lo, hi, device="cuda") % K), f"labels of points {lo}..{hi}"
+    counts = torch.tensor([(N - k + K - 1) // K for k in range(K)], dtype=torch.float64, device="cuda")
+    assert torch.equal(reduced[:, D].double(), counts)                    # counts are exact
+    assert bool((contrib == P).all())
+    want = sums / counts[:, None]
+    assert float((cents.double() - want).abs().max()) < 1e-4 * 20.0
+    assert km.tc_status() == 0
+    km.destroy()
