@@ -333,6 +333,16 @@ int ec_kmeans_get(ec_kmeans_t* km, float* centroids, int32_t* labels, float* red
  * after this call is a full one.  EC_ERR_INVALID for every < 1. */
 int ec_kmeans_set_refresh(ec_kmeans_t* km, int every);
 
+/* Distance bounds (on by default; tensor-core kernel only).  Between full passes the driver keeps, for every
+ * point, an upper bound on the distance to its own centroid and a lower bound on the distance to every other
+ * one, and for every centroid how far it has moved since.  A tile of 128 points whose bounds show that no label
+ * can change is not read in that iteration (triangle inequality; all roundings directed, and a margin far above
+ * the rounding of the exact form), so labels, sums and centroids are the same as without the bounds; only the
+ * time changes: an iteration in which the centroids barely move reads 12 bytes per point instead of the points.
+ * enable = 0 searches every tile in every iteration.  The paper has no counterpart (its K-means-like workloads
+ * are not described at this level); the bounds are those of the textbook accelerations of Lloyd's algorithm. */
+int ec_kmeans_set_bounds(ec_kmeans_t* km, int enable);
+
 /* Expert knob: which kernel ec_kmeans_iterate / ec_kmeans_assign use.
  *   0  automatic: the fastest one that covers the shape (default);
  *   1  fp32 fused kernel: candidate search by one FMA per (point, centroid, coordinate);

@@ -48,6 +48,7 @@ SYMBOLS = {
     "ec_kmeans_get": (_i, [_vp, _vp, _vp, _vp, _vp, _vp]),
     "ec_kmeans_set_path": (_i, [_vp, _i]),
     "ec_kmeans_set_refresh": (_i, [_vp, _i]),
+    "ec_kmeans_set_bounds": (_i, [_vp, _i]),
     "ec_kmeans_tc_status": (_i, [_vp, _vp, _vp]),
     "ec_kmeans_destroy": (_i, [_vp]),
     "ec_kmeans_partials_static": (_i, [_vp, _vp, _sz, _i, _i, _i, _vp, _vp]),
@@ -255,6 +256,10 @@ class KMeans:
     def set_refresh(self, every: int) -> None:
         """Every `every`-th iteration sums all points afresh (1 = each one does; default 32)."""
         _check(lib().ec_kmeans_set_refresh(self._h, every), "ec_kmeans_set_refresh")
+
+    def set_bounds(self, enable: bool) -> None:
+        """Distance bounds that let an iteration skip tiles whose labels cannot change (on by default)."""
+        _check(lib().ec_kmeans_set_bounds(self._h, 1 if enable else 0), "ec_kmeans_set_bounds")
 
     def set_path(self, path: int) -> None:
         """0 automatic, 1 fp32 fused kernel, 2 tensor-core fused kernel."""

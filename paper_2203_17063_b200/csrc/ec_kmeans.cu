@@ -251,6 +251,42 @@ __global__ void update_kernel(const float* __restrict__ reduced, int D, int K, f
     if (pts > 0.0f) centroids[i] = __fdiv_rn(reduced[(size_t)k * (D + 4) + d], pts);
 }
 
+// The same update in one block, which also keeps the drift sums the assignment's distance bounds rest on:
+// drift[k] += |c_k(new) - c_k(old)|, drift[K] += max_k of those moves.  Every rounding goes upwards, so the sums
+// never understate how far a centroid has moved.  One warp per centroid, lanes over the coordinates.
+constexpr int UD_THREADS = 1024;
+__global__ void __launch_bounds__(UD_THREADS)
+update_drift_kernel(const float* __restrict__ reduced, int D, int K, float* __restrict__ centroids, float* __restrict__ drift) {
+    __shared__ float s_max[UD_THREADS / 32];
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    float wmax = 0.0f;
+    for (int k = wid; k < K; k += UD_THREADS / 32) {
+        const float pts = reduced[(size_t)k * (D + 4) + D];
+        float sq = 0.0f;
+        if (pts > 0.0f) {
+            for (int d = lane; d < D; d += 32) {
+                const float c_old = centroids[(size_t)k * D + d];
+                const float c_new = __fdiv_rn(reduced[(size_t)k * (D + 4) + d], pts);
+                centroids[(size_t)k * D + d] = c_new;
+                const float diff = fmaxf(fabsf(__fsub_ru(c_new, c_old)), fabsf(__fsub_rd(c_new, c_old)));
+                sq = __fadd_ru(sq, __fmul_ru(diff, diff));
+            }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) sq = __fadd_ru(sq, __shfl_xor_sync(0xffffffffu, sq, o));
+        const float move = __fsqrt_ru(sq);
+        if (lane == 0 && move > 0.0f) drift[k] = __fadd_ru(drift[k], move);
+        wmax = fmaxf(wmax, move);
+    }
+    if (lane == 0) s_max[wid] = wmax;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float m = 0.0f;
+        for (int w = 0; w < UD_THREADS / 32; ++w) m = fmaxf(m, s_max[w]);
+        if (m > 0.0f) drift[K] = __fadd_ru(drift[K], m);
+    }
+}
+
 // ---------------------------------------------------------------------------------------------
 // fused assignment + partial sums (the path ec_kmeans_iterate takes)
 // ---------------------------------------------------------------------------------------------
@@ -515,6 +551,12 @@ struct ec_kmeans {
     size_t tc_smem, tc_assign_smem;
     uint32_t* tc_status;   // device word: nonzero if a wait on the tensor core ever gave up
     uint32_t* dirty;       // [P][Cf]: delta mode, which row blocks of scratch hold changes
+    float2* bounds;        // [N]: distance bounds of every point (tensor-core path), see tc_fused_kernel
+    float* drift;          // [K + 1]: how far every centroid has moved in all, and the sum of the largest moves
+    uint32_t* need;        // [P * Cf][need_words]: delta mode with bounds, which tiles have to be searched
+    int need_words;
+    bool bounds_valid;     // the bounds belong to the labels and to the drift sums
+    bool use_bounds;       // tiles whose bounds say that no label can change are skipped
     bool state_valid;      // labels and partials belong together (an iteration has run): changes can be summed
     int since_full;        // iterations since everything was summed afresh
     int refresh;           // every refresh-th iteration sums everything afresh (1: every iteration)
@@ -525,7 +567,8 @@ using namespace ec;
 namespace {
 
 struct KmLayout {
-    size_t off_centroids, off_labels, off_partials, off_scratch, off_reduced, off_contrib, off_dirty, off_ar, total;
+    size_t off_centroids, off_labels, off_partials, off_scratch, off_reduced, off_contrib, off_dirty, off_bounds, off_drift, off_need, off_ar, total;
+    int need_words;      // tiles of the longest run (0: the distance bounds are not kept)
     int C, warps;
     int Cf;   // runs per rank for the fused assignment+partials kernel, 0 if the shape is not covered
 };
@@ -578,6 +621,15 @@ bool km_plan(size_t N, int D, int K, int P, int sms, KmLayout* L) {
     L->off_reduced = off; off = align_up(off + (size_t)K * stride * 4, 256);
     L->off_contrib = off; off = align_up(off + (size_t)K * 4 + 256, 256);   // + a status word
     L->off_dirty = off; off = align_up(off + (size_t)P * (L->Cf > 0 ? L->Cf : 1) * 4, 256);   // change flags of the row blocks
+    L->need_words = 0;
+    if (L->Cf > 0 && tc_capable(D, K)) {
+        const size_t maxrun = (N / (size_t)P + 1) / (size_t)L->Cf + 2;
+        const size_t nw = (maxrun + 127) / 128 + 1;
+        if (nw <= (size_t)tc::NEED_WORDS_MAX) L->need_words = (int)nw;     // longer runs: no bounds, every tile is searched
+    }
+    L->off_bounds = off; off = align_up(off + (L->need_words > 0 ? N * 8 : 0), 256);   // distance bounds of the points
+    L->off_drift = off; off = align_up(off + ((size_t)K + 1) * 4, 256);
+    L->off_need = off; off = align_up(off + (size_t)P * (L->Cf > 0 ? L->Cf : 1) * (size_t)L->need_words * 4, 256);
     L->off_ar = off; off = align_up(off + ec_allreduce_workspace_bytes(P, (size_t)K * stride, stride), 256);
     L->total = off;
     return true;
@@ -609,21 +661,33 @@ int km_fused_launch(ec_kmeans* km, bool partials, const float* centroids, int32_
 template <int D>
 int km_tc_launch(ec_kmeans* km, bool partials, const float* centroids, int32_t* labels, cudaStream_t st, bool delta) {
     const float tau_scale = 0.015625f;     // 2^-6: four times the bound 2^-8 (|x|^2 + |c|max^2) of one candidate's error
+    // the distance bounds describe the context's own labels against its own centroids: an iteration keeps them,
+    // a stand-alone call on other arrays leaves them alone
+    const bool own = centroids == km->centroids && labels == km->labels && km->bounds != nullptr;
+    const bool skip = partials && delta && own && km->bounds_valid && km->use_bounds;
+    if (skip) {      // which tiles can still change a label: one byte per 32 points
+        tc::bounds_check_kernel<<<(unsigned)(km->P * km->Cf), tc::BC_THREADS, 0, st>>>(
+            km->N, km->P, km->Cf, km->K, labels, km->bounds, km->drift, km->need, km->need_words);
+        EC_CUDA(cudaGetLastError());
+    }
     if (partials) {
         if (delta)
             tc::tc_fused_kernel<D, true, true><<<(unsigned)(km->P * km->Cf), tc::THREADS, km->tc_smem, st>>>(
-                km->points, km->N, km->P, km->Cf, centroids, km->K, labels, km->scratch, tau_scale, km->tc_status, km->dirty);
+                km->points, km->N, km->P, km->Cf, centroids, km->K, labels, km->scratch, tau_scale, km->tc_status, km->dirty,
+                own ? km->bounds : nullptr, km->drift, skip ? km->need : nullptr, km->need_words);
         else
             tc::tc_fused_kernel<D, true, false><<<(unsigned)(km->P * km->Cf), tc::THREADS, km->tc_smem, st>>>(
                 km->points, km->N, km->P, km->Cf, centroids, km->K, labels, km->Cf == 1 ? km->partials : km->scratch,
-                tau_scale, km->tc_status, km->dirty);
+                tau_scale, km->tc_status, km->dirty, own ? km->bounds : nullptr, km->drift, nullptr, 0);
     } else {
         size_t runs = (km->N + 2047) / 2048;
         if (runs > 0x7fffffffull) return EC_ERR_CAPACITY;
         tc::tc_fused_kernel<D, false, false><<<(unsigned)runs, tc::THREADS, km->tc_assign_smem, st>>>(
-            km->points, km->N, 1, (int)runs, centroids, km->K, labels, nullptr, tau_scale, km->tc_status, nullptr);
+            km->points, km->N, 1, (int)runs, centroids, km->K, labels, nullptr, tau_scale, km->tc_status, nullptr,
+            nullptr, nullptr, nullptr, 0);
     }
     EC_CUDA(cudaGetLastError());
+    if (partials && own) km->bounds_valid = true;       // every tile searched in this launch has fresh bounds, the others kept valid ones
     return EC_OK;
 }
 
@@ -751,6 +815,12 @@ int ec_kmeans_init(ec_kmeans_t** out, const float* points, size_t N, int D, int 
     km->tc_assign_smem = tc::layout_of(D, K, false).total;
     km->tc_status = reinterpret_cast<uint32_t*>(base + L.off_contrib + align_up((size_t)K * 4, 256));
     km->dirty = reinterpret_cast<uint32_t*>(base + L.off_dirty);
+    km->bounds = km->tc_ok && L.need_words > 0 ? reinterpret_cast<float2*>(base + L.off_bounds) : nullptr;
+    km->need = reinterpret_cast<uint32_t*>(base + L.off_need);
+    km->need_words = L.need_words;
+    km->drift = reinterpret_cast<float*>(base + L.off_drift);
+    km->bounds_valid = false;
+    km->use_bounds = true;
     // centroid chunk for the assignment: as many as fit in 64 KB, all of them if possible
     int kc = (int)((64 * 1024) / ((size_t)D * 4));
     if (kc > K) kc = K;
@@ -779,6 +849,7 @@ int ec_kmeans_init(ec_kmeans_t** out, const float* points, size_t N, int D, int 
     if (e == cudaSuccess && km->tc_ok)
         e = D == 16 ? km_tc_attr<16>() : km_tc_attr<32>();
     if (e == cudaSuccess) e = cudaMemsetAsync(km->tc_status, 0, 4, 0);
+    if (e == cudaSuccess) e = cudaMemsetAsync(km->drift, 0, ((size_t)K + 1) * 4, 0);
     if (e == cudaSuccess) e = cudaMemcpyAsync(km->centroids, init_centroids, (size_t)K * D * 4, cudaMemcpyDeviceToDevice, 0);
     if (e == cudaSuccess) e = cudaStreamSynchronize(0);
     if (e != cudaSuccess) rc = cuda_fail(e);
@@ -853,8 +924,12 @@ int km_iterate_rounds(ec_kmeans_t* km, const uint64_t* const* masks, int rounds,
                                 km->reduced, km->contrib, stream);
         if (rc != EC_OK) return rc;
     }
-    const int total = km->K * km->D;
-    update_kernel<<<(total + 255) / 256, 256, 0, stream>>>(km->reduced, km->D, km->K, km->centroids);
+    if (km->bounds != nullptr) {
+        update_drift_kernel<<<1, UD_THREADS, 0, stream>>>(km->reduced, km->D, km->K, km->centroids, km->drift);
+    } else {
+        const int total = km->K * km->D;
+        update_kernel<<<(total + 255) / 256, 256, 0, stream>>>(km->reduced, km->D, km->K, km->centroids);
+    }
     EC_CUDA(cudaGetLastError());
     return EC_OK;
 }
@@ -863,6 +938,7 @@ int km_iterate_rounds(ec_kmeans_t* km, const uint64_t* const* masks, int rounds,
 int ec_kmeans_set_centroids(ec_kmeans_t* km, const float* centroids, ec_stream_t stream) {
     if (!km || !centroids) return EC_ERR_INVALID;
     EC_CUDA(cudaMemcpyAsync(km->centroids, centroids, (size_t)km->K * km->D * 4, cudaMemcpyDeviceToDevice, stream));
+    km->bounds_valid = false;       // the centroids moved without the drift sums knowing: the next iteration searches every tile
     return EC_OK;
 }
 
@@ -880,6 +956,12 @@ int ec_kmeans_set_refresh(ec_kmeans_t* km, int every) {
     if (!km || every < 1) return EC_ERR_INVALID;
     km->refresh = every;
     km->state_valid = false;        // the next iteration sums everything afresh
+    return EC_OK;
+}
+
+int ec_kmeans_set_bounds(ec_kmeans_t* km, int enable) {
+    if (!km) return EC_ERR_INVALID;
+    km->use_bounds = enable != 0;
     return EC_OK;
 }
 

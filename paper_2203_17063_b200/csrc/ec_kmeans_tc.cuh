@@ -155,7 +155,7 @@ __host__ __device__ inline Layout layout_of(int D, int K, bool partials) {
     Layout L;
     L.x = 0;
     L.cn = 6 * (size_t)XCHUNK;                       // npad floats (at most 256) ...
-    L.xn = L.cn + 1024;                               // ... then 128 floats; both inside columns 6-7 (at least 4160 bytes)
+    L.xn = L.cn + 1024;                               // ... then 128 floats, then npad floats of centroid drift; all inside columns 6-7 (at least 4160 bytes)
     L.b = 14 * (size_t)XCHUNK;                        // centroid operand: npad rows x (kch + 2) chunks of 16 bytes
     size_t off = L.b + npad * (kch + 2) * 16;
     if (off < 16 * (size_t)XCHUNK) off = 16 * (size_t)XCHUNK;   // all 16 columns lie inside the allocation
@@ -204,11 +204,58 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     return u;
 }
 
+// Which tiles of a delta-mode pass have to be searched (see the bounds in tc_fused_kernel).  Same runs as the
+// fused kernel (block = run c of rank r), but nothing else to carry, so the SMs are full of warps: a warp takes
+// 32 consecutive points at a time and leaves one byte, nonzero if the bounds of one of them no longer hold.
+// need: [blocks][need_words] words; byte p of a block's words = points [32p, 32p + 32) of its run, so a word is a
+// tile of the fused kernel.
+constexpr int BC_THREADS = 256;
+constexpr int NEED_WORDS_MAX = 256;
+__global__ void __launch_bounds__(BC_THREADS)
+bounds_check_kernel(size_t N, int P, int C, int K, const int32_t* __restrict__ labels, const float2* __restrict__ bounds,
+                    const float* __restrict__ drift, uint32_t* __restrict__ need, int need_words) {
+    __shared__ float s_d[1024 + 1];
+    const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
+    for (int k = tid; k <= K; k += BC_THREADS) s_d[k] = drift[k];
+    __syncthreads();
+    const float dmax = s_d[K];
+    const int r = blockIdx.x / C, c = blockIdx.x - r * C;
+    const size_t j0 = (size_t)r * N / P, j1 = (size_t)(r + 1) * N / P;
+    const size_t len = j1 - j0;
+    const size_t b0 = j0 + len * c / C, b1 = j0 + len * (c + 1) / C;
+    unsigned char* out = reinterpret_cast<unsigned char*>(need + (size_t)blockIdx.x * need_words);
+    const int pieces = (int)((b1 - b0 + 31) / 32), slots = need_words * 4;
+    for (int p0 = w; p0 < slots; p0 += 2 * (BC_THREADS / 32)) {      // two pieces per warp in flight
+        bool fail[2];
+        float2 bd[2];
+        int lb[2];
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+            const int p = p0 + q * (BC_THREADS / 32);
+            const size_t j = b0 + (size_t)p * 32 + lane;
+            lb[q] = -2;
+            if (p < pieces && j < b1) {
+                lb[q] = labels[j];
+                bd[q] = bounds[j];
+            }
+        }
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+            const int p = p0 + q * (BC_THREADS / 32);
+            fail[q] = lb[q] == -1;                               // a point without a label
+            if (lb[q] >= 0) fail[q] = !(__fmul_ru(__fadd_ru(bd[q].x, s_d[lb[q]]), 1.001f) < __fsub_rd(bd[q].y, dmax));
+            const bool any = __any_sync(0xffffffffu, fail[q]);
+            if (lane == 0 && p < slots) out[p] = any ? 1 : 0;    // bytes beyond the run are cleared, too
+        }
+    }
+}
+
 template <int D, bool PARTIALS, bool DELTA>
 __global__ void __launch_bounds__(THREADS, EC_TC_MINB)
 tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const float* __restrict__ centroids, int K,
                 int32_t* __restrict__ labels, float* __restrict__ scratch, float tau_scale, uint32_t* __restrict__ status,
-                uint32_t* __restrict__ dirty) {
+                uint32_t* __restrict__ dirty, float2* __restrict__ bounds, const float* __restrict__ drift,
+                const uint32_t* __restrict__ need, int need_words) {
     constexpr bool delta = DELTA;                        // sum only what changed since the labels were written last
     constexpr int KCH = D / 8;                           // 16-byte chunks of coordinates per point
     static_assert(D % 16 == 0 && KCH + 2 <= 8 && (KCH & (KCH - 1)) == 0, "D is 16 or 32");
@@ -220,6 +267,7 @@ tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const 
     unsigned char* s_x = smem_raw + L.x;
     float* s_cn = reinterpret_cast<float*>(smem_raw + L.cn);
     float* s_xn = reinterpret_cast<float*>(smem_raw + L.xn);
+    float* s_drift = s_xn + TILE;                        // [npad]: how far every centroid has moved in all (bounds only)
     unsigned char* s_b = smem_raw + L.b;
     unsigned char* s_oh = smem_raw + L.oh;
     uint64_t* s_bar = reinterpret_cast<uint64_t*>(smem_raw + L.bar);
@@ -229,6 +277,27 @@ tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const 
     const uint32_t ncols = tmem_cols_of(D, K, PARTIALS);
     const uint32_t bar1 = smem_u32(s_bar), bar2 = smem_u32(s_bar + 1);
 
+    const int r = blockIdx.x / C, c = blockIdx.x - r * C;
+    const size_t j0 = (size_t)r * N / P, j1 = (size_t)(r + 1) * N / P;
+    const size_t len = j1 - j0;
+    const size_t b0 = j0 + len * c / C, b1 = j0 + len * (c + 1) / C;
+    // Delta mode with distance bounds: bounds_check_kernel has looked at every point of the run and left one byte
+    // per 32 points, nonzero if one of them may change its label; a word is a tile.  A run without such a tile
+    // is done before anything is set up: once the centroids have settled that is every block.
+    const bool skipping = DELTA && PARTIALS && need != nullptr;
+    uint32_t* s_need = reinterpret_cast<uint32_t*>(s_xn + TILE + 256);   // [need_words] (at most 256), after the drift table
+    if (skipping) {
+        bool any = false;
+        for (int q = tid; q < need_words; q += THREADS) {
+            const uint32_t wd = need[(size_t)blockIdx.x * need_words + q];
+            s_need[q] = wd;
+            any = any || wd != 0u;
+        }
+        if (!__syncthreads_or(any ? 1 : 0)) {
+            if (tid == 0) dirty[blockIdx.x] = 0u;            // the row block is left alone
+            return;
+        }
+    }
     if (w == 0) tmem_alloc(smem_u32(s_tmem), ncols);
     if (tid == 0) {
         mbar_init(bar1, 1);
@@ -259,6 +328,8 @@ tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const 
         *reinterpret_cast<uint4*>(s_b + (size_t)kc * npad * 16 + (size_t)n * 16) =
             make_uint4(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]), pack_bf16(v[4], v[5]), pack_bf16(v[6], v[7]));
     }
+    if (PARTIALS && bounds != nullptr)
+        for (int k = tid; k < npad; k += THREADS) s_drift[k] = k < K ? drift[k] : 0.0f;
     // constant chunk columns of the point tile
     *reinterpret_cast<uint4*>(s_x + (size_t)KCH * XCHUNK + (size_t)tid * 16) = make_uint4(0x3F803F80u, 0u, 0u, 0u);   // [1, 1, 0, ...]
     *reinterpret_cast<uint4*>(s_x + (size_t)(KCH + 1) * XCHUNK + (size_t)tid * 16) = make_uint4(0u, 0u, 0u, 0u);
@@ -280,10 +351,6 @@ tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const 
     const uint32_t idesc_sum = instr_desc(MROWS, npad, true);
     const uint32_t b_base = smem_u32(s_b), x_base = smem_u32(s_x), oh_base = smem_u32(s_oh);
 
-    const int r = blockIdx.x / C, c = blockIdx.x - r * C;
-    const size_t j0 = (size_t)r * N / P, j1 = (size_t)(r + 1) * N / P;
-    const size_t len = j1 - j0;
-    const size_t b0 = j0 + len * c / C, b1 = j0 + len * (c + 1) / C;
     const int stride = D + 4;
     float* row_block = PARTIALS ? scratch + ((size_t)r * C + c) * (size_t)K * stride : nullptr;
     uint32_t phase1 = 0, phase2 = 0;
@@ -314,11 +381,30 @@ tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const 
             }
         }
     };
-    issue_loads(b0);
+    // Bounds (delta mode): for every point an upper bound u on the distance to its own centroid and a lower
+    // bound l on the distance to any other, both taken when the point was last searched and stored relative to
+    // the drift sums of then (u - drift[label], l + drift_max).  Centroid k has since moved by at most
+    // drift[k] - (its value then), any centroid by at most drift_max - (its value then), so u + drift[label] still
+    // bounds the one distance from above and l - drift_max the others from below (triangle inequality; all
+    // roundings directed).  A tile in which every point has u < l by a margin far above the rounding of the
+    // exact form keeps its labels: it is not read at all.
+    const bool keep_bounds = PARTIALS && bounds != nullptr;
+    const float drift_max = keep_bounds ? drift[K] : 0.0f;
+    bool pts_ready = false;                              // the registers hold the loads of the tile at hand
+    if (!skipping) {
+        issue_loads(b0);
+        pts_ready = true;
+    }
 
     for (size_t base = b0; base < b1; base += TILE) {
+        if (skipping && s_need[(base - b0) / TILE] == 0u) {  // nothing in this tile can change
+            pts_ready = false;
+            continue;
+        }
         const size_t j = base + tid;
         const bool live = j < b1;
+        if (!pts_ready) issue_loads(base);               // the tile before was skipped: its points are fetched now
+        pts_ready = false;
         const int old = (delta && live) ? labels[j] : -1;   // delta mode: the label this point had (asked for early: used after the search)
         if (PARTIALS && sums_pending) {
             // the previous tile's sums MMA still reads the tile: wait for it (its latency hid behind the search)
@@ -363,7 +449,10 @@ tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const 
             for (int o = 1; o < KCH; o <<= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
             if (kc == 0) s_xn[row] = sq;
         }
-        if (base + TILE < b1) issue_loads(base + TILE);
+        if (base + TILE < b1) {      // this tile had to be searched: the next one probably has to be, too
+            issue_loads(base + TILE);
+            pts_ready = true;
+        }
         fence_async_smem();          // the tensor core reads shared memory through the async proxy
         healthy = __syncthreads_and(healthy) != 0;
         if (tid == 0 && healthy) {
@@ -428,6 +517,17 @@ tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const 
         }
         const bool changed = live && !(delta && old == kb);
         if (changed) labels[j] = kb;
+        if (keep_bounds && live) {
+            float2 w = make_float2(__int_as_float(0x7f800000), 0.0f);      // decided by the exact form: searched again next time
+            if (done && !redo) {
+                // |x - c|^2 = |x|^2 + v; the search knows v to within tau
+                const float xn = s_xn[tid];
+                const float u = __fsqrt_ru(fmaxf(__fadd_ru(__fadd_ru(xn, m1), tau), 0.0f));
+                const float l = __fsqrt_rd(fmaxf(__fsub_rd(__fadd_rd(xn, m2), tau), 0.0f));
+                w = make_float2(__fsub_ru(u, s_drift[kb]), __fadd_rd(l, drift_max));
+            }
+            bounds[j] = w;
+        }
         if (PARTIALS && done) {
             if (changed) {
                 // one-hot row of this point: 16-byte chunk kb/8, bf16 1.0 at position kb%8 (and -1.0 for the old label)
