@@ -549,6 +549,7 @@ struct ec_kmeans {
     bool tc_ok;            // the tensor-core candidate search covers this shape
     int path;              // 0 = automatic, 1 = fp32 fused kernel, 2 = tensor-core fused kernel
     size_t tc_smem, tc_assign_smem;
+    int tc_wave_full, tc_wave_delta, tc_wave_assign;   // resident blocks of the tensor-core kernels on the whole device
     uint32_t* tc_status;   // device word: nonzero if a wait on the tensor core ever gave up
     uint32_t* dirty;       // [P][Cf]: delta mode, which row blocks of scratch hold changes
     float2* bounds;        // [N]: distance bounds of every point (tensor-core path), see tc_fused_kernel
@@ -672,17 +673,17 @@ int km_tc_launch(ec_kmeans* km, bool partials, const float* centroids, int32_t* 
     }
     if (partials) {
         if (delta)
-            tc::tc_fused_kernel<D, true, true><<<(unsigned)(km->P * km->Cf), tc::THREADS, km->tc_smem, st>>>(
+            tc::tc_fused_kernel<D, true, true><<<(unsigned)(km->P * km->Cf < km->tc_wave_delta ? km->P * km->Cf : km->tc_wave_delta), tc::THREADS, km->tc_smem, st>>>(
                 km->points, km->N, km->P, km->Cf, centroids, km->K, labels, km->scratch, tau_scale, km->tc_status, km->dirty,
                 own ? km->bounds : nullptr, km->drift, skip ? km->need : nullptr, km->need_words);
         else
-            tc::tc_fused_kernel<D, true, false><<<(unsigned)(km->P * km->Cf), tc::THREADS, km->tc_smem, st>>>(
+            tc::tc_fused_kernel<D, true, false><<<(unsigned)(km->P * km->Cf < km->tc_wave_full ? km->P * km->Cf : km->tc_wave_full), tc::THREADS, km->tc_smem, st>>>(
                 km->points, km->N, km->P, km->Cf, centroids, km->K, labels, km->Cf == 1 ? km->partials : km->scratch,
                 tau_scale, km->tc_status, km->dirty, own ? km->bounds : nullptr, km->drift, nullptr, 0);
     } else {
         size_t runs = (km->N + 2047) / 2048;
         if (runs > 0x7fffffffull) return EC_ERR_CAPACITY;
-        tc::tc_fused_kernel<D, false, false><<<(unsigned)runs, tc::THREADS, km->tc_assign_smem, st>>>(
+        tc::tc_fused_kernel<D, false, false><<<(unsigned)(runs < (size_t)km->tc_wave_assign ? runs : (size_t)km->tc_wave_assign), tc::THREADS, km->tc_assign_smem, st>>>(
             km->points, km->N, 1, (int)runs, centroids, km->K, labels, nullptr, tau_scale, km->tc_status, nullptr,
             nullptr, nullptr, nullptr, 0);
     }
@@ -691,13 +692,26 @@ int km_tc_launch(ec_kmeans* km, bool partials, const float* centroids, int32_t* 
     return EC_OK;
 }
 
+// Raises the kernels' shared-memory limit and asks how many blocks of each stay resident on an SM: a launch is
+// one wave of resident blocks that work through the runs in turn.
 template <int D>
-cudaError_t km_tc_attr() {
+cudaError_t km_tc_attr(ec_kmeans* km) {
     cudaError_t e = cudaFuncSetAttribute(tc::tc_fused_kernel<D, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BUDGET);
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(tc::tc_fused_kernel<D, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BUDGET);
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(tc::tc_fused_kernel<D, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BUDGET);
+    // Resident blocks per SM, from the kernels' own budgets (the occupancy query depends on the shared-memory
+    // carve-out of the moment): 128 threads x 128 registers, shared memory + 1 KB per block, tensor-memory columns.
+    auto per_sm = [](size_t smem, uint32_t cols) {
+        int n = 65536 / (tc::THREADS * 128);
+        const int by_smem = (int)(233472 / (smem + 1024)), by_tmem = (int)(512u / cols);
+        if (by_smem < n) n = by_smem;
+        if (by_tmem < n) n = by_tmem;
+        return n < 1 ? 1 : n;
+    };
+    km->tc_wave_full = km->tc_wave_delta = km->sms * per_sm(km->tc_smem, tc::tmem_cols_of(D, km->K, true));
+    km->tc_wave_assign = km->sms * per_sm(km->tc_assign_smem, tc::tmem_cols_of(D, km->K, false));
     return e;
 }
 
@@ -847,7 +861,7 @@ int ec_kmeans_init(ec_kmeans_t** out, const float* points, size_t N, int D, int 
     if (e == cudaSuccess && km->Cf > 0)
         e = D == 8 ? km_fused_attr<8>() : D == 16 ? km_fused_attr<16>() : D == 32 ? km_fused_attr<32>() : km_fused_attr<64>();
     if (e == cudaSuccess && km->tc_ok)
-        e = D == 16 ? km_tc_attr<16>() : km_tc_attr<32>();
+        e = D == 16 ? km_tc_attr<16>(km) : km_tc_attr<32>(km);
     if (e == cudaSuccess) e = cudaMemsetAsync(km->tc_status, 0, 4, 0);
     if (e == cudaSuccess) e = cudaMemsetAsync(km->drift, 0, ((size_t)K + 1) * 4, 0);
     if (e == cudaSuccess) e = cudaMemcpyAsync(km->centroids, init_centroids, (size_t)K * D * 4, cudaMemcpyDeviceToDevice, 0);

@@ -225,12 +225,13 @@ bounds_check_kernel(size_t N, int P, int C, int K, const int32_t* __restrict__ l
     const size_t b0 = j0 + len * c / C, b1 = j0 + len * (c + 1) / C;
     unsigned char* out = reinterpret_cast<unsigned char*>(need + (size_t)blockIdx.x * need_words);
     const int pieces = (int)((b1 - b0 + 31) / 32), slots = need_words * 4;
-    for (int p0 = w; p0 < slots; p0 += 2 * (BC_THREADS / 32)) {      // two pieces per warp in flight
-        bool fail[2];
-        float2 bd[2];
-        int lb[2];
+    constexpr int BC_U = 4;                                            // pieces a warp has in flight
+    for (int p0 = w; p0 < slots; p0 += BC_U * (BC_THREADS / 32)) {
+        bool fail[BC_U];
+        float2 bd[BC_U];
+        int lb[BC_U];
 #pragma unroll
-        for (int q = 0; q < 2; ++q) {
+        for (int q = 0; q < BC_U; ++q) {
             const int p = p0 + q * (BC_THREADS / 32);
             const size_t j = b0 + (size_t)p * 32 + lane;
             lb[q] = -2;
@@ -240,7 +241,7 @@ bounds_check_kernel(size_t N, int P, int C, int K, const int32_t* __restrict__ l
             }
         }
 #pragma unroll
-        for (int q = 0; q < 2; ++q) {
+        for (int q = 0; q < BC_U; ++q) {
             const int p = p0 + q * (BC_THREADS / 32);
             fail[q] = lb[q] == -1;                               // a point without a label
             if (lb[q] >= 0) fail[q] = !(__fmul_ru(__fadd_ru(bd[q].x, s_d[lb[q]]), 1.001f) < __fsub_rd(bd[q].y, dmax));
@@ -277,24 +278,21 @@ tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const 
     const uint32_t ncols = tmem_cols_of(D, K, PARTIALS);
     const uint32_t bar1 = smem_u32(s_bar), bar2 = smem_u32(s_bar + 1);
 
-    const int r = blockIdx.x / C, c = blockIdx.x - r * C;
-    const size_t j0 = (size_t)r * N / P, j1 = (size_t)(r + 1) * N / P;
-    const size_t len = j1 - j0;
-    const size_t b0 = j0 + len * c / C, b1 = j0 + len * (c + 1) / C;
-    // Delta mode with distance bounds: bounds_check_kernel has looked at every point of the run and left one byte
-    // per 32 points, nonzero if one of them may change its label; a word is a tile.  A run without such a tile
-    // is done before anything is set up: once the centroids have settled that is every block.
+    // A block works through the runs blockIdx.x, blockIdx.x + gridDim.x, ... (run = (rank r, part c) of the points;
+    // the grid is one wave of resident blocks), so the set-up below is paid once per block.
+    const int runs = P * C;
+    // Delta mode with distance bounds: bounds_check_kernel has looked at every point and left one byte per 32
+    // points, nonzero if one of them may change its label; a word is a tile.  A run without such a tile is
+    // done at once, and a block none of whose runs has one before anything is set up: once the centroids have
+    // settled that is every block.
     const bool skipping = DELTA && PARTIALS && need != nullptr;
     uint32_t* s_need = reinterpret_cast<uint32_t*>(s_xn + TILE + 256);   // [need_words] (at most 256), after the drift table
     if (skipping) {
         bool any = false;
-        for (int q = tid; q < need_words; q += THREADS) {
-            const uint32_t wd = need[(size_t)blockIdx.x * need_words + q];
-            s_need[q] = wd;
-            any = any || wd != 0u;
-        }
+        for (int run = blockIdx.x; run < runs; run += gridDim.x)
+            for (int q = tid; q < need_words; q += THREADS) any = any || need[(size_t)run * need_words + q] != 0u;
         if (!__syncthreads_or(any ? 1 : 0)) {
-            if (tid == 0) dirty[blockIdx.x] = 0u;            // the row block is left alone
+            for (int run = blockIdx.x + tid * gridDim.x; run < runs; run += THREADS * gridDim.x) dirty[run] = 0u;   // the row blocks are left alone
             return;
         }
     }
@@ -352,9 +350,35 @@ tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const 
     const uint32_t b_base = smem_u32(s_b), x_base = smem_u32(s_x), oh_base = smem_u32(s_oh);
 
     const int stride = D + 4;
-    float* row_block = PARTIALS ? scratch + ((size_t)r * C + c) * (size_t)K * stride : nullptr;
     uint32_t phase1 = 0, phase2 = 0;
     bool healthy = true;             // false once a wait on the tensor core gave up: plain fp32 from then on
+    bool oh_clean = true;            // the one-hot tile is all zeros
+    const bool keep_bounds = PARTIALS && bounds != nullptr;
+    const float drift_max = keep_bounds ? drift[K] : 0.0f;
+
+    for (int run = blockIdx.x; run < runs; run += gridDim.x) {
+    const int r = run / C, c = run - r * C;
+    const size_t j0 = (size_t)r * N / P, j1 = (size_t)(r + 1) * N / P;
+    const size_t len = j1 - j0;
+    const size_t b0 = j0 + len * c / C, b1 = j0 + len * (c + 1) / C;
+    if (skipping) {
+        bool any = false;
+        for (int q = tid; q < need_words; q += THREADS) {
+            const uint32_t wd = need[(size_t)run * need_words + q];
+            s_need[q] = wd;
+            any = any || wd != 0u;
+        }
+        if (!__syncthreads_or(any ? 1 : 0)) {
+            if (tid == 0) dirty[run] = 0u;               // the row block is left alone
+            continue;
+        }
+    }
+    float* row_block = PARTIALS ? scratch + (size_t)run * (size_t)K * stride : nullptr;
+    if (PARTIALS && !oh_clean) {     // the run before used the one-hot tile as scratch for its sums
+        for (int ch = 0; ch < npad / 8; ++ch)
+            *reinterpret_cast<uint4*>(s_oh + (size_t)ch * OCHUNK + (size_t)tid * 16) = make_uint4(0u, 0u, 0u, 0u);
+        oh_clean = true;
+    }
     bool sums_started = false;       // a sums MMA has been issued (the accumulator holds data)
     bool sums_pending = false;       // ... and its completion has not been waited for yet
     int prev_chunk = -1;             // one-hot chunk this thread set in the previous tile
@@ -388,8 +412,6 @@ tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const 
     // bounds the one distance from above and l - drift_max the others from below (triangle inequality; all
     // roundings directed).  A tile in which every point has u < l by a margin far above the rounding of the
     // exact form keeps its labels: it is not read at all.
-    const bool keep_bounds = PARTIALS && bounds != nullptr;
-    const float drift_max = keep_bounds ? drift[K] : 0.0f;
     bool pts_ready = false;                              // the registers hold the loads of the tile at hand
     if (!skipping) {
         issue_loads(b0);
@@ -593,7 +615,12 @@ tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const 
     }
     if (PARTIALS) {
         bool ok = true;
-        if (sums_pending) ok = mbar_wait_bounded(bar2, phase2);
+        if (sums_pending) {
+            ok = mbar_wait_bounded(bar2, phase2);
+            phase2 ^= 1u;                        // the block goes on with its next run
+            sums_pending = false;
+            if (!ok) healthy = false;
+        }
         ok = __syncthreads_and(ok) != 0;
         fence_after_sync();
         if (!ok && tid == 0 && status != nullptr) atomicOr(status, 1u);
@@ -602,6 +629,7 @@ tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const 
         // The low rows go through shared memory (the one-hot tile is free now) to the thread of their coordinate.
         if (ok && sums_started) {
             float* s_lo = reinterpret_cast<float*>(s_oh);          // [npad][D] floats <= npad/8 * 2048 bytes for D <= 32... (D*4 <= 256)
+            oh_clean = false;
             const bool is_hi = tid < D, is_cnt = tid == D, is_pad = tid > D && tid < D + 4, is_lo = tid >= 64 && tid < 64 + D;
             for (int ch = 0; ch < npad / 32; ++ch) {
                 uint32_t v[32];
@@ -627,11 +655,17 @@ tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const 
             }
         }
     }
-    if (PARTIALS && delta) {                     // delta mode: a block without changes leaves its row block alone and says so
-        if (tid == 0) dirty[blockIdx.x] = (sums_started || by_hand) ? 1u : 0u;
+    if (PARTIALS && delta) {                     // delta mode: a run without changes leaves its row block alone and says so
+        if (tid == 0) dirty[run] = (sums_started || by_hand) ? 1u : 0u;
     } else if (PARTIALS && !sums_started && !by_hand) {   // an empty run: its row block is all zeros
         for (int i = tid; i < K * stride; i += THREADS) row_block[i] = 0.0f;
     }
+    if (prev_chunk >= 0) *reinterpret_cast<uint4*>(s_oh + (size_t)prev_chunk * OCHUNK + (size_t)tid * 16) = make_uint4(0u, 0u, 0u, 0u);
+    if (prev_chunk2 >= 0) *reinterpret_cast<uint4*>(s_oh + (size_t)prev_chunk2 * OCHUNK + (size_t)tid * 16) = make_uint4(0u, 0u, 0u, 0u);
+    fence_before_sync();
+    __syncthreads();                             // the run's shared memory (sums scratch, tile flags) is free for the next one
+    fence_after_sync();
+    }   // runs
     fence_before_sync();
     __syncthreads();
     if (w == 0) tmem_dealloc(tmem_base, ncols);

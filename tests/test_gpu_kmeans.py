@@ -220,3 +220,50 @@ def test_running_sums_follow_label_changes_over_many_iterations(N, D, K, P, iter
     assert moved > (iters // 2) * N // 10                                         # the test did exercise the changes
     km.destroy()
     full.destroy()
+
+
+def test_distance_bounds_change_nothing_but_the_time():
+    """The same iterations with and without the distance bounds: labels, counts and centroids must be the same,
+    whether tiles are skipped (separated clusters), searched again (two clusters that overlap and keep
+    exchanging points) or the centroids are replaced from outside (two of them swapped: every bound is void)."""
+    N, D, K, P, iters = 40000 + 77, 32, 16, 5, 12
+    rng = np.random.default_rng(31)
+    centres = rng.uniform(-10, 10, size=(K, D)).astype(np.float32)
+    centres[1] = centres[0] + 0.3                                       # clusters 0 and 1 overlap almost entirely
+    comp = rng.integers(0, K, size=N)
+    points = (centres[comp] + rng.standard_normal((N, D))).astype(np.float32)
+    init = (centres + 0.5 * rng.standard_normal((K, D))).astype(np.float32)
+    masks = [to_dev(np.ascontiguousarray(m).view(np.int64)) for m in inputs.kmeans_masks(77, iters, P, K, 0.8)]
+    d_points = to_dev(points)
+    out = []
+    for use_bounds in (True, False):
+        km = ec.KMeans(d_points, K, P, to_dev(init))
+        km.set_bounds(use_bounds)
+        trace = []
+        for t in range(iters):
+            if t == 7:                                                  # swap two centroids behind the driver's back
+                c = torch.empty(K, D, device="cuda")
+                km.get(c)
+                c[[2, 3]] = c[[3, 2]]
+                km.set_centroids(c.contiguous())
+            km.iterate(masks[t])
+            c = torch.empty(K, D, device="cuda")
+            lab = torch.empty(N, dtype=torch.int32, device="cuda")
+            red = torch.empty(K, D + 4, device="cuda")
+            km.get(c, lab, red)
+            trace.append((to_host(c), to_host(lab), to_host(red)))
+        assert km.tc_status() == 0
+        km.destroy()
+        out.append(trace)
+    changed = 0
+    for t in range(iters):
+        (c1, l1, r1), (c0, l0, r0) = out[0][t], out[1][t]
+        assert np.array_equal(l1, l0), f"labels differ in iteration {t}"
+        assert np.array_equal(r1[:, D], r0[:, D]), f"counts differ in iteration {t}"
+        assert np.allclose(c1, c0, rtol=1e-6, atol=1e-6), f"centroids differ in iteration {t}"
+        if t:
+            changed += int((out[1][t][1] != out[1][t - 1][1]).sum())
+    assert changed > 100                                                # the overlapping clusters did keep moving points
+    # and the labels are the checker's for the centroids the last iteration started from
+    c_prev = out[0][iters - 2][0]
+    check_labels(out[0][iters - 1][1], points, c_prev)
