@@ -664,7 +664,7 @@ int km_tc_launch(ec_kmeans* km, bool partials, const float* centroids, int32_t* 
     const float tau_scale = 0.015625f;     // 2^-6: four times the bound 2^-8 (|x|^2 + |c|max^2) of one candidate's error
     // the distance bounds describe the context's own labels against its own centroids: an iteration keeps them,
     // a stand-alone call on other arrays leaves them alone
-    const bool own = centroids == km->centroids && labels == km->labels && km->bounds != nullptr;
+    const bool own = centroids == km->centroids && labels == km->labels && km->bounds != nullptr && km->use_bounds;
     const bool skip = partials && delta && own && km->bounds_valid && km->use_bounds;
     if (skip) {      // which tiles can still change a label: one byte per 32 points
         tc::bounds_check_kernel<<<(unsigned)(km->P * km->Cf), tc::BC_THREADS, 0, st>>>(
@@ -976,6 +976,7 @@ int ec_kmeans_set_refresh(ec_kmeans_t* km, int every) {
 int ec_kmeans_set_bounds(ec_kmeans_t* km, int enable) {
     if (!km) return EC_ERR_INVALID;
     km->use_bounds = enable != 0;
+    km->bounds_valid = false;       // kept only while they are in use: the next iteration searches every tile and renews them
     return EC_OK;
 }
 
