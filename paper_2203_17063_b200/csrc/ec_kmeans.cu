@@ -19,7 +19,9 @@
 //             walks a run of points with lane = coordinate into its own [K][D] slab.  These also
 //             serve ec_kmeans_partials (and ec_kmeans_assign for shapes the fused kernels skip).
 //   partials_fold_kernel  folds the row blocks of a rank in index order;
-//   update_kernel         centroid = sum / points where points > 0.
+//   update_kernel         centroid = sum / points where points > 0;
+//   update_drift_kernel   the same in one block, and how far every centroid has moved in all (what the distance
+//                         bounds of the tensor-core path rest on).
 // No floating-point atomics on any of these paths: sums are the same bits run after run.
 
 #include <new>

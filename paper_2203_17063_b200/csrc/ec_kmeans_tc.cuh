@@ -26,10 +26,15 @@
 // block without one leaves its row block unwritten and says so in a flag.  Once the clustering has settled
 // an iteration is the search alone.
 //
-// Block (r, c) covers the c-th of C runs of rank r's points and writes one [K][D+4] row block of
-// scratch; the rows of a rank are folded in order afterwards.  Every wait on the tensor core is
-// bounded; if one gives up, the block finishes in plain fp32 (exact form, atomic adds into its row
-// block) and a status word records it.
+// Distance bounds (delta mode): every point also carries an upper bound on the distance to its own centroid and
+// a lower bound on the distance to any other, every centroid the sum of its moves; bounds_check_kernel marks the
+// tiles in which a label can still change and only those are searched (details at the tile loop).
+//
+// Run (r, c) is the c-th of C parts of rank r's points and yields one [K][D+4] row block of scratch; the rows of
+// a rank are folded in order afterwards.  The grid is one wave of resident blocks; block b takes the runs b,
+// b + gridDim.x, ..., so the set-up (centroid operand, tensor memory) is paid once per block.  Every wait on
+// the tensor core is bounded; if one gives up, the block finishes in plain fp32 (exact form, atomic adds into
+// its row block) and a status word records it.
 #pragma once
 
 #include <cuda_bf16.h>
