@@ -223,7 +223,9 @@ partials_kernel(const float* __restrict__ points, const int32_t* __restrict__ la
 // (accumulate: the row blocks hold changes, which are added to what partials holds)
 __global__ void partials_fold_kernel(const float* __restrict__ scratch, int C, size_t row_elems, size_t total,
                                      float* __restrict__ partials, int accumulate = 0,
-                                     const uint32_t* __restrict__ dirty = nullptr) {
+                                     const uint32_t* __restrict__ dirty = nullptr,
+                                     const uint32_t* __restrict__ any_work = nullptr) {
+    if (any_work != nullptr && *any_work == 0u) return;      // the bounds check found no tile to search: nothing was written
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
         const size_t r = i / row_elems, e = i - r * row_elems;
         const float* src = scratch + r * (size_t)C * row_elems + e;
@@ -286,6 +288,7 @@ update_drift_kernel(const float* __restrict__ reduced, int D, int K, float* __re
         float m = 0.0f;
         for (int w = 0; w < UD_THREADS / 32; ++w) m = fmaxf(m, s_max[w]);
         if (m > 0.0f) drift[K] = __fadd_ru(drift[K], m);
+        reinterpret_cast<uint32_t*>(drift)[K + 1] = 0u;      // "some tile has to be searched": set by the next bounds check
     }
 }
 
@@ -558,6 +561,7 @@ struct ec_kmeans {
     float* drift;          // [K + 1]: how far every centroid has moved in all, and the sum of the largest moves
     uint32_t* need;        // [P * Cf][need_words]: delta mode with bounds, which tiles have to be searched
     int need_words;
+    bool skipped;          // the last pass of the tensor-core kernel ran behind a bounds check
     bool bounds_valid;     // the bounds belong to the labels and to the drift sums
     bool use_bounds;       // tiles whose bounds say that no label can change are skipped
     bool state_valid;      // labels and partials belong together (an iteration has run): changes can be summed
@@ -631,7 +635,7 @@ bool km_plan(size_t N, int D, int K, int P, int sms, KmLayout* L) {
         if (nw <= (size_t)tc::NEED_WORDS_MAX) L->need_words = (int)nw;     // longer runs: no bounds, every tile is searched
     }
     L->off_bounds = off; off = align_up(off + (L->need_words > 0 ? N * 8 : 0), 256);   // distance bounds of the points
-    L->off_drift = off; off = align_up(off + ((size_t)K + 1) * 4, 256);
+    L->off_drift = off; off = align_up(off + ((size_t)K + 2) * 4, 256);    // drift sums, their maximum's sum, the check's flag word
     L->off_need = off; off = align_up(off + (size_t)P * (L->Cf > 0 ? L->Cf : 1) * (size_t)L->need_words * 4, 256);
     L->off_ar = off; off = align_up(off + ec_allreduce_workspace_bytes(P, (size_t)K * stride, stride), 256);
     L->total = off;
@@ -670,7 +674,8 @@ int km_tc_launch(ec_kmeans* km, bool partials, const float* centroids, int32_t* 
     const bool skip = partials && delta && own && km->bounds_valid && km->use_bounds;
     if (skip) {      // which tiles can still change a label: one byte per 32 points
         tc::bounds_check_kernel<<<(unsigned)(km->P * km->Cf), tc::BC_THREADS, 0, st>>>(
-            km->N, km->P, km->Cf, km->K, labels, km->bounds, km->drift, km->need, km->need_words);
+            km->N, km->P, km->Cf, km->K, labels, km->bounds, km->drift, km->need, km->need_words, km->dirty,
+            reinterpret_cast<uint32_t*>(km->drift) + km->K + 1);
         EC_CUDA(cudaGetLastError());
     }
     if (partials) {
@@ -690,6 +695,7 @@ int km_tc_launch(ec_kmeans* km, bool partials, const float* centroids, int32_t* 
             nullptr, nullptr, nullptr, 0);
     }
     EC_CUDA(cudaGetLastError());
+    km->skipped = skip;
     if (partials && own) km->bounds_valid = true;       // every tile searched in this launch has fresh bounds, the others kept valid ones
     return EC_OK;
 }
@@ -865,7 +871,7 @@ int ec_kmeans_init(ec_kmeans_t** out, const float* points, size_t N, int D, int 
     if (e == cudaSuccess && km->tc_ok)
         e = D == 16 ? km_tc_attr<16>(km) : km_tc_attr<32>(km);
     if (e == cudaSuccess) e = cudaMemsetAsync(km->tc_status, 0, 4, 0);
-    if (e == cudaSuccess) e = cudaMemsetAsync(km->drift, 0, ((size_t)K + 1) * 4, 0);
+    if (e == cudaSuccess) e = cudaMemsetAsync(km->drift, 0, ((size_t)K + 2) * 4, 0);
     if (e == cudaSuccess) e = cudaMemcpyAsync(km->centroids, init_centroids, (size_t)K * D * 4, cudaMemcpyDeviceToDevice, 0);
     if (e == cudaSuccess) e = cudaStreamSynchronize(0);
     if (e != cudaSuccess) rc = cuda_fail(e);
@@ -921,7 +927,8 @@ int km_iterate_rounds(ec_kmeans_t* km, const uint64_t* const* masks, int rounds,
         if (km->Cf > 1 || delta) {
             const size_t row = (size_t)km->K * (km->D + 4), total = row * km->P;
             partials_fold_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(km->scratch, km->Cf, row, total,
-                                                                                      km->partials, delta ? 1 : 0, km->dirty);
+                                                                                      km->partials, delta ? 1 : 0, km->dirty,
+                                                                                      delta && km->skipped ? reinterpret_cast<const uint32_t*>(km->drift) + km->K + 1 : nullptr);
             EC_CUDA(cudaGetLastError());
         }
         km->state_valid = true;

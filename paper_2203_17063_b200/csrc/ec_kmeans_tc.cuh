@@ -218,7 +218,8 @@ constexpr int BC_THREADS = 256;
 constexpr int NEED_WORDS_MAX = 256;
 __global__ void __launch_bounds__(BC_THREADS)
 bounds_check_kernel(size_t N, int P, int C, int K, const int32_t* __restrict__ labels, const float2* __restrict__ bounds,
-                    const float* __restrict__ drift, uint32_t* __restrict__ need, int need_words) {
+                    const float* __restrict__ drift, uint32_t* __restrict__ need, int need_words,
+                    uint32_t* __restrict__ dirty, uint32_t* __restrict__ any_work) {
     __shared__ float s_d[1024 + 1];
     const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
     for (int k = tid; k <= K; k += BC_THREADS) s_d[k] = drift[k];
@@ -230,6 +231,7 @@ bounds_check_kernel(size_t N, int P, int C, int K, const int32_t* __restrict__ l
     const size_t b0 = j0 + len * c / C, b1 = j0 + len * (c + 1) / C;
     unsigned char* out = reinterpret_cast<unsigned char*>(need + (size_t)blockIdx.x * need_words);
     const int pieces = (int)((b1 - b0 + 31) / 32), slots = need_words * 4;
+    bool mine = false;                                                 // one of this thread's points may change its label
     constexpr int BC_U = 4;                                            // pieces a warp has in flight
     for (int p0 = w; p0 < slots; p0 += BC_U * (BC_THREADS / 32)) {
         bool fail[BC_U];
@@ -252,7 +254,15 @@ bounds_check_kernel(size_t N, int P, int C, int K, const int32_t* __restrict__ l
             if (lb[q] >= 0) fail[q] = !(__fmul_ru(__fadd_ru(bd[q].x, s_d[lb[q]]), 1.001f) < __fsub_rd(bd[q].y, dmax));
             const bool any = __any_sync(0xffffffffu, fail[q]);
             if (lane == 0 && p < slots) out[p] = any ? 1 : 0;    // bytes beyond the run are cleared, too
+            mine = mine || fail[q];
         }
+    }
+    // A run without a marked tile is settled here (its row block is left alone); if there is none at all,
+    // *any_work (cleared by the update kernel of the iteration before) stays 0 and the fused kernel's blocks leave at once.
+    const bool any_run = __syncthreads_or(mine ? 1 : 0) != 0;
+    if (tid == 0) {
+        if (any_run) atomicOr(any_work, 1u);
+        else dirty[blockIdx.x] = 0u;
     }
 }
 
@@ -293,6 +303,7 @@ tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const 
     const bool skipping = DELTA && PARTIALS && need != nullptr;
     uint32_t* s_need = reinterpret_cast<uint32_t*>(s_xn + TILE + 256);   // [need_words] (at most 256), after the drift table
     if (skipping) {
+        if (reinterpret_cast<const uint32_t*>(drift)[K + 1] == 0u) return;   // no tile anywhere: the check has settled every run
         bool any = false;
         for (int run = blockIdx.x; run < runs; run += gridDim.x)
             for (int q = tid; q < need_words; q += THREADS) any = any || need[(size_t)run * need_words + q] != 0u;
