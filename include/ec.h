@@ -309,7 +309,9 @@ int ec_kmeans_partials(ec_kmeans_t* km, const int32_t* labels, float* partials, 
  * the sums only what changed - +x for the cluster a point joins, -x for the one
  * it leaves - and every 32nd iteration sums everything afresh, which bounds the
  * rounding the running sums collect (about 2^-24 of a sum per iteration; counts
- * stay exact).  Results repeat bit for bit from run to run either way. */
+ * stay exact).  Those iterations also skip the search of points whose label
+ * provably cannot change (ec_kmeans_set_bounds below).  Results repeat bit for
+ * bit from run to run either way. */
 int ec_kmeans_iterate(ec_kmeans_t* km, const uint64_t* arrival_mask, ec_stream_t stream);
 
 /* The same iteration with the combine step spread over several rounds: one allreduce epoch with
@@ -318,7 +320,8 @@ int ec_kmeans_iterate(ec_kmeans_t* km, const uint64_t* arrival_mask, ec_stream_t
  * rows that are late in round 1 still count if a later round of the same iteration sees them. */
 int ec_kmeans_iterate_rounds(ec_kmeans_t* km, const uint64_t* const* arrival_masks, int rounds, ec_stream_t stream);
 
-/* Replace the context's centroids (device [K][D]); used for lock-step checks. */
+/* Replace the context's centroids (device [K][D]); used for lock-step checks.  The next iteration
+ * searches every point again (the distance bounds do not know how far the centroids were moved). */
 int ec_kmeans_set_centroids(ec_kmeans_t* km, const float* centroids, ec_stream_t stream);
 
 /* Copy out (device to device, on `stream`) whichever outputs are non-NULL:
