@@ -676,8 +676,9 @@ tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const 
     } else if (PARTIALS && !sums_started && !by_hand) {   // an empty run: its row block is all zeros
         for (int i = tid; i < K * stride; i += THREADS) row_block[i] = 0.0f;
     }
-    if (prev_chunk >= 0) *reinterpret_cast<uint4*>(s_oh + (size_t)prev_chunk * OCHUNK + (size_t)tid * 16) = make_uint4(0u, 0u, 0u, 0u);
-    if (prev_chunk2 >= 0) *reinterpret_cast<uint4*>(s_oh + (size_t)prev_chunk2 * OCHUNK + (size_t)tid * 16) = make_uint4(0u, 0u, 0u, 0u);
+    // A run that issued a sums MMA leaves entries in the one-hot tile (the last tile's, and the sums scratch above):
+    // the next run clears the whole tile before it uses it.  (Not here: other warps may still be reading the scratch.)
+    if (sums_started) oh_clean = false;
     fence_before_sync();
     __syncthreads();                             // the run's shared memory (sums scratch, tile flags) is free for the next one
     fence_after_sync();

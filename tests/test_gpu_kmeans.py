@@ -259,8 +259,9 @@ def test_distance_bounds_change_nothing_but_the_time():
     for t in range(iters):
         (c1, l1, r1), (c0, l0, r0) = out[0][t], out[1][t]
         assert np.array_equal(l1, l0), f"labels differ in iteration {t}"
-        assert np.array_equal(r1[:, D], r0[:, D]), f"counts differ in iteration {t}"
-        assert np.allclose(c1, c0, rtol=1e-6, atol=1e-6), f"centroids differ in iteration {t}"
+        # the same tiles issue the same sums in the same order either way: not a bit may differ
+        assert np.array_equal(r1, r0), f"reduced sums differ in iteration {t}"
+        assert np.array_equal(c1, c0), f"centroids differ in iteration {t}"
         if t:
             changed += int((out[1][t][1] != out[1][t - 1][1]).sum())
     assert changed > 100                                                # the overlapping clusters did keep moving points
