@@ -268,3 +268,45 @@ def test_distance_bounds_change_nothing_but_the_time():
     # and the labels are the checker's for the centroids the last iteration started from
     c_prev = out[0][iters - 2][0]
     check_labels(out[0][iters - 1][1], points, c_prev)
+
+
+def test_many_runs_per_block_with_churn():
+    """More runs than resident blocks, so that a block works through several runs, on clusters that keep exchanging
+    points: with the bounds, without them, and with every iteration summing all points afresh the labels and counts
+    must agree, the first two to the bit, the running sums with the fresh ones to rounding."""
+    N, D, K, P, iters = (1 << 21) + 1234, 32, 64, 64, 6
+    g = torch.Generator(device="cuda").manual_seed(99)
+    centres = (torch.rand(K, D, device="cuda", generator=g) - 0.5) * 4.0          # sigma 1 around centres 4 wide: heavy overlap
+    comp = torch.randint(0, K, (N,), device="cuda", generator=g)
+    points = (centres[comp] + torch.randn(N, D, device="cuda", generator=g)).contiguous()
+    init = points[torch.randperm(N, device="cuda", generator=g)[:K]].contiguous()
+    masks = [to_dev(np.ascontiguousarray(m).view(np.int64)) for m in inputs.kmeans_masks(123, iters, P, K, 0.8)]
+    traces = []
+    for mode in ("bounds", "no bounds", "fresh sums"):
+        km = ec.KMeans(points, K, P, init)
+        km.set_bounds(mode == "bounds")
+        if mode == "fresh sums":
+            km.set_refresh(1)
+        tr = []
+        for t in range(iters):
+            km.iterate(masks[t])
+            c = torch.empty(K, D, device="cuda")
+            lab = torch.empty(N, dtype=torch.int32, device="cuda")
+            red = torch.empty(K, D + 4, device="cuda")
+            km.get(c, lab, red)
+            tr.append((c.clone(), lab.clone(), red.clone()))
+        assert km.tc_status() == 0
+        km.destroy()
+        traces.append(tr)
+    moved = 0
+    for t in range(iters):
+        (c1, l1, r1), (c0, l0, r0), (cf, lf, rf) = traces[0][t], traces[1][t], traces[2][t]
+        assert torch.equal(l1, l0) and torch.equal(r1, r0) and torch.equal(c1, c0), f"bounds on / off differ in iteration {t}"
+        # fresh sums: the centroids of the iteration before differ by rounding, so a few near-tie labels may differ
+        same = (l1 == lf).float().mean().item()
+        assert same > 0.9999, f"labels of running and fresh sums: {same}"
+        err = (r1[:, :D].double() - rf[:, :D].double()).norm(dim=1) / rf[:, :D].double().norm(dim=1).clamp_min(1e-30)
+        assert float(err.max()) < 2e-4, f"running sums drifted from fresh ones in iteration {t}: {float(err.max())}"
+        if t:
+            moved += int((l0 != traces[1][t - 1][1]).sum())
+    assert moved > 10000
