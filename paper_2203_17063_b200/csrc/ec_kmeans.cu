@@ -947,7 +947,7 @@ int km_iterate_rounds(ec_kmeans_t* km, const uint64_t* const* masks, int rounds,
                                 km->reduced, km->contrib, stream);
         if (rc != EC_OK) return rc;
     }
-    if (km->bounds != nullptr) {
+    if (km->bounds != nullptr && km->use_bounds) {   // (bounds switched on again later are all renewed first: no drift sums needed meanwhile)
         update_drift_kernel<<<1, UD_THREADS, 0, stream>>>(km->reduced, km->D, km->K, km->centroids, km->drift);
     } else {
         const int total = km->K * km->D;
