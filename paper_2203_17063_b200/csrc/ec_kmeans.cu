@@ -679,18 +679,29 @@ int km_tc_launch(ec_kmeans* km, bool partials, const float* centroids, int32_t* 
         EC_CUDA(cudaGetLastError());
     }
     if (partials) {
-        if (delta)
-            tc::tc_fused_kernel<D, true, true><<<(unsigned)(km->P * km->Cf < km->tc_wave_delta ? km->P * km->Cf : km->tc_wave_delta), tc::THREADS, km->tc_smem, st>>>(
+        const unsigned gd = (unsigned)(km->P * km->Cf < km->tc_wave_delta ? km->P * km->Cf : km->tc_wave_delta);
+        const unsigned gf = (unsigned)(km->P * km->Cf < km->tc_wave_full ? km->P * km->Cf : km->tc_wave_full);
+        float* full_out = km->Cf == 1 ? km->partials : km->scratch;
+        if (delta && own)
+            tc::tc_fused_kernel<D, true, true, true><<<gd, tc::THREADS, km->tc_smem, st>>>(
                 km->points, km->N, km->P, km->Cf, centroids, km->K, labels, km->scratch, tau_scale, km->tc_status, km->dirty,
-                own ? km->bounds : nullptr, km->drift, skip ? km->need : nullptr, km->need_words);
+                km->bounds, km->drift, skip ? km->need : nullptr, km->need_words);
+        else if (delta)
+            tc::tc_fused_kernel<D, true, true, false><<<gd, tc::THREADS, km->tc_smem, st>>>(
+                km->points, km->N, km->P, km->Cf, centroids, km->K, labels, km->scratch, tau_scale, km->tc_status, km->dirty,
+                nullptr, nullptr, nullptr, 0);
+        else if (own)
+            tc::tc_fused_kernel<D, true, false, true><<<gf, tc::THREADS, km->tc_smem, st>>>(
+                km->points, km->N, km->P, km->Cf, centroids, km->K, labels, full_out, tau_scale, km->tc_status, km->dirty,
+                km->bounds, km->drift, nullptr, 0);
         else
-            tc::tc_fused_kernel<D, true, false><<<(unsigned)(km->P * km->Cf < km->tc_wave_full ? km->P * km->Cf : km->tc_wave_full), tc::THREADS, km->tc_smem, st>>>(
-                km->points, km->N, km->P, km->Cf, centroids, km->K, labels, km->Cf == 1 ? km->partials : km->scratch,
-                tau_scale, km->tc_status, km->dirty, own ? km->bounds : nullptr, km->drift, nullptr, 0);
+            tc::tc_fused_kernel<D, true, false, false><<<gf, tc::THREADS, km->tc_smem, st>>>(
+                km->points, km->N, km->P, km->Cf, centroids, km->K, labels, full_out, tau_scale, km->tc_status, km->dirty,
+                nullptr, nullptr, nullptr, 0);
     } else {
         size_t runs = (km->N + 2047) / 2048;
         if (runs > 0x7fffffffull) return EC_ERR_CAPACITY;
-        tc::tc_fused_kernel<D, false, false><<<(unsigned)(runs < (size_t)km->tc_wave_assign ? runs : (size_t)km->tc_wave_assign), tc::THREADS, km->tc_assign_smem, st>>>(
+        tc::tc_fused_kernel<D, false, false, false><<<(unsigned)(runs < (size_t)km->tc_wave_assign ? runs : (size_t)km->tc_wave_assign), tc::THREADS, km->tc_assign_smem, st>>>(
             km->points, km->N, 1, (int)runs, centroids, km->K, labels, nullptr, tau_scale, km->tc_status, nullptr,
             nullptr, nullptr, nullptr, 0);
     }
@@ -704,11 +715,15 @@ int km_tc_launch(ec_kmeans* km, bool partials, const float* centroids, int32_t* 
 // one wave of resident blocks that work through the runs in turn.
 template <int D>
 cudaError_t km_tc_attr(ec_kmeans* km) {
-    cudaError_t e = cudaFuncSetAttribute(tc::tc_fused_kernel<D, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BUDGET);
+    cudaError_t e = cudaFuncSetAttribute(tc::tc_fused_kernel<D, true, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BUDGET);
     if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(tc::tc_fused_kernel<D, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BUDGET);
+        e = cudaFuncSetAttribute(tc::tc_fused_kernel<D, true, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BUDGET);
     if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(tc::tc_fused_kernel<D, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BUDGET);
+        e = cudaFuncSetAttribute(tc::tc_fused_kernel<D, true, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BUDGET);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(tc::tc_fused_kernel<D, true, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BUDGET);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(tc::tc_fused_kernel<D, false, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BUDGET);
     // Resident blocks per SM, from the kernels' own budgets (the occupancy query depends on the shared-memory
     // carve-out of the moment): 128 threads x 128 registers, shared memory + 1 KB per block, tensor-memory columns.
     auto per_sm = [](size_t smem, uint32_t cols) {

@@ -266,7 +266,7 @@ bounds_check_kernel(size_t N, int P, int C, int K, const int32_t* __restrict__ l
     }
 }
 
-template <int D, bool PARTIALS, bool DELTA>
+template <int D, bool PARTIALS, bool DELTA, bool BOUNDS>
 __global__ void __launch_bounds__(THREADS, EC_TC_MINB)
 tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const float* __restrict__ centroids, int K,
                 int32_t* __restrict__ labels, float* __restrict__ scratch, float tau_scale, uint32_t* __restrict__ status,
@@ -300,7 +300,7 @@ tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const 
     // points, nonzero if one of them may change its label; a word is a tile.  A run without such a tile is
     // done at once, and a block none of whose runs has one before anything is set up: once the centroids have
     // settled that is every block.
-    const bool skipping = DELTA && PARTIALS && need != nullptr;
+    const bool skipping = DELTA && PARTIALS && BOUNDS && need != nullptr;
     uint32_t* s_need = reinterpret_cast<uint32_t*>(s_xn + TILE + 256);   // [need_words] (at most 256), after the drift table
     if (skipping) {
         if (reinterpret_cast<const uint32_t*>(drift)[K + 1] == 0u) return;   // no tile anywhere: the check has settled every run
@@ -342,7 +342,7 @@ tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const 
         *reinterpret_cast<uint4*>(s_b + (size_t)kc * npad * 16 + (size_t)n * 16) =
             make_uint4(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]), pack_bf16(v[4], v[5]), pack_bf16(v[6], v[7]));
     }
-    if (PARTIALS && bounds != nullptr)
+    if (PARTIALS && BOUNDS)
         for (int k = tid; k < npad; k += THREADS) s_drift[k] = k < K ? drift[k] : 0.0f;
     // constant chunk columns of the point tile
     *reinterpret_cast<uint4*>(s_x + (size_t)KCH * XCHUNK + (size_t)tid * 16) = make_uint4(0x3F803F80u, 0u, 0u, 0u);   // [1, 1, 0, ...]
@@ -369,7 +369,7 @@ tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const 
     uint32_t phase1 = 0, phase2 = 0;
     bool healthy = true;             // false once a wait on the tensor core gave up: plain fp32 from then on
     bool oh_clean = true;            // the one-hot tile is all zeros
-    const bool keep_bounds = PARTIALS && bounds != nullptr;
+    constexpr bool keep_bounds = PARTIALS && BOUNDS;     // (the host passes the arrays whenever it picks this instantiation)
     const float drift_max = keep_bounds ? drift[K] : 0.0f;
 
     for (int run = blockIdx.x; run < runs; run += gridDim.x) {
