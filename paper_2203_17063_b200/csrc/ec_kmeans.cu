@@ -267,10 +267,11 @@ update_drift_kernel(const float* __restrict__ reduced, int D, int K, float* __re
     for (int k = wid; k < K; k += UD_THREADS / 32) {
         const float pts = reduced[(size_t)k * (D + 4) + D];
         float sq = 0.0f;
-        if (pts > 0.0f) {
-            for (int d = lane; d < D; d += 32) {
-                const float c_old = centroids[(size_t)k * D + d];
-                const float c_new = __fdiv_rn(reduced[(size_t)k * (D + 4) + d], pts);
+        for (int d = lane; d < D; d += 32) {             // the loads do not wait for the count
+            const float c_old = centroids[(size_t)k * D + d];
+            const float sum = reduced[(size_t)k * (D + 4) + d];
+            if (pts > 0.0f) {
+                const float c_new = __fdiv_rn(sum, pts);
                 centroids[(size_t)k * D + d] = c_new;
                 const float diff = fmaxf(fabsf(__fsub_ru(c_new, c_old)), fabsf(__fsub_rd(c_new, c_old)));
                 sq = __fadd_ru(sq, __fmul_ru(diff, diff));
