@@ -375,7 +375,7 @@ int ec_kmeans_destroy(ec_kmeans_t* km);
  *
  * It computes exactly what ec_kmeans_partials computes (same kernels, same
  * order of additions, same bits) from
- *   points    device fp32 [N][D], 16-byte aligned
+ *   points    device fp32 [N][D]
  *   labels    device int32 [N]
  *   partials  device fp32 [P][K][D+4], written
  * with the same limits on N, D, K, P as the K-means driver.  The per-block
@@ -388,7 +388,8 @@ int ec_kmeans_destroy(ec_kmeans_t* km);
  * The call itself allocates nothing: no cudaMalloc, no cudaFree, no allocating
  * library routine.  The first call on each device looks up the device address
  * of the array and raises the kernel's shared-memory limit; make that first
- * call before starting any stream capture.
+ * call before starting any stream capture.  Host threads may make their first
+ * calls at the same time: the set-up is serialised by a lock inside the library.
  * All calls on a device share the one array.  A call overwrites every element
  * it later reads, so no clearing is needed and nothing leaks from the previous
  * call; but two calls that run on the GPU at the same time (different streams,

@@ -655,7 +655,7 @@ apply_bulk_kernel(const ApplyArgs a, const __grid_constant__ PtrTable<64> tbl) {
     __shared__ const char* s_ptr[64];
     __shared__ uint16_t s_rank[64];
     __shared__ uint64_t s_new[MAX_W];
-    __shared__ int s_m, s_fresh;
+    __shared__ int s_m, s_fresh, s_gave_up;
     __shared__ __align__(8) uint64_t s_bar[BK_STAGES];
 
     const unsigned s = blockIdx.x / a.tiles_per_seg;
@@ -665,6 +665,7 @@ apply_bulk_kernel(const ApplyArgs a, const __grid_constant__ PtrTable<64> tbl) {
     if (seg_hi > a.n) seg_hi = a.n;
     const int tid = threadIdx.x;
     if (tid == 0) {
+        s_gave_up = 0;
 #pragma unroll
         for (int q = 0; q < BK_STAGES; ++q)
             asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bk_smem(&s_bar[q])) : "memory");
@@ -712,19 +713,27 @@ apply_bulk_kernel(const ApplyArgs a, const __grid_constant__ PtrTable<64> tbl) {
             load_acc<Acc, VEC>(res + (size_t)v * VEC, acc[p], rpol_ld);
         }
     }
-    unsigned late_mask = 0;                                               // stages whose copy did not report in time
+    // A wait that runs out (never expected) ends the staging for the whole block: the thread that saw it reads its
+    // vectors of that rank directly and raises s_gave_up; after the barrier that closes the rank every thread sees
+    // the flag, no further copy is issued and the remaining ranks are read directly.  So no barrier is ever armed a
+    // second time inside a phase that did not complete, and a late copy can only land in a stage nobody reads again.
+    bool direct = false;
+    int issued = m < BK_STAGES ? m : BK_STAGES;                           // copies issued so far (thread 0's count)
     if (bytes != 0) {
         for (int j = 0; j < m; ++j) {
             const int st = j % BK_STAGES;
-            const bool arrived = bk_wait(bk_smem(&s_bar[st]), (uint32_t)(j / BK_STAGES) & 1u);
-            if (!arrived) late_mask |= 1u << st;
+            bool arrived = false;
+            if (!direct) {
+                arrived = bk_wait(bk_smem(&s_bar[st]), (uint32_t)(j / BK_STAGES) & 1u);
+                if (!arrived) *reinterpret_cast<volatile int*>(&s_gave_up) = 1;
+            }
             const unsigned char* src = bk_stage + (size_t)st * BK_STAGE_BYTES;
 #pragma unroll
             for (int p = 0; p < BK_VPT; ++p) {
                 const int v = p * BK_THREADS + tid;
                 if (v < nvec) {
                     const uint4 raw = arrived ? *reinterpret_cast<const uint4*>(src + (size_t)v * 16)
-                                              : ld_stream16(s_ptr[j] + (size_t)v * 16, pol);     // the copy never reported: read directly
+                                              : ld_stream16(s_ptr[j] + (size_t)v * 16, pol);     // no copy to read from: read directly
                     Acc x[VEC];
                     E::unpack(raw, x);
 #pragma unroll
@@ -732,8 +741,11 @@ apply_bulk_kernel(const ApplyArgs a, const __grid_constant__ PtrTable<64> tbl) {
                 }
             }
             __syncthreads();                                             // everybody is done with this stage
-            if (tid == 0 && j + BK_STAGES < m)
+            if (!direct && *reinterpret_cast<volatile int*>(&s_gave_up) != 0) direct = true;
+            if (tid == 0 && !direct && j + BK_STAGES < m) {
                 bk_copy(bk_smem(bk_stage + (size_t)st * BK_STAGE_BYTES), s_ptr[j + BK_STAGES], bytes, bk_smem(&s_bar[st]), pol);
+                ++issued;
+            }
         }
 #pragma unroll
         for (int p = 0; p < BK_VPT; ++p) {
@@ -747,12 +759,11 @@ apply_bulk_kernel(const ApplyArgs a, const __grid_constant__ PtrTable<64> tbl) {
         for (int j = 0; j < m; ++j) x = comb<OP>(x, E::widen(reinterpret_cast<const In*>(s_ptr[j])[i]));
         res[i] = x;
     }
-    // a copy that was given up on may still be on its way into this block's shared memory: give it one more
-    // bounded wait before the block retires (the last use of stage st was rank j with j % BK_STAGES == st)
-    if (late_mask != 0) {
-        for (int st = 0; st < BK_STAGES; ++st) {
-            if (!((late_mask >> st) & 1u) || st >= m) continue;
-            const int last_j = st + ((m - 1 - st) / BK_STAGES) * BK_STAGES;
+    // Copies that were given up on, or issued ahead and never read, may still be on their way into this block's
+    // shared memory: thread 0 gives the last copy of every stage one more bounded wait before the block retires.
+    if (direct && tid == 0 && bytes != 0) {
+        for (int st = 0; st < BK_STAGES && st < issued; ++st) {
+            const int last_j = st + ((issued - 1 - st) / BK_STAGES) * BK_STAGES;
             bk_wait(bk_smem(&s_bar[st]), (uint32_t)(last_j / BK_STAGES) & 1u);
         }
     }

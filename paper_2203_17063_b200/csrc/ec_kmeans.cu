@@ -24,6 +24,7 @@
 //                         bounds of the tensor-core path rest on).
 // No floating-point atomics on any of these paths: sums are the same bits run after run.
 
+#include <mutex>
 #include <new>
 
 #include "ec_common.cuh"
@@ -668,7 +669,9 @@ int km_fused_launch(ec_kmeans* km, bool partials, const float* centroids, int32_
 
 template <int D>
 int km_tc_launch(ec_kmeans* km, bool partials, const float* centroids, int32_t* labels, cudaStream_t st, bool delta) {
-    const float tau_scale = 0.015625f;     // 2^-6: four times the bound 2^-8 (|x|^2 + |c|max^2) of one candidate's error
+    // 2^-6 + 2^-10: the bf16 search's two candidates are off by less than 2^-7 (|x|^2 + |c|^2) each (derivation at the
+    // kernel's use of tau); the 2^-10 on top covers the fp32 accumulation and the split of |c|^2
+    const float tau_scale = 0.015625f + 0.0009765625f;
     // the distance bounds describe the context's own labels against its own centroids: an iteration keeps them,
     // a stand-alone call on other arrays leaves them alone
     const bool own = centroids == km->centroids && labels == km->labels && km->bounds != nullptr && km->use_bounds;
@@ -1052,12 +1055,14 @@ struct StaticDeviceState {
     int sms;
 };
 StaticDeviceState g_static_state[MAX_DEVICES];   // host side, indexed by device ordinal; zero-initialised
+std::mutex g_static_mutex;                        // host threads making their first calls at the same time take turns
 
 // Once per device, with that device current.  In host code `g_static_scratch` is only a handle of
 // the symbol, not an address the GPU understands: the device address has to be asked for.
 int static_setup(int dev, StaticDeviceState** out) {
     if (dev < 0 || dev >= MAX_DEVICES) return EC_ERR_CAPACITY;
     StaticDeviceState* st = &g_static_state[dev];
+    std::lock_guard<std::mutex> guard(g_static_mutex);
     if (!st->ready) {
         void* addr = nullptr;
         EC_CUDA(cudaGetSymbolAddress(&addr, g_static_scratch));

@@ -493,6 +493,7 @@ tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const 
         }
         fence_async_smem();          // the tensor core reads shared memory through the async proxy
         healthy = __syncthreads_and(healthy) != 0;
+        const float xn = s_xn[tid];  // taken now: a warp that runs ahead stages the next tile's norms over this array
         if (tid == 0 && healthy) {
             fence_after_sync();
 #pragma unroll
@@ -532,8 +533,15 @@ tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const 
             atomicOr(status, 1u);    // the tensor core did not answer in time
         }
         fence_before_sync();         // accumulator reads are done before the next tile's MMA may overwrite it
-        // rounding to bf16 perturbs v by at most 2^-7 |x||c| <= 2^-8 (|x|^2 + |c|max^2) per candidate
-        const float tau = tau_scale * (s_xn[tid] + cmax);
+        // Error of the search.  bf16 keeps 8 significant bits: rounding to nearest changes a number by a factor
+        // (1 + e) with |e| <= u/(1+u), u = 2^-8, so a product of two rounded numbers is off by less than 2u of
+        // itself and the term -2 x.c_k by less than 4u sum_d |x_d c_kd| <= 4u |x||c_k| <= 2u (|x|^2 + |c_k|^2):
+        // one candidate's v is wrong by less than 2^-7 (|x|^2 + |c_k|^2), the difference of two candidates' v by less
+        // than 2^-6 (|x|^2 + |c|max^2).  The rest is far smaller: |c_k|^2 enters as hi + lo with 16 significant bits
+        // (2^-16 |c_k|^2) and the D + 2 products, exact in fp32, are added up in fp32 (at most (D+2) 2^-23 of the
+        // largest partial sum).  tau = (2^-6 + 2^-10)(|x|^2 + |c|max^2) covers the first part exactly and leaves
+        // 2^-10 (|x|^2 + |c|max^2), 64 times the rest for D = 32, for the second.
+        const float tau = tau_scale * (xn + cmax);
         const bool redo = live && (!done || !(m2 - m1 > tau));
         // Delta mode: the row block receives only what changed since the labels were written last: +x for the
         // cluster a point joins, -x for the one it leaves (old label < 0: it was in none).  A tile in which no
@@ -559,7 +567,6 @@ tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const 
             float2 w = make_float2(__int_as_float(0x7f800000), 0.0f);      // decided by the exact form: searched again next time
             if (done && !redo) {
                 // |x - c|^2 = |x|^2 + v; the search knows v to within tau
-                const float xn = s_xn[tid];
                 const float u = __fsqrt_ru(fmaxf(__fadd_ru(__fadd_ru(xn, m1), tau), 0.0f));
                 const float l = __fsqrt_rd(fmaxf(__fsub_rd(__fadd_rd(xn, m2), tau), 0.0f));
                 w = make_float2(__fsub_ru(u, s_drift[kb]), __fadd_rd(l, drift_max));

@@ -49,6 +49,30 @@ def sentinel(dtype_out, n):
     return np.full(n, np.nan, dtype=dtype_out)
 
 
+GUARD = 64          # guard elements on either side of an output (256 or 512 bytes: alignment is kept)
+GUARD_COUNT = 0x5EA1ED
+
+
+def guarded(values: np.ndarray, offset_elems: int = 0):
+    """Upload `values` with GUARD sentinel elements before and after it (compute-sanitizer's stand-in: a kernel that
+    writes outside its output is caught by check_guards).  Returns (whole allocation, view of the values)."""
+    t = torch.from_numpy(values)
+    lead = GUARD + offset_elems
+    big = torch.empty(lead + t.numel() + GUARD, dtype=t.dtype, device="cuda")
+    fill = GUARD_COUNT if not t.dtype.is_floating_point else float("inf")
+    big.fill_(fill)
+    view = big[lead:lead + t.numel()]
+    view.copy_(t)
+    return big, view
+
+
+def check_guards(big: torch.Tensor, view: torch.Tensor, what: str) -> None:
+    lead = view.storage_offset() - big.storage_offset()
+    fill = GUARD_COUNT if not big.dtype.is_floating_point else float("inf")
+    ok = bool((big[:lead] == fill).all()) and bool((big[lead + view.numel():] == fill).all())
+    assert ok, f"{what}: bytes outside the output were written"
+
+
 def run_schedule(P, n, seg, dtype, op, bufs, masks, order=ec.ORDER_FIXED, offset_elems=0, result_offset=0,
                  tile=None, poison=None, oracle_threads=4, compare=True, path=None):
     """Apply the cumulative masks one round after the other on GPU and CPU.
@@ -67,8 +91,8 @@ def run_schedule(P, n, seg, dtype, op, bufs, masks, order=ec.ORDER_FIXED, offset
     ref = oracle.Allreduce(P, n, dtype, op, seg)
     d_bufs = [to_dev(b, offset_elems) for b in bufs]
     res_np = sentinel(NP_OUT[dtype], n)
-    d_res = to_dev(res_np.copy(), result_offset)
-    d_cnt = torch.full((S,), 0xFFFFFFF, dtype=torch.int32, device="cuda")
+    res_all, d_res = guarded(res_np.copy(), result_offset)
+    cnt_all, d_cnt = guarded(np.full(S, 0xFFFFFFF, dtype=np.int32))
     c_res = res_np.copy()
     c_cnt = np.full(S, 0xFFFFFFF, dtype=np.uint32)
     out = []
@@ -87,6 +111,8 @@ def run_schedule(P, n, seg, dtype, op, bufs, masks, order=ec.ORDER_FIXED, offset
         d_mask = None if m is None else to_dev(np.ascontiguousarray(m, dtype=np.uint64))
         ar.apply(d_bufs, d_mask, d_res, d_cnt)
         torch.cuda.synchronize()
+        check_guards(res_all, d_res, f"round {t}: result")
+        check_guards(cnt_all, d_cnt, f"round {t}: contrib_count")
         ref.apply(bufs, m, c_res, c_cnt, order=order, threads=oracle_threads)
         g_res = to_host(d_res)
         g_cnt = d_cnt.cpu().numpy().view(np.uint32)

@@ -11,7 +11,7 @@ pytestmark = pytest.mark.gpu
 
 import oracle
 from paper_2203_17063_b200 import inputs
-from tests.gpu_util import ec, to_dev, to_host
+from tests.gpu_util import check_guards, ec, guarded, to_dev, to_host
 
 
 @pytest.fixture(autouse=True)
@@ -41,8 +41,9 @@ def lockstep(N, D, K, P, iters, seed, p_arrive=0.75):
     masks = inputs.kmeans_masks(seed + 1000, iters, P, K, p_arrive)
     d_points = to_dev(points)
     km = ec.KMeans(d_points, K, P, to_dev(cents))
-    d_labels = torch.empty(N, dtype=torch.int32, device="cuda")
-    d_part = torch.empty(P, K, D + 4, device="cuda")
+    lab_all, d_labels = guarded(np.zeros(N, dtype=np.int32))           # sentinels on either side of the outputs
+    part_all, d_part = guarded(np.zeros(P * K * (D + 4), dtype=np.float32))
+    d_part = d_part.view(P, K, D + 4)
     d_cent = torch.empty(K, D, device="cuda")
     d_red = torch.empty(K, D + 4, device="cuda")
     d_cnt = torch.empty(K, dtype=torch.int32, device="cuda")
@@ -51,10 +52,12 @@ def lockstep(N, D, K, P, iters, seed, p_arrive=0.75):
         km.set_centroids(to_dev(cents))
         km.assign(to_dev(cents), d_labels)
         g_labels = to_host(d_labels)
+        check_guards(lab_all, d_labels, "labels")
         c_labels, nmis = check_labels(g_labels, points, cents)
         # partials from the checker's labels: sums within tolerance, counts exact
         km.partials(to_dev(c_labels), d_part)
         g_part = to_host(d_part)
+        check_guards(part_all, d_part.view(-1), "partials")
         c_part = oracle.kmeans_partials(points, c_labels, K, P, 8)
         assert np.array_equal(g_part[:, :, D], c_part[:, :, D])
         assert (g_part[:, :, D + 1:] == 0).all()
