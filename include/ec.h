@@ -349,9 +349,15 @@ int ec_kmeans_set_bounds(ec_kmeans_t* km, int enable);
 /* Expert knob: which kernel ec_kmeans_iterate / ec_kmeans_assign use.
  *   0  automatic: the fastest one that covers the shape (default);
  *   1  fp32 fused kernel: candidate search by one FMA per (point, centroid, coordinate);
- *   2  tensor-core fused kernel: candidate search as a bf16 GEMM on tcgen05 (D in {16, 32, 64}, K <= 256).
- * Both decide every point whose two best candidates lie within the error bound of the search again
+ *   2  tensor cores (D in {16, 32}, K <= 256): for K <= 128 the warp-specialised kernel - the fp32 points go from
+ *      global to shared memory by bulk tensor copies and are multiplied as they lie (tcgen05, tf32) - otherwise
+ *      the kernel of 3;
+ *   3  tensor cores, register-staged form: points converted to bf16 by the threads, candidate search as a bf16 GEMM.
+ * All decide every point whose two best candidates lie within the error bound of the search again
  * by the exact form sum_d (x-c)^2 in fp32, so labels do not depend on the choice; speed does.
+ * ec_kmeans_tc_status reads a word that is nonzero if a bounded wait inside a tensor-core kernel ever gave up:
+ * bit 0 - the kernel of 3 finished that tile in plain fp32 (results valid); bit 1 - the warp-specialised kernel
+ * stopped early (the results of that call are not valid; the other bits say which wait it was).
  * EC_ERR_UNSUPPORTED if the shape is not covered by the requested kernel. */
 int ec_kmeans_set_path(ec_kmeans_t* km, int path);
 

@@ -220,30 +220,55 @@ partials_kernel(const float* __restrict__ points, const int32_t* __restrict__ la
     }
 }
 
-// partials[r][k][d] = scratch[r][0][k][d] + scratch[r][1][k][d] + ... in index order
-// (accumulate: the row blocks hold changes, which are added to what partials holds)
+// partials[r][k][d] = scratch[r][0][k][d] + scratch[r][1][k][d] + ... in index order, one warp per row (r, k).
+// accumulate: the row blocks hold changes, which are added to what partials holds; only the row blocks that hold
+// changes (dirty) were written.  The point counts stay exact integers under such updates, the coordinate sums
+// collect rounding: a row whose count comes back to zero is an empty cluster and its sums are set to zero exactly.
 __global__ void partials_fold_kernel(const float* __restrict__ scratch, int C, size_t row_elems, size_t total,
-                                     float* __restrict__ partials, int accumulate = 0,
+                                     float* __restrict__ partials, int stride, int accumulate = 0,
                                      const uint32_t* __restrict__ dirty = nullptr,
                                      const uint32_t* __restrict__ any_work = nullptr) {
     if (any_work != nullptr && *any_work == 0u) return;      // the bounds check found no tile to search: nothing was written
-    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
-        const size_t r = i / row_elems, e = i - r * row_elems;
-        const float* src = scratch + r * (size_t)C * row_elems + e;
-        if (accumulate) {                        // only the row blocks that hold changes (dirty) were written
-            float v = partials[i];
-            bool any = false;
-            for (int c = 0; c < C; ++c) {
-                if (dirty[r * (size_t)C + c]) {
-                    v = __fadd_rn(v, src[(size_t)c * row_elems]);
-                    any = true;
-                }
+    const int lane = threadIdx.x & 31;
+    const size_t rows = total / (size_t)stride;
+    const size_t per_rank = row_elems / (size_t)stride;      // K
+    constexpr int U = 8;                                      // loads in flight per lane
+    for (size_t row = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5; row < rows; row += ((size_t)gridDim.x * blockDim.x) >> 5) {
+        const size_t r = row / per_rank;
+        const float* src = scratch + r * (size_t)C * row_elems + (row - r * per_rank) * (size_t)stride;
+        float* dst = partials + row * (size_t)stride;
+        if (accumulate) {
+            // which row blocks of this rank hold changes: 32 flags per ballot (C is at most 64)
+            unsigned long long mask = 0;
+            for (int c0 = 0; c0 < C; c0 += 32) {
+                const int c = c0 + lane;
+                const unsigned m = __ballot_sync(0xffffffffu, c < C && dirty[r * (size_t)C + c] != 0u);
+                mask |= (unsigned long long)m << c0;
             }
-            if (any) partials[i] = v;
+            if (mask == 0) continue;
+            const int D = stride - 4;
+            float cnt = dst[D];                               // every lane folds the count: it decides what the others write
+            for (unsigned long long m = mask; m; m &= m - 1) cnt = __fadd_rn(cnt, src[(size_t)(__ffsll((long long)m) - 1) * row_elems + D]);
+            __syncwarp();                                     // all lanes have read the old count before lane D % 32 replaces it
+            for (int e = lane; e < stride; e += 32) {
+                float v = dst[e];
+                for (unsigned long long m = mask; m; m &= m - 1) v = __fadd_rn(v, src[(size_t)(__ffsll((long long)m) - 1) * row_elems + e]);
+                dst[e] = (cnt == 0.0f && e < D) ? 0.0f : v;
+            }
         } else {
-            float v = src[0];
-            for (int c = 1; c < C; ++c) v = __fadd_rn(v, src[(size_t)c * row_elems]);
-            partials[i] = v;
+            for (int e = lane; e < stride; e += 32) {
+                float v = src[e];
+                int c = 1;
+                for (; c + U <= C; c += U) {                  // the loads of U row blocks together, the additions in index order
+                    float t[U];
+#pragma unroll
+                    for (int u = 0; u < U; ++u) t[u] = src[(size_t)(c + u) * row_elems + e];
+#pragma unroll
+                    for (int u = 0; u < U; ++u) v = __fadd_rn(v, t[u]);
+                }
+                for (; c < C; ++c) v = __fadd_rn(v, src[(size_t)c * row_elems + e]);
+                dst[e] = v;
+            }
         }
     }
 }
@@ -519,6 +544,7 @@ fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const flo
 }  // namespace ec
 
 #include "ec_kmeans_tc.cuh"
+#include "ec_kmeans_ws.cuh"
 
 namespace ec {
 namespace {
@@ -554,7 +580,10 @@ struct ec_kmeans {
     int Cf;                // runs per rank of the fused kernel; 0 = shape not covered by it
     size_t fused_smem, fused_assign_smem;
     bool tc_ok;            // the tensor-core candidate search covers this shape
-    int path;              // 0 = automatic, 1 = fp32 fused kernel, 2 = tensor-core fused kernel
+    bool ws_ok;            // ... and so does its warp-specialised form (K <= 128, tensor map of the points made)
+    CUtensorMap pmap;      // the points as a 2-D tensor [N][D] of fp32, tiles of 128 rows, swizzled rows
+    ec::ws::Plan ws_plan, ws_plan_assign;
+    int path;              // 0 = automatic, 1 = fp32 fused kernel, 2 = tensor cores, 3 = tensor cores, register-staged form
     size_t tc_smem, tc_assign_smem;
     int tc_wave_full, tc_wave_delta, tc_wave_assign;   // resident blocks of the tensor-core kernels on the whole device
     uint32_t* tc_status;   // device word: nonzero if a wait on the tensor core ever gave up
@@ -742,7 +771,103 @@ cudaError_t km_tc_attr(ec_kmeans* km) {
     return e;
 }
 
+// Shapes the warp-specialised tensor-core kernel covers: a row of D floats is one 64- or 128-byte swizzle span, the
+// accumulators of at least two epilogue groups and of two runs fit in tensor memory, row indices fit the copy's int32.
+bool ws_capable(size_t N, int D, int K) {
+    if (D != 16 && D != 32) return false;
+    if (tc::npad_of(K) > 128) return false;
+    if (N >= 0x7fffff00ull) return false;
+    return ws::plan_of(D, K, true).total <= 227 * 1024 && ws::plan_of(D, K, true).stages >= 3;
+}
+
+// The tensor map of the points (driver entry point taken through the runtime: the library links no libcuda).
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+bool km_make_point_map(ec_kmeans* km) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres = cudaDriverEntryPointSymbolNotFound;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || fn == nullptr ||
+        qres != cudaDriverEntryPointSuccess) {
+        cudaGetLastError();
+        return false;
+    }
+    const cuuint64_t dims[2] = {(cuuint64_t)km->D, (cuuint64_t)km->N};
+    const cuuint64_t strides[1] = {(cuuint64_t)km->D * 4};
+    const cuuint32_t box[2] = {(cuuint32_t)km->D, (cuuint32_t)ws::TILE};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = reinterpret_cast<EncodeTiledFn>(fn)(
+        &km->pmap, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(km->points), dims, strides, box, estr,
+        CU_TENSOR_MAP_INTERLEAVE_NONE, km->D == 32 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
+        CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+template <int D>
+cudaError_t km_ws_attr(ec_kmeans* km) {
+    const int full = (int)km->ws_plan.total, asg = (int)km->ws_plan_assign.total;
+    cudaError_t e = cudaFuncSetAttribute(ws::ws_fused_kernel<D, true, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(ws::ws_fused_kernel<D, true, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(ws::ws_fused_kernel<D, true, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(ws::ws_fused_kernel<D, true, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(ws::ws_fused_kernel<D, false, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    (void)full; (void)asg;
+    return e;
+}
+
+template <int D>
+int km_ws_launch(ec_kmeans* km, bool partials, const float* centroids, int32_t* labels, cudaStream_t st, bool delta) {
+    const bool own = centroids == km->centroids && labels == km->labels && km->bounds != nullptr && km->use_bounds;
+    const bool skip = partials && delta && own && km->bounds_valid && km->use_bounds;
+    if (skip) {      // which tiles can still change a label: one byte per 32 points
+        tc::bounds_check_kernel<<<(unsigned)(km->P * km->Cf), tc::BC_THREADS, 0, st>>>(
+            km->N, km->P, km->Cf, km->K, labels, km->bounds, km->drift, km->need, km->need_words, km->dirty,
+            reinterpret_cast<uint32_t*>(km->drift) + km->K + 1);
+        EC_CUDA(cudaGetLastError());
+    }
+    if (partials) {
+        const int runs = km->P * km->Cf;
+        const unsigned grid = (unsigned)(runs < km->sms ? runs : km->sms);
+        const unsigned thr = (unsigned)ws::threads_of(km->ws_plan);
+        const size_t smem = km->ws_plan.total;
+        float* full_out = km->Cf == 1 ? km->partials : km->scratch;
+        if (delta && own)
+            ws::ws_fused_kernel<D, true, true, true><<<grid, thr, smem, st>>>(
+                km->pmap, km->points, km->N, km->P, km->Cf, centroids, km->K, labels, km->scratch, km->tc_status, km->dirty,
+                km->bounds, km->drift, skip ? km->need : nullptr, km->need_words);
+        else if (delta)
+            ws::ws_fused_kernel<D, true, true, false><<<grid, thr, smem, st>>>(
+                km->pmap, km->points, km->N, km->P, km->Cf, centroids, km->K, labels, km->scratch, km->tc_status, km->dirty,
+                nullptr, nullptr, nullptr, 0);
+        else if (own)
+            ws::ws_fused_kernel<D, true, false, true><<<grid, thr, smem, st>>>(
+                km->pmap, km->points, km->N, km->P, km->Cf, centroids, km->K, labels, full_out, km->tc_status, km->dirty,
+                km->bounds, km->drift, nullptr, 0);
+        else
+            ws::ws_fused_kernel<D, true, false, false><<<grid, thr, smem, st>>>(
+                km->pmap, km->points, km->N, km->P, km->Cf, centroids, km->K, labels, full_out, km->tc_status, km->dirty,
+                nullptr, nullptr, nullptr, 0);
+    } else {
+        size_t runs = (km->N + 2047) / 2048;
+        if (runs > 0x7fffffffull) return EC_ERR_CAPACITY;
+        const unsigned grid = (unsigned)(runs < (size_t)km->sms ? runs : (size_t)km->sms);
+        ws::ws_fused_kernel<D, false, false, false><<<grid, (unsigned)ws::threads_of(km->ws_plan_assign), km->ws_plan_assign.total, st>>>(
+            km->pmap, km->points, km->N, 1, (int)runs, centroids, km->K, labels, nullptr, km->tc_status, nullptr,
+            nullptr, nullptr, nullptr, 0);
+    }
+    EC_CUDA(cudaGetLastError());
+    km->skipped = skip;
+    if (partials && own) km->bounds_valid = true;       // every tile searched in this launch has fresh bounds, the others kept valid ones
+    return EC_OK;
+}
+
 int km_fused(ec_kmeans* km, bool partials, const float* centroids, int32_t* labels, cudaStream_t st, bool delta = false) {
+    if (km->ws_ok && km->path != 1 && km->path != 3) {
+        switch (km->D) {
+            case 16: return km_ws_launch<16>(km, partials, centroids, labels, st, delta);
+            case 32: return km_ws_launch<32>(km, partials, centroids, labels, st, delta);
+        }
+    }
     if (km->tc_ok && km->path != 1) {
         switch (km->D) {
             case 16: return km_tc_launch<16>(km, partials, centroids, labels, st, delta);
@@ -797,8 +922,8 @@ int km_partials(ec_kmeans* km, const int32_t* labels, float* partials, cudaStrea
     EC_CUDA(cudaGetLastError());
     if (km->C > 1) {
         const size_t row = (size_t)km->K * (km->D + 4), total = row * km->P;
-        const unsigned grid = (unsigned)((total + 255) / 256);
-        partials_fold_kernel<<<grid, 256, 0, st>>>(km->scratch, km->C, row, total, partials);
+        const unsigned grid = (unsigned)((total / (km->D + 4) * 32 + 255) / 256);   // one warp per row
+        partials_fold_kernel<<<grid, 256, 0, st>>>(km->scratch, km->C, row, total, partials, km->D + 4);
         EC_CUDA(cudaGetLastError());
     }
     return EC_OK;
@@ -889,6 +1014,12 @@ int ec_kmeans_init(ec_kmeans_t** out, const float* points, size_t N, int D, int 
         e = D == 8 ? km_fused_attr<8>() : D == 16 ? km_fused_attr<16>() : D == 32 ? km_fused_attr<32>() : km_fused_attr<64>();
     if (e == cudaSuccess && km->tc_ok)
         e = D == 16 ? km_tc_attr<16>(km) : km_tc_attr<32>(km);
+    km->ws_ok = km->tc_ok && ws_capable(N, D, K) && km_make_point_map(km);
+    if (km->ws_ok) {
+        km->ws_plan = ws::plan_of(D, K, true);
+        km->ws_plan_assign = ws::plan_of(D, K, false);
+        if (e == cudaSuccess) e = D == 16 ? km_ws_attr<16>(km) : km_ws_attr<32>(km);
+    }
     if (e == cudaSuccess) e = cudaMemsetAsync(km->tc_status, 0, 4, 0);
     if (e == cudaSuccess) e = cudaMemsetAsync(km->drift, 0, ((size_t)K + 2) * 4, 0);
     if (e == cudaSuccess) e = cudaMemcpyAsync(km->centroids, init_centroids, (size_t)K * D * 4, cudaMemcpyDeviceToDevice, 0);
@@ -945,8 +1076,8 @@ int km_iterate_rounds(ec_kmeans_t* km, const uint64_t* const* masks, int rounds,
         if (rc != EC_OK) return rc;
         if (km->Cf > 1 || delta) {
             const size_t row = (size_t)km->K * (km->D + 4), total = row * km->P;
-            partials_fold_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(km->scratch, km->Cf, row, total,
-                                                                                      km->partials, delta ? 1 : 0, km->dirty,
+            partials_fold_kernel<<<(unsigned)(((size_t)km->P * km->K * 32 + 255) / 256), 256, 0, stream>>>(km->scratch, km->Cf, row, total,
+                                                                                      km->partials, km->D + 4, delta ? 1 : 0, km->dirty,
                                                                                       delta && km->skipped ? reinterpret_cast<const uint32_t*>(km->drift) + km->K + 1 : nullptr);
             EC_CUDA(cudaGetLastError());
         }
@@ -1009,8 +1140,8 @@ int ec_kmeans_set_bounds(ec_kmeans_t* km, int enable) {
 }
 
 int ec_kmeans_set_path(ec_kmeans_t* km, int path) {
-    if (!km || path < 0 || path > 2) return EC_ERR_INVALID;
-    if (path == 2 && !km->tc_ok) return EC_ERR_UNSUPPORTED;
+    if (!km || path < 0 || path > 3) return EC_ERR_INVALID;
+    if ((path == 2 || path == 3) && !km->tc_ok) return EC_ERR_UNSUPPORTED;
     if (path == 1 && km->Cf == 0) return EC_ERR_UNSUPPORTED;
     km->path = path;
     km->state_valid = false;        // the next iteration sums everything afresh
@@ -1099,7 +1230,7 @@ extern "C" int ec_kmeans_partials_static(const float* points, const int32_t* lab
     EC_CUDA(cudaGetLastError());
     if (L.C > 1) {
         const size_t total = row * P;
-        partials_fold_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(st->scratch, L.C, row, total, partials);
+        partials_fold_kernel<<<(unsigned)(((size_t)P * K * 32 + 255) / 256), 256, 0, stream>>>(st->scratch, L.C, row, total, partials, D + 4);
         EC_CUDA(cudaGetLastError());
     }
     return EC_OK;

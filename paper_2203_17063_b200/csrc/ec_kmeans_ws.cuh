@@ -1,0 +1,822 @@
+// K-means assignment + partial sums, warp-specialised: the form ec_kmeans_iterate takes for D in {16, 32}, K <= 128.
+//
+// One persistent block per SM.  The fp32 points never pass through registers on their way to the tensor core:
+//
+//   producer (one thread)    walks the block's runs and, for every tile of 128 points that has to be searched,
+//                            issues one bulk tensor copy (cp.async.bulk.tensor.2d, 128-byte swizzle, no multicast,
+//                            this GPU's memory only) into a ring of shared-memory stages, each with its mbarrier;
+//   search issuer (one thread) multiplies a landed tile, as it lies, with the centroid operand: tcgen05.mma kind::tf32,
+//                            A = the stage (128 points x D floats, K-major), B = -2 c rounded to tf32 (K-major, same
+//                            swizzle), plus one step of a constant [1,1,1,0..] chunk against [hi, mid, lo](|c|^2), so
+//                            the accumulator in tensor memory holds v_k = |c_k|^2 - 2 x.c_k for 128 points x all
+//                            centroids.  One accumulator per epilogue group, so tiles overlap;
+//   epilogue groups (4 warps each, tile i goes to group i mod G): read the scores with tcgen05.ld (one point per
+//                            thread), find the best two by a tournament of min/max pairs whose low mantissa bits carry
+//                            the column index, decide (exact fp32 form from the staged row whenever the two are closer
+//                            than the search's error bound tau), write label and distance bounds, and - only for a tile in
+//                            which a label changed - convert the staged rows to bf16 high + low parts and set the
+//                            one-hot rows for the sums GEMM;
+//   sums issuer (one thread)  sums[d][k] += sum_j x[j][d] onehot[j][k] as tcgen05.mma kind::f16 over such tiles, in
+//                            tile order (so the sums repeat bit for bit), accumulator in tensor memory per run, double
+//                            buffered so that a run is written out while the next one accumulates.
+//
+// Every wait (mbarrier) is bounded; a wait that gives up raises an abort flag that every role polls, the block sets a
+// status word, waits (bounded) for its copies in flight, frees its tensor memory and returns.  The results of a launch
+// whose status word is nonzero are not valid.
+//
+// Error of the search (kind::tf32).  The tensor core keeps 11 significant bits of an fp32 operand; whether it rounds
+// or truncates, a point's coordinate is changed by a factor (1 + e), |e| <= 2^-10.  The centroids are rounded to
+// nearest here, |e| <= 2^-11.  A product is off by less than 1.5001 * 2^-10 of itself, the term -2 x.c_k by less
+// than 3.0002 * 2^-10 |x||c_k| <= 1.5001 * 2^-10 (|x|^2 + |c_k|^2); |c_k|^2 enters exactly (three tf32 terms), the
+// products are exact in fp32 and the few additions cost at most (D/8 + 2) 2^-23 of the largest partial sum.  Tagging a
+// score with its column (7 low mantissa bits) moves it by less than 2^-16 |v| <= 2^-15 (|x|^2 + |c|^2).  The
+// difference of two candidates' scores is therefore known to within 3.0002 * 2^-10 + 2^-14 + ... < 3.1 * 2^-10 of
+// (|x|^2 + |c|max^2); tau = 2^-8 = 4 * 2^-10 of it.  One score alone is within tau / 2.
+#pragma once
+
+#include <cuda.h>
+#ifdef EC_WS_DEBUG
+#include <cstdio>
+#endif
+
+#ifndef EC_WS_HINT
+#define EC_WS_HINT 20000
+#endif
+
+namespace ec {
+namespace ws {
+
+using tc::fence_after_sync;
+using tc::fence_async_smem;
+using tc::fence_before_sync;
+using tc::mbar_init;
+using tc::mma_commit;
+using tc::npad_of;
+using tc::pack_bf16;
+using tc::smem_desc;
+using tc::smem_u32;
+using tc::tmem_alloc;
+using tc::tmem_dealloc;
+
+constexpr int TILE = 128;                       // points per tile = rows of an accumulator
+constexpr int MAX_GROUPS = 4;                   // epilogue groups of four warps
+constexpr int MAX_STAGES = 8;
+constexpr int SLOTS = 2;                        // operand buffers of the sums GEMM
+constexpr int MAX_THREADS = (4 * MAX_GROUPS + 3) * 32;
+constexpr uint32_t WAIT_LIMIT = 1u << 24;
+constexpr uint32_t OCHUNK = TILE * 16;          // one-hot tile: bytes between chunks of 8 centroids
+constexpr float TAU_SCALE = 0.00390625f;        // 2^-8, see above
+// bf16 operand of the sums GEMM: bytes between chunk columns (8 coordinates x 128 points x 2 bytes, padded so that
+// consecutive columns start in different banks)
+__host__ __device__ constexpr uint32_t xchunk_of(int D) { return TILE * 16 + 1024u / (uint32_t)D; }
+
+// Shared memory of a block (byte offsets from a 1024-byte aligned base) and its tensor-memory columns.
+struct Plan {
+    int groups, stages;
+    uint32_t tmem_cols;
+    uint32_t stage_bytes, slot_bytes, oh_off;       // oh_off: one-hot tile inside a slot
+    uint32_t stage, b, ones, cnb, slot, prev, cn, drift, need, desc, ctrl, bar, total;
+};
+__host__ __device__ inline Plan plan_of(int D, int K, bool partials) {
+    Plan p;
+    const uint32_t npad = (uint32_t)npad_of(K), XC = xchunk_of(D);
+    const uint32_t acc = partials ? 2u : 0u;
+    int g = (int)(512u / npad) - (int)acc;
+    p.groups = g > MAX_GROUPS ? MAX_GROUPS : g < 1 ? 1 : g;
+    uint32_t need = ((uint32_t)p.groups + acc) * npad, cols = 32;
+    while (cols < need) cols <<= 1;
+    p.tmem_cols = cols;
+    p.stage_bytes = (uint32_t)TILE * (uint32_t)D * 4u;
+    const uint32_t kch = (uint32_t)D / 8u;
+    p.oh_off = ((2u * kch + 1u) * XC + 127u) & ~127u;   // high/low columns interleaved, then the ones column
+    uint32_t slot = p.oh_off + npad / 8u * OCHUNK;
+    if (slot < 16u * XC) slot = 16u * XC;            // the sums MMA reads 128 rows = 16 chunk columns from the slot's start
+    p.slot_bytes = (slot + 127u) & ~127u;
+    uint32_t off = 0;
+    const uint32_t fixed_after_stages = npad * (uint32_t)D * 4u + 1024u   // b (1024-aligned)
+        + 4096u + npad * 32u                                              // ones, cnb
+        + (partials ? SLOTS * p.slot_bytes + SLOTS * TILE * 2u : 0u)      // slots, previous one-hot chunks
+        + npad * 8u + 1024u + 4096u;                                       // cn, drift, need words, descriptors, control, barriers
+    int st = (int)((226u * 1024u - fixed_after_stages) / p.stage_bytes);
+    p.stages = st > MAX_STAGES ? MAX_STAGES : st;
+    p.stage = off; off += (uint32_t)p.stages * p.stage_bytes;
+    off = (off + 1023u) & ~1023u;
+    p.b = off; off += npad * (uint32_t)D * 4u;       // -2 c, tf32, K-major, swizzled like the stages
+    p.ones = off; off += 4096u;                      // [2 chunks][128 rows][16 bytes]: (1,1,1,0 | 0,0,0,0), no swizzle
+    p.cnb = off; off += npad * 32u;                  // [2 chunks][npad rows][16 bytes]: (hi, mid, lo, 0 | 0...) of |c|^2
+    off = (off + 127u) & ~127u;
+    p.slot = off; off += partials ? SLOTS * p.slot_bytes : 0u;
+    p.prev = off; off += partials ? SLOTS * TILE * 2u : 0u;
+    p.cn = off; off += npad * 4u;
+    p.drift = off; off += npad * 4u;
+    p.need = off; off += 1024u;
+    p.desc = off; off += MAX_STAGES * 32u;
+    p.ctrl = off; off += 256u;
+    p.bar = off; off += 512u;
+    p.total = off + 1024u;                           // slack to align the base
+    return p;
+}
+inline int threads_of(const Plan& p) { return (4 * p.groups + 3) * 32; }
+
+// What the producer says about the tile in a stage.
+struct TileDesc {
+    unsigned long long base;     // index of the tile's first point
+    unsigned long long end;      // one past the run's last point
+    int run;                     // run index (row block), -1: no more tiles
+    int run_seq;                 // how many runs with tiles this block has started before this tile's run
+    int last;                    // the run's last tile
+    int pad;
+};
+
+// One try; the thread may sleep in hardware until the phase completes or the hinted time (nanoseconds) has passed, so
+// a waiting warp costs few issue slots.
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n"
+        "selp.u32 %0, 1, 0, p;\n"
+        "}\n"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity), "r"((uint32_t)EC_WS_HINT)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void tma_tile_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+// Bounded wait (in tries and in time: about two seconds); gives up early when another role has raised the abort flag.
+__device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, volatile int* abort_flag, int where) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 63u) == 63u) {
+            if (*abort_flag != 0) return false;
+            if (clock64() - t0 > 4000000000LL) break;
+        }
+    }
+    if (*abort_flag == 0) *abort_flag = where;               // which wait gave up first (reported in the status word)
+    return false;
+}
+__device__ __forceinline__ void mma_tf32(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "setp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n"
+        "}\n" ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// K-major operand whose rows are one swizzle span wide (128 bytes for D = 32, 64 bytes for D = 16): groups of 8 rows
+// are 8 spans apart.
+template <int D>
+__device__ __forceinline__ uint64_t swz_desc(uint32_t saddr) {
+    constexpr uint32_t span = D * 4;
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)1 << 16;                                   // leading byte offset: not used by swizzled K-major operands
+    d |= (uint64_t)((8u * span) >> 4) << 32;                  // stride between groups of 8 rows
+    d |= 1ull << 46;
+    d |= (uint64_t)(span == 128 ? 2 : 4) << 61;               // 128-byte / 64-byte swizzle
+    return d;
+}
+__host__ __device__ inline uint32_t idesc_tf32(int M, int N) {
+    return (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+// byte offset of logical 16-byte chunk q of row r inside a swizzled tile
+template <int D>
+__device__ __forceinline__ uint32_t swz_off(int r, int q) {
+    if (D == 32) return (uint32_t)r * 128u + (uint32_t)((q ^ (r & 7)) << 4);
+    return (uint32_t)r * 64u + (uint32_t)((q ^ ((r >> 1) & 3)) << 4);
+}
+__device__ __forceinline__ float min3(float a, float b, float c) {
+    float d;
+    asm("min.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+__device__ __forceinline__ void tmem_ld32_nowait(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Best two of 32 scores whose low 7 mantissa bits have been replaced by their column index: sorted pairs, then the
+// same again on the smaller halves; the second best is the smallest of all the larger halves (the partner of the
+// winner is among them, and every other larger half is at least the second best of the smaller ones).
+__device__ __forceinline__ void best_two_of_32(const uint32_t (&raw)[32], float& c1, float& c2) {
+    float lo[16], hi_min;
+    {
+        float hi[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const float a = __uint_as_float((raw[2 * i] & 0xFFFFFF80u) | (uint32_t)(2 * i));
+            const float b = __uint_as_float((raw[2 * i + 1] & 0xFFFFFF80u) | (uint32_t)(2 * i + 1));
+            lo[i] = fminf(a, b);
+            hi[i] = fmaxf(a, b);
+        }
+        float t[6];
+#pragma unroll
+        for (int i = 0; i < 5; ++i) t[i] = min3(hi[3 * i], hi[3 * i + 1], hi[3 * i + 2]);
+        hi_min = min3(min3(t[0], t[1], t[2]), min3(t[3], t[4], hi[15]), t[0]);
+    }
+    float l8[8];
+    {
+        float h8[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            l8[i] = fminf(lo[2 * i], lo[2 * i + 1]);
+            h8[i] = fmaxf(lo[2 * i], lo[2 * i + 1]);
+        }
+        hi_min = min3(hi_min, min3(h8[0], h8[1], h8[2]), min3(h8[3], h8[4], h8[5]));
+        hi_min = min3(hi_min, h8[6], h8[7]);
+    }
+    float l4[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        l4[i] = fminf(l8[2 * i], l8[2 * i + 1]);
+        hi_min = fminf(hi_min, fmaxf(l8[2 * i], l8[2 * i + 1]));
+    }
+    const float a = fminf(l4[0], l4[1]), b = fminf(l4[2], l4[3]);
+    hi_min = min3(hi_min, fmaxf(l4[0], l4[1]), fmaxf(l4[2], l4[3]));
+    c1 = fminf(a, b);
+    c2 = fminf(hi_min, fmaxf(a, b));
+}
+
+__device__ __forceinline__ void tmem_ld16_nowait(uint32_t taddr, uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr)
+        : "memory");
+}
+// The same for 16 scores (tags 0..15), so that the next 16 can be on their way from tensor memory meanwhile.
+__device__ __forceinline__ void best_two_of_16(const uint32_t (&raw)[16], float& c1, float& c2) {
+    float lo[8], hi[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const float a = __uint_as_float((raw[2 * i] & 0xFFFFFF80u) | (uint32_t)(2 * i));
+        const float b = __uint_as_float((raw[2 * i + 1] & 0xFFFFFF80u) | (uint32_t)(2 * i + 1));
+        lo[i] = fminf(a, b);
+        hi[i] = fmaxf(a, b);
+    }
+    float hi_min = min3(min3(hi[0], hi[1], hi[2]), min3(hi[3], hi[4], hi[5]), fminf(hi[6], hi[7]));
+    float l4[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) l4[i] = fminf(lo[2 * i], lo[2 * i + 1]);
+    hi_min = min3(hi_min, fmaxf(lo[0], lo[1]), fmaxf(lo[2], lo[3]));
+    hi_min = min3(hi_min, fmaxf(lo[4], lo[5]), fmaxf(lo[6], lo[7]));
+    const float a = fminf(l4[0], l4[1]), b = fminf(l4[2], l4[3]);
+    hi_min = min3(hi_min, fmaxf(l4[0], l4[1]), fmaxf(l4[2], l4[3]));
+    c1 = fminf(a, b);
+    c2 = fminf(hi_min, fmaxf(a, b));
+}
+
+template <int D, bool PARTIALS, bool DELTA, bool BOUNDS>
+__global__ void __launch_bounds__(MAX_THREADS, 1)
+ws_fused_kernel(const __grid_constant__ CUtensorMap pmap, const float* __restrict__ points, size_t N, int P, int C,
+                const float* __restrict__ centroids, int K, int32_t* __restrict__ labels, float* __restrict__ scratch,
+                uint32_t* __restrict__ status, uint32_t* __restrict__ dirty, float2* __restrict__ bounds,
+                const float* __restrict__ drift, const uint32_t* __restrict__ need, int need_words) {
+    constexpr int KCH = D / 8;                              // 16-byte bf16 chunks (8 coordinates) per point
+    constexpr int Q = D / 4;                                // 16-byte fp32 chunks per point
+    constexpr uint32_t XC = xchunk_of(D);
+    static_assert(D == 16 || D == 32, "a row is one 64- or 128-byte swizzle span");
+    extern __shared__ unsigned char ws_smem_raw[];
+    const Plan pl = plan_of(D, K, PARTIALS);
+    const int npad = npad_of(K);
+    const int G = pl.groups, NST = pl.stages;
+    unsigned char* sm = ws_smem_raw + ((1024u - (smem_u32(ws_smem_raw) & 1023u)) & 1023u);
+    const uint32_t sm_u = smem_u32(sm);
+    float* s_cn = reinterpret_cast<float*>(sm + pl.cn);
+    float* s_drift = reinterpret_cast<float*>(sm + pl.drift);
+    uint32_t* s_need = reinterpret_cast<uint32_t*>(sm + pl.need);
+    TileDesc* s_desc = reinterpret_cast<TileDesc*>(sm + pl.desc);
+    // control words: [0..3] what a group says about its tile (CTRL_*), [4..5] run had sums, [6] tensor-memory address,
+    // [7] abort, [8 + 3 g + n % 3] "a label changed" votes of group g's n-th tile, [25] runs whose end the sums issuer has
+    // signalled, [26] tiles it is through with, [28..29] sums GEMMs issued from each slot, [32 + 4 slot + w] rows of warp w
+    // of the slot's last user have one-hot entries set
+    volatile int* s_ctrl = reinterpret_cast<volatile int*>(sm + pl.ctrl);
+    volatile int* s_abort = s_ctrl + 7;
+    volatile int* s_vote = s_ctrl + 8;
+    constexpr int CTRL_SUMS = 1, CTRL_LAST = 2, CTRL_PAR = 4, CTRL_END = 8;
+    // barriers (8 bytes each)
+    const uint32_t bar0 = sm_u + pl.bar;
+    auto B_full = [&](int s) { return bar0 + 8u * (uint32_t)s; };
+    auto B_empty = [&](int s) { return bar0 + 8u * (uint32_t)(MAX_STAGES + s); };
+    auto B_accfull = [&](int g) { return bar0 + 8u * (uint32_t)(2 * MAX_STAGES + g); };
+    auto B_accempty = [&](int g) { return bar0 + 8u * (uint32_t)(2 * MAX_STAGES + MAX_GROUPS + g); };
+    auto B_decided = [&](int g) { return bar0 + 8u * (uint32_t)(2 * MAX_STAGES + 2 * MAX_GROUPS + g); };
+    auto B_tiledone = [&](int g) { return bar0 + 8u * (uint32_t)(2 * MAX_STAGES + 3 * MAX_GROUPS + g); };
+    auto B_rundone = [&](int p) { return bar0 + 8u * (uint32_t)(2 * MAX_STAGES + 4 * MAX_GROUPS + p); };
+    auto B_drained = [&](int p) { return bar0 + 8u * (uint32_t)(2 * MAX_STAGES + 4 * MAX_GROUPS + 2 + p); };
+    auto B_vote = [&](int g) { return bar0 + 8u * (uint32_t)(2 * MAX_STAGES + 4 * MAX_GROUPS + 4 + g); };
+    auto B_slotfree = [&](int sl) { return bar0 + 8u * (uint32_t)(2 * MAX_STAGES + 5 * MAX_GROUPS + 4 + sl); };
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int nthreads = (4 * G + 3) * 32;
+    if (tid >= nthreads) return;                             // (the launch uses exactly nthreads; kept for safety)
+    const int runs = P * C;
+    const bool skipping = DELTA && PARTIALS && BOUNDS && need != nullptr;
+    if (skipping) {
+        if (reinterpret_cast<const uint32_t*>(drift)[K + 1] == 0u) return;   // no tile anywhere: the check has settled every run
+        bool any = false;
+        for (int run = blockIdx.x; run < runs; run += gridDim.x)
+            for (int q = tid; q < need_words; q += nthreads) any = any || need[(size_t)run * need_words + q] != 0u;
+        if (!__syncthreads_or(any ? 1 : 0)) {
+            for (int run = blockIdx.x + tid * gridDim.x; run < runs; run += nthreads * gridDim.x) dirty[run] = 0u;
+            return;
+        }
+    }
+    // ---- set-up, all threads ------------------------------------------------------------------------------------
+    if (warp == 4 * G + 1) tmem_alloc(smem_u32(const_cast<int*>(s_ctrl + 6)), pl.tmem_cols);
+    if (tid == 0) {
+        for (int s = 0; s < NST; ++s) { mbar_init(B_full(s), 1); mbar_init(B_empty(s), 4); }
+        for (int g = 0; g < G; ++g) {
+            mbar_init(B_accfull(g), 1); mbar_init(B_accempty(g), 4); mbar_init(B_decided(g), 4); mbar_init(B_vote(g), 4);
+        }
+        for (int q = 0; q < 3 * MAX_GROUPS; ++q) s_vote[q] = 0;
+        for (int g = 0; g < G; ++g) mbar_init(B_tiledone(g), 1);
+        for (int sl = 0; sl < SLOTS; ++sl) mbar_init(B_slotfree(sl), 1);
+        s_ctrl[0] = 0; s_ctrl[1] = 0; s_ctrl[2] = 0; s_ctrl[3] = 0;
+        s_ctrl[25] = 0; s_ctrl[26] = 0; s_ctrl[28] = 0; s_ctrl[29] = 0;
+        for (int q = 32; q < 40; ++q) s_ctrl[q] = 0;
+        for (int p = 0; p < 2; ++p) { mbar_init(B_rundone(p), 1); mbar_init(B_drained(p), 4); }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        *s_abort = 0;
+    }
+    for (int k = tid; k < npad; k += nthreads) {
+        float s = 3.0e38f;
+        if (k < K) {
+            s = 0.0f;
+            for (int d = 0; d < D; ++d) s = fmaf(centroids[(size_t)k * D + d], centroids[(size_t)k * D + d], s);
+        }
+        s_cn[k] = s;
+        // |c|^2 as three numbers of 11 significant bits each: exact, and exact in tf32 whether it rounds or truncates
+        const float hi = __uint_as_float(__float_as_uint(s) & 0xFFFFE000u);
+        const float r1 = s - hi;
+        const float mid = __uint_as_float(__float_as_uint(r1) & 0xFFFFE000u);
+        const float lo = r1 - mid;
+        *reinterpret_cast<float4*>(sm + pl.cnb + (size_t)k * 16) = make_float4(hi, mid, lo, 0.0f);
+        *reinterpret_cast<float4*>(sm + pl.cnb + (size_t)npad * 16 + (size_t)k * 16) = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+        if (PARTIALS && BOUNDS) s_drift[k] = k < K ? drift[k] : 0.0f;
+    }
+    for (int i = tid; i < npad * Q; i += nthreads) {          // -2 c rounded to 11 significant bits (nearest, ties away)
+        const int n = i / Q, q = i - n * Q;
+        float v[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const float c = n < K ? -2.0f * centroids[(size_t)n * D + q * 4 + e] : 0.0f;
+            v[e] = __uint_as_float((__float_as_uint(c) + 0x1000u) & 0xFFFFE000u);
+        }
+        *reinterpret_cast<float4*>(sm + pl.b + swz_off<D>(n, q)) = make_float4(v[0], v[1], v[2], v[3]);
+    }
+    for (int r = tid; r < TILE; r += nthreads) {
+        *reinterpret_cast<float4*>(sm + pl.ones + (size_t)r * 16) = make_float4(1.0f, 1.0f, 1.0f, 0.0f);
+        *reinterpret_cast<float4*>(sm + pl.ones + 2048 + (size_t)r * 16) = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+    }
+    if (PARTIALS) {
+        for (int i = tid; i < (int)(SLOTS * pl.slot_bytes / 16); i += nthreads)
+            *reinterpret_cast<uint4*>(sm + pl.slot + (size_t)i * 16) = make_uint4(0u, 0u, 0u, 0u);
+        for (int i = tid; i < SLOTS * TILE; i += nthreads) reinterpret_cast<uint16_t*>(sm + pl.prev)[i] = 0xFFFFu;
+        __syncthreads();                                     // (other threads' zeros must not land on top of the ones)
+        for (int s = 0; s < SLOTS; ++s)                      // the ones column of a slot: [1, 1, 0, ...] for every point
+            for (int r = tid; r < TILE; r += nthreads)
+                *reinterpret_cast<uint4*>(sm + pl.slot + (size_t)s * pl.slot_bytes + (size_t)(2 * KCH) * XC + (size_t)r * 16) = make_uint4(0x3F803F80u, 0u, 0u, 0u);
+    }
+    fence_async_smem();
+    fence_before_sync();
+    __syncthreads();
+    fence_after_sync();
+    const uint32_t tmem_base = (uint32_t)s_ctrl[6];
+    const uint32_t sums_col0 = (uint32_t)(G * npad);
+    bool ok = true;                                           // this thread has seen no wait give up
+
+    if (warp == 4 * G) {
+        // ---- producer ---------------------------------------------------------------------------------------------
+        // (all lanes walk the runs: they fetch the run's tile marks together; lane 0 does the rest)
+        int i = 0, run_seq = 0;
+        for (int run = blockIdx.x; run < runs; run += gridDim.x) {
+            ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+            if (!ok) break;
+            if (skipping) {
+                __syncwarp();
+                for (int q = lane; q < need_words; q += 32) s_need[q] = need[(size_t)run * need_words + q];
+                __syncwarp();
+            }
+            if (lane != 0) continue;
+            const int r = run / C, c = run - r * C;
+            const size_t j0 = (size_t)r * N / P, j1 = (size_t)(r + 1) * N / P;
+            const size_t len = j1 - j0;
+            const size_t b0 = j0 + len * c / C, b1 = j0 + len * (c + 1) / C;
+            const size_t ntiles = (b1 - b0 + TILE - 1) / TILE;
+            size_t t = 0;                                    // first tile that has to be searched
+            if (skipping) while (t < ntiles && s_need[t] == 0u) ++t;
+            if (t >= ntiles) {                               // nothing to do in this run
+                if (PARTIALS && DELTA) dirty[run] = 0u;
+                else if (PARTIALS) for (int q = 0; q < K * (D + 4); ++q) scratch[(size_t)run * K * (D + 4) + q] = 0.0f;   // an empty run
+                continue;
+            }
+            while (t < ntiles) {
+                size_t tn = t + 1;
+                if (skipping) while (tn < ntiles && s_need[tn] == 0u) ++tn;
+                const int s = i % NST, use = i / NST;
+                if (use > 0 && !wait_or_abort(B_empty(s), (uint32_t)(use - 1) & 1u, s_abort, 1)) { ok = false; break; }
+                TileDesc d;
+                d.base = b0 + t * TILE; d.end = b1; d.run = run; d.run_seq = run_seq; d.last = tn >= ntiles ? 1 : 0; d.pad = 0;
+                s_desc[s] = d;
+                mbar_expect_tx(B_full(s), pl.stage_bytes);
+                tma_tile_2d(sm_u + pl.stage + (uint32_t)s * pl.stage_bytes, &pmap, 0, (int)(b0 + t * TILE), B_full(s));
+                ++i;
+                t = tn;
+            }
+            ++run_seq;
+        }
+        if (lane == 0) {
+            for (int e = 0; e < G && ok; ++e) {               // end markers: one for every epilogue group
+                const int s = i % NST, use = i / NST;
+                if (use > 0 && !wait_or_abort(B_empty(s), (uint32_t)(use - 1) & 1u, s_abort, 1)) { ok = false; break; }
+                TileDesc d;
+                d.base = 0; d.end = 0; d.run = -1; d.run_seq = e; d.last = 0; d.pad = 0;
+                s_desc[s] = d;
+                mbar_arrive(B_full(s));
+                ++i;
+            }
+            if (!ok) {                                        // copies still in flight must land before the block may go
+                for (int back = 1; back <= NST && back <= i; ++back) {
+                    const int ii = i - back;
+                    for (uint32_t it = 0; it < WAIT_LIMIT; ++it)
+                        if (mbar_try_wait(B_full(ii % NST), (uint32_t)(ii / NST) & 1u)) break;
+                }
+            }
+        }
+    } else if (warp == 4 * G + 1) {
+        // ---- search issuer -------------------------------------------------------------------------------------------
+        if (lane == 0) {
+            // Everything that does not change from tile to tile is made once: this one thread's instruction stream is
+            // what every tile waits for.  A descriptor's address field counts 16-byte units, so a step of 32 bytes adds 2
+            // and the next stage adds stage_bytes / 16.
+            const uint32_t idesc = idesc_tf32(TILE, npad);
+            uint64_t bdesc[D / 8];
+#pragma unroll
+            for (int ks = 0; ks < D / 8; ++ks) bdesc[ks] = swz_desc<D>(sm_u + pl.b + ks * 32);
+            const uint64_t adesc0 = swz_desc<D>(sm_u + pl.stage);
+            const uint64_t ones_desc = smem_desc(sm_u + pl.ones, 2048, 128), cnb_desc = smem_desc(sm_u + pl.cnb, (uint32_t)npad * 16, 128);
+            const uint32_t stage_units = pl.stage_bytes >> 4;
+            int s = 0, g = 0;
+            uint32_t full_par = 0, empty_par = 1;            // parities of the next waits on full[s] and accempty[g]
+            bool first_round = true;                          // the accumulators start out free
+            for (;;) {
+                if (!wait_or_abort(B_full(s), full_par, s_abort, 3)) { ok = false; break; }
+                if (s_desc[s].run < 0) break;
+                if (!first_round && !wait_or_abort(B_accempty(g), empty_par, s_abort, 4)) { ok = false; break; }
+                fence_after_sync();
+                const uint32_t acc = tmem_base + (uint32_t)(g * npad);
+                const uint64_t adesc = adesc0 + (uint64_t)((uint32_t)s * stage_units);
+#pragma unroll
+                for (int ks = 0; ks < D / 8; ++ks)             // 8 coordinates (32 bytes) per step
+                    mma_tf32(acc, adesc + (uint64_t)(2 * ks), bdesc[ks], idesc, ks > 0 ? 1u : 0u);
+                mma_tf32(acc, ones_desc, cnb_desc, idesc, 1u);
+                mma_commit(B_accfull(g));
+                if (++s == NST) { s = 0; full_par ^= 1u; }
+                if (++g == G) { g = 0; empty_par ^= 1u; first_round = false; }
+            }
+        }
+    } else if (warp == 4 * G + 2) {
+        // ---- sums issuer -----------------------------------------------------------------------------------------------
+        if (PARTIALS && lane == 0) {
+            const uint32_t idesc = tc::instr_desc(TILE, npad, true);
+            const uint64_t xdesc0 = smem_desc(sm_u + pl.slot, 128, XC), odesc0 = smem_desc(sm_u + pl.slot + pl.oh_off, 128, OCHUNK);
+            const uint32_t slot_units = pl.slot_bytes >> 4;
+            bool started = false, run_checked = false;
+            int nruns[2] = {0, 0};                            // runs finished on each accumulator so far
+            int uses[SLOTS] = {0, 0};                         // sums GEMMs issued from each slot so far
+            int g = 0;
+            uint32_t dec_par = 0;
+            for (int i = 0;; ++i) {
+                const int slot = i & (SLOTS - 1);
+                if (!wait_or_abort(B_decided(g), dec_par, s_abort, 5 | (i << 8))) { ok = false; break; }
+                const int ctrl = atomicExch(const_cast<int*>(s_ctrl + g), 0);   // taken and cleared: the warps or their flags in
+                mbar_arrive(B_tiledone(g));                    // the group's control word may be written again
+                if (ctrl & CTRL_END) break;
+                const int par = (ctrl & CTRL_PAR) ? 1 : 0, last = ctrl & CTRL_LAST;
+                if (!run_checked && (ctrl & (CTRL_SUMS | CTRL_LAST))) {
+                    // the run before last used this accumulator and this "had sums" word: its last tile's group must be
+                    // through with both (it says so after writing the sums out, or after seeing that there were none)
+                    if (nruns[par] > 0 && !wait_or_abort(B_drained(par), (uint32_t)(nruns[par] - 1) & 1u, s_abort, 6)) { ok = false; break; }
+                    run_checked = true;
+                }
+                if (ctrl & CTRL_SUMS) {
+                    fence_after_sync();
+                    const uint32_t acc = tmem_base + sums_col0 + (uint32_t)(par * npad);
+                    const uint64_t xd = xdesc0 + (uint64_t)((uint32_t)slot * slot_units), od = odesc0 + (uint64_t)((uint32_t)slot * slot_units);
+#pragma unroll
+                    for (int ks = 0; ks < TILE / 16; ++ks)     // 16 points (256 bytes) per step, both operands MN-major
+                        tc::mma_bf16(acc, xd + (uint64_t)(16 * ks), od + (uint64_t)(16 * ks), idesc, (started || ks > 0) ? 1u : 0u);
+                    started = true;
+                    mma_commit(B_slotfree(slot));
+                    s_ctrl[28 + slot] = ++uses[slot];
+                }
+                s_ctrl[26] = i + 1;                            // through with tile i (its sums GEMM, if any, is on its way)
+                if (last) {
+                    s_ctrl[4 + par] = started ? 1 : 0;
+                    __threadfence_block();
+                    if (started) mma_commit(B_rundone(par));
+                    else mbar_arrive(B_rundone(par));
+                    ++nruns[par];
+                    s_ctrl[25] = nruns[0] + nruns[1];          // runs whose end has been signalled
+                    started = false;
+                    run_checked = false;
+                }
+                if (++g == G) { g = 0; dec_par ^= 1u; }
+            }
+        }
+    } else {
+        // ---- epilogue groups ------------------------------------------------------------------------------------------
+        const int g = warp >> 2, t = tid & 127;              // t: this thread's point of the tile = row of the accumulator
+        const uint32_t lane_base = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
+        const int stride = D + 4;
+        float cmax = 0.0f;
+        for (int k = 0; k < K; ++k) cmax = fmaxf(cmax, s_cn[k]);
+        const float drift_max = (PARTIALS && BOUNDS) ? drift[K] : 0.0f;
+        // One lane per warp waits and arrives for its warp (the barriers of the groups count warps, not threads):
+        // 32 times fewer barrier operations, and the warp's other lanes are ordered behind lane 0 by the shuffle.
+        auto wwait = [&](uint32_t bar, uint32_t par, int where) -> bool {
+            int r = 1;
+            if (lane == 0) r = wait_or_abort(bar, par, s_abort, where) ? 1 : 0;
+            return __shfl_sync(0xffffffffu, r, 0) != 0;
+        };
+        auto warrive = [&](uint32_t bar) {
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar);
+        };
+#ifdef EC_WS_DEBUG
+        long long dbg_t[6] = {0, 0, 0, 0, 0, 0}; long long dbg_c = clock64(); int dbg_n = 0;
+#define DBG_LAP(k) { const long long now__ = clock64(); dbg_t[k] += now__ - dbg_c; dbg_c = now__; }
+#else
+#define DBG_LAP(k)
+#endif
+        // tile i = g, g + G, ...: stage s = i mod stages on its lap-th use, this group's n-th tile, slot i mod 2
+        int s = g % NST, n = 0;
+        uint32_t lap = (uint32_t)(g / NST);
+        for (int i = g; ok; i += G, ++n) {
+            const int slot = i & (SLOTS - 1);
+            if (n > 0) {
+                s += G;
+                while (s >= NST) { s -= NST; ++lap; }
+            }
+            DBG_LAP(5)
+            if (!wwait(B_full(s), lap & 1u, 3)) { ok = false; break; }
+            DBG_LAP(0)
+            const TileDesc td = s_desc[s];
+            if (td.run < 0) {                                // no more tiles: the sums issuer hears it from the first group that does
+                if (PARTIALS && td.run_seq == 0) {          // (the first of the G end markers)
+                    if (n > 0 && !wwait(B_tiledone(g), (uint32_t)(n - 1) & 1u, 12 | (i << 8))) { ok = false; break; }
+                    if (t == 0) atomicOr(const_cast<int*>(s_ctrl + g), CTRL_END);
+                    warrive(B_decided(g));
+                }
+                break;
+            }
+            const size_t j = (size_t)td.base + (size_t)t;
+            const bool live = j < (size_t)td.end;
+            const int old = (DELTA && live) ? labels[j] : -1;
+            const unsigned char* row = sm + pl.stage + (size_t)s * pl.stage_bytes;
+            float xn;
+            {
+                float n0 = 0.0f, n1 = 0.0f, n2 = 0.0f, n3 = 0.0f;   // four chains
+#ifdef EC_WS_EXP_NOXN
+                n0 = 1000.0f;
+#else
+#pragma unroll
+                for (int q = 0; q < Q; ++q) {
+                    const float4 v = *reinterpret_cast<const float4*>(row + swz_off<D>(t, q));
+                    n0 = fmaf(v.x, v.x, n0); n1 = fmaf(v.y, v.y, n1); n2 = fmaf(v.z, v.z, n2); n3 = fmaf(v.w, v.w, n3);
+                }
+#endif
+                xn = (n0 + n1) + (n2 + n3);
+            }
+            DBG_LAP(1)
+            if (!wwait(B_accfull(g), (uint32_t)n & 1u, 8)) { ok = false; break; }
+            DBG_LAP(2)
+            fence_after_sync();
+            float m1 = __int_as_float(0x7f800000), m2 = m1;
+            {
+                // 16 columns at a time, the next 16 on their way while these are looked at (npad / 16 is even)
+                const uint32_t col0 = lane_base + (uint32_t)(g * npad);
+                uint32_t va[16], vb[16];
+                tmem_ld16_nowait(col0, va);
+                for (int ch = 0; ch < npad / 16; ch += 2) {
+                    float c1, c2;
+                    tmem_ld_wait();
+                    tmem_ld16_nowait(col0 + (uint32_t)(ch * 16 + 16), vb);
+                    best_two_of_16(va, c1, c2);              // tags 0..15; bits 4-6 (zero so far) take the chunk number
+                    c1 = __uint_as_float(__float_as_uint(c1) | (uint32_t)(ch << 4));
+                    m2 = min3(m2, c2, fmaxf(m1, c1));
+                    m1 = fminf(m1, c1);
+                    tmem_ld_wait();
+                    if (ch + 2 < npad / 16) tmem_ld16_nowait(col0 + (uint32_t)(ch * 16 + 32), va);
+                    best_two_of_16(vb, c1, c2);
+                    c1 = __uint_as_float(__float_as_uint(c1) | (uint32_t)((ch + 1) << 4));
+                    m2 = min3(m2, c2, fmaxf(m1, c1));
+                    m1 = fminf(m1, c1);
+                }
+            }
+            fence_before_sync();
+            DBG_LAP(3)
+            warrive(B_accempty(g));                      // the accumulator may take the group's next tile
+            int kb = (int)(__float_as_uint(m1) & 127u);
+            const float tau = TAU_SCALE * (xn + cmax);
+            const bool redo = live && !(m2 - m1 > tau);
+            if (redo) {
+                float x[D];
+#pragma unroll
+                for (int q = 0; q < Q; ++q) {
+                    const float4 v = *reinterpret_cast<const float4*>(row + swz_off<D>(t, q));
+                    x[4 * q] = v.x; x[4 * q + 1] = v.y; x[4 * q + 2] = v.z; x[4 * q + 3] = v.w;
+                }
+                kb = tc::exact_argmin_global<D>(x, centroids, K);
+            }
+            const bool changed = live && !(DELTA && old == kb);
+            if (changed) labels[j] = kb;
+            if (PARTIALS && BOUNDS && live) {
+                float2 w = make_float2(__int_as_float(0x7f800000), 0.0f);      // decided by the exact form: searched again next time
+                if (!redo) {
+                    // |x - c|^2 = |x|^2 + v; the search knows v to within tau (tags included)
+                    const float u = __fsqrt_ru(fmaxf(__fadd_ru(__fadd_ru(xn, m1), tau), 0.0f));
+                    const float l = __fsqrt_rd(fmaxf(__fsub_rd(__fadd_rd(xn, m2), tau), 0.0f));
+                    w = make_float2(__fsub_ru(u, s_drift[kb]), __fadd_rd(l, drift_max));
+                }
+                bounds[j] = w;
+            }
+            if (PARTIALS) {
+                // Every warp goes its own way: no meeting of the group's four warps.  A warp tells the sums issuer whether one
+                // of its points changed the sums (flags or-ed into the group's control word, which the issuer takes and
+                // clears); only a thread whose label changed converts its row and sets its one-hot row - the other rows of
+                // the slot keep whatever finite numbers they hold, against one-hot rows that are zero.
+                const bool any_w = __any_sync(0xffffffffu, changed);
+                // the sums issuer must have taken what the group said about its previous tile
+                if (n > 0 && !wwait(B_tiledone(g), (uint32_t)(n - 1) & 1u, 10 | (i << 8))) { ok = false; break; }
+                // Two groups take turns on a slot.  Once the sums issuer is through with tile i - SLOTS (the slot's last possible
+                // user before this tile) the slot's book-keeping is final: whether the rows of this warp's position still have
+                // one-hot entries set (they must be cleared before the slot's next GEMM), and how many GEMMs were issued from
+                // the slot, which says which phase of its barrier to wait for before the operands may be touched - at most one
+                // phase back, because every user waits for its predecessor.
+                int info = 0;                                        // bit 0: stale rows, bits 1..: GEMMs issued from the slot
+                if (lane == 0 && i >= SLOTS) {
+                    const long long t0 = clock64();
+                    while (s_ctrl[26] < i - SLOTS + 1) {
+                        if (*s_abort != 0 || clock64() - t0 > 4000000000LL) { if (*s_abort == 0) *s_abort = 14; info = -1; break; }
+                    }
+                    if (info == 0) info = (s_ctrl[32 + 4 * slot + (warp & 3)] != 0 ? 1 : 0) | (s_ctrl[28 + slot] << 1);
+                }
+                info = __shfl_sync(0xffffffffu, info, 0);
+                if (info < 0) { ok = false; break; }
+                const bool stale = (info & 1) != 0;
+                if (any_w || stale) {
+                    const int uses = info >> 1;
+                    if (uses > 0 && !wwait(B_slotfree(slot), (uint32_t)(uses - 1) & 1u, 7)) { ok = false; break; }
+                    unsigned char* xs = sm + pl.slot + (size_t)slot * pl.slot_bytes;
+                    unsigned char* oh = xs + pl.oh_off;
+                    uint16_t* prev = reinterpret_cast<uint16_t*>(sm + pl.prev) + slot * TILE + t;
+                    const uint16_t pv = *prev;
+                    if ((pv & 0xFFu) != 0xFFu) *reinterpret_cast<uint4*>(oh + (size_t)(pv & 0xFFu) * OCHUNK + (size_t)t * 16) = make_uint4(0u, 0u, 0u, 0u);
+                    if ((pv >> 8) != 0xFFu) *reinterpret_cast<uint4*>(oh + (size_t)(pv >> 8) * OCHUNK + (size_t)t * 16) = make_uint4(0u, 0u, 0u, 0u);
+                    uint16_t nv = 0xFFFFu;
+                    if (changed) {
+                        // one-hot row of this point: 16-byte chunk kb/8, bf16 1.0 at position kb%8 (and -1.0 for the label it leaves)
+                        uint32_t wv[4] = {0u, 0u, 0u, 0u};
+                        wv[(kb & 7) >> 1] = 0x3F80u << (16 * (kb & 1));
+                        const int ck = kb >> 3;
+                        if (old >= 0 && (old >> 3) == ck) wv[(old & 7) >> 1] |= 0xBF80u << (16 * (old & 1));
+                        *reinterpret_cast<uint4*>(oh + (size_t)ck * OCHUNK + (size_t)t * 16) = make_uint4(wv[0], wv[1], wv[2], wv[3]);
+                        nv = (uint16_t)(0xFF00u | (uint32_t)ck);
+                        if (old >= 0 && (old >> 3) != ck) {
+                            uint32_t wo[4] = {0u, 0u, 0u, 0u};
+                            wo[(old & 7) >> 1] = 0xBF80u << (16 * (old & 1));
+                            *reinterpret_cast<uint4*>(oh + (size_t)(old >> 3) * OCHUNK + (size_t)t * 16) = make_uint4(wo[0], wo[1], wo[2], wo[3]);
+                            nv = (uint16_t)(((uint32_t)(old >> 3) << 8) | (uint32_t)ck);
+                        }
+                        // bf16 high and low parts of the row (low = bf16(x - high)): chunk column 2 kc resp. 2 kc + 1
+#pragma unroll
+                        for (int kc = 0; kc < KCH; ++kc) {
+                            const float4 va = *reinterpret_cast<const float4*>(row + swz_off<D>(t, 2 * kc));
+                            const float4 vb = *reinterpret_cast<const float4*>(row + swz_off<D>(t, 2 * kc + 1));
+                            const float v[8] = {va.x, va.y, va.z, va.w, vb.x, vb.y, vb.z, vb.w};
+                            uint32_t hw[4], lw[4];
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                hw[e] = pack_bf16(v[2 * e], v[2 * e + 1]);
+                                const float ah = __uint_as_float(hw[e] << 16), bh = __uint_as_float(hw[e] & 0xFFFF0000u);
+                                lw[e] = pack_bf16(v[2 * e] - ah, v[2 * e + 1] - bh);
+                            }
+                            *reinterpret_cast<uint4*>(xs + (size_t)(2 * kc) * XC + (size_t)t * 16) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
+                            *reinterpret_cast<uint4*>(xs + (size_t)(2 * kc + 1) * XC + (size_t)t * 16) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
+                        }
+                    }
+                    *prev = nv;
+                    if (lane == 0) s_ctrl[32 + 4 * slot + (warp & 3)] = any_w ? 1 : 0;
+                    fence_async_smem();                      // the tensor core reads shared memory through the async proxy
+                }
+                if (lane == 0) {
+                    const int flags = (any_w ? CTRL_SUMS : 0) |
+                                      ((warp & 3) == 0 ? (td.last ? CTRL_LAST : 0) | ((td.run_seq & 1) ? CTRL_PAR : 0) : 0);
+                    if (flags) atomicOr(const_cast<int*>(s_ctrl + g), flags);
+                }
+                fence_before_sync();
+                warrive(B_decided(g));
+            }
+            warrive(B_empty(s));                         // the stage may take another tile
+            DBG_LAP(4)
+#ifdef EC_WS_DEBUG
+            ++dbg_n;
+#endif
+            if (PARTIALS && td.last) {
+                // the run's last tile: its group writes the run's sums out once the sums issuer is through the run
+                // (first until the sums issuer has signalled the end of this run: it has then seen the run before last written
+                // out, so the barrier is at most one phase behind this wait - different runs' ends are waited for by
+                // different groups, none of which sees every phase)
+                const int par = td.run_seq & 1;
+                {
+                    const long long t0 = clock64();
+                    while (s_ctrl[25] <= td.run_seq) {
+                        if (*s_abort != 0 || clock64() - t0 > 4000000000LL) { if (*s_abort == 0) *s_abort = 13; ok = false; break; }
+                    }
+                    if (!ok) break;
+                }
+                if (!wwait(B_rundone(par), (uint32_t)(td.run_seq >> 1) & 1u, 11)) { ok = false; break; }
+                fence_after_sync();
+                const bool had_sums = s_ctrl[4 + par] != 0;
+                float* row_block = scratch + (size_t)td.run * (size_t)K * stride;
+                if (had_sums) {
+                    // Accumulator rows: 16 (d / 8) + d % 8 holds the high-part sums of coordinate d, 8 rows further on the
+                    // low-part sums (same warp, 8 lanes up), row 2 D the counts.  Columns are the centroids.
+                    const int d_of = (t >> 4) * 8 + (t & 7);
+                    const bool is_hi = (t & 8) == 0 && t < 2 * D, is_cnt = t == 2 * D;
+                    for (int ch = 0; ch < npad / 32; ++ch) {
+                        uint32_t v[32];
+                        tmem_ld32_nowait(lane_base + sums_col0 + (uint32_t)(par * npad + ch * 32), v);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) {
+                            const float lo = __shfl_down_sync(0xffffffffu, __uint_as_float(v[e]), 8);
+                            const int k = ch * 32 + e;
+                            if (k < K) {
+                                if (is_hi) row_block[(size_t)k * stride + d_of] = __fadd_rn(__uint_as_float(v[e]), lo);
+                                if (is_cnt) {
+                                    row_block[(size_t)k * stride + D] = __uint_as_float(v[e]);
+                                    row_block[(size_t)k * stride + D + 1] = 0.0f;
+                                    row_block[(size_t)k * stride + D + 2] = 0.0f;
+                                    row_block[(size_t)k * stride + D + 3] = 0.0f;
+                                }
+                            }
+                        }
+                    }
+                    fence_before_sync();
+                } else if (!DELTA) {
+                    for (int q = t; q < K * stride; q += TILE) row_block[q] = 0.0f;
+                }
+                warrive(B_drained(par));                 // the accumulator and the "had sums" word may serve another run
+                if (DELTA && t == 0) dirty[td.run] = had_sums ? 1u : 0u;
+            }
+        }
+#ifdef EC_WS_DEBUG
+        if (blockIdx.x == 0 && (tid & 127) == 5)
+            printf("group %d tiles %d: wait full %lld, xn %lld, wait acc %lld, ld+track %lld, rest %lld, loop %lld (cycles per tile)\n", g, dbg_n,
+                   dbg_t[0] / (dbg_n + 1), dbg_t[1] / (dbg_n + 1), dbg_t[2] / (dbg_n + 1), dbg_t[3] / (dbg_n + 1), dbg_t[4] / (dbg_n + 1), dbg_t[5] / (dbg_n + 1));
+#endif
+    }
+    if (!ok && *s_abort == 0) *s_abort = 15;
+    fence_before_sync();
+    __syncthreads();
+    if (tid == 0 && *s_abort != 0 && status != nullptr) atomicCAS(status, 0u, 2u | (((uint32_t)*s_abort & 0xFFFu) << 4) | ((uint32_t)s_ctrl[24] << 16));   // the first block to report stays
+#ifdef EC_WS_DEBUG
+    if (tid == 0 && *s_abort != 0)
+        printf("block %d abort %x ctrl %d %d %d %d had %d %d sums %x votes %d %d %d | %d %d %d\n", blockIdx.x, *s_abort, s_ctrl[0], s_ctrl[1], s_ctrl[2],
+               s_ctrl[3], s_ctrl[4], s_ctrl[5], s_ctrl[24], s_vote[0], s_vote[1], s_vote[2], s_vote[6], s_vote[7], s_vote[8]);
+#endif
+    if (warp == 4 * G + 1) {
+        fence_after_sync();
+        tmem_dealloc(tmem_base, pl.tmem_cols);
+    }
+}
+
+}  // namespace ws
+}  // namespace ec
