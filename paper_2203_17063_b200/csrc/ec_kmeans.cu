@@ -582,7 +582,7 @@ struct ec_kmeans {
     bool tc_ok;            // the tensor-core candidate search covers this shape
     bool ws_ok;            // ... and so does its warp-specialised form (K <= 128, tensor map of the points made)
     CUtensorMap pmap;      // the points as a 2-D tensor [N][D] of fp32, tiles of 128 rows, swizzled rows
-    ec::ws::Plan ws_plan, ws_plan_assign;
+    ec::ws::Plan ws_plan, ws_plan_delta, ws_plan_assign;
     int path;              // 0 = automatic, 1 = fp32 fused kernel, 2 = tensor cores, 3 = tensor cores, register-staged form
     size_t tc_smem, tc_assign_smem;
     int tc_wave_full, tc_wave_delta, tc_wave_assign;   // resident blocks of the tensor-core kernels on the whole device
@@ -777,7 +777,8 @@ bool ws_capable(size_t N, int D, int K) {
     if (D != 16 && D != 32) return false;
     if (tc::npad_of(K) > 128) return false;
     if (N >= 0x7fffff00ull) return false;
-    return ws::plan_of(D, K, true).total <= 227 * 1024 && ws::plan_of(D, K, true).stages >= 3;
+    return ws::plan_of(D, K, true, false).total <= 227 * 1024 && ws::plan_of(D, K, true, false).stages >= 3 &&
+           ws::plan_of(D, K, true, true).total <= 227 * 1024;
 }
 
 // The tensor map of the points (driver entry point taken through the runtime: the library links no libcuda).
@@ -828,8 +829,9 @@ int km_ws_launch(ec_kmeans* km, bool partials, const float* centroids, int32_t* 
     if (partials) {
         const int runs = km->P * km->Cf;
         const unsigned grid = (unsigned)(runs < km->sms ? runs : km->sms);
-        const unsigned thr = (unsigned)ws::threads_of(km->ws_plan);
-        const size_t smem = km->ws_plan.total;
+        const ws::Plan& plan = delta ? km->ws_plan_delta : km->ws_plan;
+        const unsigned thr = (unsigned)ws::threads_of(plan);
+        const size_t smem = plan.total;
         float* full_out = km->Cf == 1 ? km->partials : km->scratch;
         if (delta && own)
             ws::ws_fused_kernel<D, true, true, true><<<grid, thr, smem, st>>>(
@@ -1016,8 +1018,9 @@ int ec_kmeans_init(ec_kmeans_t** out, const float* points, size_t N, int D, int 
         e = D == 16 ? km_tc_attr<16>(km) : km_tc_attr<32>(km);
     km->ws_ok = km->tc_ok && ws_capable(N, D, K) && km_make_point_map(km);
     if (km->ws_ok) {
-        km->ws_plan = ws::plan_of(D, K, true);
-        km->ws_plan_assign = ws::plan_of(D, K, false);
+        km->ws_plan = ws::plan_of(D, K, true, false);
+        km->ws_plan_delta = ws::plan_of(D, K, true, true);
+        km->ws_plan_assign = ws::plan_of(D, K, false, false);
         if (e == cudaSuccess) e = D == 16 ? km_ws_attr<16>(km) : km_ws_attr<32>(km);
     }
     if (e == cudaSuccess) e = cudaMemsetAsync(km->tc_status, 0, 4, 0);

@@ -11,11 +11,12 @@
 //                            the accumulator in tensor memory holds v_k = |c_k|^2 - 2 x.c_k for 128 points x all
 //                            centroids.  One accumulator per epilogue group, so tiles overlap;
 //   epilogue groups (4 warps each, tile i goes to group i mod G): read the scores with tcgen05.ld (one point per
-//                            thread), find the best two by a tournament of min/max pairs whose low mantissa bits carry
-//                            the column index, decide (exact fp32 form from the staged row whenever the two are closer
-//                            than the search's error bound tau), write label and distance bounds, and - only for a tile in
-//                            which a label changed - convert the staged rows to bf16 high + low parts and set the
-//                            one-hot rows for the sums GEMM;
+//                            thread, 16 columns at a time with the next 16 on their way), find the best two by a
+//                            tournament of min/max pairs whose low mantissa bits carry the column index, decide (exact
+//                            fp32 form from the staged row whenever the two are closer than the search's error bound tau),
+//                            write label and distance bounds, and - only a thread whose label changed - convert the
+//                            staged row to bf16 high + low parts and set the one-hot row for the sums GEMM.  The warps
+//                            of a group never meet: each waits and arrives for itself (one lane per warp);
 //   sums issuer (one thread)  sums[d][k] += sum_j x[j][d] onehot[j][k] as tcgen05.mma kind::f16 over such tiles, in
 //                            tile order (so the sums repeat bit for bit), accumulator in tensor memory per run, double
 //                            buffered so that a run is written out while the next one accumulates.
@@ -35,9 +36,6 @@
 #pragma once
 
 #include <cuda.h>
-#ifdef EC_WS_DEBUG
-#include <cstdio>
-#endif
 
 #ifndef EC_WS_HINT
 #define EC_WS_HINT 20000
@@ -61,7 +59,7 @@ using tc::tmem_dealloc;
 constexpr int TILE = 128;                       // points per tile = rows of an accumulator
 constexpr int MAX_GROUPS = 4;                   // epilogue groups of four warps
 constexpr int MAX_STAGES = 8;
-constexpr int SLOTS = 2;                        // operand buffers of the sums GEMM
+constexpr int MAX_SLOTS = 4;                    // operand buffers of the sums GEMM: 2 when only changes are summed, else 3
 constexpr int MAX_THREADS = (4 * MAX_GROUPS + 3) * 32;
 constexpr uint32_t WAIT_LIMIT = 1u << 24;
 constexpr uint32_t OCHUNK = TILE * 16;          // one-hot tile: bytes between chunks of 8 centroids
@@ -72,13 +70,15 @@ __host__ __device__ constexpr uint32_t xchunk_of(int D) { return TILE * 16 + 102
 
 // Shared memory of a block (byte offsets from a 1024-byte aligned base) and its tensor-memory columns.
 struct Plan {
-    int groups, stages;
+    int groups, stages, slots;
     uint32_t tmem_cols;
     uint32_t stage_bytes, slot_bytes, oh_off;       // oh_off: one-hot tile inside a slot
     uint32_t stage, b, ones, cnb, slot, prev, cn, drift, need, desc, ctrl, bar, total;
 };
-__host__ __device__ inline Plan plan_of(int D, int K, bool partials) {
+__host__ __device__ inline Plan plan_of(int D, int K, bool partials, bool delta) {
     Plan p;
+    p.slots = partials ? (delta ? 2 : 3) : 0;
+    const uint32_t SLOTS = (uint32_t)p.slots;
     const uint32_t npad = (uint32_t)npad_of(K), XC = xchunk_of(D);
     const uint32_t acc = partials ? 2u : 0u;
     int g = (int)(512u / npad) - (int)acc;
@@ -95,7 +95,7 @@ __host__ __device__ inline Plan plan_of(int D, int K, bool partials) {
     uint32_t off = 0;
     const uint32_t fixed_after_stages = npad * (uint32_t)D * 4u + 1024u   // b (1024-aligned)
         + 4096u + npad * 32u                                              // ones, cnb
-        + (partials ? SLOTS * p.slot_bytes + SLOTS * TILE * 2u : 0u)      // slots, previous one-hot chunks
+        + SLOTS * p.slot_bytes + SLOTS * TILE * 2u                        // slots, previous one-hot chunks
         + npad * 8u + 1024u + 4096u;                                       // cn, drift, need words, descriptors, control, barriers
     int st = (int)((226u * 1024u - fixed_after_stages) / p.stage_bytes);
     p.stages = st > MAX_STAGES ? MAX_STAGES : st;
@@ -105,8 +105,8 @@ __host__ __device__ inline Plan plan_of(int D, int K, bool partials) {
     p.ones = off; off += 4096u;                      // [2 chunks][128 rows][16 bytes]: (1,1,1,0 | 0,0,0,0), no swizzle
     p.cnb = off; off += npad * 32u;                  // [2 chunks][npad rows][16 bytes]: (hi, mid, lo, 0 | 0...) of |c|^2
     off = (off + 127u) & ~127u;
-    p.slot = off; off += partials ? SLOTS * p.slot_bytes : 0u;
-    p.prev = off; off += partials ? SLOTS * TILE * 2u : 0u;
+    p.slot = off; off += SLOTS * p.slot_bytes;
+    p.prev = off; off += SLOTS * TILE * 2u;
     p.cn = off; off += npad * 4u;
     p.drift = off; off += npad * 4u;
     p.need = off; off += 1024u;
@@ -218,48 +218,6 @@ __device__ __forceinline__ void tmem_ld32_nowait(uint32_t taddr, uint32_t (&r)[3
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
-// Best two of 32 scores whose low 7 mantissa bits have been replaced by their column index: sorted pairs, then the
-// same again on the smaller halves; the second best is the smallest of all the larger halves (the partner of the
-// winner is among them, and every other larger half is at least the second best of the smaller ones).
-__device__ __forceinline__ void best_two_of_32(const uint32_t (&raw)[32], float& c1, float& c2) {
-    float lo[16], hi_min;
-    {
-        float hi[16];
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-            const float a = __uint_as_float((raw[2 * i] & 0xFFFFFF80u) | (uint32_t)(2 * i));
-            const float b = __uint_as_float((raw[2 * i + 1] & 0xFFFFFF80u) | (uint32_t)(2 * i + 1));
-            lo[i] = fminf(a, b);
-            hi[i] = fmaxf(a, b);
-        }
-        float t[6];
-#pragma unroll
-        for (int i = 0; i < 5; ++i) t[i] = min3(hi[3 * i], hi[3 * i + 1], hi[3 * i + 2]);
-        hi_min = min3(min3(t[0], t[1], t[2]), min3(t[3], t[4], hi[15]), t[0]);
-    }
-    float l8[8];
-    {
-        float h8[8];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            l8[i] = fminf(lo[2 * i], lo[2 * i + 1]);
-            h8[i] = fmaxf(lo[2 * i], lo[2 * i + 1]);
-        }
-        hi_min = min3(hi_min, min3(h8[0], h8[1], h8[2]), min3(h8[3], h8[4], h8[5]));
-        hi_min = min3(hi_min, h8[6], h8[7]);
-    }
-    float l4[4];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        l4[i] = fminf(l8[2 * i], l8[2 * i + 1]);
-        hi_min = fminf(hi_min, fmaxf(l8[2 * i], l8[2 * i + 1]));
-    }
-    const float a = fminf(l4[0], l4[1]), b = fminf(l4[2], l4[3]);
-    hi_min = min3(hi_min, fmaxf(l4[0], l4[1]), fmaxf(l4[2], l4[3]));
-    c1 = fminf(a, b);
-    c2 = fminf(hi_min, fmaxf(a, b));
-}
-
 __device__ __forceinline__ void tmem_ld16_nowait(uint32_t taddr, uint32_t (&r)[16]) {
     asm volatile(
         "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
@@ -268,7 +226,10 @@ __device__ __forceinline__ void tmem_ld16_nowait(uint32_t taddr, uint32_t (&r)[1
         : "r"(taddr)
         : "memory");
 }
-// The same for 16 scores (tags 0..15), so that the next 16 can be on their way from tensor memory meanwhile.
+// Best two of 16 scores whose low 7 mantissa bits are replaced by their column index (here: 0..15 in the low four; the
+// caller adds the number of the group of 16): sorted pairs, then the same again on the smaller halves; the second best
+// is the smallest of all the larger halves (the partner of the winner is among them, and every other larger half is at
+// least the second best of the smaller ones).  16 at a time, so that the next 16 can be on their way from tensor memory.
 __device__ __forceinline__ void best_two_of_16(const uint32_t (&raw)[16], float& c1, float& c2) {
     float lo[8], hi[8];
 #pragma unroll
@@ -301,7 +262,8 @@ ws_fused_kernel(const __grid_constant__ CUtensorMap pmap, const float* __restric
     constexpr uint32_t XC = xchunk_of(D);
     static_assert(D == 16 || D == 32, "a row is one 64- or 128-byte swizzle span");
     extern __shared__ unsigned char ws_smem_raw[];
-    const Plan pl = plan_of(D, K, PARTIALS);
+    const Plan pl = plan_of(D, K, PARTIALS, DELTA);
+    const int SLOTS = pl.slots;
     const int npad = npad_of(K);
     const int G = pl.groups, NST = pl.stages;
     unsigned char* sm = ws_smem_raw + ((1024u - (smem_u32(ws_smem_raw) & 1023u)) & 1023u);
@@ -311,12 +273,11 @@ ws_fused_kernel(const __grid_constant__ CUtensorMap pmap, const float* __restric
     uint32_t* s_need = reinterpret_cast<uint32_t*>(sm + pl.need);
     TileDesc* s_desc = reinterpret_cast<TileDesc*>(sm + pl.desc);
     // control words: [0..3] what a group says about its tile (CTRL_*), [4..5] run had sums, [6] tensor-memory address,
-    // [7] abort, [8 + 3 g + n % 3] "a label changed" votes of group g's n-th tile, [25] runs whose end the sums issuer has
-    // signalled, [26] tiles it is through with, [28..29] sums GEMMs issued from each slot, [32 + 4 slot + w] rows of warp w
+    // [7] abort, [25] runs whose end the sums issuer has
+    // signalled, [26] tiles it is through with, [28..31] sums GEMMs issued from each slot, [32 + 4 slot + w] rows of warp w
     // of the slot's last user have one-hot entries set
     volatile int* s_ctrl = reinterpret_cast<volatile int*>(sm + pl.ctrl);
     volatile int* s_abort = s_ctrl + 7;
-    volatile int* s_vote = s_ctrl + 8;
     constexpr int CTRL_SUMS = 1, CTRL_LAST = 2, CTRL_PAR = 4, CTRL_END = 8;
     // barriers (8 bytes each)
     const uint32_t bar0 = sm_u + pl.bar;
@@ -328,8 +289,7 @@ ws_fused_kernel(const __grid_constant__ CUtensorMap pmap, const float* __restric
     auto B_tiledone = [&](int g) { return bar0 + 8u * (uint32_t)(2 * MAX_STAGES + 3 * MAX_GROUPS + g); };
     auto B_rundone = [&](int p) { return bar0 + 8u * (uint32_t)(2 * MAX_STAGES + 4 * MAX_GROUPS + p); };
     auto B_drained = [&](int p) { return bar0 + 8u * (uint32_t)(2 * MAX_STAGES + 4 * MAX_GROUPS + 2 + p); };
-    auto B_vote = [&](int g) { return bar0 + 8u * (uint32_t)(2 * MAX_STAGES + 4 * MAX_GROUPS + 4 + g); };
-    auto B_slotfree = [&](int sl) { return bar0 + 8u * (uint32_t)(2 * MAX_STAGES + 5 * MAX_GROUPS + 4 + sl); };
+    auto B_slotfree = [&](int sl) { return bar0 + 8u * (uint32_t)(2 * MAX_STAGES + 5 * MAX_GROUPS + 4 + sl); };   // (MAX_SLOTS of them)
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int nthreads = (4 * G + 3) * 32;
@@ -351,14 +311,13 @@ ws_fused_kernel(const __grid_constant__ CUtensorMap pmap, const float* __restric
     if (tid == 0) {
         for (int s = 0; s < NST; ++s) { mbar_init(B_full(s), 1); mbar_init(B_empty(s), 4); }
         for (int g = 0; g < G; ++g) {
-            mbar_init(B_accfull(g), 1); mbar_init(B_accempty(g), 4); mbar_init(B_decided(g), 4); mbar_init(B_vote(g), 4);
+            mbar_init(B_accfull(g), 1); mbar_init(B_accempty(g), 4); mbar_init(B_decided(g), 4);
         }
-        for (int q = 0; q < 3 * MAX_GROUPS; ++q) s_vote[q] = 0;
         for (int g = 0; g < G; ++g) mbar_init(B_tiledone(g), 1);
-        for (int sl = 0; sl < SLOTS; ++sl) mbar_init(B_slotfree(sl), 1);
+        for (int sl = 0; sl < MAX_SLOTS; ++sl) mbar_init(B_slotfree(sl), 1);
         s_ctrl[0] = 0; s_ctrl[1] = 0; s_ctrl[2] = 0; s_ctrl[3] = 0;
-        s_ctrl[25] = 0; s_ctrl[26] = 0; s_ctrl[28] = 0; s_ctrl[29] = 0;
-        for (int q = 32; q < 40; ++q) s_ctrl[q] = 0;
+        s_ctrl[25] = 0; s_ctrl[26] = 0; s_ctrl[28] = 0; s_ctrl[29] = 0; s_ctrl[30] = 0; s_ctrl[31] = 0;
+        for (int q = 32; q < 48; ++q) s_ctrl[q] = 0;
         for (int p = 0; p < 2; ++p) { mbar_init(B_rundone(p), 1); mbar_init(B_drained(p), 4); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         *s_abort = 0;
@@ -508,11 +467,10 @@ ws_fused_kernel(const __grid_constant__ CUtensorMap pmap, const float* __restric
             const uint32_t slot_units = pl.slot_bytes >> 4;
             bool started = false, run_checked = false;
             int nruns[2] = {0, 0};                            // runs finished on each accumulator so far
-            int uses[SLOTS] = {0, 0};                         // sums GEMMs issued from each slot so far
+            int slot = 0;
             int g = 0;
             uint32_t dec_par = 0;
             for (int i = 0;; ++i) {
-                const int slot = i & (SLOTS - 1);
                 if (!wait_or_abort(B_decided(g), dec_par, s_abort, 5 | (i << 8))) { ok = false; break; }
                 const int ctrl = atomicExch(const_cast<int*>(s_ctrl + g), 0);   // taken and cleared: the warps or their flags in
                 mbar_arrive(B_tiledone(g));                    // the group's control word may be written again
@@ -533,7 +491,7 @@ ws_fused_kernel(const __grid_constant__ CUtensorMap pmap, const float* __restric
                         tc::mma_bf16(acc, xd + (uint64_t)(16 * ks), od + (uint64_t)(16 * ks), idesc, (started || ks > 0) ? 1u : 0u);
                     started = true;
                     mma_commit(B_slotfree(slot));
-                    s_ctrl[28 + slot] = ++uses[slot];
+                    s_ctrl[28 + slot] = s_ctrl[28 + slot] + 1;
                 }
                 s_ctrl[26] = i + 1;                            // through with tile i (its sums GEMM, if any, is on its way)
                 if (last) {
@@ -547,6 +505,7 @@ ws_fused_kernel(const __grid_constant__ CUtensorMap pmap, const float* __restric
                     run_checked = false;
                 }
                 if (++g == G) { g = 0; dec_par ^= 1u; }
+                if (++slot == SLOTS) slot = 0;
             }
         }
     } else {
@@ -568,24 +527,20 @@ ws_fused_kernel(const __grid_constant__ CUtensorMap pmap, const float* __restric
             __syncwarp();
             if (lane == 0) mbar_arrive(bar);
         };
-#ifdef EC_WS_DEBUG
-        long long dbg_t[6] = {0, 0, 0, 0, 0, 0}; long long dbg_c = clock64(); int dbg_n = 0;
-#define DBG_LAP(k) { const long long now__ = clock64(); dbg_t[k] += now__ - dbg_c; dbg_c = now__; }
-#else
-#define DBG_LAP(k)
-#endif
         // tile i = g, g + G, ...: stage s = i mod stages on its lap-th use, this group's n-th tile, slot i mod 2
         int s = g % NST, n = 0;
         uint32_t lap = (uint32_t)(g / NST);
+        int slot = PARTIALS ? g % SLOTS : 0;
         for (int i = g; ok; i += G, ++n) {
-            const int slot = i & (SLOTS - 1);
             if (n > 0) {
                 s += G;
                 while (s >= NST) { s -= NST; ++lap; }
+                if (PARTIALS) {
+                    slot += G;
+                    while (slot >= SLOTS) slot -= SLOTS;
+                }
             }
-            DBG_LAP(5)
             if (!wwait(B_full(s), lap & 1u, 3)) { ok = false; break; }
-            DBG_LAP(0)
             const TileDesc td = s_desc[s];
             if (td.run < 0) {                                // no more tiles: the sums issuer hears it from the first group that does
                 if (PARTIALS && td.run_seq == 0) {          // (the first of the G end markers)
@@ -602,20 +557,14 @@ ws_fused_kernel(const __grid_constant__ CUtensorMap pmap, const float* __restric
             float xn;
             {
                 float n0 = 0.0f, n1 = 0.0f, n2 = 0.0f, n3 = 0.0f;   // four chains
-#ifdef EC_WS_EXP_NOXN
-                n0 = 1000.0f;
-#else
 #pragma unroll
                 for (int q = 0; q < Q; ++q) {
                     const float4 v = *reinterpret_cast<const float4*>(row + swz_off<D>(t, q));
                     n0 = fmaf(v.x, v.x, n0); n1 = fmaf(v.y, v.y, n1); n2 = fmaf(v.z, v.z, n2); n3 = fmaf(v.w, v.w, n3);
                 }
-#endif
                 xn = (n0 + n1) + (n2 + n3);
             }
-            DBG_LAP(1)
             if (!wwait(B_accfull(g), (uint32_t)n & 1u, 8)) { ok = false; break; }
-            DBG_LAP(2)
             fence_after_sync();
             float m1 = __int_as_float(0x7f800000), m2 = m1;
             {
@@ -640,7 +589,6 @@ ws_fused_kernel(const __grid_constant__ CUtensorMap pmap, const float* __restric
                 }
             }
             fence_before_sync();
-            DBG_LAP(3)
             warrive(B_accempty(g));                      // the accumulator may take the group's next tile
             int kb = (int)(__float_as_uint(m1) & 127u);
             const float tau = TAU_SCALE * (xn + cmax);
@@ -674,7 +622,7 @@ ws_fused_kernel(const __grid_constant__ CUtensorMap pmap, const float* __restric
                 const bool any_w = __any_sync(0xffffffffu, changed);
                 // the sums issuer must have taken what the group said about its previous tile
                 if (n > 0 && !wwait(B_tiledone(g), (uint32_t)(n - 1) & 1u, 10 | (i << 8))) { ok = false; break; }
-                // Two groups take turns on a slot.  Once the sums issuer is through with tile i - SLOTS (the slot's last possible
+                // The groups take turns on the slots.  Once the sums issuer is through with tile i - SLOTS (the slot's last possible
                 // user before this tile) the slot's book-keeping is final: whether the rows of this warp's position still have
                 // one-hot entries set (they must be cleared before the slot's next GEMM), and how many GEMMs were issued from
                 // the slot, which says which phase of its barrier to wait for before the operands may be touched - at most one
@@ -744,10 +692,6 @@ ws_fused_kernel(const __grid_constant__ CUtensorMap pmap, const float* __restric
                 warrive(B_decided(g));
             }
             warrive(B_empty(s));                         // the stage may take another tile
-            DBG_LAP(4)
-#ifdef EC_WS_DEBUG
-            ++dbg_n;
-#endif
             if (PARTIALS && td.last) {
                 // the run's last tile: its group writes the run's sums out once the sums issuer is through the run
                 // (first until the sums issuer has signalled the end of this run: it has then seen the run before last written
@@ -797,21 +741,11 @@ ws_fused_kernel(const __grid_constant__ CUtensorMap pmap, const float* __restric
                 if (DELTA && t == 0) dirty[td.run] = had_sums ? 1u : 0u;
             }
         }
-#ifdef EC_WS_DEBUG
-        if (blockIdx.x == 0 && (tid & 127) == 5)
-            printf("group %d tiles %d: wait full %lld, xn %lld, wait acc %lld, ld+track %lld, rest %lld, loop %lld (cycles per tile)\n", g, dbg_n,
-                   dbg_t[0] / (dbg_n + 1), dbg_t[1] / (dbg_n + 1), dbg_t[2] / (dbg_n + 1), dbg_t[3] / (dbg_n + 1), dbg_t[4] / (dbg_n + 1), dbg_t[5] / (dbg_n + 1));
-#endif
     }
     if (!ok && *s_abort == 0) *s_abort = 15;
     fence_before_sync();
     __syncthreads();
     if (tid == 0 && *s_abort != 0 && status != nullptr) atomicCAS(status, 0u, 2u | (((uint32_t)*s_abort & 0xFFFu) << 4) | ((uint32_t)s_ctrl[24] << 16));   // the first block to report stays
-#ifdef EC_WS_DEBUG
-    if (tid == 0 && *s_abort != 0)
-        printf("block %d abort %x ctrl %d %d %d %d had %d %d sums %x votes %d %d %d | %d %d %d\n", blockIdx.x, *s_abort, s_ctrl[0], s_ctrl[1], s_ctrl[2],
-               s_ctrl[3], s_ctrl[4], s_ctrl[5], s_ctrl[24], s_vote[0], s_vote[1], s_vote[2], s_vote[6], s_vote[7], s_vote[8]);
-#endif
     if (warp == 4 * G + 1) {
         fence_after_sync();
         tmem_dealloc(tmem_base, pl.tmem_cols);
