@@ -251,6 +251,58 @@ __device__ __forceinline__ void best_two_of_16(const uint32_t (&raw)[16], float&
     c2 = fminf(hi_min, fmaxf(a, b));
 }
 
+// The search cannot separate the best candidates of some point of this warp (redo: of this thread's point).  The true
+// nearest centroid's score is within tau of the best score (each score is within tau / 2 of its exact value), so the
+// exact form sum_d (x - c)^2 decides among the columns with v <= lim = best + tau alone.  The scores are read once more
+// (all lanes: the read is warp-wide) and every thread notes its candidates, up to four column numbers packed in a word;
+// then each thread works through its own list - no thread waits for another's columns.  Candidates are taken in
+// ascending order with strict <, so the lowest index wins an exact tie as it does over all centroids; a point with
+// more than four candidates is decided over all centroids.
+template <int D>
+__device__ __noinline__ int redecide(bool redo, int kb, float lim, const unsigned char* row0, int t, uint32_t col0, int npad,
+                                     const float* __restrict__ centroids, int K) {
+    constexpr int Q = D / 4;
+    uint32_t cand = 0;
+    int cnt = 0;
+    for (int ch = 0; ch < npad / 16; ++ch) {
+        uint32_t vv[16];
+        tmem_ld16_nowait(col0 + (uint32_t)(ch * 16), vv);
+        tmem_ld_wait();
+#pragma unroll
+        for (int e = 0; e < 16; ++e) {
+            const bool in = __uint_as_float(vv[e]) <= lim && ch * 16 + e < K;
+            cand = in ? (cand << 8) | (uint32_t)(ch * 16 + e) : cand;     // (column numbers are below 128)
+            cnt += in ? 1 : 0;
+        }
+    }
+    if (!redo) return kb;
+    float x[D];
+    const unsigned char* row = row0 - swz_off<D>(t, 0);
+#pragma unroll
+    for (int q = 0; q < Q; ++q) {
+        const float4 v = *reinterpret_cast<const float4*>(row + swz_off<D>(t, q));
+        x[4 * q] = v.x; x[4 * q + 1] = v.y; x[4 * q + 2] = v.z; x[4 * q + 3] = v.w;
+    }
+    if (cnt > 4 || cnt == 0) return tc::exact_argmin_global<D>(x, centroids, K);
+    float best = __int_as_float(0x7f800000);
+    for (int s = cnt - 1; s >= 0; --s) {                 // the first candidate noted sits highest in the word
+        const int k = (int)((cand >> (8 * s)) & 0xFFu);
+        const float4* c = reinterpret_cast<const float4*>(centroids + (size_t)k * D);
+        float d0 = 0.0f;
+#pragma unroll
+        for (int q = 0; q < Q; ++q) {
+            const float4 a = __ldg(c + q);
+            float u;
+            u = x[4 * q] - a.x; d0 = fmaf(u, u, d0);
+            u = x[4 * q + 1] - a.y; d0 = fmaf(u, u, d0);
+            u = x[4 * q + 2] - a.z; d0 = fmaf(u, u, d0);
+            u = x[4 * q + 3] - a.w; d0 = fmaf(u, u, d0);
+        }
+        if (d0 < best) { best = d0; kb = k; }
+    }
+    return kb;
+}
+
 template <int D, bool PARTIALS, bool DELTA, bool BOUNDS>
 __global__ void __launch_bounds__(MAX_THREADS, 1)
 ws_fused_kernel(const __grid_constant__ CUtensorMap pmap, const float* __restrict__ points, size_t N, int P, int C,
@@ -588,20 +640,13 @@ ws_fused_kernel(const __grid_constant__ CUtensorMap pmap, const float* __restric
                     m1 = fminf(m1, c1);
                 }
             }
-            fence_before_sync();
-            warrive(B_accempty(g));                      // the accumulator may take the group's next tile
             int kb = (int)(__float_as_uint(m1) & 127u);
             const float tau = TAU_SCALE * (xn + cmax);
             const bool redo = live && !(m2 - m1 > tau);
-            if (redo) {
-                float x[D];
-#pragma unroll
-                for (int q = 0; q < Q; ++q) {
-                    const float4 v = *reinterpret_cast<const float4*>(row + swz_off<D>(t, q));
-                    x[4 * q] = v.x; x[4 * q + 1] = v.y; x[4 * q + 2] = v.z; x[4 * q + 3] = v.w;
-                }
-                kb = tc::exact_argmin_global<D>(x, centroids, K);
-            }
+            if (__any_sync(0xffffffffu, redo))            // rare on separated data: kept out of line, away from this loop's registers
+                kb = redecide<D>(redo, kb, m1 + tau, row + swz_off<D>(t, 0), t, lane_base + (uint32_t)(g * npad), npad, centroids, K);
+            fence_before_sync();
+            warrive(B_accempty(g));                      // the accumulator may take the group's next tile
             const bool changed = live && !(DELTA && old == kb);
             if (changed) labels[j] = kb;
             if (PARTIALS && BOUNDS && live) {
