@@ -202,8 +202,8 @@ int ec_allreduce_epoch_host(ec_ctx_t* ctx, const void* const* host_rank_bufs, co
 int ec_allreduce_set_tile(ec_ctx_t* ctx, int threads, size_t tile_elems);
 
 /* Expert knob: 1 = the tiles of the rank buffers are staged through shared memory
- * by bulk asynchronous copies (the default for up to 64 ranks in fixed or ring
- * order; EC_ERR_UNSUPPORTED for other contexts); 0 = they are read with direct
+ * by bulk asynchronous copies (the default for up to 64 ranks, in every order;
+ * EC_ERR_UNSUPPORTED for more ranks); 0 = they are read with direct
  * 128-bit loads.  Calls that cannot take the 128-bit path, and short segments,
  * use the direct kernels whatever the setting.  Affects speed only, never results. */
 int ec_allreduce_set_path(ec_ctx_t* ctx, int path);

@@ -769,6 +769,280 @@ apply_bulk_kernel(const ApplyArgs a, const __grid_constant__ PtrTable<64> tbl) {
     }
 }
 
+// ---------------------------------------------------------------------------------------------
+// the pairwise tree with bulk-copy staging: up to 64 ranks on the 128-bit path
+// ---------------------------------------------------------------------------------------------
+// The same balanced tree over the rank index as apply_kernel's pairwise branch (leaves eight ranks at a time, the
+// subtrees merged by a binary counter: the additions of the recursive halving tree, bit for bit), but no load is held in
+// a register.  A stage of shared memory takes the tiles (2 KB each) of the new ranks of one leaf block of eight, fetched
+// by bulk asynchronous copies that report to the stage's mbarrier; the next leaf block's stage is under way while the
+// threads reduce the one at hand out of shared memory and push it onto their binary counter.  Every wait is bounded;
+// once one gives up the block stops staging and reads the remaining leaf blocks directly.  Shape by measurement on
+// 32 bf16 ranks x 2^25 and 16 fp32 ranks x 2^24, all at once (threads / tile bytes / stages -> GB/s): 128/2048/2 6033
+// and 6642; 64/1024/2 5702, 6733; 128/2048/3 5322, 5253; 256/4096/3 5203, 5115; 256/4096/2 5112, 6530; one stage 4133,
+// 4682; all tiles of a block behind one barrier (no pipeline) 3290, 3915; the direct-load tree 4640, 6106.
+#ifndef EC_PW_THREADS
+#define EC_PW_THREADS 128
+#endif
+#ifndef EC_PW_TILE_BYTES
+#define EC_PW_TILE_BYTES 2048
+#endif
+#ifndef EC_PW_STAGES
+#define EC_PW_STAGES 2
+#endif
+constexpr int PW_THREADS = EC_PW_THREADS;
+constexpr int PW_TILE_BYTES = EC_PW_TILE_BYTES;
+constexpr int PW_STAGES = EC_PW_STAGES;
+constexpr int PW_SMEM = PW_STAGES * 8 * PW_TILE_BYTES;
+
+// One tree, rank by rank from global memory: fetch(r, out) delivers the PVU values of new rank r.
+template <class Acc, int PVU, class Fetch>
+__device__ __forceinline__ void pw_tree(uint64_t word, int P, Fetch fetch, Acc (&node)[PVU]) {
+    int P2 = 1;
+    while (P2 < P) P2 <<= 1;
+    const int leaf = P2 < 8 ? P2 : 8;
+    const int nblk = P2 / leaf;
+    int nlev = 0;
+    while ((1 << nlev) < nblk) ++nlev;
+    Acc stack[3][PVU];
+    for (int blk = 0; blk < nblk; ++blk) {
+        const int r0 = blk * leaf;
+        const unsigned byte = (unsigned)(word >> r0) & ((1u << leaf) - 1u);
+        Acc lv[8][PVU];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+#pragma unroll
+            for (int e = 0; e < PVU; ++e) lv[u][e] = ident<EC_SUM>(Acc());
+            if ((byte >> u) & 1u) fetch(r0 + u, lv[u]);
+        }
+#pragma unroll
+        for (int e = 0; e < PVU; ++e) {
+            if (leaf == 8)
+                node[e] = comb<EC_SUM>(comb<EC_SUM>(comb<EC_SUM>(lv[0][e], lv[1][e]), comb<EC_SUM>(lv[2][e], lv[3][e])),
+                                       comb<EC_SUM>(comb<EC_SUM>(lv[4][e], lv[5][e]), comb<EC_SUM>(lv[6][e], lv[7][e])));
+            else if (leaf == 4)
+                node[e] = comb<EC_SUM>(comb<EC_SUM>(lv[0][e], lv[1][e]), comb<EC_SUM>(lv[2][e], lv[3][e]));
+            else if (leaf == 2)
+                node[e] = comb<EC_SUM>(lv[0][e], lv[1][e]);
+            else
+                node[e] = lv[0][e];
+        }
+        bool carry = true;
+#pragma unroll
+        for (int l = 0; l < 3; ++l) {
+            if (l < nlev && carry) {
+                if ((blk >> l) & 1) {
+#pragma unroll
+                    for (int e = 0; e < PVU; ++e) node[e] = comb<EC_SUM>(stack[l][e], node[e]);
+                } else {
+#pragma unroll
+                    for (int e = 0; e < PVU; ++e) stack[l][e] = node[e];
+                    carry = false;
+                }
+            }
+        }
+    }
+}
+
+template <int DT>
+__global__ void __launch_bounds__(PW_THREADS)
+apply_pw_bulk_kernel(const ApplyArgs a, const __grid_constant__ PtrTable<64> tbl) {
+    typedef Elem<DT> E;
+    typedef typename E::In In;
+    typedef typename E::Acc Acc;
+    constexpr int PV = E::VEC > 4 ? 4 : E::VEC;                        // elements per tree walk (at most four accumulators per node)
+    constexpr int UNIT_BYTES = PV * (int)sizeof(In);
+    constexpr int UPT = PW_TILE_BYTES / UNIT_BYTES / PW_THREADS;       // units per thread: 1 (fp32, fp64) or 2 (bf16)
+    static_assert(UPT >= 1 && UPT * UNIT_BYTES * PW_THREADS == PW_TILE_BYTES, "a tile is a whole number of units per thread");
+
+    extern __shared__ __align__(128) unsigned char pw_stage[];         // [PW_STAGES][8 ranks][PW_TILE_BYTES]
+    __shared__ uint16_t s_rank[64];
+    __shared__ uint64_t s_new[MAX_W];
+    __shared__ int s_m, s_fresh, s_gave_up;
+    __shared__ __align__(8) uint64_t s_bar[PW_STAGES];
+
+    const unsigned s = blockIdx.x / a.tiles_per_seg;
+    const unsigned t = blockIdx.x - s * a.tiles_per_seg;
+    const size_t lo = (size_t)s * a.seg + (size_t)t * a.tile;
+    size_t seg_hi = (size_t)(s + 1) * a.seg;
+    if (seg_hi > a.n) seg_hi = a.n;
+    const int tid = threadIdx.x;
+    if (tid == 0) {
+        s_gave_up = 0;
+#pragma unroll
+        for (int q = 0; q < PW_STAGES; ++q)
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bk_smem(&s_bar[q])) : "memory");
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (tid < 32) block_prologue(a, s, t, s_rank, s_new, &s_m, &s_fresh);
+    __syncthreads();
+    const int m = s_m;
+    const bool fresh = s_fresh != 0;
+    if (m == 0 && !(fresh && a.first_apply)) return;
+    if (lo >= seg_hi) return;
+    size_t hi = lo + a.tile;
+    if (hi > seg_hi) hi = seg_hi;
+    const size_t cnt = hi - lo;
+    const uint32_t bytes = (uint32_t)(cnt * sizeof(In) / 16) * 16u;    // staged part of a rank's tile: whole 16-byte vectors
+    const int nunits = (int)(bytes / UNIT_BYTES);
+    Acc* res = reinterpret_cast<Acc*>(a.result) + lo;
+    const uint64_t pol = evict_first_policy();
+    const uint64_t rpol_ld = result_policy(1), rpol_st = result_policy(a.res_hint == 2 ? 2 : 1);
+    const uint64_t word = s_new[0];
+    int P2 = 1;
+    while (P2 < a.P) P2 <<= 1;
+    const int leaf = P2 < 8 ? P2 : 8;
+    const int nblk = P2 / leaf;
+    int nlev = 0;
+    while ((1 << nlev) < nblk) ++nlev;
+
+    // thread 0 issues, for leaf block b, one copy per new rank of the block into stage b % PW_STAGES, side by side
+    auto issue = [&](int b) {
+        const int r0 = b * leaf;
+        const unsigned byte = (unsigned)(word >> r0) & ((1u << leaf) - 1u);
+        if (byte == 0u || bytes == 0u) return;
+        const uint32_t bar = bk_smem(&s_bar[b % PW_STAGES]);
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes * (uint32_t)__popc(byte)) : "memory");
+        unsigned char* dst = pw_stage + (size_t)(b % PW_STAGES) * 8 * PW_TILE_BYTES;
+        for (unsigned rest = byte; rest != 0u; rest &= rest - 1u) {
+            const int u = __ffs((int)rest) - 1;
+            asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+                         ::"r"(bk_smem(dst)), "l"(reinterpret_cast<const char*>(tbl.p[r0 + u]) + lo * sizeof(In)), "r"(bytes), "r"(bar), "l"(pol)
+                         : "memory");
+            dst += PW_TILE_BYTES;
+        }
+    };
+    if (tid == 0)
+        for (int b = 0; b < nblk && b < PW_STAGES; ++b) issue(b);
+
+    Acc node[UPT][PV], stack[UPT][3][PV];
+    bool direct = false;
+    uint32_t waits[PW_STAGES];                                          // completed phases of every stage's barrier so far
+#pragma unroll
+    for (int q = 0; q < PW_STAGES; ++q) waits[q] = 0u;
+    for (int blk = 0; blk < nblk; ++blk) {
+        const int r0 = blk * leaf, st = blk % PW_STAGES;
+        const unsigned byte = (unsigned)(word >> r0) & ((1u << leaf) - 1u);
+        bool staged = false;
+        if (byte != 0u && bytes != 0u && !direct) {
+            uint32_t par = 0u;
+#pragma unroll
+            for (int q = 0; q < PW_STAGES; ++q)
+                if (q == st) { par = waits[q] & 1u; ++waits[q]; }
+            staged = bk_wait(bk_smem(&s_bar[st]), par);
+            if (!staged) *reinterpret_cast<volatile int*>(&s_gave_up) = 1;
+        }
+        const unsigned char* sbase = pw_stage + (size_t)st * 8 * PW_TILE_BYTES;
+#pragma unroll
+        for (int q = 0; q < UPT; ++q) {
+            const int w = q * PW_THREADS + tid;
+            Acc lv[8][PV];
+            if (w < nunits) {
+                auto from_stage = [&](int slot, Acc (&out)[PV]) {
+                    const unsigned char* src = sbase + (size_t)slot * PW_TILE_BYTES + (size_t)w * UNIT_BYTES;
+                    if constexpr (DT == EC_BF16) {
+                        const uint2 r = *reinterpret_cast<const uint2*>(src);
+                        out[0] = __uint_as_float(r.x << 16); out[1] = __uint_as_float(r.x & 0xFFFF0000u);
+                        out[2] = __uint_as_float(r.y << 16); out[3] = __uint_as_float(r.y & 0xFFFF0000u);
+                    } else {
+                        E::unpack(*reinterpret_cast<const uint4*>(src), out);
+                    }
+                };
+                auto from_global = [&](int r, Acc (&out)[PV]) {
+                    const char* src = reinterpret_cast<const char*>(tbl.p[r]) + lo * sizeof(In) + (size_t)w * UNIT_BYTES;
+                    if constexpr (DT == EC_BF16) {
+                        const uint2 v = ld_stream8(src, pol);
+                        out[0] = __uint_as_float(v.x << 16); out[1] = __uint_as_float(v.x & 0xFFFF0000u);
+                        out[2] = __uint_as_float(v.y << 16); out[3] = __uint_as_float(v.y & 0xFFFF0000u);
+                    } else {
+                        E::unpack(ld_stream16(src, pol), out);
+                    }
+                };
+                if (staged && leaf == 8 && byte == 0xFFu) {             // all eight ranks new: the usual case in a first apply
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) from_stage(u, lv[u]);
+                } else {
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+#pragma unroll
+                        for (int e = 0; e < PV; ++e) lv[u][e] = ident<EC_SUM>(Acc());
+                        if ((byte >> u) & 1u) {
+                            if (staged) from_stage(__popc(byte & ((1u << u) - 1u)), lv[u]);
+                            else from_global(r0 + u, lv[u]);
+                        }
+                    }
+                }
+#pragma unroll
+                for (int e = 0; e < PV; ++e) {
+                    if (leaf == 8)
+                        node[q][e] = comb<EC_SUM>(comb<EC_SUM>(comb<EC_SUM>(lv[0][e], lv[1][e]), comb<EC_SUM>(lv[2][e], lv[3][e])),
+                                                  comb<EC_SUM>(comb<EC_SUM>(lv[4][e], lv[5][e]), comb<EC_SUM>(lv[6][e], lv[7][e])));
+                    else if (leaf == 4)
+                        node[q][e] = comb<EC_SUM>(comb<EC_SUM>(lv[0][e], lv[1][e]), comb<EC_SUM>(lv[2][e], lv[3][e]));
+                    else if (leaf == 2)
+                        node[q][e] = comb<EC_SUM>(lv[0][e], lv[1][e]);
+                    else
+                        node[q][e] = lv[0][e];
+                }
+                bool carry = true;
+#pragma unroll
+                for (int l = 0; l < 3; ++l) {
+                    if (l < nlev && carry) {
+                        if ((blk >> l) & 1) {
+#pragma unroll
+                            for (int e = 0; e < PV; ++e) node[q][e] = comb<EC_SUM>(stack[q][l][e], node[q][e]);
+                        } else {
+#pragma unroll
+                            for (int e = 0; e < PV; ++e) stack[q][l][e] = node[q][e];
+                            carry = false;
+                        }
+                    }
+                }
+            }
+        }
+        if (blk + 1 < nblk) {
+            __syncthreads();                                            // everybody is done with this stage
+            if (!direct && *reinterpret_cast<volatile int*>(&s_gave_up) != 0) direct = true;
+            if (tid == 0 && !direct && blk + PW_STAGES < nblk) issue(blk + PW_STAGES);
+        }
+    }
+    // node is the root now
+#pragma unroll
+    for (int q = 0; q < UPT; ++q) {
+        const int w = q * PW_THREADS + tid;
+        if (w < nunits) {
+            if (!fresh) {
+                Acc acc[PV];
+                load_acc<Acc, PV>(res + (size_t)w * PV, acc, rpol_ld);
+#pragma unroll
+                for (int e = 0; e < PV; ++e) node[q][e] = comb<EC_SUM>(acc[e], node[q][e]);
+            }
+            store_acc<Acc, PV>(res + (size_t)w * PV, node[q], rpol_st);
+        }
+    }
+    // elements after the last whole vector of a ragged tile: the same tree, element by element, from the rank buffers
+    for (size_t i = (size_t)nunits * PV + tid; i < cnt; i += PW_THREADS) {
+        Acc root[1];
+        pw_tree<Acc, 1>(word, a.P, [&](int r, Acc (&out)[1]) { out[0] = E::widen(reinterpret_cast<const In*>(tbl.p[r])[lo + i]); }, root);
+        res[i] = fresh ? root[0] : comb<EC_SUM>(res[i], root[0]);
+    }
+    // copies that were given up on, or issued ahead and never read, may still be on their way into this block's
+    // shared memory: thread 0 gives every stage's barrier one more bounded wait before the block retires
+    if (tid == 0 && *reinterpret_cast<volatile int*>(&s_gave_up) != 0) {
+#pragma unroll
+        for (int q = 0; q < PW_STAGES; ++q) bk_wait(bk_smem(&s_bar[q]), waits[q] & 1u);
+    }
+}
+
+template <int DT>
+int launch_pw_bulk(const ApplyArgs& a, const void* const* bufs, unsigned grid, cudaStream_t st) {
+    PtrTable<64> tbl;
+    for (int r = 0; r < 64; ++r) tbl.p[r] = r < a.P ? bufs[r] : nullptr;
+    apply_pw_bulk_kernel<DT><<<grid, PW_THREADS, PW_SMEM, st>>>(a, tbl);
+    EC_CUDA(cudaGetLastError());
+    return EC_OK;
+}
+
 template <int DT, int OP, bool VECTOR, int ORDER>
 int launch_cap(const ApplyArgs& a, const void* const* bufs, unsigned grid, int threads, bool short_seg, cudaStream_t st) {
     if (a.P <= 64) {
@@ -919,7 +1193,13 @@ int ec_allreduce_init(ec_ctx_t** out, int P, size_t n, ec_dtype_t dtype, ec_op_t
     }
     // Few ranks: many small blocks overlap their start-up latency best.  Hundreds of ranks: a block
     // lives long anyway and wider blocks read longer contiguous runs of each buffer (both measured).
-    c->path = (order != EC_ORDER_PAIRWISE && P <= 64) ? 1 : 0;
+    c->path = P <= 64 ? 1 : 0;
+    if (order == EC_ORDER_PAIRWISE && P <= 64 && PW_SMEM > 48 * 1024) {   // the limit of dynamic shared memory has to be raised
+        cudaError_t e2 = cudaFuncSetAttribute(apply_pw_bulk_kernel<EC_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, PW_SMEM);
+        if (e2 == cudaSuccess) e2 = cudaFuncSetAttribute(apply_pw_bulk_kernel<EC_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, PW_SMEM);
+        if (e2 == cudaSuccess) e2 = cudaFuncSetAttribute(apply_pw_bulk_kernel<EC_F64>, cudaFuncAttributeMaxDynamicSharedMemorySize, PW_SMEM);
+        if (e2 != cudaSuccess) { cudaGetLastError(); c->path = 0; }
+    }
     c->threads = P > 64 ? 256 : 128;
     c->tile = dtype == EC_BF16 ? 2048 : 8192 / in_bytes(dtype);   // 8 KB of every rank buffer per block (4 KB for bf16), measured
     *out = c;
@@ -928,7 +1208,7 @@ int ec_allreduce_init(ec_ctx_t** out, int P, size_t n, ec_dtype_t dtype, ec_op_t
 
 int ec_allreduce_set_path(ec_ctx_t* c, int path) {
     if (!c || (path != 0 && path != 1)) return EC_ERR_INVALID;
-    if (path == 1 && (c->order == EC_ORDER_PAIRWISE || c->P > 64)) return EC_ERR_UNSUPPORTED;
+    if (path == 1 && c->P > 64) return EC_ERR_UNSUPPORTED;
     c->path = path;
     return EC_OK;
 }
@@ -984,6 +1264,19 @@ int apply_common(ec_ctx_t* c, const void* const* rank_bufs, int P, size_t n, ec_
         if (btiles * c->S > 0x7fffffffull) return EC_ERR_CAPACITY;
         a.tiles_per_seg = (unsigned)btiles;
         return launch_bulk(a, rank_bufs, c->dtype, c->op, (unsigned)(btiles * c->S), stream);
+    }
+    if (c->path == 1 && vector && c->order == EC_ORDER_PAIRWISE && c->P <= 64 && a.notif_clock == nullptr) {
+        // the pairwise tree out of bulk-staged tiles: 2 KB of every rank per block
+        a.tile = PW_TILE_BYTES / in_bytes(c->dtype);
+        const size_t ptiles = (seg_len + a.tile - 1) / a.tile;
+        if (ptiles * c->S > 0x7fffffffull) return EC_ERR_CAPACITY;
+        a.tiles_per_seg = (unsigned)ptiles;
+        const unsigned pgrid = (unsigned)(ptiles * c->S);
+        switch (c->dtype) {
+            case EC_F32: return launch_pw_bulk<EC_F32>(a, rank_bufs, pgrid, stream);
+            case EC_BF16: return launch_pw_bulk<EC_BF16>(a, rank_bufs, pgrid, stream);
+            case EC_F64: return launch_pw_bulk<EC_F64>(a, rank_bufs, pgrid, stream);
+        }
     }
     switch (c->dtype) {
         case EC_F32: return launch_dt<EC_F32>(a, rank_bufs, c->op, vector, c->order, grid, c->threads, short_seg, stream);
