@@ -760,7 +760,7 @@ def mf_case(dev, stream, iters=20):
     return out
 
 
-def kmeans_case(dev, stream, reps=5, iters=20, profile_only=False):
+def kmeans_case(dev, stream, reps=5, iters=20, profile_only=False, bounds=True, refresh=32):
     """Config 5: N = 2^22 points, D = 32, K = 64, P = 64 ranks, 20 Lloyd iterations with seeded masks."""
     import torch
     from paper_2203_17063_b200 import binding as ec
@@ -773,6 +773,9 @@ def kmeans_case(dev, stream, reps=5, iters=20, profile_only=False):
     d_pts = torch.from_numpy(pts).to(dev)
     d_init = torch.from_numpy(init).to(dev)
     km = ec.KMeans(d_pts, K, P, d_init)
+    if profile_only:                 # which leg a profiler capture looks at: distance bounds on / off, sums afresh every `refresh`
+        km.set_bounds(bounds)
+        km.set_refresh(refresh)
     with torch.cuda.stream(stream):
         for t in range(3):
             km.iterate_raw(masks[t].data_ptr(), st)
@@ -780,7 +783,7 @@ def kmeans_case(dev, stream, reps=5, iters=20, profile_only=False):
         first_ms = []
         for rep in range(reps):
             km.set_centroids(d_init, stream)
-            km.set_refresh(32)          # forgets labels and running sums: every repetition is a fresh run of 20 iterations
+            km.set_refresh(refresh)     # forgets labels and running sums: every repetition is a fresh run of 20 iterations
             a, b, c = (torch.cuda.Event(enable_timing=True) for _ in range(3))
             a.record(stream)
             km.iterate_raw(masks[0].data_ptr(), st)
@@ -958,6 +961,8 @@ def main():
                     help="direct: force the direct-load apply kernel (ec_allreduce_set_path(0)) where bulk staging is the default")
     ap.add_argument("--workload", default="headline", choices=["headline", "kmeans", "mf"],
                     help="kmeans: time only the K-means driver (config 5) and print its own JSON line")
+    ap.add_argument("--kmeans-bounds", default="on", choices=["on", "off"], help="with --workload kmeans --profile-only: distance bounds")
+    ap.add_argument("--kmeans-refresh", type=int, default=32, help="with --workload kmeans --profile-only: all points summed every N-th iteration")
     ap.add_argument("--cpu-seconds", type=float, default=15.0, help="time budget of the CPU baseline leg")
     ap.add_argument("--threads", type=int, default=0, help="expert: threads per block of the apply kernel")
     ap.add_argument("--tile", type=int, default=0, help="expert: elements per block of the apply kernel")
@@ -977,7 +982,8 @@ def main():
         torch.cuda.set_device(local_rank)
         dev = torch.device("cuda", local_rank)
         print(json.dumps({"workload": "kmeans", **kmeans_case(dev, torch.cuda.Stream(device=dev), reps=max(1, min(args.steps, 5)),
-                                                               profile_only=args.profile_only)}))
+                                                               profile_only=args.profile_only, bounds=args.kmeans_bounds == "on",
+                                                               refresh=args.kmeans_refresh)}))
         return
     if args.workload == "mf":
         import torch
