@@ -230,12 +230,15 @@ __device__ __forceinline__ void tmem_ld16_nowait(uint32_t taddr, uint32_t (&r)[1
 // caller adds the number of the group of 16): sorted pairs, then the same again on the smaller halves; the second best
 // is the smallest of all the larger halves (the partner of the winner is among them, and every other larger half is at
 // least the second best of the smaller ones).  16 at a time, so that the next 16 can be on their way from tensor memory.
-__device__ __forceinline__ void best_two_of_16(const uint32_t (&raw)[16], float& c1, float& c2) {
+// (raw & mask) | tag is ONE logic instruction when the mask comes in a register (two immediates would take two).
+__device__ __forceinline__ void best_two_of_16(const uint32_t (&raw)[16], uint32_t mask, float& c1, float& c2) {
     float lo[8], hi[8];
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
-        const float a = __uint_as_float((raw[2 * i] & 0xFFFFFF80u) | (uint32_t)(2 * i));
-        const float b = __uint_as_float((raw[2 * i + 1] & 0xFFFFFF80u) | (uint32_t)(2 * i + 1));
+        uint32_t ra, rb;
+        asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(ra) : "r"(raw[2 * i]), "r"(mask), "r"((uint32_t)(2 * i)));
+        asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(rb) : "r"(raw[2 * i + 1]), "r"(mask), "r"((uint32_t)(2 * i + 1)));
+        const float a = __uint_as_float(ra), b = __uint_as_float(rb);
         lo[i] = fminf(a, b);
         hi[i] = fmaxf(a, b);
     }
@@ -568,12 +571,12 @@ ws_fused_kernel(const __grid_constant__ CUtensorMap pmap, const float* __restric
         float cmax = 0.0f;
         for (int k = 0; k < K; ++k) cmax = fmaxf(cmax, s_cn[k]);
         const float drift_max = (PARTIALS && BOUNDS) ? drift[K] : 0.0f;
-        // One lane per warp waits and arrives for its warp (the barriers of the groups count warps, not threads):
-        // 32 times fewer barrier operations, and the warp's other lanes are ordered behind lane 0 by the shuffle.
+        uint32_t tag_mask;                                    // 0xFFFFFF80, kept in a register (see best_two_of_16)
+        asm volatile("mov.u32 %0, 0xFFFFFF80;" : "=r"(tag_mask));
+        // One lane per warp arrives for its warp (the barriers of the groups count warps, not threads): 32 times fewer
+        // barrier operations; all lanes wait (the same instruction count as one lane waiting, without the divergence).
         auto wwait = [&](uint32_t bar, uint32_t par, int where) -> bool {
-            int r = 1;
-            if (lane == 0) r = wait_or_abort(bar, par, s_abort, where) ? 1 : 0;
-            return __shfl_sync(0xffffffffu, r, 0) != 0;
+            return __all_sync(0xffffffffu, wait_or_abort(bar, par, s_abort, where)) != 0;   // (all lanes: one instruction either way, no divergence)
         };
         auto warrive = [&](uint32_t bar) {
             __syncwarp();
@@ -628,13 +631,13 @@ ws_fused_kernel(const __grid_constant__ CUtensorMap pmap, const float* __restric
                     float c1, c2;
                     tmem_ld_wait();
                     tmem_ld16_nowait(col0 + (uint32_t)(ch * 16 + 16), vb);
-                    best_two_of_16(va, c1, c2);              // tags 0..15; bits 4-6 (zero so far) take the chunk number
+                    best_two_of_16(va, tag_mask, c1, c2);    // tags 0..15; bits 4-6 (zero so far) take the chunk number
                     c1 = __uint_as_float(__float_as_uint(c1) | (uint32_t)(ch << 4));
                     m2 = min3(m2, c2, fmaxf(m1, c1));
                     m1 = fminf(m1, c1);
                     tmem_ld_wait();
                     if (ch + 2 < npad / 16) tmem_ld16_nowait(col0 + (uint32_t)(ch * 16 + 32), va);
-                    best_two_of_16(vb, c1, c2);
+                    best_two_of_16(vb, tag_mask, c1, c2);
                     c1 = __uint_as_float(__float_as_uint(c1) | (uint32_t)((ch + 1) << 4));
                     m2 = min3(m2, c2, fmaxf(m1, c1));
                     m1 = fminf(m1, c1);
