@@ -25,7 +25,10 @@ namespace {
 #ifndef EC_GV_CHUNK
 #define EC_GV_CHUNK 65536
 #endif
-constexpr int GV_THREADS = 256;
+#ifndef EC_GV_THREADS
+#define EC_GV_THREADS 256
+#endif
+constexpr int GV_THREADS = EC_GV_THREADS;
 constexpr size_t GV_CHUNK_BYTES = EC_GV_CHUNK;
 constexpr int GV_BATCH = EC_GV_BATCH;  // loads in flight per thread before the stores
 
