@@ -347,7 +347,9 @@ int ec_kmeans_set_refresh(ec_kmeans_t* km, int every);
 int ec_kmeans_set_bounds(ec_kmeans_t* km, int enable);
 
 /* Expert knob: which kernel ec_kmeans_iterate / ec_kmeans_assign use.
- *   0  automatic: the fastest one that covers the shape (default);
+ *   0  automatic: the fastest one that covers the shape (default); where both tensor-core kernels do, the kernel of 2
+ *      for the assignment alone and for iterations that sum only changes, the kernel of 3 for an iteration that sums
+ *      every point;
  *   1  fp32 fused kernel: candidate search by one FMA per (point, centroid, coordinate);
  *   2  tensor cores (D in {16, 32}, K <= 256): for K <= 128 the warp-specialised kernel - the fp32 points go from
  *      global to shared memory by bulk tensor copies and are multiplied as they lie (tcgen05, tf32) - otherwise

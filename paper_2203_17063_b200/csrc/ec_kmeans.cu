@@ -864,7 +864,12 @@ int km_ws_launch(ec_kmeans* km, bool partials, const float* centroids, int32_t* 
 }
 
 int km_fused(ec_kmeans* km, bool partials, const float* centroids, int32_t* labels, cudaStream_t st, bool delta = false) {
-    if (km->ws_ok && km->path != 1 && km->path != 3) {
+    // Automatic choice between the two tensor-core kernels: the warp-specialised one for the assignment alone and for the
+    // passes that sum only changes (config 5: 0.109 against 0.136 ms, 5980 against 4851 iterations/s), the register-staged
+    // one for a pass that sums every point (0.253-0.268 against 0.313-0.320 ms: there every row has to be converted
+    // for the sums GEMM anyway, and its four independent blocks per SM overlap that better than one block's slots do).
+    const bool full_pass = partials && !delta;
+    if (km->ws_ok && km->path != 1 && km->path != 3 && !(km->path == 0 && full_pass)) {
         switch (km->D) {
             case 16: return km_ws_launch<16>(km, partials, centroids, labels, st, delta);
             case 32: return km_ws_launch<32>(km, partials, centroids, labels, st, delta);

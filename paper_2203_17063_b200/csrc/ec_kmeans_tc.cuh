@@ -266,6 +266,50 @@ bounds_check_kernel(size_t N, int P, int C, int K, const int32_t* __restrict__ l
     }
 }
 
+// Some point of this warp has its two best scores closer than the search's error bound (redo: this thread's point
+// has).  The true nearest centroid's score is within tau of the best score, so the exact form decides among the columns
+// with v <= lim = best + tau alone.  The scores are read once more from tensor memory (all lanes: the read is warp-wide),
+// every thread notes its candidates - up to four column numbers packed in a word - and then works through its own list
+// in ascending order with strict <, so the lowest index wins an exact tie as it does over all centroids; a point with
+// more than four candidates is decided over all centroids.
+template <int D>
+__device__ __noinline__ int redecide_candidates(bool redo, int kb, float lim, const float* __restrict__ points, size_t j,
+                                                uint32_t col0, int npad, const float* __restrict__ centroids, int K) {
+    uint32_t cand = 0;
+    int cnt = 0;
+    for (int ch = 0; ch < npad / 32; ++ch) {
+        uint32_t vv[32];
+        tmem_ld32(col0 + (uint32_t)(ch * 32), vv);
+#pragma unroll
+        for (int e = 0; e < 32; ++e) {
+            const bool in = __uint_as_float(vv[e]) <= lim && ch * 32 + e < K;
+            cand = in ? (cand << 8) | (uint32_t)(ch * 32 + e) : cand;
+            cnt += in ? 1 : 0;
+        }
+    }
+    if (!redo) return kb;
+    float x[D];
+    load_point<D>(points, j, x);
+    if (cnt > 4 || cnt == 0) return exact_argmin_global<D>(x, centroids, K);
+    float best = __int_as_float(0x7f800000);
+    for (int s = cnt - 1; s >= 0; --s) {                 // the first candidate noted sits highest in the word
+        const int k = (int)((cand >> (8 * s)) & 0xFFu);
+        const float4* c = reinterpret_cast<const float4*>(centroids + (size_t)k * D);
+        float d0 = 0.0f;
+#pragma unroll
+        for (int q = 0; q < D / 4; ++q) {
+            const float4 a = __ldg(c + q);
+            float u;
+            u = x[4 * q] - a.x; d0 = fmaf(u, u, d0);
+            u = x[4 * q + 1] - a.y; d0 = fmaf(u, u, d0);
+            u = x[4 * q + 2] - a.z; d0 = fmaf(u, u, d0);
+            u = x[4 * q + 3] - a.w; d0 = fmaf(u, u, d0);
+        }
+        if (d0 < best) { best = d0; kb = k; }
+    }
+    return kb;
+}
+
 template <int D, bool PARTIALS, bool DELTA, bool BOUNDS>
 __global__ void __launch_bounds__(THREADS, EC_TC_MINB)
 tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const float* __restrict__ centroids, int K,
@@ -546,10 +590,15 @@ tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const 
         // Delta mode: the row block receives only what changed since the labels were written last: +x for the
         // cluster a point joins, -x for the one it leaves (old label < 0: it was in none).  A tile in which no
         // label changed needs no sums MMA at all.  Otherwise every live point joins its cluster.
-        if (redo || (live && PARTIALS && !done)) {
+        if (done && __any_sync(0xffffffffu, redo))        // (the accumulator is still this tile's: the next MMA comes after the next barrier)
+        {
+            kb = redecide_candidates<D>(redo, kb, m1 + tau, points, j, tmem_lane, npad, centroids, K);
+            fence_before_sync();                         // these reads, too, come before the barrier that lets the next MMA start
+        }
+        if (live && !done) {
             float x[D];
-            load_point<D>(points, j, x);                 // rare: read the point again instead of keeping it in registers
-            if (redo) kb = exact_argmin_global<D>(x, centroids, K);
+            load_point<D>(points, j, x);                 // the tensor core is out of service: plain fp32 for this point
+            kb = exact_argmin_global<D>(x, centroids, K);
             if (PARTIALS && !done && !(delta && old == kb)) {   // tensor core out of service: add this point by hand
 #pragma unroll
                 for (int d = 0; d < D; ++d) atomicAdd(row_block + (size_t)kb * stride + d, x[d]);
