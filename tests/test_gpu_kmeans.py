@@ -35,12 +35,14 @@ def rows_close(g, c, rel=1e-4):
     return (num <= rel * den + 1e-30).all()
 
 
-def lockstep(N, D, K, P, iters, seed, p_arrive=0.75):
+def lockstep(N, D, K, P, iters, seed, p_arrive=0.75, path=None):
     points, comp, _ = inputs.kmeans_mixture(seed, N, D, K)
     cents = inputs.kmeans_first_of_component(points, comp, K)
     masks = inputs.kmeans_masks(seed + 1000, iters, P, K, p_arrive)
     d_points = to_dev(points)
     km = ec.KMeans(d_points, K, P, to_dev(cents))
+    if path is not None:
+        km.set_path(path)
     lab_all, d_labels = guarded(np.zeros(N, dtype=np.int32))           # sentinels on either side of the outputs
     part_all, d_part = guarded(np.zeros(P * K * (D + 4), dtype=np.float32))
     d_part = d_part.view(P, K, D + 4)
@@ -80,9 +82,19 @@ def test_lockstep_small():
 
 
 @pytest.mark.parametrize("N,D,K,P", [(5000, 8, 5, 3), (4099, 16, 7, 1), (3000, 4, 3, 7), (2048, 64, 9, 2),
-                                     (3001, 12, 6, 5), (2500, 128, 4, 2), (20000, 32, 200, 4)])
+                                     (3001, 12, 6, 5), (2500, 128, 4, 2), (20000, 32, 200, 4),
+                                     # the warp-specialised kernel with three and with two epilogue groups (96 and 128 score columns)
+                                     (9000, 32, 90, 3), (7001, 16, 128, 2), (6000, 32, 33, 5)])
 def test_lockstep_shapes(N, D, K, P):
     lockstep(N, D, K, P, iters=2, seed=77 + D)
+
+
+@pytest.mark.parametrize("path", [2, 3])
+@pytest.mark.parametrize("N,D,K,P", [(9000, 32, 90, 3), (7001, 16, 128, 2), (8000, 32, 64, 4)])
+def test_lockstep_each_tensor_core_kernel_on_its_own(N, D, K, P, path):
+    """The automatic choice mixes the two tensor-core kernels (one for passes that sum every point, one for the others);
+    here each does every kind of pass alone: 2 = warp-specialised, 3 = register-staged."""
+    lockstep(N, D, K, P, iters=3, seed=500 + K, path=path)
 
 
 def test_exact_ties_take_the_lowest_index():
@@ -183,7 +195,8 @@ def test_iteration_with_two_rounds_matches_checker():
     km.destroy()
 
 
-@pytest.mark.parametrize("N,D,K,P,iters", [(30000, 32, 16, 8, 40), (20011, 16, 200, 5, 8), (25000, 32, 64, 64, 8)])
+@pytest.mark.parametrize("N,D,K,P,iters", [(30000, 32, 16, 8, 40), (20011, 16, 200, 5, 8), (25000, 32, 64, 64, 8),
+                                           (26000, 32, 100, 4, 8), (24001, 16, 90, 3, 8)])
 def test_running_sums_follow_label_changes_over_many_iterations(N, D, K, P, iters):
     """The tensor-core path sums only what changed since the previous iteration (+x into the cluster a point joins,
     -x out of the one it leaves) and sums everything afresh every 32nd iteration.  With overlapping clusters and
