@@ -32,6 +32,22 @@
 namespace ec {
 namespace {
 
+// Programmatic dependent launch: a small kernel that follows a big one in the stream is launched while the big one's last
+// blocks are still running; it waits here, on the device, until its predecessor has completed and its writes are visible.
+// (Without the launch attribute the instruction returns at once.)
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <class... KArgs, class... Args>
+cudaError_t launch_dependent(void (*kernel)(KArgs...), unsigned grid, unsigned block, size_t smem, cudaStream_t stream, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid); cfg.blockDim = dim3(block); cfg.dynamicSmemBytes = smem; cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 constexpr int AS_THREADS = 256;
 constexpr int PT_THREADS = 256;
 constexpr int PT_WARPS = PT_THREADS / 32;
@@ -228,6 +244,7 @@ __global__ void partials_fold_kernel(const float* __restrict__ scratch, int C, s
                                      float* __restrict__ partials, int stride, int accumulate = 0,
                                      const uint32_t* __restrict__ dirty = nullptr,
                                      const uint32_t* __restrict__ any_work = nullptr) {
+    grid_dependency_wait();                                  // (launched ahead of its predecessor's end, see launch_dependent)
     if (any_work != nullptr && *any_work == 0u) return;      // the bounds check found no tile to search: nothing was written
     const int lane = threadIdx.x & 31;
     const size_t rows = total / (size_t)stride;
@@ -274,6 +291,7 @@ __global__ void partials_fold_kernel(const float* __restrict__ scratch, int C, s
 }
 
 __global__ void update_kernel(const float* __restrict__ reduced, int D, int K, float* __restrict__ centroids) {
+    grid_dependency_wait();
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= K * D) return;
     const int k = i / D, d = i - k * D;
@@ -288,6 +306,7 @@ constexpr int UD_THREADS = 1024;
 __global__ void __launch_bounds__(UD_THREADS)
 update_drift_kernel(const float* __restrict__ reduced, int D, int K, float* __restrict__ centroids, float* __restrict__ drift) {
     __shared__ float s_max[UD_THREADS / 32];
+    grid_dependency_wait();
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     float wmax = 0.0f;
     for (int k = wid; k < K; k += UD_THREADS / 32) {
@@ -1084,10 +1103,10 @@ int km_iterate_rounds(ec_kmeans_t* km, const uint64_t* const* masks, int rounds,
         if (rc != EC_OK) return rc;
         if (km->Cf > 1 || delta) {
             const size_t row = (size_t)km->K * (km->D + 4), total = row * km->P;
-            partials_fold_kernel<<<(unsigned)(((size_t)km->P * km->K * 32 + 255) / 256), 256, 0, stream>>>(km->scratch, km->Cf, row, total,
-                                                                                      km->partials, km->D + 4, delta ? 1 : 0, km->dirty,
-                                                                                      delta && km->skipped ? reinterpret_cast<const uint32_t*>(km->drift) + km->K + 1 : nullptr);
-            EC_CUDA(cudaGetLastError());
+            EC_CUDA(launch_dependent(partials_fold_kernel, (unsigned)(((size_t)km->P * km->K * 32 + 255) / 256), 256, 0, stream,
+                                     (const float*)km->scratch, km->Cf, row, total, km->partials, km->D + 4, delta ? 1 : 0,
+                                     (const uint32_t*)km->dirty,
+                                     delta && km->skipped ? reinterpret_cast<const uint32_t*>(km->drift) + km->K + 1 : (const uint32_t*)nullptr));
         }
         km->state_valid = true;
         km->since_full = delta ? km->since_full + 1 : 0;
@@ -1106,10 +1125,10 @@ int km_iterate_rounds(ec_kmeans_t* km, const uint64_t* const* masks, int rounds,
         if (rc != EC_OK) return rc;
     }
     if (km->bounds != nullptr && km->use_bounds) {   // (bounds switched on again later are all renewed first: no drift sums needed meanwhile)
-        update_drift_kernel<<<1, UD_THREADS, 0, stream>>>(km->reduced, km->D, km->K, km->centroids, km->drift);
+        EC_CUDA(launch_dependent(update_drift_kernel, 1, UD_THREADS, 0, stream, (const float*)km->reduced, km->D, km->K, km->centroids, km->drift));
     } else {
         const int total = km->K * km->D;
-        update_kernel<<<(total + 255) / 256, 256, 0, stream>>>(km->reduced, km->D, km->K, km->centroids);
+        EC_CUDA(launch_dependent(update_kernel, (unsigned)((total + 255) / 256), 256, 0, stream, (const float*)km->reduced, km->D, km->K, km->centroids));
     }
     EC_CUDA(cudaGetLastError());
     return EC_OK;

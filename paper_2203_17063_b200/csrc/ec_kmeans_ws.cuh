@@ -57,7 +57,7 @@ using tc::tmem_alloc;
 using tc::tmem_dealloc;
 
 constexpr int TILE = 128;                       // points per tile = rows of an accumulator
-constexpr int MAX_GROUPS = 4;                   // epilogue groups of four warps
+constexpr int MAX_GROUPS = 4;                   // epilogue groups of four warps (3: the same speed; 5, 6: slower, registers spill)
 constexpr int MAX_STAGES = 8;
 constexpr int MAX_SLOTS = 4;                    // operand buffers of the sums GEMM: 2 when only changes are summed, else 3
 constexpr int MAX_THREADS = (4 * MAX_GROUPS + 3) * 32;
