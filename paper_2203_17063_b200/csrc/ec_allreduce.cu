@@ -153,6 +153,7 @@ struct ApplyArgs {
     uint32_t* seg_clock;         // [S] or nullptr: smallest clock among the accepted, 0 if none
     uint32_t* wait_count;        // [S] or nullptr: ranks whose contribution is too stale
     size_t ring_chunk;           // ring order: elements per 1/P chunk of the vector (0 = plain rank order)
+    int dependent;               // host side only: launch as a programmatic dependent of the stream's previous kernel
 };
 
 // Shape of the streaming loop, chosen by measurement on B200 (config 2 and 3 epochs): what counts
@@ -340,6 +341,7 @@ __device__ __forceinline__ int block_prologue(const ApplyArgs& a, unsigned s, un
 template <int DT, int OP, bool VECTOR, int CAP, int ORDER>
 __global__ void __launch_bounds__(EC_MAXT, (ORDER != EC_ORDER_FIXED ? (CAP > 64 ? 2 : EC_PW_MINB) : CAP > 64 ? 4 : EC_MINB))   // tree and wide-table variants need more registers
 apply_kernel(const ApplyArgs a, const __grid_constant__ PtrTable<CAP> tbl) {
+    grid_dependency_wait();            // (a no-op unless launched as a programmatic dependent)
     typedef Elem<DT> E;
     typedef typename E::In In;
     typedef typename E::Acc Acc;
@@ -532,6 +534,7 @@ constexpr int STAGE = 512;           // 16-byte items staged per pass
 template <int DT, int OP, int CAP>
 __global__ void __launch_bounds__(EC_MAXT)
 apply_short_kernel(const ApplyArgs a, const __grid_constant__ PtrTable<CAP> tbl) {
+    grid_dependency_wait();            // (a no-op unless launched as a programmatic dependent)
     typedef Elem<DT> E;
     typedef typename E::In In;
     typedef typename E::Acc Acc;
@@ -646,6 +649,7 @@ __device__ __forceinline__ void bk_copy(uint32_t dst, const void* src, uint32_t 
 template <int DT, int OP, bool LATE>
 __global__ void __launch_bounds__(BK_THREADS)
 apply_bulk_kernel(const ApplyArgs a, const __grid_constant__ PtrTable<64> tbl) {
+    grid_dependency_wait();            // (a no-op unless launched as a programmatic dependent)
     typedef Elem<DT> E;
     typedef typename E::In In;
     typedef typename E::Acc Acc;
@@ -847,6 +851,7 @@ __device__ __forceinline__ void pw_tree(uint64_t word, int P, Fetch fetch, Acc (
 template <int DT>
 __global__ void __launch_bounds__(PW_THREADS)
 apply_pw_bulk_kernel(const ApplyArgs a, const __grid_constant__ PtrTable<64> tbl) {
+    grid_dependency_wait();            // (a no-op unless launched as a programmatic dependent)
     typedef Elem<DT> E;
     typedef typename E::In In;
     typedef typename E::Acc Acc;
@@ -1038,7 +1043,8 @@ template <int DT>
 int launch_pw_bulk(const ApplyArgs& a, const void* const* bufs, unsigned grid, cudaStream_t st) {
     PtrTable<64> tbl;
     for (int r = 0; r < 64; ++r) tbl.p[r] = r < a.P ? bufs[r] : nullptr;
-    apply_pw_bulk_kernel<DT><<<grid, PW_THREADS, PW_SMEM, st>>>(a, tbl);
+    if (a.dependent) EC_CUDA(launch_dependent(apply_pw_bulk_kernel<DT>, grid, PW_THREADS, PW_SMEM, st, a, tbl));
+    else apply_pw_bulk_kernel<DT><<<grid, PW_THREADS, PW_SMEM, st>>>(a, tbl);
     EC_CUDA(cudaGetLastError());
     return EC_OK;
 }
@@ -1050,16 +1056,19 @@ int launch_cap(const ApplyArgs& a, const void* const* bufs, unsigned grid, int t
         for (int r = 0; r < 64; ++r) tbl.p[r] = r < a.P ? bufs[r] : nullptr;
         if constexpr (VECTOR && ORDER == EC_ORDER_FIXED) {
             if (short_seg) {
-                apply_short_kernel<DT, OP, 64><<<grid, threads, 0, st>>>(a, tbl);
+                if (a.dependent) EC_CUDA(launch_dependent(apply_short_kernel<DT, OP, 64>, grid, (unsigned)threads, 0, st, a, tbl));
+                else apply_short_kernel<DT, OP, 64><<<grid, threads, 0, st>>>(a, tbl);
                 EC_CUDA(cudaGetLastError());
                 return EC_OK;
             }
         }
-        apply_kernel<DT, OP, VECTOR, 64, ORDER><<<grid, threads, 0, st>>>(a, tbl);
+        if (a.dependent) EC_CUDA(launch_dependent(apply_kernel<DT, OP, VECTOR, 64, ORDER>, grid, (unsigned)threads, 0, st, a, tbl));
+        else apply_kernel<DT, OP, VECTOR, 64, ORDER><<<grid, threads, 0, st>>>(a, tbl);
     } else {
         PtrTable<EC_MAX_RANKS> tbl;
         for (int r = 0; r < EC_MAX_RANKS; ++r) tbl.p[r] = r < a.P ? bufs[r] : nullptr;
-        apply_kernel<DT, OP, VECTOR, EC_MAX_RANKS, ORDER><<<grid, threads, 0, st>>>(a, tbl);
+        if (a.dependent) EC_CUDA(launch_dependent(apply_kernel<DT, OP, VECTOR, EC_MAX_RANKS, ORDER>, grid, (unsigned)threads, 0, st, a, tbl));
+        else apply_kernel<DT, OP, VECTOR, EC_MAX_RANKS, ORDER><<<grid, threads, 0, st>>>(a, tbl);
     }
     EC_CUDA(cudaGetLastError());
     return EC_OK;
@@ -1092,7 +1101,10 @@ template <int DT, int OP>
 int launch_bulk_op(const ApplyArgs& a, const void* const* bufs, unsigned grid, cudaStream_t st) {
     PtrTable<64> tbl;
     for (int r = 0; r < 64; ++r) tbl.p[r] = r < a.P ? bufs[r] : nullptr;
-    if (a.first_apply) apply_bulk_kernel<DT, OP, false><<<grid, BK_THREADS, BK_STAGES * BK_STAGE_BYTES, st>>>(a, tbl);
+    if (a.dependent) {
+        if (a.first_apply) EC_CUDA(launch_dependent(apply_bulk_kernel<DT, OP, false>, grid, BK_THREADS, BK_STAGES * BK_STAGE_BYTES, st, a, tbl));
+        else EC_CUDA(launch_dependent(apply_bulk_kernel<DT, OP, true>, grid, BK_THREADS, BK_STAGES * BK_STAGE_BYTES, st, a, tbl));
+    } else if (a.first_apply) apply_bulk_kernel<DT, OP, false><<<grid, BK_THREADS, BK_STAGES * BK_STAGE_BYTES, st>>>(a, tbl);
     else apply_bulk_kernel<DT, OP, true><<<grid, BK_THREADS, BK_STAGES * BK_STAGE_BYTES, st>>>(a, tbl);
     EC_CUDA(cudaGetLastError());
     return EC_OK;
@@ -1141,7 +1153,12 @@ struct ec_ctx {
     size_t tile;       // elements per block
     int res_hint;      // L2 policy of the result accesses
     int path;          // 1: bulk-copy staging where it applies (the default when the context allows it), 0: direct loads
+    bool dependent;    // apply kernels are launched as programmatic dependents (set by the drivers, see ec_common.cuh)
 };
+
+void ec::allreduce_set_dependent_launch(ec_ctx* ctx, bool on) {
+    if (ctx) ctx->dependent = on;
+}
 
 using namespace ec;
 
@@ -1185,6 +1202,7 @@ int ec_allreduce_init(ec_ctx_t** out, int P, size_t n, ec_dtype_t dtype, ec_op_t
     c->applied[1] = reinterpret_cast<uint64_t*>(reinterpret_cast<char*>(c->ws) + need / 2);
     c->cur = 0;
     c->first_apply = true;
+    c->dependent = false;
     {
         int dev = 0, l2 = 0;
         if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&l2, cudaDevAttrL2CacheSize, dev) != cudaSuccess)
@@ -1246,6 +1264,7 @@ int apply_common(ec_ctx_t* c, const void* const* rank_bufs, int P, size_t n, ec_
     a.tiles_per_seg = (unsigned)tiles;
     a.P = c->P; a.W = c->W;
     a.res_hint = c->res_hint;
+    a.dependent = c->dependent ? 1 : 0;
     a.ring_chunk = c->order == EC_ORDER_RING ? (c->n + (size_t)c->P - 1) / (size_t)c->P : 0;
     unsigned grid = (unsigned)(tiles * c->S);
     // short segments and more ranks than the streaming fold keeps in flight: one block per segment, staged fold

@@ -6,9 +6,31 @@
 
 #include "ec.h"
 
+struct ec_ctx;
+
 namespace ec {
 
 extern thread_local int g_last_cuda_error;
+
+// Internal (the K-means and matrix-factorisation drivers): launch this context's apply kernels as programmatic dependents
+// of whatever precedes them in the stream - they start while their predecessor's last blocks still run and wait on the
+// device (griddepcontrol.wait) until it has completed.  Results do not change.
+void allreduce_set_dependent_launch(ec_ctx* ctx, bool on);
+
+// Programmatic dependent launch: the device-side wait (returns at once in a kernel launched the ordinary way) ...
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+// ... and the launch.
+template <class... KArgs, class... Args>
+inline cudaError_t launch_dependent(void (*kernel)(KArgs...), unsigned grid, unsigned block, size_t smem, cudaStream_t stream, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid); cfg.blockDim = dim3(block); cfg.dynamicSmemBytes = smem; cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
 
 inline int cuda_fail(cudaError_t e) {
     g_last_cuda_error = (int)e;

@@ -32,22 +32,6 @@
 namespace ec {
 namespace {
 
-// Programmatic dependent launch: a small kernel that follows a big one in the stream is launched while the big one's last
-// blocks are still running; it waits here, on the device, until its predecessor has completed and its writes are visible.
-// (Without the launch attribute the instruction returns at once.)
-__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
-
-template <class... KArgs, class... Args>
-cudaError_t launch_dependent(void (*kernel)(KArgs...), unsigned grid, unsigned block, size_t smem, cudaStream_t stream, Args... args) {
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(grid); cfg.blockDim = dim3(block); cfg.dynamicSmemBytes = smem; cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr; cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
-}
-
 constexpr int AS_THREADS = 256;
 constexpr int PT_THREADS = 256;
 constexpr int PT_WARPS = PT_THREADS / 32;
@@ -725,10 +709,9 @@ int km_tc_launch(ec_kmeans* km, bool partials, const float* centroids, int32_t* 
     const bool own = centroids == km->centroids && labels == km->labels && km->bounds != nullptr && km->use_bounds;
     const bool skip = partials && delta && own && km->bounds_valid && km->use_bounds;
     if (skip) {      // which tiles can still change a label: one byte per 32 points
-        tc::bounds_check_kernel<<<(unsigned)(km->P * km->Cf), tc::BC_THREADS, 0, st>>>(
-            km->N, km->P, km->Cf, km->K, labels, km->bounds, km->drift, km->need, km->need_words, km->dirty,
-            reinterpret_cast<uint32_t*>(km->drift) + km->K + 1);
-        EC_CUDA(cudaGetLastError());
+        EC_CUDA(launch_dependent(tc::bounds_check_kernel, (unsigned)(km->P * km->Cf), tc::BC_THREADS, 0, st,
+                                 km->N, km->P, km->Cf, km->K, (const int32_t*)labels, (const float2*)km->bounds, (const float*)km->drift,
+                                 km->need, km->need_words, km->dirty, reinterpret_cast<uint32_t*>(km->drift) + km->K + 1));
     }
     if (partials) {
         const unsigned gd = (unsigned)(km->P * km->Cf < km->tc_wave_delta ? km->P * km->Cf : km->tc_wave_delta);
@@ -840,10 +823,9 @@ int km_ws_launch(ec_kmeans* km, bool partials, const float* centroids, int32_t* 
     const bool own = centroids == km->centroids && labels == km->labels && km->bounds != nullptr && km->use_bounds;
     const bool skip = partials && delta && own && km->bounds_valid && km->use_bounds;
     if (skip) {      // which tiles can still change a label: one byte per 32 points
-        tc::bounds_check_kernel<<<(unsigned)(km->P * km->Cf), tc::BC_THREADS, 0, st>>>(
-            km->N, km->P, km->Cf, km->K, labels, km->bounds, km->drift, km->need, km->need_words, km->dirty,
-            reinterpret_cast<uint32_t*>(km->drift) + km->K + 1);
-        EC_CUDA(cudaGetLastError());
+        EC_CUDA(launch_dependent(tc::bounds_check_kernel, (unsigned)(km->P * km->Cf), tc::BC_THREADS, 0, st,
+                                 km->N, km->P, km->Cf, km->K, (const int32_t*)labels, (const float2*)km->bounds, (const float*)km->drift,
+                                 km->need, km->need_words, km->dirty, reinterpret_cast<uint32_t*>(km->drift) + km->K + 1));
     }
     if (partials) {
         const int runs = km->P * km->Cf;
@@ -853,28 +835,28 @@ int km_ws_launch(ec_kmeans* km, bool partials, const float* centroids, int32_t* 
         const size_t smem = plan.total;
         float* full_out = km->Cf == 1 ? km->partials : km->scratch;
         if (delta && own)
-            ws::ws_fused_kernel<D, true, true, true><<<grid, thr, smem, st>>>(
+            EC_CUDA(launch_dependent(ws::ws_fused_kernel<D, true, true, true>, grid, thr, smem, st,
                 km->pmap, km->points, km->N, km->P, km->Cf, centroids, km->K, labels, km->scratch, km->tc_status, km->dirty,
-                km->bounds, km->drift, skip ? km->need : nullptr, km->need_words);
+                km->bounds, km->drift, skip ? km->need : nullptr, km->need_words));
         else if (delta)
-            ws::ws_fused_kernel<D, true, true, false><<<grid, thr, smem, st>>>(
+            EC_CUDA(launch_dependent(ws::ws_fused_kernel<D, true, true, false>, grid, thr, smem, st,
                 km->pmap, km->points, km->N, km->P, km->Cf, centroids, km->K, labels, km->scratch, km->tc_status, km->dirty,
-                nullptr, nullptr, nullptr, 0);
+                nullptr, nullptr, nullptr, 0));
         else if (own)
-            ws::ws_fused_kernel<D, true, false, true><<<grid, thr, smem, st>>>(
+            EC_CUDA(launch_dependent(ws::ws_fused_kernel<D, true, false, true>, grid, thr, smem, st,
                 km->pmap, km->points, km->N, km->P, km->Cf, centroids, km->K, labels, full_out, km->tc_status, km->dirty,
-                km->bounds, km->drift, nullptr, 0);
+                km->bounds, km->drift, nullptr, 0));
         else
-            ws::ws_fused_kernel<D, true, false, false><<<grid, thr, smem, st>>>(
+            EC_CUDA(launch_dependent(ws::ws_fused_kernel<D, true, false, false>, grid, thr, smem, st,
                 km->pmap, km->points, km->N, km->P, km->Cf, centroids, km->K, labels, full_out, km->tc_status, km->dirty,
-                nullptr, nullptr, nullptr, 0);
+                nullptr, nullptr, nullptr, 0));
     } else {
         size_t runs = (km->N + 2047) / 2048;
         if (runs > 0x7fffffffull) return EC_ERR_CAPACITY;
         const unsigned grid = (unsigned)(runs < (size_t)km->sms ? runs : (size_t)km->sms);
-        ws::ws_fused_kernel<D, false, false, false><<<grid, (unsigned)ws::threads_of(km->ws_plan_assign), km->ws_plan_assign.total, st>>>(
-            km->pmap, km->points, km->N, 1, (int)runs, centroids, km->K, labels, nullptr, km->tc_status, nullptr,
-            nullptr, nullptr, nullptr, 0);
+        EC_CUDA(launch_dependent(ws::ws_fused_kernel<D, false, false, false>, grid, (unsigned)ws::threads_of(km->ws_plan_assign), km->ws_plan_assign.total, st,
+                km->pmap, km->points, km->N, 1, (int)runs, centroids, km->K, labels, nullptr, km->tc_status, nullptr,
+            nullptr, nullptr, nullptr, 0));
     }
     EC_CUDA(cudaGetLastError());
     km->skipped = skip;
@@ -1061,6 +1043,7 @@ int ec_kmeans_init(ec_kmeans_t** out, const float* points, size_t N, int D, int 
         return rc;
     }
     for (int r = 0; r < P; ++r) km->bufs[r] = km->partials + (size_t)r * K * stride;
+    allreduce_set_dependent_launch(km->ar, true);        // the small allreduce follows the fold kernel closely
     *out = km;
     return EC_OK;
 }

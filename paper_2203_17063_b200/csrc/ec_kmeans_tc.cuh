@@ -221,6 +221,7 @@ bounds_check_kernel(size_t N, int P, int C, int K, const int32_t* __restrict__ l
                     const float* __restrict__ drift, uint32_t* __restrict__ need, int need_words,
                     uint32_t* __restrict__ dirty, uint32_t* __restrict__ any_work) {
     __shared__ float s_d[1024 + 1];
+    grid_dependency_wait();                              // (launched as a programmatic dependent of the centroid update)
     const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
     for (int k = tid; k <= K; k += BC_THREADS) s_d[k] = drift[k];
     __syncthreads();
@@ -316,6 +317,7 @@ tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const 
                 int32_t* __restrict__ labels, float* __restrict__ scratch, float tau_scale, uint32_t* __restrict__ status,
                 uint32_t* __restrict__ dirty, float2* __restrict__ bounds, const float* __restrict__ drift,
                 const uint32_t* __restrict__ need, int need_words) {
+    grid_dependency_wait();                              // (a no-op unless launched as a programmatic dependent)
     constexpr bool delta = DELTA;                        // sum only what changed since the labels were written last
     constexpr int KCH = D / 8;                           // 16-byte chunks of coordinates per point
     static_assert(D % 16 == 0 && KCH + 2 <= 8 && (KCH & (KCH - 1)) == 0, "D is 16 or 32");

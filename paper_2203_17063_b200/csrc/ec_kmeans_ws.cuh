@@ -312,6 +312,7 @@ ws_fused_kernel(const __grid_constant__ CUtensorMap pmap, const float* __restric
                 const float* __restrict__ centroids, int K, int32_t* __restrict__ labels, float* __restrict__ scratch,
                 uint32_t* __restrict__ status, uint32_t* __restrict__ dirty, float2* __restrict__ bounds,
                 const float* __restrict__ drift, const uint32_t* __restrict__ need, int need_words) {
+    grid_dependency_wait();                                 // (a no-op unless launched as a programmatic dependent)
     constexpr int KCH = D / 8;                              // 16-byte bf16 chunks (8 coordinates) per point
     constexpr int Q = D / 4;                                // 16-byte fp32 chunks per point
     constexpr uint32_t XC = xchunk_of(D);
