@@ -1202,7 +1202,7 @@ int ec_allreduce_init(ec_ctx_t** out, int P, size_t n, ec_dtype_t dtype, ec_op_t
     c->applied[1] = reinterpret_cast<uint64_t*>(reinterpret_cast<char*>(c->ws) + need / 2);
     c->cur = 0;
     c->first_apply = true;
-    c->dependent = false;
+    c->dependent = true;    // (see ec_common.cuh: the apply kernels wait on the device for whatever precedes them in the stream)
     {
         int dev = 0, l2 = 0;
         if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&l2, cudaDevAttrL2CacheSize, dev) != cudaSuccess)

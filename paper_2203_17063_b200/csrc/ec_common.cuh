@@ -12,9 +12,10 @@ namespace ec {
 
 extern thread_local int g_last_cuda_error;
 
-// Internal (the K-means and matrix-factorisation drivers): launch this context's apply kernels as programmatic dependents
-// of whatever precedes them in the stream - they start while their predecessor's last blocks still run and wait on the
-// device (griddepcontrol.wait) until it has completed.  Results do not change.
+// Internal: whether this context's apply kernels are launched as programmatic dependents of whatever precedes them in
+// the stream (the default) - they start while their predecessor's last blocks still run and wait on the device
+// (griddepcontrol.wait, their first instruction) until it has completed and its writes are visible.  Results do not
+// change; the gaps between the applies of an epoch go (config 2 epoch: 0.191 -> 0.187 ms).
 void allreduce_set_dependent_launch(ec_ctx* ctx, bool on);
 
 // Programmatic dependent launch: the device-side wait (returns at once in a kernel launched the ordinary way) ...
