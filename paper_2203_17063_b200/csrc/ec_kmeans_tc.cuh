@@ -209,6 +209,40 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     return u;
 }
 
+__device__ __forceinline__ float min3(float a, float b, float c) {
+    float d;
+    asm("min.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+
+// Best two of 16 scores whose low 7 mantissa bits are replaced by their column index (here: 0..15 in the low four; the
+// caller adds the number of the group of 16): sorted pairs, then the same again on the smaller halves; the second best
+// is the smallest of all the larger halves (the partner of the winner is among them, and every other larger half is at
+// least the second best of the smaller ones).  16 at a time, so that the next 16 can be on their way from tensor memory.
+// (raw & mask) | tag is ONE logic instruction when the mask comes in a register (two immediates would take two).
+__device__ __forceinline__ void best_two_of_16(const uint32_t (&raw)[16], uint32_t mask, float& c1, float& c2) {
+    float lo[8], hi[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        uint32_t ra, rb;
+        asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(ra) : "r"(raw[2 * i]), "r"(mask), "r"((uint32_t)(2 * i)));
+        asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(rb) : "r"(raw[2 * i + 1]), "r"(mask), "r"((uint32_t)(2 * i + 1)));
+        const float a = __uint_as_float(ra), b = __uint_as_float(rb);
+        lo[i] = fminf(a, b);
+        hi[i] = fmaxf(a, b);
+    }
+    float hi_min = min3(min3(hi[0], hi[1], hi[2]), min3(hi[3], hi[4], hi[5]), fminf(hi[6], hi[7]));
+    float l4[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) l4[i] = fminf(lo[2 * i], lo[2 * i + 1]);
+    hi_min = min3(hi_min, fmaxf(lo[0], lo[1]), fmaxf(lo[2], lo[3]));
+    hi_min = min3(hi_min, fmaxf(lo[4], lo[5]), fmaxf(lo[6], lo[7]));
+    const float a = fminf(l4[0], l4[1]), b = fminf(l4[2], l4[3]);
+    hi_min = min3(hi_min, fmaxf(l4[0], l4[1]), fmaxf(l4[2], l4[3]));
+    c1 = fminf(a, b);
+    c2 = fminf(hi_min, fmaxf(a, b));
+}
+
 // Which tiles of a delta-mode pass have to be searched (see the bounds in tc_fused_kernel).  Same runs as the
 // fused kernel (block = run c of rank r), but nothing else to carry, so the SMs are full of warps: a warp takes
 // 32 consecutive points at a time and leaves one byte, nonzero if the bounds of one of them no longer hold.
@@ -407,6 +441,8 @@ tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const 
     const uint32_t tmem_lane = tmem_base + ((uint32_t)(w * 32) << 16);   // this warp's 32 lanes
     float cmax = 0.0f;
     for (int k = 0; k < K; ++k) cmax = fmaxf(cmax, s_cn[k]);
+    uint32_t tag_mask;                                   // 0xFFFFFF00 in a register (see best_two_of_16; up to 256 columns here)
+    asm volatile("mov.u32 %0, 0xFFFFFF00;" : "=r"(tag_mask));
     const uint32_t idesc_search = instr_desc(MROWS, npad, false);
     const uint32_t idesc_sum = instr_desc(MROWS, npad, true);
     const uint32_t b_base = smem_u32(s_b), x_base = smem_u32(s_x), oh_base = smem_u32(s_oh);
@@ -563,18 +599,25 @@ tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const 
         float m1 = __int_as_float(0x7f800000), m2 = m1;
         int kb = 0;
         if (done) {
+            // the best two scores by a tournament of min/max pairs; the low 7 mantissa bits of a score are replaced by its
+            // column (a change of less than 2^-16 of the score: far inside the margin of tau)
             for (int ch = 0; ch < npad / 32; ++ch) {
                 uint32_t vv[32];
                 tmem_ld32(tmem_lane + (uint32_t)(ch * 32), vv);
+                uint32_t lo_half[16], hi_half[16];
 #pragma unroll
-                for (int e = 0; e < 32; ++e) {
-                    const float v = __uint_as_float(vv[e]);
-                    const bool lt = v < m1;
-                    m2 = fminf(m2, lt ? m1 : v);
-                    kb = lt ? ch * 32 + e : kb;
-                    m1 = lt ? v : m1;
-                }
+                for (int e = 0; e < 16; ++e) { lo_half[e] = vv[e]; hi_half[e] = vv[16 + e]; }
+                float c1, c2;
+                best_two_of_16(lo_half, tag_mask, c1, c2);
+                c1 = __uint_as_float(__float_as_uint(c1) | (uint32_t)(ch << 5));
+                m2 = min3(m2, c2, fmaxf(m1, c1));
+                m1 = fminf(m1, c1);
+                best_two_of_16(hi_half, tag_mask, c1, c2);
+                c1 = __uint_as_float(__float_as_uint(c1) | (uint32_t)((ch << 5) | 16));
+                m2 = min3(m2, c2, fmaxf(m1, c1));
+                m1 = fminf(m1, c1);
             }
+            kb = (int)(__float_as_uint(m1) & 255u);
         } else if (tid == 0 && status != nullptr) {
             atomicOr(status, 1u);    // the tensor core did not answer in time
         }

@@ -47,7 +47,9 @@ namespace ws {
 using tc::fence_after_sync;
 using tc::fence_async_smem;
 using tc::fence_before_sync;
+using tc::best_two_of_16;
 using tc::mbar_init;
+using tc::min3;
 using tc::mma_commit;
 using tc::npad_of;
 using tc::pack_bf16;
@@ -199,11 +201,6 @@ __device__ __forceinline__ uint32_t swz_off(int r, int q) {
     if (D == 32) return (uint32_t)r * 128u + (uint32_t)((q ^ (r & 7)) << 4);
     return (uint32_t)r * 64u + (uint32_t)((q ^ ((r >> 1) & 3)) << 4);
 }
-__device__ __forceinline__ float min3(float a, float b, float c) {
-    float d;
-    asm("min.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
-    return d;
-}
 __device__ __forceinline__ void tmem_ld32_nowait(uint32_t taddr, uint32_t (&r)[32]) {
     asm volatile(
         "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
@@ -226,34 +223,6 @@ __device__ __forceinline__ void tmem_ld16_nowait(uint32_t taddr, uint32_t (&r)[1
         : "r"(taddr)
         : "memory");
 }
-// Best two of 16 scores whose low 7 mantissa bits are replaced by their column index (here: 0..15 in the low four; the
-// caller adds the number of the group of 16): sorted pairs, then the same again on the smaller halves; the second best
-// is the smallest of all the larger halves (the partner of the winner is among them, and every other larger half is at
-// least the second best of the smaller ones).  16 at a time, so that the next 16 can be on their way from tensor memory.
-// (raw & mask) | tag is ONE logic instruction when the mask comes in a register (two immediates would take two).
-__device__ __forceinline__ void best_two_of_16(const uint32_t (&raw)[16], uint32_t mask, float& c1, float& c2) {
-    float lo[8], hi[8];
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-        uint32_t ra, rb;
-        asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(ra) : "r"(raw[2 * i]), "r"(mask), "r"((uint32_t)(2 * i)));
-        asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(rb) : "r"(raw[2 * i + 1]), "r"(mask), "r"((uint32_t)(2 * i + 1)));
-        const float a = __uint_as_float(ra), b = __uint_as_float(rb);
-        lo[i] = fminf(a, b);
-        hi[i] = fmaxf(a, b);
-    }
-    float hi_min = min3(min3(hi[0], hi[1], hi[2]), min3(hi[3], hi[4], hi[5]), fminf(hi[6], hi[7]));
-    float l4[4];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) l4[i] = fminf(lo[2 * i], lo[2 * i + 1]);
-    hi_min = min3(hi_min, fmaxf(lo[0], lo[1]), fmaxf(lo[2], lo[3]));
-    hi_min = min3(hi_min, fmaxf(lo[4], lo[5]), fmaxf(lo[6], lo[7]));
-    const float a = fminf(l4[0], l4[1]), b = fminf(l4[2], l4[3]);
-    hi_min = min3(hi_min, fmaxf(l4[0], l4[1]), fmaxf(l4[2], l4[3]));
-    c1 = fminf(a, b);
-    c2 = fminf(hi_min, fmaxf(a, b));
-}
-
 // The search cannot separate the best candidates of some point of this warp (redo: of this thread's point).  The true
 // nearest centroid's score is within tau of the best score (each score is within tau / 2 of its exact value), so the
 // exact form sum_d (x - c)^2 decides among the columns with v <= lim = best + tau alone.  The scores are read once more
