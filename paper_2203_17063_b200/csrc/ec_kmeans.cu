@@ -274,6 +274,19 @@ __global__ void partials_fold_kernel(const float* __restrict__ scratch, int C, s
     }
 }
 
+// |x|^2 of every point (four chains, the order the fused kernels used to take), once per context.
+__global__ void point_norm_kernel(const float* __restrict__ points, size_t N, int D, float* __restrict__ xnorm) {
+    for (size_t j = (size_t)blockIdx.x * blockDim.x + threadIdx.x; j < N; j += (size_t)gridDim.x * blockDim.x) {
+        const float4* row = reinterpret_cast<const float4*>(points + j * D);
+        float n0 = 0.0f, n1 = 0.0f, n2 = 0.0f, n3 = 0.0f;
+        for (int q = 0; q < D / 4; ++q) {
+            const float4 v = __ldg(row + q);
+            n0 = fmaf(v.x, v.x, n0); n1 = fmaf(v.y, v.y, n1); n2 = fmaf(v.z, v.z, n2); n3 = fmaf(v.w, v.w, n3);
+        }
+        xnorm[j] = (n0 + n1) + (n2 + n3);
+    }
+}
+
 __global__ void update_kernel(const float* __restrict__ reduced, int D, int K, float* __restrict__ centroids) {
     grid_dependency_wait();
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
@@ -592,6 +605,7 @@ struct ec_kmeans {
     uint32_t* tc_status;   // device word: nonzero if a wait on the tensor core ever gave up
     uint32_t* dirty;       // [P][Cf]: delta mode, which row blocks of scratch hold changes
     float2* bounds;        // [N]: distance bounds of every point (tensor-core path), see tc_fused_kernel
+    float* xnorm;          // [N]: |x|^2 of every point, made once (the points do not change under a context)
     float* drift;          // [K + 1]: how far every centroid has moved in all, and the sum of the largest moves
     uint32_t* need;        // [P * Cf][need_words]: delta mode with bounds, which tiles have to be searched
     int need_words;
@@ -608,7 +622,7 @@ using namespace ec;
 namespace {
 
 struct KmLayout {
-    size_t off_centroids, off_labels, off_partials, off_scratch, off_reduced, off_contrib, off_dirty, off_bounds, off_drift, off_need, off_ar, total;
+    size_t off_centroids, off_labels, off_partials, off_scratch, off_reduced, off_contrib, off_dirty, off_bounds, off_drift, off_need, off_xnorm, off_ar, total;
     int need_words;      // tiles of the longest run (0: the distance bounds are not kept)
     int C, warps;
     int Cf;   // runs per rank for the fused assignment+partials kernel, 0 if the shape is not covered
@@ -671,6 +685,7 @@ bool km_plan(size_t N, int D, int K, int P, int sms, KmLayout* L) {
     L->off_bounds = off; off = align_up(off + (L->need_words > 0 ? N * 8 : 0), 256);   // distance bounds of the points
     L->off_drift = off; off = align_up(off + ((size_t)K + 2) * 4, 256);    // drift sums, their maximum's sum, the check's flag word
     L->off_need = off; off = align_up(off + (size_t)P * (L->Cf > 0 ? L->Cf : 1) * (size_t)L->need_words * 4, 256);
+    L->off_xnorm = off; off = align_up(off + ((L->Cf > 0 && tc_capable(D, K)) ? N * 4 : 0), 256);   // |x|^2 of every point
     L->off_ar = off; off = align_up(off + ec_allreduce_workspace_bytes(P, (size_t)K * stride, stride), 256);
     L->total = off;
     return true;
@@ -836,26 +851,26 @@ int km_ws_launch(ec_kmeans* km, bool partials, const float* centroids, int32_t* 
         float* full_out = km->Cf == 1 ? km->partials : km->scratch;
         if (delta && own)
             EC_CUDA(launch_dependent(ws::ws_fused_kernel<D, true, true, true>, grid, thr, smem, st,
-                km->pmap, km->points, km->N, km->P, km->Cf, centroids, km->K, labels, km->scratch, km->tc_status, km->dirty,
+                km->pmap, km->points, (const float*)km->xnorm, km->N, km->P, km->Cf, centroids, km->K, labels, km->scratch, km->tc_status, km->dirty,
                 km->bounds, km->drift, skip ? km->need : nullptr, km->need_words));
         else if (delta)
             EC_CUDA(launch_dependent(ws::ws_fused_kernel<D, true, true, false>, grid, thr, smem, st,
-                km->pmap, km->points, km->N, km->P, km->Cf, centroids, km->K, labels, km->scratch, km->tc_status, km->dirty,
+                km->pmap, km->points, (const float*)km->xnorm, km->N, km->P, km->Cf, centroids, km->K, labels, km->scratch, km->tc_status, km->dirty,
                 nullptr, nullptr, nullptr, 0));
         else if (own)
             EC_CUDA(launch_dependent(ws::ws_fused_kernel<D, true, false, true>, grid, thr, smem, st,
-                km->pmap, km->points, km->N, km->P, km->Cf, centroids, km->K, labels, full_out, km->tc_status, km->dirty,
+                km->pmap, km->points, (const float*)km->xnorm, km->N, km->P, km->Cf, centroids, km->K, labels, full_out, km->tc_status, km->dirty,
                 km->bounds, km->drift, nullptr, 0));
         else
             EC_CUDA(launch_dependent(ws::ws_fused_kernel<D, true, false, false>, grid, thr, smem, st,
-                km->pmap, km->points, km->N, km->P, km->Cf, centroids, km->K, labels, full_out, km->tc_status, km->dirty,
+                km->pmap, km->points, (const float*)km->xnorm, km->N, km->P, km->Cf, centroids, km->K, labels, full_out, km->tc_status, km->dirty,
                 nullptr, nullptr, nullptr, 0));
     } else {
         size_t runs = (km->N + 2047) / 2048;
         if (runs > 0x7fffffffull) return EC_ERR_CAPACITY;
         const unsigned grid = (unsigned)(runs < (size_t)km->sms ? runs : (size_t)km->sms);
         EC_CUDA(launch_dependent(ws::ws_fused_kernel<D, false, false, false>, grid, (unsigned)ws::threads_of(km->ws_plan_assign), km->ws_plan_assign.total, st,
-                km->pmap, km->points, km->N, 1, (int)runs, centroids, km->K, labels, nullptr, km->tc_status, nullptr,
+                km->pmap, km->points, (const float*)km->xnorm, km->N, 1, (int)runs, centroids, km->K, labels, nullptr, km->tc_status, nullptr,
             nullptr, nullptr, nullptr, 0));
     }
     EC_CUDA(cudaGetLastError());
@@ -991,6 +1006,7 @@ int ec_kmeans_init(ec_kmeans_t** out, const float* points, size_t N, int D, int 
     km->dirty = reinterpret_cast<uint32_t*>(base + L.off_dirty);
     km->bounds = km->tc_ok && L.need_words > 0 ? reinterpret_cast<float2*>(base + L.off_bounds) : nullptr;
     km->need = reinterpret_cast<uint32_t*>(base + L.off_need);
+    km->xnorm = km->tc_ok ? reinterpret_cast<float*>(base + L.off_xnorm) : nullptr;
     km->need_words = L.need_words;
     km->drift = reinterpret_cast<float*>(base + L.off_drift);
     km->bounds_valid = false;
@@ -1031,6 +1047,10 @@ int ec_kmeans_init(ec_kmeans_t** out, const float* points, size_t N, int D, int 
     }
     if (e == cudaSuccess) e = cudaMemsetAsync(km->tc_status, 0, 4, 0);
     if (e == cudaSuccess) e = cudaMemsetAsync(km->drift, 0, ((size_t)K + 2) * 4, 0);
+    if (e == cudaSuccess && km->xnorm != nullptr) {
+        point_norm_kernel<<<(unsigned)(sms * 8), 256>>>(points, N, D, km->xnorm);
+        e = cudaGetLastError();
+    }
     if (e == cudaSuccess) e = cudaMemcpyAsync(km->centroids, init_centroids, (size_t)K * D * 4, cudaMemcpyDeviceToDevice, 0);
     if (e == cudaSuccess) e = cudaStreamSynchronize(0);
     if (e != cudaSuccess) rc = cuda_fail(e);

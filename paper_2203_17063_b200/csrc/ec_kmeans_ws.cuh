@@ -231,7 +231,7 @@ __device__ __forceinline__ void tmem_ld16_nowait(uint32_t taddr, uint32_t (&r)[1
 // ascending order with strict <, so the lowest index wins an exact tie as it does over all centroids; a point with
 // more than four candidates is decided over all centroids.
 template <int D>
-__device__ __noinline__ int redecide(bool redo, int kb, float lim, const unsigned char* row0, int t, uint32_t col0, int npad,
+__device__ __noinline__ int redecide(bool redo, int kb, float lim, const float* __restrict__ xrow, uint32_t col0, int npad,
                                      const float* __restrict__ centroids, int K) {
     constexpr int Q = D / 4;
     uint32_t cand = 0;
@@ -248,11 +248,10 @@ __device__ __noinline__ int redecide(bool redo, int kb, float lim, const unsigne
         }
     }
     if (!redo) return kb;
-    float x[D];
-    const unsigned char* row = row0 - swz_off<D>(t, 0);
+    float x[D];                                          // the point, from global memory (its stage went back after the search)
 #pragma unroll
     for (int q = 0; q < Q; ++q) {
-        const float4 v = *reinterpret_cast<const float4*>(row + swz_off<D>(t, q));
+        const float4 v = __ldg(reinterpret_cast<const float4*>(xrow) + q);
         x[4 * q] = v.x; x[4 * q + 1] = v.y; x[4 * q + 2] = v.z; x[4 * q + 3] = v.w;
     }
     if (cnt > 4 || cnt == 0) return tc::exact_argmin_global<D>(x, centroids, K);
@@ -277,7 +276,8 @@ __device__ __noinline__ int redecide(bool redo, int kb, float lim, const unsigne
 
 template <int D, bool PARTIALS, bool DELTA, bool BOUNDS>
 __global__ void __launch_bounds__(MAX_THREADS, 1)
-ws_fused_kernel(const __grid_constant__ CUtensorMap pmap, const float* __restrict__ points, size_t N, int P, int C,
+ws_fused_kernel(const __grid_constant__ CUtensorMap pmap, const float* __restrict__ points, const float* __restrict__ xnorm,
+                size_t N, int P, int C,
                 const float* __restrict__ centroids, int K, int32_t* __restrict__ labels, float* __restrict__ scratch,
                 uint32_t* __restrict__ status, uint32_t* __restrict__ dirty, float2* __restrict__ bounds,
                 const float* __restrict__ drift, const uint32_t* __restrict__ need, int need_words) {
@@ -334,7 +334,7 @@ ws_fused_kernel(const __grid_constant__ CUtensorMap pmap, const float* __restric
     // ---- set-up, all threads ------------------------------------------------------------------------------------
     if (warp == 4 * G + 1) tmem_alloc(smem_u32(const_cast<int*>(s_ctrl + 6)), pl.tmem_cols);
     if (tid == 0) {
-        for (int s = 0; s < NST; ++s) { mbar_init(B_full(s), 1); mbar_init(B_empty(s), 4); }
+        for (int s = 0; s < NST; ++s) { mbar_init(B_full(s), 1); mbar_init(B_empty(s), 5); }   // empty: the search's commit + the four warps that read the descriptor
         for (int g = 0; g < G; ++g) {
             mbar_init(B_accfull(g), 1); mbar_init(B_accempty(g), 4); mbar_init(B_decided(g), 4);
         }
@@ -480,6 +480,7 @@ ws_fused_kernel(const __grid_constant__ CUtensorMap pmap, const float* __restric
                     mma_tf32(acc, adesc + (uint64_t)(2 * ks), bdesc[ks], idesc, ks > 0 ? 1u : 0u);
                 mma_tf32(acc, ones_desc, cnb_desc, idesc, 1u);
                 mma_commit(B_accfull(g));
+                mma_commit(B_empty(s));                        // the tile has been read: its stage goes back to the producer
                 if (++s == NST) { s = 0; full_par ^= 1u; }
                 if (++g == G) { g = 0; empty_par ^= 1u; first_round = false; }
             }
@@ -575,20 +576,13 @@ ws_fused_kernel(const __grid_constant__ CUtensorMap pmap, const float* __restric
                 }
                 break;
             }
+            // The stage goes back to the producer once the search has read the tile (the issuer's commit) and this group's
+            // four warps have taken the descriptor (here): the epilogue itself reads nothing of the staged tile.
+            warrive(B_empty(s));
             const size_t j = (size_t)td.base + (size_t)t;
             const bool live = j < (size_t)td.end;
             const int old = (DELTA && live) ? labels[j] : -1;
-            const unsigned char* row = sm + pl.stage + (size_t)s * pl.stage_bytes;
-            float xn;
-            {
-                float n0 = 0.0f, n1 = 0.0f, n2 = 0.0f, n3 = 0.0f;   // four chains
-#pragma unroll
-                for (int q = 0; q < Q; ++q) {
-                    const float4 v = *reinterpret_cast<const float4*>(row + swz_off<D>(t, q));
-                    n0 = fmaf(v.x, v.x, n0); n1 = fmaf(v.y, v.y, n1); n2 = fmaf(v.z, v.z, n2); n3 = fmaf(v.w, v.w, n3);
-                }
-                xn = (n0 + n1) + (n2 + n3);
-            }
+            const float xn = live ? __ldg(xnorm + j) : 0.0f;      // |x|^2, made once per context: the staged tile is the tensor core's alone
             if (!wwait(B_accfull(g), (uint32_t)n & 1u, 8)) { ok = false; break; }
             fence_after_sync();
             float m1 = __int_as_float(0x7f800000), m2 = m1;
@@ -617,7 +611,7 @@ ws_fused_kernel(const __grid_constant__ CUtensorMap pmap, const float* __restric
             const float tau = TAU_SCALE * (xn + cmax);
             const bool redo = live && !(m2 - m1 > tau);
             if (__any_sync(0xffffffffu, redo))            // rare on separated data: kept out of line, away from this loop's registers
-                kb = redecide<D>(redo, kb, m1 + tau, row + swz_off<D>(t, 0), t, lane_base + (uint32_t)(g * npad), npad, centroids, K);
+                kb = redecide<D>(redo, kb, m1 + tau, points + j * D, lane_base + (uint32_t)(g * npad), npad, centroids, K);
             fence_before_sync();
             warrive(B_accempty(g));                      // the accumulator may take the group's next tile
             const bool changed = live && !(DELTA && old == kb);
@@ -683,8 +677,8 @@ ws_fused_kernel(const __grid_constant__ CUtensorMap pmap, const float* __restric
                         // bf16 high and low parts of the row (low = bf16(x - high)): chunk column 2 kc resp. 2 kc + 1
 #pragma unroll
                         for (int kc = 0; kc < KCH; ++kc) {
-                            const float4 va = *reinterpret_cast<const float4*>(row + swz_off<D>(t, 2 * kc));
-                            const float4 vb = *reinterpret_cast<const float4*>(row + swz_off<D>(t, 2 * kc + 1));
+                            const float4 va = __ldg(reinterpret_cast<const float4*>(points + j * D) + 2 * kc);   // (from L2: the tile was just read)
+                            const float4 vb = __ldg(reinterpret_cast<const float4*>(points + j * D) + 2 * kc + 1);
                             const float v[8] = {va.x, va.y, va.z, va.w, vb.x, vb.y, vb.z, vb.w};
                             uint32_t hw[4], lw[4];
 #pragma unroll
@@ -709,7 +703,6 @@ ws_fused_kernel(const __grid_constant__ CUtensorMap pmap, const float* __restric
                 fence_before_sync();
                 warrive(B_decided(g));
             }
-            warrive(B_empty(s));                         // the stage may take another tile
             if (PARTIALS && td.last) {
                 // the run's last tile: its group writes the run's sums out once the sums issuer is through the run
                 // (first until the sums issuer has signalled the end of this run: it has then seen the run before last written
