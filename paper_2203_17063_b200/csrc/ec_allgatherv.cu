@@ -31,6 +31,7 @@ namespace {
 constexpr int GV_THREADS = EC_GV_THREADS;
 constexpr size_t GV_CHUNK_BYTES = EC_GV_CHUNK;
 constexpr int GV_BATCH = EC_GV_BATCH;  // loads in flight per thread before the stores
+constexpr unsigned GV_MAX_BLOCKS = 16384;
 
 struct GatherArgs {
     const int64_t* counts;
@@ -95,6 +96,13 @@ allgatherv_kernel(const GatherArgs a, const __grid_constant__ PtrTable<CAP> tbl)
     const int P = a.P;
 
     if (tid == 0) s_bad = 0;
+    // the counts and the arrival words are fetched together (one trip to memory, not two in a row)
+    long long cnt[ITEMS];
+#pragma unroll
+    for (int i = 0; i < ITEMS; ++i) {
+        const int r = tid * ITEMS + i;
+        cnt[i] = (r < P && r < CAP) ? a.counts[r] : 0;
+    }
     for (int w = tid; w < (CAP + 63) / 64; w += GV_THREADS) {
         uint64_t word = 0;
         if (w * 64 < P) {
@@ -105,13 +113,12 @@ allgatherv_kernel(const GatherArgs a, const __grid_constant__ PtrTable<CAP> tbl)
     }
     __syncthreads();
     // exclusive scan: thread-local prefix, warp shuffle scan of the thread totals, scan of the warp totals
-    long long cnt[ITEMS];
     long long local = 0;
     bool neg = false;
 #pragma unroll
     for (int i = 0; i < ITEMS; ++i) {
         const int r = tid * ITEMS + i;
-        long long c = (r < P && r < CAP) ? a.counts[r] : 0;
+        long long c = cnt[i];
         if (a.compact && r < P && !((s_arr[r >> 6] >> (r & 63)) & 1ull)) c = 0;   // compact reading: no slot for a missing rank
         if (c < 0) { neg = true; c = 0; }
         cnt[i] = c;
@@ -190,41 +197,8 @@ allgatherv_kernel(const GatherArgs a, const __grid_constant__ PtrTable<CAP> tbl)
     }
 }
 
-int sm_count() {
-    static thread_local int cached_dev = -1, cached = 0;
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
-    if (dev != cached_dev) {
-        int n = 0;
-        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
-        cached = n;
-        cached_dev = dev;
-    }
-    return cached;
-}
-
-// Resident blocks of the kernel on the whole device (the blocks loop over the chunks, so more would only repeat
-// the scan in a second wave).
-template <int CAP>
-unsigned resident_blocks() {
-    static thread_local int cached_dev = -1;
-    static thread_local unsigned cached = 0;
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return 148 * 4;
-    if (dev != cached_dev) {
-        int per_sm = 0;
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, allgatherv_kernel<CAP>, GV_THREADS, 0) != cudaSuccess || per_sm < 1)
-            per_sm = 1;
-        cached = (unsigned)(sm_count() * per_sm);
-        cached_dev = dev;
-    }
-    return cached;
-}
-
 template <int CAP>
 void launch(const GatherArgs& a, const void* const* bufs, unsigned grid, cudaStream_t stream) {
-    const unsigned cap_blocks = resident_blocks<CAP>();
-    if (grid > cap_blocks) grid = cap_blocks;
     PtrTable<CAP> tbl;
     for (int r = 0; r < CAP; ++r) tbl.p[r] = r < a.P ? bufs[r] : nullptr;
     allgatherv_kernel<CAP><<<grid, GV_THREADS, 0, stream>>>(a, tbl);
@@ -250,10 +224,10 @@ int gather_common(const void* const* bufs, const int64_t* counts, int P, ec_dtyp
     GatherArgs a;
     a.counts = counts; a.arrival = arrival_mask; a.displs = displs; a.out = reinterpret_cast<char*>(out);
     a.status = status; a.capacity = out_capacity_elems; a.P = P; a.esize = es; a.compact = compact;
-    // enough blocks for every chunk the capacity allows, at most one wave of resident blocks (the blocks loop)
+    // One block per chunk the capacity allows; beyond GV_MAX_BLOCKS chunks the blocks loop.
     size_t chunks = (out_capacity_elems * (size_t)es + GV_CHUNK_BYTES - 1) / GV_CHUNK_BYTES;
     if (chunks < 1) chunks = 1;
-    const unsigned grid = (unsigned)(chunks < 0x7fffffffull ? chunks : 0x7fffffffull);
+    const unsigned grid = (unsigned)(chunks < (size_t)GV_MAX_BLOCKS ? chunks : (size_t)GV_MAX_BLOCKS);
     if (P <= 64) launch<64>(a, bufs, grid, stream);
     else if (P <= 256) launch<256>(a, bufs, grid, stream);
     else launch<EC_MAX_RANKS>(a, bufs, grid, stream);
