@@ -61,7 +61,7 @@ using tc::tmem_dealloc;
 constexpr int TILE = 128;                       // points per tile = rows of an accumulator
 constexpr int MAX_GROUPS = 4;                   // epilogue groups of four warps (3: the same speed; 5, 6: slower, registers spill)
 constexpr int MAX_STAGES = 8;
-constexpr int MAX_SLOTS = 4;                    // operand buffers of the sums GEMM: 2 when only changes are summed, else 3
+constexpr int MAX_SLOTS = 4;                    // operand buffers of the sums GEMM: 2 when only changes are summed, else 4
 constexpr int MAX_THREADS = (4 * MAX_GROUPS + 3) * 32;
 constexpr uint32_t WAIT_LIMIT = 1u << 24;
 constexpr uint32_t OCHUNK = TILE * 16;          // one-hot tile: bytes between chunks of 8 centroids
@@ -79,12 +79,16 @@ struct Plan {
 };
 __host__ __device__ inline Plan plan_of(int D, int K, bool partials, bool delta) {
     Plan p;
-    p.slots = partials ? (delta ? 2 : 3) : 0;
+    p.slots = partials ? (delta ? 2 : 4) : 0;
     const uint32_t SLOTS = (uint32_t)p.slots;
     const uint32_t npad = (uint32_t)npad_of(K), XC = xchunk_of(D);
     const uint32_t acc = partials ? 2u : 0u;
     int g = (int)(512u / npad) - (int)acc;
     p.groups = g > MAX_GROUPS ? MAX_GROUPS : g < 1 ? 1 : g;
+    // All points summed: four slots for three groups, so that the slot a group converts into was last used by another
+    // group's tile, decided a whole tile earlier - its sums GEMM is over (measured on N = 2^22, D = 32, K = 64: 269 us per
+    // iteration; four groups on four slots 314, four groups on three slots with the rows converted after the decision 375).
+    if (partials && !delta && p.groups > 3) p.groups = 3;
     uint32_t need = ((uint32_t)p.groups + acc) * npad, cols = 32;
     while (cols < need) cols <<= 1;
     p.tmem_cols = cols;
@@ -576,11 +580,57 @@ ws_fused_kernel(const __grid_constant__ CUtensorMap pmap, const float* __restric
                 }
                 break;
             }
-            // The stage goes back to the producer once the search has read the tile (the issuer's commit) and this group's
-            // four warps have taken the descriptor (here): the epilogue itself reads nothing of the staged tile.
-            warrive(B_empty(s));
             const size_t j = (size_t)td.base + (size_t)t;
             const bool live = j < (size_t)td.end;
+            // The groups take turns on the slots.  Once the sums issuer is through with tile i - SLOTS (the slot's last possible
+            // user before this tile) the slot's book-keeping is final: whether the rows of this warp's position still have
+            // one-hot entries set (they must be cleared before the slot's next GEMM), and how many GEMMs were issued from
+            // the slot, which says which phase of its barrier to wait for before the operands may be touched - at most one
+            // phase back, because every user waits for its predecessor.
+            int info = 0;                                        // bit 0: stale rows, bits 1..: GEMMs issued from the slot
+            auto slot_info = [&]() -> bool {
+                // the sums issuer must have taken what the group said about its previous tile
+                if (n > 0 && !wwait(B_tiledone(g), (uint32_t)(n - 1) & 1u, 10 | (i << 8))) return false;
+                if (lane == 0 && i >= SLOTS) {
+                    const long long t0 = clock64();
+                    while (s_ctrl[26] < i - SLOTS + 1) {
+                        if (*s_abort != 0 || clock64() - t0 > 4000000000LL) { if (*s_abort == 0) *s_abort = 14; info = -1; break; }
+                    }
+                    if (info == 0) info = (s_ctrl[32 + 4 * slot + (warp & 3)] != 0 ? 1 : 0) | (s_ctrl[28 + slot] << 1);
+                }
+                info = __shfl_sync(0xffffffffu, info, 0);
+                return info >= 0;
+            };
+            if (PARTIALS && !DELTA) {
+                // All points are summed: the operand rows do not depend on the labels, so they are made now, out of the staged
+                // tile, while the search's MMAs run - bf16 high and low parts of the row (low = bf16(x - high)): chunk column
+                // 2 kc resp. 2 kc + 1 of the slot.
+                if (!slot_info()) { ok = false; break; }
+                const int uses = info >> 1;
+                if (uses > 0 && !wwait(B_slotfree(slot), (uint32_t)(uses - 1) & 1u, 7)) { ok = false; break; }
+                if (live) {
+                    const unsigned char* row = sm + pl.stage + (size_t)s * pl.stage_bytes;
+                    unsigned char* xs = sm + pl.slot + (size_t)slot * pl.slot_bytes;
+#pragma unroll
+                    for (int kc = 0; kc < KCH; ++kc) {
+                        const float4 va = *reinterpret_cast<const float4*>(row + swz_off<D>(t, 2 * kc));
+                        const float4 vb = *reinterpret_cast<const float4*>(row + swz_off<D>(t, 2 * kc + 1));
+                        const float v[8] = {va.x, va.y, va.z, va.w, vb.x, vb.y, vb.z, vb.w};
+                        uint32_t hw[4], lw[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            hw[e] = pack_bf16(v[2 * e], v[2 * e + 1]);
+                            const float ah = __uint_as_float(hw[e] << 16), bh = __uint_as_float(hw[e] & 0xFFFF0000u);
+                            lw[e] = pack_bf16(v[2 * e] - ah, v[2 * e + 1] - bh);
+                        }
+                        *reinterpret_cast<uint4*>(xs + (size_t)(2 * kc) * XC + (size_t)t * 16) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
+                        *reinterpret_cast<uint4*>(xs + (size_t)(2 * kc + 1) * XC + (size_t)t * 16) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
+                    }
+                }
+            }
+            // The stage goes back to the producer once the search has read the tile (the issuer's commit) and this group's
+            // four warps are through with it (here): the descriptor taken and, when all points are summed, the rows converted.
+            warrive(B_empty(s));
             const int old = (DELTA && live) ? labels[j] : -1;
             const float xn = live ? __ldg(xnorm + j) : 0.0f;      // |x|^2, made once per context: the staged tile is the tensor core's alone
             if (!wwait(B_accfull(g), (uint32_t)n & 1u, 8)) { ok = false; break; }
@@ -632,27 +682,11 @@ ws_fused_kernel(const __grid_constant__ CUtensorMap pmap, const float* __restric
                 // clears); only a thread whose label changed converts its row and sets its one-hot row - the other rows of
                 // the slot keep whatever finite numbers they hold, against one-hot rows that are zero.
                 const bool any_w = __any_sync(0xffffffffu, changed);
-                // the sums issuer must have taken what the group said about its previous tile
-                if (n > 0 && !wwait(B_tiledone(g), (uint32_t)(n - 1) & 1u, 10 | (i << 8))) { ok = false; break; }
-                // The groups take turns on the slots.  Once the sums issuer is through with tile i - SLOTS (the slot's last possible
-                // user before this tile) the slot's book-keeping is final: whether the rows of this warp's position still have
-                // one-hot entries set (they must be cleared before the slot's next GEMM), and how many GEMMs were issued from
-                // the slot, which says which phase of its barrier to wait for before the operands may be touched - at most one
-                // phase back, because every user waits for its predecessor.
-                int info = 0;                                        // bit 0: stale rows, bits 1..: GEMMs issued from the slot
-                if (lane == 0 && i >= SLOTS) {
-                    const long long t0 = clock64();
-                    while (s_ctrl[26] < i - SLOTS + 1) {
-                        if (*s_abort != 0 || clock64() - t0 > 4000000000LL) { if (*s_abort == 0) *s_abort = 14; info = -1; break; }
-                    }
-                    if (info == 0) info = (s_ctrl[32 + 4 * slot + (warp & 3)] != 0 ? 1 : 0) | (s_ctrl[28 + slot] << 1);
-                }
-                info = __shfl_sync(0xffffffffu, info, 0);
-                if (info < 0) { ok = false; break; }
+                if (DELTA && !slot_info()) { ok = false; break; }
                 const bool stale = (info & 1) != 0;
                 if (any_w || stale) {
                     const int uses = info >> 1;
-                    if (uses > 0 && !wwait(B_slotfree(slot), (uint32_t)(uses - 1) & 1u, 7)) { ok = false; break; }
+                    if (DELTA && uses > 0 && !wwait(B_slotfree(slot), (uint32_t)(uses - 1) & 1u, 7)) { ok = false; break; }
                     unsigned char* xs = sm + pl.slot + (size_t)slot * pl.slot_bytes;
                     unsigned char* oh = xs + pl.oh_off;
                     uint16_t* prev = reinterpret_cast<uint16_t*>(sm + pl.prev) + slot * TILE + t;
@@ -676,7 +710,7 @@ ws_fused_kernel(const __grid_constant__ CUtensorMap pmap, const float* __restric
                         }
                         // bf16 high and low parts of the row (low = bf16(x - high)): chunk column 2 kc resp. 2 kc + 1
 #pragma unroll
-                        for (int kc = 0; kc < KCH; ++kc) {
+                        for (int kc = 0; DELTA && kc < KCH; ++kc) {
                             const float4 va = __ldg(reinterpret_cast<const float4*>(points + j * D) + 2 * kc);   // (from L2: the tile was just read)
                             const float4 vb = __ldg(reinterpret_cast<const float4*>(points + j * D) + 2 * kc + 1);
                             const float v[8] = {va.x, va.y, va.z, va.w, vb.x, vb.y, vb.z, vb.w};
