@@ -79,15 +79,14 @@ struct Plan {
 };
 __host__ __device__ inline Plan plan_of(int D, int K, bool partials, bool delta) {
     Plan p;
-    p.slots = partials ? (delta ? 2 : 4) : 0;
-    const uint32_t SLOTS = (uint32_t)p.slots;
     const uint32_t npad = (uint32_t)npad_of(K), XC = xchunk_of(D);
     const uint32_t acc = partials ? 2u : 0u;
     int g = (int)(512u / npad) - (int)acc;
     p.groups = g > MAX_GROUPS ? MAX_GROUPS : g < 1 ? 1 : g;
     // All points summed: four slots for three groups, so that the slot a group converts into was last used by another
     // group's tile, decided a whole tile earlier - its sums GEMM is over (measured on N = 2^22, D = 32, K = 64: 269 us per
-    // iteration; four groups on four slots 314, four groups on three slots with the rows converted after the decision 375).
+    // iteration; four groups on four slots 314, four groups on three slots with the rows converted after the decision 375;
+    // a group converting the next group's tile instead of its own: 310 with four groups, 325 with three).
     if (partials && !delta && p.groups > 3) p.groups = 3;
     uint32_t need = ((uint32_t)p.groups + acc) * npad, cols = 32;
     while (cols < need) cols <<= 1;
@@ -98,13 +97,22 @@ __host__ __device__ inline Plan plan_of(int D, int K, bool partials, bool delta)
     uint32_t slot = p.oh_off + npad / 8u * OCHUNK;
     if (slot < 16u * XC) slot = 16u * XC;            // the sums MMA reads 128 rows = 16 chunk columns from the slot's start
     p.slot_bytes = (slot + 127u) & ~127u;
+    // Slots: two when only changes are summed (few tiles have a GEMM at all); when all points are summed four if that
+    // leaves three stages, else three.
+    p.slots = partials ? (delta ? 2 : MAX_SLOTS) : 0;
     uint32_t off = 0;
-    const uint32_t fixed_after_stages = npad * (uint32_t)D * 4u + 1024u   // b (1024-aligned)
-        + 4096u + npad * 32u                                              // ones, cnb
-        + SLOTS * p.slot_bytes + SLOTS * TILE * 2u                        // slots, previous one-hot chunks
-        + npad * 8u + 1024u + 4096u;                                       // cn, drift, need words, descriptors, control, barriers
-    int st = (int)((226u * 1024u - fixed_after_stages) / p.stage_bytes);
-    p.stages = st > MAX_STAGES ? MAX_STAGES : st;
+    for (;;) {
+        const uint32_t SLOTS = (uint32_t)p.slots;
+        const uint32_t fixed_after_stages = npad * (uint32_t)D * 4u + 1024u   // b (1024-aligned)
+            + 4096u + npad * 32u                                              // ones, cnb
+            + SLOTS * p.slot_bytes + SLOTS * TILE * 2u                        // slots, previous one-hot chunks
+            + npad * 8u + 1024u + 4096u;                                       // cn, drift, need words, descriptors, control, barriers
+        const int st = fixed_after_stages < 226u * 1024u ? (int)((226u * 1024u - fixed_after_stages) / p.stage_bytes) : 0;
+        p.stages = st > MAX_STAGES ? MAX_STAGES : st;
+        if (partials && !delta && p.slots > 3 && p.stages < 3) { p.slots = 3; continue; }
+        break;
+    }
+    const uint32_t SLOTS = (uint32_t)p.slots;
     p.stage = off; off += (uint32_t)p.stages * p.stage_bytes;
     off = (off + 1023u) & ~1023u;
     p.b = off; off += npad * (uint32_t)D * 4u;       // -2 c, tf32, K-major, swizzled like the stages
