@@ -241,16 +241,22 @@ def run_ours(args, rank, world, local_rank):
         barrier()
         t_host0 = time.perf_counter()
         K = args.steps
-        # Every SAMPLE-th step carries per-launch events (kernel durations for the roofline, step times for the
-        # confidence interval); the steps in between run without them, so the events do not weigh on `value`.
+        # The timed region: exactly K steps between two events, nothing else in the stream (an event between two launches
+        # keeps the second from starting as a programmatic dependent of the first and costs about a tenth of a step).
+        t_all0 = torch.cuda.Event(enable_timing=True)
+        t_all1 = torch.cuda.Event(enable_timing=True)
+        t_all0.record(stream)
+        for k in range(K):
+            epoch()
+        t_all1.record(stream)
+        barrier()
+        # Right after it, the same steps once more with an event around every launch and every step: kernel durations
+        # for the roofline, step times for the confidence interval.  Every step when K <= 32, else every 8th.
         SAMPLE = 1 if K <= 32 else 8
         sampled = [k for k in range(K) if k % SAMPLE == 0]
         step_ev = {k: (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for k in sampled}
         apply_ev = {k: [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
                         for _ in d_masks] for k in sampled}
-        t_all0 = torch.cuda.Event(enable_timing=True)
-        t_all1 = torch.cuda.Event(enable_timing=True)
-        t_all0.record(stream)
         for k in range(K):
             if k in step_ev:
                 step_ev[k][0].record(stream)
@@ -258,7 +264,6 @@ def run_ours(args, rank, world, local_rank):
                 step_ev[k][1].record(stream)
             else:
                 epoch()
-        t_all1.record(stream)
         barrier()
         t_host1 = time.perf_counter()
     if args.profile_only:
@@ -357,8 +362,10 @@ def run_ours(args, rank, world, local_rank):
             "l2": "rank buffers (1 GiB) exceed L2 every step; the 64 MiB result is carried between rounds as in the workload",
             "ms_per_step_mean_ci95": [round(m_step, 5), round(ci_step, 5)],
             "ms_per_step_median_min": [round(statistics.median(steps_ms), 5), round(min(steps_ms), 5)],
-            "timing": f"value: two events around all {K} steps; per-launch and per-step events on every "
-                      + ("step" if SAMPLE == 1 else f"{SAMPLE}th step"),
+            "timing": f"value: two events around the {K} timed steps, nothing else in the stream; the per-launch and per-step "
+                      f"events (roofline, confidence interval) come from the same {K} steps run once more right after, "
+                      + ("an event pair on every step" if SAMPLE == 1 else f"an event pair on every {SAMPLE}th step")
+                      + " (events between the launches cost about a tenth of a step: ms_per_step_mean_ci95 includes them)",
             "ms_per_round_mean": [round(statistics.fmean(r[t] for r in round_ms), 5) for t in range(len(d_masks))],
             "GBps_per_round": [round(per_round_bytes[t] / (statistics.fmean(r[t] for r in round_ms) * 1e-3) / 1e9, 1)
                                for t in range(len(d_masks))],
