@@ -248,7 +248,10 @@ __device__ __forceinline__ void best_two_of_16(const uint32_t (&raw)[16], uint32
 // 32 consecutive points at a time and leaves one byte, nonzero if the bounds of one of them no longer hold.
 // need: [blocks][need_words] words; byte p of a block's words = points [32p, 32p + 32) of its run, so a word is a
 // tile of the fused kernel.
-constexpr int BC_THREADS = 256;
+#ifndef EC_BC_THREADS
+#define EC_BC_THREADS 128
+#endif
+constexpr int BC_THREADS = EC_BC_THREADS;
 constexpr int NEED_WORDS_MAX = 256;
 __global__ void __launch_bounds__(BC_THREADS)
 bounds_check_kernel(size_t N, int P, int C, int K, const int32_t* __restrict__ labels, const float2* __restrict__ bounds,
@@ -267,7 +270,10 @@ bounds_check_kernel(size_t N, int P, int C, int K, const int32_t* __restrict__ l
     unsigned char* out = reinterpret_cast<unsigned char*>(need + (size_t)blockIdx.x * need_words);
     const int pieces = (int)((b1 - b0 + 31) / 32), slots = need_words * 4;
     bool mine = false;                                                 // one of this thread's points may change its label
-    constexpr int BC_U = 4;                                            // pieces a warp has in flight
+#ifndef EC_BC_U
+#define EC_BC_U 4
+#endif
+    constexpr int BC_U = EC_BC_U;                                            // pieces a warp has in flight
     for (int p0 = w; p0 < slots; p0 += BC_U * (BC_THREADS / 32)) {
         bool fail[BC_U];
         float2 bd[BC_U];
