@@ -17,7 +17,8 @@
  *     default stream).  Buffers and notification words must stay valid and
  *     unmodified until that work has completed.  Notification words are read on
  *     the device when the kernel runs, so a producer may set bits in stream
- *     order right up to the call ("write early, check late", Sec. II).
+ *     order right up to the call (Sec. II: data is written as soon as it exists and
+ *     its arrival is looked at as late as possible).
  *   - A context is not thread-safe and expects its calls in one stream order;
  *     distinct contexts are independent.
  *
@@ -155,8 +156,8 @@ int ec_allreduce_apply(ec_ctx_t* ctx, const void* const* rank_bufs, int P, size_
  *                  notif_clock >= clock - slack (slack = 0 is the classic synchronous allreduce).
  *   contrib_count  device uint32 [S] or NULL: number of contributions used.
  *   seg_clock      device uint32 [S] or NULL: the clock of the reduction = the smallest clock among
- *                  the contributions used (0 if none): "the result ... is associated with the
- *                  minimum clock of both contributions".
+ *                  the contributions used (0 if none): Sec. III-A gives a reduction the smaller of
+ *                  the clocks of what went into it.
  *   wait_count     device uint32 [S] or NULL: contributions that were too stale (or absent).  The
  *                  paper's process blocks on those; this call never waits - it reports them, and
  *                  the caller applies again once they have been refreshed.
@@ -488,11 +489,11 @@ int ec_mf_destroy(ec_mf_t* mf);
 int ec_bcast(const void* src, void* const* dst_bufs, int P, int root, size_t n, ec_dtype_t dtype,
              size_t segment_size, double data_fraction, uint64_t* notify, ec_stream_t stream);
 
-/* Strategy 1, "send less data": the first ceil(fraction * S) segments of every rank count as
+/* Strategy 1 of Sec. III-B, less data from everybody: the first ceil(fraction * S) segments of every rank count as
  * arrived, the others do not.  0 <= fraction <= 1. */
 int ec_mask_data_fraction(int P, size_t S, double fraction, uint64_t* host_mask);
 
-/* Strategy 2, "send all data but leave processes out": the binomial spanning tree works in stages
+/* Strategy 2 of Sec. III-B, all the data of fewer processes: the binomial spanning tree works in stages
  * that double the number of involved processes (stage k brings in ranks 2^k .. 2^(k+1)-1); whole
  * stages are added until at least fraction * P processes take part.  Ranks 0 .. *ranks_included-1
  * count as arrived for every segment.  The last stage alone adds half of the processes, so
