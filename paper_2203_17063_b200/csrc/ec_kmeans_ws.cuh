@@ -9,7 +9,8 @@
 //                            A = the stage (128 points x D floats, K-major), B = -2 c rounded to tf32 (K-major, same
 //                            swizzle), plus one step of a constant [1,1,1,0..] chunk against [hi, mid, lo](|c|^2), so
 //                            the accumulator in tensor memory holds v_k = |c_k|^2 - 2 x.c_k for 128 points x all
-//                            centroids.  One accumulator per epilogue group, so tiles overlap;
+//                            centroids.  Tile i goes to accumulator i mod A, A = as many as tensor memory holds beside
+//                            the sums (six for K = 64), so the search runs ahead of the groups;
 //   epilogue groups (4 warps each, tile i goes to group i mod G): read the scores with tcgen05.ld (one point per
 //                            thread, 16 columns at a time with the next 16 on their way), find the best two by a
 //                            tournament of min/max pairs whose low mantissa bits carry the column index, decide (exact
@@ -61,6 +62,7 @@ using tc::tmem_dealloc;
 constexpr int TILE = 128;                       // points per tile = rows of an accumulator
 constexpr int MAX_GROUPS = 4;                   // epilogue groups of four warps (3: the same speed; 5, 6: slower, registers spill)
 constexpr int MAX_STAGES = 8;
+constexpr int MAX_ACCS = 8;
 constexpr int MAX_SLOTS = 4;                    // operand buffers of the sums GEMM: 2 when only changes are summed, else 4
 constexpr int MAX_THREADS = (4 * MAX_GROUPS + 3) * 32;
 constexpr uint32_t WAIT_LIMIT = 1u << 24;
@@ -72,7 +74,7 @@ __host__ __device__ constexpr uint32_t xchunk_of(int D) { return TILE * 16 + 102
 
 // Shared memory of a block (byte offsets from a 1024-byte aligned base) and its tensor-memory columns.
 struct Plan {
-    int groups, stages, slots;
+    int groups, stages, slots, accs;                // accs: search accumulators in tensor memory (tile i uses i mod accs)
     uint32_t tmem_cols;
     uint32_t stage_bytes, slot_bytes, oh_off;       // oh_off: one-hot tile inside a slot
     uint32_t stage, b, ones, cnb, slot, prev, cn, drift, need, desc, ctrl, bar, total;
@@ -88,7 +90,14 @@ __host__ __device__ inline Plan plan_of(int D, int K, bool partials, bool delta)
     // iteration; four groups on four slots 314, four groups on three slots with the rows converted after the decision 375;
     // a group converting the next group's tile instead of its own: 310 with four groups, 325 with three).
     if (partials && !delta && p.groups > 3) p.groups = 3;
-    uint32_t need = ((uint32_t)p.groups + acc) * npad, cols = 32;
+    // Search accumulators: as many as tensor memory holds beside the two of the sums (at most MAX_ACCS), so that the search
+    // of a group's next tile is over before the group asks for it, whatever else the tensor core had queued.
+#ifndef EC_WS_ACCS
+#define EC_WS_ACCS MAX_ACCS
+#endif
+    int a = (int)(512u / npad) - (int)acc;
+    p.accs = a > EC_WS_ACCS ? EC_WS_ACCS : a < p.groups ? p.groups : a;
+    uint32_t need = ((uint32_t)p.accs + acc) * npad, cols = 32;
     while (cols < need) cols <<= 1;
     p.tmem_cols = cols;
     p.stage_bytes = (uint32_t)TILE * (uint32_t)D * 4u;
@@ -302,7 +311,7 @@ ws_fused_kernel(const __grid_constant__ CUtensorMap pmap, const float* __restric
     const Plan pl = plan_of(D, K, PARTIALS, DELTA);
     const int SLOTS = pl.slots;
     const int npad = npad_of(K);
-    const int G = pl.groups, NST = pl.stages;
+    const int G = pl.groups, NST = pl.stages, A = pl.accs;
     unsigned char* sm = ws_smem_raw + ((1024u - (smem_u32(ws_smem_raw) & 1023u)) & 1023u);
     const uint32_t sm_u = smem_u32(sm);
     float* s_cn = reinterpret_cast<float*>(sm + pl.cn);
@@ -320,13 +329,14 @@ ws_fused_kernel(const __grid_constant__ CUtensorMap pmap, const float* __restric
     const uint32_t bar0 = sm_u + pl.bar;
     auto B_full = [&](int s) { return bar0 + 8u * (uint32_t)s; };
     auto B_empty = [&](int s) { return bar0 + 8u * (uint32_t)(MAX_STAGES + s); };
-    auto B_accfull = [&](int g) { return bar0 + 8u * (uint32_t)(2 * MAX_STAGES + g); };
-    auto B_accempty = [&](int g) { return bar0 + 8u * (uint32_t)(2 * MAX_STAGES + MAX_GROUPS + g); };
-    auto B_decided = [&](int g) { return bar0 + 8u * (uint32_t)(2 * MAX_STAGES + 2 * MAX_GROUPS + g); };
-    auto B_tiledone = [&](int g) { return bar0 + 8u * (uint32_t)(2 * MAX_STAGES + 3 * MAX_GROUPS + g); };
-    auto B_rundone = [&](int p) { return bar0 + 8u * (uint32_t)(2 * MAX_STAGES + 4 * MAX_GROUPS + p); };
-    auto B_drained = [&](int p) { return bar0 + 8u * (uint32_t)(2 * MAX_STAGES + 4 * MAX_GROUPS + 2 + p); };
-    auto B_slotfree = [&](int sl) { return bar0 + 8u * (uint32_t)(2 * MAX_STAGES + 5 * MAX_GROUPS + 4 + sl); };   // (MAX_SLOTS of them)
+    auto B_accfull = [&](int a) { return bar0 + 8u * (uint32_t)(2 * MAX_STAGES + a); };
+    auto B_accempty = [&](int a) { return bar0 + 8u * (uint32_t)(2 * MAX_STAGES + MAX_ACCS + a); };
+    constexpr int BAR_GROUPS = 2 * MAX_STAGES + 2 * MAX_ACCS;     // index of the first per-group barrier
+    auto B_decided = [&](int g) { return bar0 + 8u * (uint32_t)(BAR_GROUPS + g); };
+    auto B_tiledone = [&](int g) { return bar0 + 8u * (uint32_t)(BAR_GROUPS + MAX_GROUPS + g); };
+    auto B_rundone = [&](int p) { return bar0 + 8u * (uint32_t)(BAR_GROUPS + 2 * MAX_GROUPS + p); };
+    auto B_drained = [&](int p) { return bar0 + 8u * (uint32_t)(BAR_GROUPS + 2 * MAX_GROUPS + 2 + p); };
+    auto B_slotfree = [&](int sl) { return bar0 + 8u * (uint32_t)(BAR_GROUPS + 2 * MAX_GROUPS + 4 + sl); };   // (MAX_SLOTS of them: 48 barriers in all)
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int nthreads = (4 * G + 3) * 32;
@@ -347,9 +357,8 @@ ws_fused_kernel(const __grid_constant__ CUtensorMap pmap, const float* __restric
     if (warp == 4 * G + 1) tmem_alloc(smem_u32(const_cast<int*>(s_ctrl + 6)), pl.tmem_cols);
     if (tid == 0) {
         for (int s = 0; s < NST; ++s) { mbar_init(B_full(s), 1); mbar_init(B_empty(s), 5); }   // empty: the search's commit + the four warps that read the descriptor
-        for (int g = 0; g < G; ++g) {
-            mbar_init(B_accfull(g), 1); mbar_init(B_accempty(g), 4); mbar_init(B_decided(g), 4);
-        }
+        for (int a = 0; a < A; ++a) { mbar_init(B_accfull(a), 1); mbar_init(B_accempty(a), 4); }
+        for (int g = 0; g < G; ++g) mbar_init(B_decided(g), 4);
         for (int g = 0; g < G; ++g) mbar_init(B_tiledone(g), 1);
         for (int sl = 0; sl < MAX_SLOTS; ++sl) mbar_init(B_slotfree(sl), 1);
         s_ctrl[0] = 0; s_ctrl[1] = 0; s_ctrl[2] = 0; s_ctrl[3] = 0;
@@ -403,7 +412,7 @@ ws_fused_kernel(const __grid_constant__ CUtensorMap pmap, const float* __restric
     __syncthreads();
     fence_after_sync();
     const uint32_t tmem_base = (uint32_t)s_ctrl[6];
-    const uint32_t sums_col0 = (uint32_t)(G * npad);
+    const uint32_t sums_col0 = (uint32_t)(A * npad);
     bool ok = true;                                           // this thread has seen no wait give up
 
     if (warp == 4 * G) {
@@ -477,24 +486,24 @@ ws_fused_kernel(const __grid_constant__ CUtensorMap pmap, const float* __restric
             const uint64_t adesc0 = swz_desc<D>(sm_u + pl.stage);
             const uint64_t ones_desc = smem_desc(sm_u + pl.ones, 2048, 128), cnb_desc = smem_desc(sm_u + pl.cnb, (uint32_t)npad * 16, 128);
             const uint32_t stage_units = pl.stage_bytes >> 4;
-            int s = 0, g = 0;
-            uint32_t full_par = 0, empty_par = 1;            // parities of the next waits on full[s] and accempty[g]
+            int s = 0, a = 0;                                 // tile i: stage i mod stages, accumulator i mod accs
+            uint32_t full_par = 0, empty_par = 1;            // parities of the next waits on full[s] and accempty[a]
             bool first_round = true;                          // the accumulators start out free
             for (;;) {
                 if (!wait_or_abort(B_full(s), full_par, s_abort, 3)) { ok = false; break; }
                 if (s_desc[s].run < 0) break;
-                if (!first_round && !wait_or_abort(B_accempty(g), empty_par, s_abort, 4)) { ok = false; break; }
+                if (!first_round && !wait_or_abort(B_accempty(a), empty_par, s_abort, 4)) { ok = false; break; }
                 fence_after_sync();
-                const uint32_t acc = tmem_base + (uint32_t)(g * npad);
+                const uint32_t acc = tmem_base + (uint32_t)(a * npad);
                 const uint64_t adesc = adesc0 + (uint64_t)((uint32_t)s * stage_units);
 #pragma unroll
                 for (int ks = 0; ks < D / 8; ++ks)             // 8 coordinates (32 bytes) per step
                     mma_tf32(acc, adesc + (uint64_t)(2 * ks), bdesc[ks], idesc, ks > 0 ? 1u : 0u);
                 mma_tf32(acc, ones_desc, cnb_desc, idesc, 1u);
-                mma_commit(B_accfull(g));
+                mma_commit(B_accfull(a));
                 mma_commit(B_empty(s));                        // the tile has been read: its stage goes back to the producer
                 if (++s == NST) { s = 0; full_par ^= 1u; }
-                if (++g == G) { g = 0; empty_par ^= 1u; first_round = false; }
+                if (++a == A) { a = 0; empty_par ^= 1u; first_round = false; }
             }
         }
     } else if (warp == 4 * G + 2) {
@@ -569,10 +578,14 @@ ws_fused_kernel(const __grid_constant__ CUtensorMap pmap, const float* __restric
         int s = g % NST, n = 0;
         uint32_t lap = (uint32_t)(g / NST);
         int slot = PARTIALS ? g % SLOTS : 0;
+        int a = g % A;                                        // the tile's search accumulator, on its lapa-th use
+        uint32_t lapa = (uint32_t)(g / A);
         for (int i = g; ok; i += G, ++n) {
             if (n > 0) {
                 s += G;
                 while (s >= NST) { s -= NST; ++lap; }
+                a += G;
+                while (a >= A) { a -= A; ++lapa; }
                 if (PARTIALS) {
                     slot += G;
                     while (slot >= SLOTS) slot -= SLOTS;
@@ -641,12 +654,12 @@ ws_fused_kernel(const __grid_constant__ CUtensorMap pmap, const float* __restric
             warrive(B_empty(s));
             const int old = (DELTA && live) ? labels[j] : -1;
             const float xn = live ? __ldg(xnorm + j) : 0.0f;      // |x|^2, made once per context: the staged tile is the tensor core's alone
-            if (!wwait(B_accfull(g), (uint32_t)n & 1u, 8)) { ok = false; break; }
+            if (!wwait(B_accfull(a), lapa & 1u, 8)) { ok = false; break; }
             fence_after_sync();
             float m1 = __int_as_float(0x7f800000), m2 = m1;
             {
                 // 16 columns at a time, the next 16 on their way while these are looked at (npad / 16 is even)
-                const uint32_t col0 = lane_base + (uint32_t)(g * npad);
+                const uint32_t col0 = lane_base + (uint32_t)(a * npad);
                 uint32_t va[16], vb[16];
                 tmem_ld16_nowait(col0, va);
                 for (int ch = 0; ch < npad / 16; ch += 2) {
@@ -669,9 +682,9 @@ ws_fused_kernel(const __grid_constant__ CUtensorMap pmap, const float* __restric
             const float tau = TAU_SCALE * (xn + cmax);
             const bool redo = live && !(m2 - m1 > tau);
             if (__any_sync(0xffffffffu, redo))            // rare on separated data: kept out of line, away from this loop's registers
-                kb = redecide<D>(redo, kb, m1 + tau, points + j * D, lane_base + (uint32_t)(g * npad), npad, centroids, K);
+                kb = redecide<D>(redo, kb, m1 + tau, points + j * D, lane_base + (uint32_t)(a * npad), npad, centroids, K);
             fence_before_sync();
-            warrive(B_accempty(g));                      // the accumulator may take the group's next tile
+            warrive(B_accempty(a));                      // the accumulator may take another tile
             const bool changed = live && !(DELTA && old == kb);
             if (changed) labels[j] = kb;
             if (PARTIALS && BOUNDS && live) {
