@@ -3,7 +3,7 @@
 // One persistent block per SM.  The fp32 points never pass through registers on their way to the tensor core:
 //
 //   producer (one thread)    walks the block's runs and, for every tile of 128 points that has to be searched,
-//                            issues one bulk tensor copy (cp.async.bulk.tensor.2d, 128-byte swizzle, no multicast,
+//                            issues one bulk tensor copy (cp.async.bulk.tensor.2d, 128-byte swizzle, this block only,
 //                            this GPU's memory only) into a ring of shared-memory stages, each with its mbarrier;
 //   search issuer (one thread) multiplies a landed tile, as it lies, with the centroid operand: tcgen05.mma kind::tf32,
 //                            A = the stage (128 points x D floats, K-major), B = -2 c rounded to tf32 (K-major, same
