@@ -5,7 +5,8 @@
 //   producer (one thread)    walks the block's runs and, for every tile of 128 points that has to be searched,
 //                            issues one bulk tensor copy (cp.async.bulk.tensor.2d, 128-byte swizzle, this block only,
 //                            this GPU's memory only) into a ring of shared-memory stages, each with its mbarrier;
-//   search issuer (one thread) multiplies a landed tile, as it lies, with the centroid operand: tcgen05.mma kind::tf32,
+//   search issuers (two threads: even tiles, odd tiles) multiply a landed tile, as it lies, with the centroid
+//                            operand: tcgen05.mma kind::tf32,
 //                            A = the stage (128 points x D floats, K-major), B = -2 c rounded to tf32 (K-major, same
 //                            swizzle), plus one step of a constant [1,1,1,0..] chunk against [hi, mid, lo](|c|^2), so
 //                            the accumulator in tensor memory holds v_k = |c_k|^2 - 2 x.c_k for 128 points x all
@@ -64,7 +65,7 @@ constexpr int MAX_GROUPS = 4;                   // epilogue groups of four warps
 constexpr int MAX_STAGES = 8;
 constexpr int MAX_ACCS = 8;
 constexpr int MAX_SLOTS = 4;                    // operand buffers of the sums GEMM: 2 when only changes are summed, else 4
-constexpr int MAX_THREADS = (4 * MAX_GROUPS + 3) * 32;
+constexpr int MAX_THREADS = (4 * MAX_GROUPS + 4) * 32;
 constexpr uint32_t WAIT_LIMIT = 1u << 24;
 constexpr uint32_t OCHUNK = TILE * 16;          // one-hot tile: bytes between chunks of 8 centroids
 constexpr float TAU_SCALE = 0.00390625f;        // 2^-8, see above
@@ -142,7 +143,7 @@ __host__ __device__ inline Plan plan_of(int D, int K, bool partials, bool delta)
     p.total = off + 1024u;                           // slack to align the base
     return p;
 }
-inline int threads_of(const Plan& p) { return (4 * p.groups + 3) * 32; }
+inline int threads_of(const Plan& p) { return (4 * p.groups + 4) * 32; }
 
 // What the producer says about the tile in a stage.
 struct TileDesc {
@@ -342,7 +343,7 @@ ws_fused_kernel(const __grid_constant__ CUtensorMap pmap, const float* __restric
     auto B_slotfree = [&](int sl) { return bar0 + 8u * (uint32_t)(BAR_GROUPS + 2 * MAX_GROUPS + 4 + sl); };   // (MAX_SLOTS of them: 48 barriers in all)
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int nthreads = (4 * G + 3) * 32;
+    const int nthreads = (4 * G + 4) * 32;
     if (tid >= nthreads) return;                             // (the launch uses exactly nthreads; kept for safety)
     const int runs = P * C;
     const bool skipping = DELTA && PARTIALS && BOUNDS && need != nullptr;
@@ -476,8 +477,11 @@ ws_fused_kernel(const __grid_constant__ CUtensorMap pmap, const float* __restric
                 }
             }
         }
-    } else if (warp == 4 * G + 1) {
-        // ---- search issuer -------------------------------------------------------------------------------------------
+    } else if (warp == 4 * G + 1 || warp == 4 * G + 3) {
+        // ---- search issuers --------------------------------------------------------------------------------------------
+        // Two of them, one for the even tiles and one for the odd ones: a thread gets a small MMA issued every 72 cycles
+        // at best, the tensor core takes one every 48, and five per tile from one thread alone were what the epilogue
+        // groups waited for (assignment of N = 2^22, D = 32, K = 64: 1400 of a group's 3250 cycles per tile).
         if (lane == 0) {
             // Everything that does not change from tile to tile is made once: this one thread's instruction stream is
             // what every tile waits for.  A descriptor's address field counts 16-byte units, so a step of 32 bytes adds 2
@@ -489,13 +493,14 @@ ws_fused_kernel(const __grid_constant__ CUtensorMap pmap, const float* __restric
             const uint64_t adesc0 = swz_desc<D>(sm_u + pl.stage);
             const uint64_t ones_desc = smem_desc(sm_u + pl.ones, 2048, 128), cnb_desc = smem_desc(sm_u + pl.cnb, (uint32_t)npad * 16, 128);
             const uint32_t stage_units = pl.stage_bytes >> 4;
-            int s = 0, a = 0;                                 // tile i: stage i mod stages, accumulator i mod accs
-            uint32_t full_par = 0, empty_par = 1;            // parities of the next waits on full[s] and accempty[a]
-            bool first_round = true;                          // the accumulators start out free
+            // tile i = first, first + 2, ...: stage i mod stages on its laps-th use, accumulator i mod accs on its lapa-th
+            const int first = warp == 4 * G + 1 ? 0 : 1;
+            int s = first % NST, a = first % A;
+            uint32_t laps = (uint32_t)(first / NST), lapa = (uint32_t)(first / A);
             for (;;) {
-                if (!wait_or_abort(B_full(s), full_par, s_abort, 3)) { ok = false; break; }
+                if (!wait_or_abort(B_full(s), laps & 1u, s_abort, 3)) { ok = false; break; }
                 if (s_desc[s].run < 0) break;
-                if (!first_round && !wait_or_abort(B_accempty(a), empty_par, s_abort, 4)) { ok = false; break; }
+                if (lapa > 0 && !wait_or_abort(B_accempty(a), (lapa - 1u) & 1u, s_abort, 4)) { ok = false; break; }
                 fence_after_sync();
                 const uint32_t acc = tmem_base + (uint32_t)(a * npad);
                 const uint64_t adesc = adesc0 + (uint64_t)((uint32_t)s * stage_units);
@@ -505,8 +510,10 @@ ws_fused_kernel(const __grid_constant__ CUtensorMap pmap, const float* __restric
                 mma_tf32(acc, ones_desc, cnb_desc, idesc, 1u);
                 mma_commit(B_accfull(a));
                 mma_commit(B_empty(s));                        // the tile has been read: its stage goes back to the producer
-                if (++s == NST) { s = 0; full_par ^= 1u; }
-                if (++a == A) { a = 0; empty_par ^= 1u; first_round = false; }
+                s += 2;
+                while (s >= NST) { s -= NST; ++laps; }
+                a += 2;
+                while (a >= A) { a -= A; ++lapa; }
             }
         }
     } else if (warp == 4 * G + 2) {
