@@ -719,6 +719,37 @@ def extras(args, dev, stream, peak):
                                                        "frac_measured": round(gbytes8 / m / 1e6 / peak, 4), "bytes": gbytes8}
     del db, d_out, g_sets, big, d_out8
 
+    # The allreduce inside a config 5 iteration on its own: 64 ranks x 64 centroid rows of 36 floats (590 KB), one row a
+    # segment, arrival probability 0.75.  Warm (everything in L2, as between the kernels of an iteration) and cold (a
+    # buffer of twice the L2 size is overwritten before every timed call).
+    P, Kc, Dc = 64, 64, 32
+    n5, seg5 = Kc * (Dc + 4), Dc + 4
+    rows5 = torch.randn(P, n5, device=dev)
+    tab5 = (C.c_void_p * P)(*[rows5[r].data_ptr() for r in range(P)])
+    mask5 = torch.from_numpy(inputs.pack_mask(inputs.bernoulli_mask(2005, 0, P, Kc, 0.75)).view(np.int64)).to(dev)
+    res5 = torch.empty(n5, device=dev)
+    cnt5 = torch.empty(Kc, dtype=torch.int32, device=dev)
+    ar5 = ec.Allreduce(P, n5, ec.F32, ec.SUM, seg5, device=dev)
+    call5 = lambda: ar5.apply_raw(tab5, mask5.data_ptr(), res5.data_ptr(), cnt5.data_ptr(), st)
+    reset5 = lambda: L.ec_allreduce_reset(ar5._h, st)
+    bytes5 = int(0.75 * P * n5 * 4) + n5 * 4 + Kc * 4
+    entry = {"bytes_about": bytes5}
+    ms = time_rotating(stream, [call5], reps, before=reset5)
+    m, ci = mean_ci(ms)
+    entry["warm"] = {"us": round(m * 1e3, 2), "ci95_us": round(ci * 1e3, 2), "GBps": round(bytes5 / m / 1e6, 1)}
+    flush = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device=dev)
+    def cold_before():
+        flush.fill_(1)
+        reset5()
+    ms = time_rotating(stream, [call5], reps, before=cold_before)
+    m, ci = mean_ci(ms)
+    entry["cold"] = {"us": round(m * 1e3, 2), "ci95_us": round(ci * 1e3, 2), "GBps": round(bytes5 / m / 1e6, 1),
+                     "how": "252 MB written before every timed call"}
+    entry["note"] = "a launch with three dependent trips to memory: latency, not bandwidth"
+    out["config5_allreduce_P64_K64_D32"] = entry
+    ar5.destroy()
+    del flush, rows5
+
     out["config5_kmeans_N2^22_D32_K64_P64"] = kmeans_case(dev, stream, reps=5)
     out["mf_ssp_U2^17_I2^14_k32_nnz2^23_P16"] = mf_case(dev, stream)
     return out
