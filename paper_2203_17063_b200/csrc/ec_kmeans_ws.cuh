@@ -98,6 +98,7 @@ __host__ __device__ inline Plan plan_of(int D, int K, bool partials, bool delta)
 #endif
     int a = (int)(512u / npad) - (int)acc;
     p.accs = a > EC_WS_ACCS ? EC_WS_ACCS : a < p.groups ? p.groups : a;
+    if (p.accs > p.groups && (p.accs & 1)) --p.accs;   // even, if that costs no group its accumulator: both search issuers can work
     uint32_t need = ((uint32_t)p.accs + acc) * npad, cols = 32;
     while (cols < need) cols <<= 1;
     p.tmem_cols = cols;
@@ -493,11 +494,15 @@ ws_fused_kernel(const __grid_constant__ CUtensorMap pmap, const float* __restric
             const uint64_t adesc0 = swz_desc<D>(sm_u + pl.stage);
             const uint64_t ones_desc = smem_desc(sm_u + pl.ones, 2048, 128), cnb_desc = smem_desc(sm_u + pl.cnb, (uint32_t)npad * 16, 128);
             const uint32_t stage_units = pl.stage_bytes >> 4;
-            // tile i = first, first + 2, ...: stage i mod stages on its laps-th use, accumulator i mod accs on its lapa-th
+            // tile i = first, first + step, ...: stage i mod stages on its laps-th use, accumulator i mod accs on its lapa-th.
+            // Both take part only when the numbers of stages and of accumulators are even: a stage and an accumulator then
+            // always meet the same issuer, which sees every phase of their barriers - an issuer that skipped a phase (the
+            // other one's) could find the barrier two phases back and take its parity for "done".
+            const int step = (NST % 2 == 0 && A % 2 == 0) ? 2 : 1;
             const int first = warp == 4 * G + 1 ? 0 : 1;
             int s = first % NST, a = first % A;
             uint32_t laps = (uint32_t)(first / NST), lapa = (uint32_t)(first / A);
-            for (;;) {
+            for (; first < step;) {
                 if (!wait_or_abort(B_full(s), laps & 1u, s_abort, 3)) { ok = false; break; }
                 if (s_desc[s].run < 0) break;
                 if (lapa > 0 && !wait_or_abort(B_accempty(a), (lapa - 1u) & 1u, s_abort, 4)) { ok = false; break; }
@@ -510,9 +515,9 @@ ws_fused_kernel(const __grid_constant__ CUtensorMap pmap, const float* __restric
                 mma_tf32(acc, ones_desc, cnb_desc, idesc, 1u);
                 mma_commit(B_accfull(a));
                 mma_commit(B_empty(s));                        // the tile has been read: its stage goes back to the producer
-                s += 2;
+                s += step;
                 while (s >= NST) { s -= NST; ++laps; }
-                a += 2;
+                a += step;
                 while (a >= A) { a -= A; ++lapa; }
             }
         }

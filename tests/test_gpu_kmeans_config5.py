@@ -106,9 +106,11 @@ def blocky_mixture(seed, N, D, K):
     return np.ascontiguousarray(points), np.ascontiguousarray(init.astype(np.float32))
 
 
+@pytest.mark.parametrize("N,K", [((1 << 21) + 1234, 64),       # four epilogue groups, a sums slot each
+                                 ((1 << 20) + 777, 90)])        # 96 score columns: three groups, three search accumulators
 @pytest.mark.parametrize("fed_by", ["checker", "library"])
-def test_many_runs_per_block_with_churn_against_the_checker(fed_by):
-    N, D, K, P, iters = (1 << 21) + 1234, 32, 64, 64, 5
+def test_many_runs_per_block_with_churn_against_the_checker(fed_by, N, K):
+    D, P, iters = 32, 64, 5
     points, init = blocky_mixture(4242, N, D, K)
     masks = inputs.kmeans_masks(4243, iters, P, K, 0.8)
     km = ec.KMeans(to_dev(points), K, P, to_dev(init))
@@ -139,5 +141,5 @@ def test_many_runs_per_block_with_churn_against_the_checker(fed_by):
         prev_labels = g_labels
         cents = new if fed_by == "checker" else to_host(d_cent)
     assert km.tc_status() == 0
-    assert moved > 10000                                        # labels did keep moving
+    assert moved > 5000                                         # labels did keep moving
     km.destroy()
