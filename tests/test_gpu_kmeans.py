@@ -97,6 +97,16 @@ def test_lockstep_each_tensor_core_kernel_on_its_own(N, D, K, P, path):
     lockstep(N, D, K, P, iters=3, seed=500 + K, path=path)
 
 
+@pytest.mark.parametrize("path", [0, 2, 3])
+@pytest.mark.parametrize("N,D,K,P", [(600011, 16, 128, 7), (500000, 32, 96, 5), (450001, 16, 33, 3), (700001, 32, 17, 9),
+                                     (520000, 16, 90, 64)])
+def test_lockstep_at_a_size_where_every_block_takes_many_tiles(N, D, K, P, path):
+    """The shapes with three and two epilogue groups, odd and even numbers of search accumulators and of stages, at sizes
+    where a thread block works through dozens of tiles and several runs (the small cases above leave most blocks with one
+    tile or none)."""
+    lockstep(N, D, K, P, iters=2, seed=900 + K + D, path=path)
+
+
 def test_exact_ties_take_the_lowest_index():
     pts = np.zeros((300, 4), dtype=np.float32)
     cents = np.array([[1, 0, 0, 0], [0, 1, 0, 0], [-1, 0, 0, 0], [0, 0, 0, 0.5]], dtype=np.float32)

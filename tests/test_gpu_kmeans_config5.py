@@ -106,11 +106,13 @@ def blocky_mixture(seed, N, D, K):
     return np.ascontiguousarray(points), np.ascontiguousarray(init.astype(np.float32))
 
 
-@pytest.mark.parametrize("N,K", [((1 << 21) + 1234, 64),       # four epilogue groups, a sums slot each
-                                 ((1 << 20) + 777, 90)])        # 96 score columns: three groups, three search accumulators
+@pytest.mark.parametrize("N,K,D", [((1 << 21) + 1234, 64, 32),    # four epilogue groups, a sums slot each
+                                   ((1 << 20) + 777, 90, 32),     # 96 score columns: three groups, three search accumulators
+                                   ((1 << 20) + 555, 128, 16),    # 128 score columns: two groups, two accumulators
+                                   ((1 << 20) + 333, 24, 16)])    # 32 score columns, 64-byte rows
 @pytest.mark.parametrize("fed_by", ["checker", "library"])
-def test_many_runs_per_block_with_churn_against_the_checker(fed_by, N, K):
-    D, P, iters = 32, 64, 5
+def test_many_runs_per_block_with_churn_against_the_checker(fed_by, N, K, D):
+    P, iters = 64, 5
     points, init = blocky_mixture(4242, N, D, K)
     masks = inputs.kmeans_masks(4243, iters, P, K, 0.8)
     km = ec.KMeans(to_dev(points), K, P, to_dev(init))
