@@ -39,11 +39,13 @@ def _rows_close(got, want, tol):
     return bool((err <= tol * np.linalg.norm(want, axis=1) + 1e-12).all())
 
 
-@pytest.mark.parametrize("k,P,slack", [(32, 8, 2), (64, 5, 1), (32, 1, 0), (32, 70, 3)])
-def test_lock_step_iterations(cuda_device, k, P, slack):
-    U, I, nnz, seg = 1500, 200, 30000, 16
+@pytest.mark.parametrize("k,P,slack,U,I,nnz,seg,iters", [(32, 8, 2, 1500, 200, 30000, 16, 6), (64, 5, 1, 1500, 200, 30000, 16, 6),
+                                                         (32, 1, 0, 1500, 200, 30000, 16, 6), (32, 70, 3, 1500, 200, 30000, 16, 6),
+                                                         # more rows than resident warps, item segments of the bench's size
+                                                         (32, 16, 1, 24000, 3000, 400000, 64, 2)])
+def test_lock_step_iterations(cuda_device, k, P, slack, U, I, nnz, seg, iters):
     d, gpu, ref = _setup(U, I, k, nnz, P, seg, 21 + P)
-    masks = inputs.mf_refresh_masks(31, 6, P, gpu.S, 0.5)
+    masks = inputs.mf_refresh_masks(31, iters, P, gpu.S, 0.5)
     for t, m in enumerate(masks):
         # both sides start the iteration from the checker's factors (rounded to fp32)
         gpu.set_factors(torch.from_numpy(ref.pu.astype(np.float32)).cuda(), torch.from_numpy(ref.qi.astype(np.float32)).cuda())
