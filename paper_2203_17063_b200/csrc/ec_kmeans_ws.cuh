@@ -153,7 +153,7 @@ struct TileDesc {
     int run;                     // run index (row block), -1: no more tiles
     int run_seq;                 // how many runs with tiles this block has started before this tile's run
     int last;                    // the run's last tile
-    int pad;
+    int pad;                     // the tile's number in the block's sequence (what a reader expects to find)
 };
 
 // One try; the thread may sleep in hardware until the phase completes or the hinted time (nanoseconds) has passed, so
@@ -451,7 +451,7 @@ ws_fused_kernel(const __grid_constant__ CUtensorMap pmap, const float* __restric
                 const int s = i % NST, use = i / NST;
                 if (use > 0 && !wait_or_abort(B_empty(s), (uint32_t)(use - 1) & 1u, s_abort, 1)) { ok = false; break; }
                 TileDesc d;
-                d.base = b0 + t * TILE; d.end = b1; d.run = run; d.run_seq = run_seq; d.last = tn >= ntiles ? 1 : 0; d.pad = 0;
+                d.base = b0 + t * TILE; d.end = b1; d.run = run; d.run_seq = run_seq; d.last = tn >= ntiles ? 1 : 0; d.pad = i;
                 s_desc[s] = d;
                 mbar_expect_tx(B_full(s), pl.stage_bytes);
                 tma_tile_2d(sm_u + pl.stage + (uint32_t)s * pl.stage_bytes, &pmap, 0, (int)(b0 + t * TILE), B_full(s));
@@ -465,7 +465,7 @@ ws_fused_kernel(const __grid_constant__ CUtensorMap pmap, const float* __restric
                 const int s = i % NST, use = i / NST;
                 if (use > 0 && !wait_or_abort(B_empty(s), (uint32_t)(use - 1) & 1u, s_abort, 1)) { ok = false; break; }
                 TileDesc d;
-                d.base = 0; d.end = 0; d.run = -1; d.run_seq = e; d.last = 0; d.pad = 0;
+                d.base = 0; d.end = 0; d.run = -1; d.run_seq = e; d.last = 0; d.pad = i;
                 s_desc[s] = d;
                 mbar_arrive(B_full(s));
                 ++i;
@@ -595,6 +595,7 @@ ws_fused_kernel(const __grid_constant__ CUtensorMap pmap, const float* __restric
         uint32_t lap = (uint32_t)(g / NST);
         int slot = PARTIALS ? g % SLOTS : 0;
         const bool own_slot = PARTIALS && DELTA && SLOTS == G;   // slot g belongs to group g alone
+        const bool seq_check = NST % G != 0;                  // a stage meets different groups in turn
         bool my_stale = false;                                // own_slot: this warp's rows of the slot have one-hot entries set
         int a = g % A;                                        // the tile's search accumulator, on its lapa-th use
         uint32_t lapa = (uint32_t)(g / A);
@@ -608,6 +609,17 @@ ws_fused_kernel(const __grid_constant__ CUtensorMap pmap, const float* __restric
                     slot += G;
                     while (slot >= SLOTS) slot -= SLOTS;
                 }
+            }
+            // When the stages do not divide evenly among the groups, the stage's previous tile was another group's and this
+            // group has not seen that phase of the barrier: it first waits until the producer has written this tile's
+            // descriptor (which it does only after the previous tile has been released, i.e. after that phase), so that the
+            // parity asked for below cannot be mistaken for the phase two back.
+            if (seq_check && lap > 0) {
+                const long long t0 = clock64();
+                while (reinterpret_cast<volatile TileDesc*>(s_desc)[s].pad != i) {
+                    if (*s_abort != 0 || clock64() - t0 > 4000000000LL) { if (*s_abort == 0) *s_abort = 2; ok = false; break; }
+                }
+                if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
             }
             if (!wwait(B_full(s), lap & 1u, 3)) { ok = false; break; }
             const TileDesc td = s_desc[s];
