@@ -248,11 +248,14 @@ def test_running_sums_follow_label_changes_over_many_iterations(N, D, K, P, iter
     full.destroy()
 
 
-def test_distance_bounds_change_nothing_but_the_time():
+@pytest.mark.parametrize("N,D,K,P", [(40000 + 77, 32, 16, 5),
+                                     # every block takes many tiles and several runs; four, three and two epilogue groups
+                                     (900001, 32, 64, 64), (700011, 32, 90, 7), (600013, 16, 128, 6)])
+def test_distance_bounds_change_nothing_but_the_time(N, D, K, P):
     """The same iterations with and without the distance bounds: labels, counts and centroids must be the same,
     whether tiles are skipped (separated clusters), searched again (two clusters that overlap and keep
     exchanging points) or the centroids are replaced from outside (two of them swapped: every bound is void)."""
-    N, D, K, P, iters = 40000 + 77, 32, 16, 5, 12
+    iters = 12
     rng = np.random.default_rng(31)
     centres = rng.uniform(-10, 10, size=(K, D)).astype(np.float32)
     centres[1] = centres[0] + 0.3                                       # clusters 0 and 1 overlap almost entirely
