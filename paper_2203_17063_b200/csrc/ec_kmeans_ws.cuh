@@ -595,7 +595,6 @@ ws_fused_kernel(const __grid_constant__ CUtensorMap pmap, const float* __restric
         uint32_t lap = (uint32_t)(g / NST);
         int slot = PARTIALS ? g % SLOTS : 0;
         const bool own_slot = PARTIALS && DELTA && SLOTS == G;   // slot g belongs to group g alone
-        const bool seq_check = NST % G != 0;                  // a stage meets different groups in turn
         bool my_stale = false;                                // own_slot: this warp's rows of the slot have one-hot entries set
         int a = g % A;                                        // the tile's search accumulator, on its lapa-th use
         uint32_t lapa = (uint32_t)(g / A);
@@ -610,19 +609,21 @@ ws_fused_kernel(const __grid_constant__ CUtensorMap pmap, const float* __restric
                     while (slot >= SLOTS) slot -= SLOTS;
                 }
             }
+            if (!wwait(B_full(s), lap & 1u, 3)) { ok = false; break; }
+            TileDesc td = s_desc[s];
             // When the stages do not divide evenly among the groups, the stage's previous tile was another group's and this
-            // group has not seen that phase of the barrier: it first waits until the producer has written this tile's
-            // descriptor (which it does only after the previous tile has been released, i.e. after that phase), so that the
-            // parity asked for below cannot be mistaken for the phase two back.
-            if (seq_check && lap > 0) {
+            // group has not seen that phase of the barrier: had that phase not been over yet, the parity asked for above
+            // would have been taken for done two phases early.  The descriptor tells: the producer writes this tile's only
+            // after the previous tile has been released, i.e. after that phase.  (Never seen to happen; one compare.)
+            if (td.pad != i) {
                 const long long t0 = clock64();
                 while (reinterpret_cast<volatile TileDesc*>(s_desc)[s].pad != i) {
                     if (*s_abort != 0 || clock64() - t0 > 4000000000LL) { if (*s_abort == 0) *s_abort = 2; ok = false; break; }
                 }
                 if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
+                if (!wwait(B_full(s), lap & 1u, 3)) { ok = false; break; }
+                td = s_desc[s];
             }
-            if (!wwait(B_full(s), lap & 1u, 3)) { ok = false; break; }
-            const TileDesc td = s_desc[s];
             if (td.run < 0) {                                // no more tiles: the sums issuer hears it from the first group that does
                 if (PARTIALS && td.run_seq == 0) {          // (the first of the G end markers)
                     if (n > 0 && !wwait(B_tiledone(g), (uint32_t)(n - 1) & 1u, 12 | (i << 8))) { ok = false; break; }
