@@ -109,7 +109,8 @@ def blocky_mixture(seed, N, D, K):
 @pytest.mark.parametrize("N,K,D", [((1 << 21) + 1234, 64, 32),    # four epilogue groups, a sums slot each
                                    ((1 << 20) + 777, 90, 32),     # 96 score columns: three groups, three search accumulators
                                    ((1 << 20) + 555, 128, 16),    # 128 score columns: two groups, two accumulators
-                                   ((1 << 20) + 333, 24, 16)])    # 32 score columns, 64-byte rows
+                                   ((1 << 20) + 333, 24, 16),     # 32 score columns, 64-byte rows
+                                   ((1 << 19) + 111, 200, 32)])   # beyond the warp-specialised kernel: the register-staged one alone
 @pytest.mark.parametrize("fed_by", ["checker", "library"])
 def test_many_runs_per_block_with_churn_against_the_checker(fed_by, N, K, D):
     P, iters = 64, 5
