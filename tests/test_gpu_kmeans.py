@@ -107,6 +107,13 @@ def test_lockstep_at_a_size_where_every_block_takes_many_tiles(N, D, K, P, path)
     lockstep(N, D, K, P, iters=2, seed=900 + K + D, path=path)
 
 
+@pytest.mark.parametrize("N,D,K,P", [(300001, 64, 9, 4), (400003, 8, 5, 3), (250001, 128, 4, 2), (200003, 12, 6, 5),
+                                     (350001, 4, 3, 7), (300007, 32, 300, 6)])
+def test_lockstep_at_that_size_on_the_fp32_kernels(N, D, K, P):
+    """Shapes outside the tensor-core kernels (other D, more than 256 centroids), many tiles per block."""
+    lockstep(N, D, K, P, iters=2, seed=700 + K + D)
+
+
 def test_exact_ties_take_the_lowest_index():
     pts = np.zeros((300, 4), dtype=np.float32)
     cents = np.array([[1, 0, 0, 0], [0, 1, 0, 0], [-1, 0, 0, 0], [0, 0, 0, 0.5]], dtype=np.float32)
