@@ -209,6 +209,15 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     return u;
 }
 
+// One 16-byte chunk of a one-hot row: the bf16 number `one` (0x3F80 = 1.0, 0xBF80 = -1.0) at position pos (0..7) of eight,
+// zeros elsewhere.  (Selects, not an array indexed by pos: that would live in local memory.)
+__device__ __forceinline__ uint4 onehot_chunk(int pos, uint32_t one) {
+    const uint32_t v = one << (16 * (pos & 1));
+    const int q = (pos & 7) >> 1;
+    return make_uint4(q == 0 ? v : 0u, q == 1 ? v : 0u, q == 2 ? v : 0u, q == 3 ? v : 0u);
+}
+__device__ __forceinline__ uint4 or4(uint4 a, uint4 b) { return make_uint4(a.x | b.x, a.y | b.y, a.z | b.z, a.w | b.w); }
+
 __device__ __forceinline__ float min3(float a, float b, float c) {
     float d;
     asm("min.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
@@ -676,16 +685,13 @@ tc_fused_kernel(const float* __restrict__ points, size_t N, int P, int C, const 
         if (PARTIALS && done) {
             if (changed) {
                 // one-hot row of this point: 16-byte chunk kb/8, bf16 1.0 at position kb%8 (and -1.0 for the old label)
-                uint32_t wv[4] = {0u, 0u, 0u, 0u};
-                wv[(kb & 7) >> 1] = 0x3F80u << (16 * (kb & 1));
+                uint4 wv = onehot_chunk(kb, 0x3F80u);
                 prev_chunk = kb >> 3;
-                if (old >= 0 && (old >> 3) == prev_chunk) wv[(old & 7) >> 1] |= 0xBF80u << (16 * (old & 1));
-                *reinterpret_cast<uint4*>(s_oh + (size_t)prev_chunk * OCHUNK + (size_t)tid * 16) = make_uint4(wv[0], wv[1], wv[2], wv[3]);
+                if (old >= 0 && (old >> 3) == prev_chunk) wv = or4(wv, onehot_chunk(old, 0xBF80u));
+                *reinterpret_cast<uint4*>(s_oh + (size_t)prev_chunk * OCHUNK + (size_t)tid * 16) = wv;
                 if (old >= 0 && (old >> 3) != prev_chunk) {
-                    uint32_t wo[4] = {0u, 0u, 0u, 0u};
-                    wo[(old & 7) >> 1] = 0xBF80u << (16 * (old & 1));
                     prev_chunk2 = old >> 3;
-                    *reinterpret_cast<uint4*>(s_oh + (size_t)prev_chunk2 * OCHUNK + (size_t)tid * 16) = make_uint4(wo[0], wo[1], wo[2], wo[3]);
+                    *reinterpret_cast<uint4*>(s_oh + (size_t)prev_chunk2 * OCHUNK + (size_t)tid * 16) = onehot_chunk(old, 0xBF80u);
                 }
             }
             fence_async_smem();

@@ -773,16 +773,13 @@ ws_fused_kernel(const __grid_constant__ CUtensorMap pmap, const float* __restric
                     uint16_t nv = 0xFFFFu;
                     if (changed) {
                         // one-hot row of this point: 16-byte chunk kb/8, bf16 1.0 at position kb%8 (and -1.0 for the label it leaves)
-                        uint32_t wv[4] = {0u, 0u, 0u, 0u};
-                        wv[(kb & 7) >> 1] = 0x3F80u << (16 * (kb & 1));
+                        uint4 wv = tc::onehot_chunk(kb, 0x3F80u);
                         const int ck = kb >> 3;
-                        if (old >= 0 && (old >> 3) == ck) wv[(old & 7) >> 1] |= 0xBF80u << (16 * (old & 1));
-                        *reinterpret_cast<uint4*>(oh + (size_t)ck * OCHUNK + (size_t)t * 16) = make_uint4(wv[0], wv[1], wv[2], wv[3]);
+                        if (old >= 0 && (old >> 3) == ck) wv = tc::or4(wv, tc::onehot_chunk(old, 0xBF80u));
+                        *reinterpret_cast<uint4*>(oh + (size_t)ck * OCHUNK + (size_t)t * 16) = wv;
                         nv = (uint16_t)(0xFF00u | (uint32_t)ck);
                         if (old >= 0 && (old >> 3) != ck) {
-                            uint32_t wo[4] = {0u, 0u, 0u, 0u};
-                            wo[(old & 7) >> 1] = 0xBF80u << (16 * (old & 1));
-                            *reinterpret_cast<uint4*>(oh + (size_t)(old >> 3) * OCHUNK + (size_t)t * 16) = make_uint4(wo[0], wo[1], wo[2], wo[3]);
+                            *reinterpret_cast<uint4*>(oh + (size_t)(old >> 3) * OCHUNK + (size_t)t * 16) = tc::onehot_chunk(old, 0xBF80u);
                             nv = (uint16_t)(((uint32_t)(old >> 3) << 8) | (uint32_t)ck);
                         }
                         // bf16 high and low parts of the row (low = bf16(x - high)): chunk column 2 kc resp. 2 kc + 1
