@@ -346,3 +346,41 @@ def test_many_runs_per_block_with_churn():
         if t:
             moved += int((l0 != traces[1][t - 1][1]).sum())
     assert moved > 10000
+
+
+def test_two_contexts_on_two_streams_do_not_disturb_each_other():
+    """Contexts are independent (ec.h): two of them iterate at the same time on two streams, on different data and
+    shapes (one per tensor-core kernel layout), and each ends where it ends when it runs alone."""
+    shapes = [(300001, 32, 64, 16, 11), (260003, 16, 128, 4, 12)]
+    data = []
+    for N, D, K, P, seed in shapes:
+        points, comp, _ = inputs.kmeans_mixture(seed, N, D, K, sigma=1.0, box=2.5)      # overlapping: labels keep moving
+        init = points[np.random.default_rng(seed).choice(N, K, replace=False)].copy()
+        masks = [to_dev(np.ascontiguousarray(m).view(np.int64)) for m in inputs.kmeans_masks(seed + 1, 6, P, K, 0.8)]
+        data.append((to_dev(points), to_dev(init), masks, N, D, K, P))
+
+    def run(order):
+        kms = [ec.KMeans(d[0], d[5], d[6], d[1]) for d in data]
+        streams = [torch.cuda.Stream(), torch.cuda.Stream()] if order == "together" else [None, None]
+        torch.cuda.synchronize()
+        for t in range(6):
+            for i, km in enumerate(kms):
+                km.iterate(data[i][2][t], stream=streams[i])
+            if order == "alone":
+                torch.cuda.synchronize()
+        torch.cuda.synchronize()
+        out = []
+        for i, km in enumerate(kms):
+            N, D, K = data[i][3], data[i][4], data[i][5]
+            c = torch.empty(K, D, device="cuda")
+            lab = torch.empty(N, dtype=torch.int32, device="cuda")
+            km.get(c, lab)
+            torch.cuda.synchronize()
+            assert km.tc_status() == 0
+            out.append((to_host(c), to_host(lab)))
+            km.destroy()
+        return out
+
+    alone, together = run("alone"), run("together")
+    for (c0, l0), (c1, l1) in zip(alone, together):
+        assert np.array_equal(l0, l1) and np.array_equal(c0, c1)
